@@ -1,0 +1,389 @@
+"""Pins for the CPU oracle: everything here checks ``oracle/`` against something other than
+itself -- hand-derived values of a worked example (Eq. 8-10), closed forms, NumPy/PyTorch
+library routines on special cases, brute-force enumeration on tiny inputs and invariants
+the paper's statements imply.  No GPU, no CUDA library."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "fig1_style_6x6.txt")
+
+
+def _load_fig1():
+    mat, nsi_rows, keep_rows = [], [], []
+    mode = None
+    for line in open(GOLDEN):
+        line = line.split("#")[0].strip()
+        if not line:
+            continue
+        tok = line.split()
+        if tok[0] == "matrix":
+            mode = "matrix"
+        elif tok[0] == "nsi":
+            nsi_rows.append((float(tok[1]), [float(t) for t in tok[2:]]))
+        elif tok[0] == "keep":
+            keep_rows.append((float(tok[1]), int(tok[2]), [int(t) for t in tok[3:]]))
+        elif mode == "matrix":
+            mat.append([float(t) for t in tok])
+    return np.array(mat, dtype=np.float32), nsi_rows, keep_rows
+
+
+# ---------------------------------------------------------------------------------------------
+# worked example (Fig. 1 style), Eq. 8-10 by hand
+# ---------------------------------------------------------------------------------------------
+
+def test_fig1_style_worked_example(oracle):
+    m, nsi_rows, keep_rows = _load_fig1()
+    assert m.shape == (6, 6)
+    shape = (6, 6, 3, 3)
+    for alpha, expected in nsi_rows:
+        ref, f32, bad = oracle.nsi(m.reshape(-1), shape, alpha)
+        assert bad == 0
+        np.testing.assert_allclose(ref, expected, atol=6e-7, rtol=0)
+        np.testing.assert_allclose(f32, expected, atol=2e-6, rtol=0)
+    for alpha, k, kept in keep_rows:
+        _, f32, _ = oracle.nsi(m.reshape(-1), shape, alpha)
+        sel, thr = oracle.select(f32, k)
+        assert sel.tolist() == kept
+        assert thr == min(f32[kept])
+
+
+def test_fig1_style_exact_closed_forms(oracle):
+    m, _, _ = _load_fig1()
+    for alpha in (0.5, 0.25, 1.0, 0.0):
+        ref, _, _ = oracle.nsi(m.reshape(-1), (6, 6, 3, 3), alpha)
+        a32 = float(np.float32(alpha))
+        n3 = np.array([-0.4, -0.3, -0.2, -0.1, 0.0, 0.1, 0.2, 0.3, 0.4], dtype=np.float32).astype(np.float64)
+        exact = [
+            a32 * 2.0,
+            a32 * 1.0 + (1 - a32) * math.sqrt(80.0 / 81.0),
+            a32 * 1.0 + (1 - a32) * math.sqrt(8.0),
+            a32 * np.abs(n3).mean() + (1 - a32) * math.sqrt(((n3 - n3.mean()) ** 2).mean()),
+        ]
+        np.testing.assert_allclose(ref, exact, rtol=1e-13)
+
+
+def test_elementwise_topk_differs_from_neighborhood_choice(oracle):
+    """The contrast the figure's caption draws: the 18 largest entries by magnitude are the 9,
+    the nine 2's and eight of the +-1's, whereas k = 2 neighborhoods keeps N0 and N2 whole."""
+    m, _, _ = _load_fig1()
+    flat = np.abs(m.reshape(-1))
+    top18 = np.argsort(-flat, kind="stable")[:18]
+    rows, cols = np.unravel_index(top18, (6, 6))
+    tiles = set(((rows // 3) * 2 + cols // 3).tolist())
+    assert tiles == {0, 1, 2}
+    _, f32, _ = oracle.nsi(m.reshape(-1), (6, 6, 3, 3), 0.5)
+    sel, _ = oracle.select(f32, 2)
+    assert sel.tolist() == [0, 2]
+
+
+# ---------------------------------------------------------------------------------------------
+# NSI against library routines and closed forms
+# ---------------------------------------------------------------------------------------------
+
+def _numpy_tile_stats(v, rows, cols, nh, nw, alpha):
+    x = v.reshape(rows, cols).astype(np.float64)
+    out = []
+    for tr in range(-(-rows // nh)):
+        for tc in range(-(-cols // nw)):
+            t = x[tr * nh:(tr + 1) * nh, tc * nw:(tc + 1) * nw]
+            out.append(alpha * np.mean(np.abs(t)) + (1 - alpha) * np.std(t))  # np.std: ddof=0
+    return np.array(out)
+
+
+@pytest.mark.parametrize("rows,cols,nh,nw", [(6, 6, 3, 3), (7, 11, 3, 3), (4, 4, 3, 3), (5, 45, 3, 3),
+                                             (12, 9, 1, 9), (1, 64, 1, 9), (10, 14, 2, 5), (3, 3, 3, 3),
+                                             (8, 6, 4, 2), (1, 1, 3, 3)])
+def test_nsi_matches_numpy_mean_and_std_per_tile(oracle, rows, cols, nh, nw):
+    rng = np.random.default_rng(rows * 1000 + cols)
+    v = (rng.standard_normal(rows * cols) * 10 ** rng.uniform(-4, 1)).astype(np.float32)
+    v += np.float32(0.3) * np.float32(np.abs(v).mean())  # non-zero mean so the mean term matters
+    for alpha in (0.5, 0.25, 0.0, 1.0):
+        a32 = float(np.float32(alpha))
+        ref, f32, bad = oracle.nsi(v, (rows, cols, nh, nw), alpha)
+        expect = _numpy_tile_stats(v, rows, cols, nh, nw, a32)
+        assert bad == 0 and ref.size == oracle.tile_count(rows, cols, nh, nw) == expect.size
+        np.testing.assert_allclose(ref, expect, rtol=1e-12, atol=0)
+        np.testing.assert_allclose(f32, expect, rtol=2e-6, atol=1e-30)
+
+
+def test_nsi_constant_tile_and_single_spike(oracle):
+    c = np.full(9, -3.25, dtype=np.float32)
+    ref, f32, _ = oracle.nsi(c, (3, 3, 3, 3), 0.5)
+    assert ref[0] == 0.5 * 3.25 and f32[0] == np.float32(0.5 * 3.25)  # std term vanishes
+    spike = np.zeros(9, dtype=np.float32)
+    spike[4] = 9.0
+    ref, f32, _ = oracle.nsi(spike, (3, 3, 3, 3), 0.25)
+    np.testing.assert_allclose(ref[0], 0.25 * 1.0 + 0.75 * math.sqrt(8.0), rtol=1e-14)
+    zeros = np.zeros(18, dtype=np.float32)
+    ref, f32, _ = oracle.nsi(zeros, (3, 6, 3, 3), 0.5)
+    assert (ref == 0).all() and (f32 == 0).all() and not np.signbit(f32).any()
+
+
+def test_nsi_1x1_tiles_reduce_to_alpha_abs(oracle):
+    rng = np.random.default_rng(3)
+    v = rng.standard_normal(50).astype(np.float32)
+    ref, f32, _ = oracle.nsi(v, (5, 10, 1, 1), 0.5)
+    np.testing.assert_array_equal(ref, 0.5 * np.abs(v.astype(np.float64)))
+    np.testing.assert_array_equal(f32, np.float32(0.5) * np.abs(v))
+
+
+def test_nsi_homogeneity_and_rms_bounds(oracle):
+    rng = np.random.default_rng(4)
+    v = rng.standard_normal(9 * 40).astype(np.float32)
+    shape = (3, 120, 3, 3)
+    ref, f32, _ = oracle.nsi(v, shape, 0.5)
+    for c in (4.0, -0.125, 1024.0):
+        ref_c, f32_c, _ = oracle.nsi(v * np.float32(c), shape, 0.5)
+        np.testing.assert_array_equal(ref_c, abs(c) * ref)      # powers of two: exact
+        np.testing.assert_array_equal(f32_c, np.float32(abs(c)) * f32)
+    ref3, _, _ = oracle.nsi(v * np.float32(3.0), shape, 0.5)
+    np.testing.assert_allclose(ref3, 3.0 * ref, rtol=1e-6)
+    # mean|v| <= rms and std <= rms, hence NSI <= rms for alpha in [0, 1]
+    rms = np.sqrt((v.reshape(3, 40, 3).astype(np.float64) ** 2).transpose(1, 0, 2).reshape(40, 9).mean(axis=1))
+    for alpha in (0.0, 0.5, 1.0):
+        r, _, _ = oracle.nsi(v, shape, alpha)
+        assert (r <= rms * (1 + 1e-12)).all()
+
+
+def test_nsi_invariant_under_permutation_inside_a_tile(oracle):
+    rng = np.random.default_rng(5)
+    tiles = rng.standard_normal((30, 9)).astype(np.float32)
+    perm = tiles.copy()
+    for t in perm:
+        rng.shuffle(t)
+    shape = (30, 9, 1, 9)
+    a, _, _ = oracle.nsi(tiles.reshape(-1), shape, 0.5)
+    b, _, _ = oracle.nsi(perm.reshape(-1), shape, 0.5)
+    np.testing.assert_allclose(a, b, rtol=1e-12)
+
+
+def test_nsi_tile_geometry_is_row_major_not_transposed(oracle):
+    """A 2x3 tiling of a 4x6 matrix with one hot entry per tile pins tile indexing."""
+    rows, cols, nh, nw = 4, 6, 2, 3
+    for i in range(rows):
+        for j in range(cols):
+            v = np.zeros(rows * cols, dtype=np.float32)
+            v[i * cols + j] = 1.0
+            ref, _, _ = oracle.nsi(v, (rows, cols, nh, nw), 1.0)
+            hot = (i // nh) * 2 + (j // nw)
+            expect = np.zeros(4)
+            expect[hot] = 1.0 / 6.0
+            np.testing.assert_allclose(ref, expect, rtol=1e-15)
+
+
+def test_nsi_nonfinite_is_counted_and_ranked_first(oracle):
+    v = np.ones(27, dtype=np.float32)
+    v[13] = np.inf
+    v[25] = np.nan
+    ref, f32, bad = oracle.nsi(v, (3, 9, 3, 3), 0.5)
+    assert bad == 2 and np.isposinf(f32[1]) and np.isposinf(f32[2]) and np.isfinite(f32[0])
+    sel, _ = oracle.select(f32, 1)
+    assert sel.tolist() == [1]
+
+
+# ---------------------------------------------------------------------------------------------
+# accumulation (Eq. 12)
+# ---------------------------------------------------------------------------------------------
+
+def test_accumulate_f32_is_one_ieee_add(oracle):
+    rng = np.random.default_rng(6)
+    g = rng.standard_normal(1000).astype(np.float32)
+    r = (rng.standard_normal(1000) * 1e-3).astype(np.float32)
+    np.testing.assert_array_equal(oracle.accumulate(g, r), g + r)
+    exact = g.astype(np.float64) + r.astype(np.float64)
+    assert (np.abs(oracle.accumulate(g, r) - exact) <= np.abs(exact) * 2.0 ** -24).all()
+
+
+def test_accumulate_bf16_widens_exactly(oracle):
+    from paper_2312_17530_b200 import synth
+
+    rng = np.random.default_rng(7)
+    x = rng.standard_normal(4096).astype(np.float32)
+    bits = synth.f32_to_bf16_bits(x)
+    t = torch.from_numpy(x).to(torch.bfloat16)
+    np.testing.assert_array_equal(bits.view(np.int16), t.view(torch.int16).numpy())  # generator == torch RNE
+    r = rng.standard_normal(4096).astype(np.float32)
+    v = oracle.accumulate(bits, r)
+    np.testing.assert_array_equal(v, (t.to(torch.float32) + torch.from_numpy(r)).numpy())
+
+
+# ---------------------------------------------------------------------------------------------
+# keep count (Eq. 11) and selection
+# ---------------------------------------------------------------------------------------------
+
+def test_keep_count_examples(oracle):
+    assert oracle.keep_count(29241, 1 / 64) == 457           # 171 x 171 tiles of a 512 x 512 matrix
+    assert oracle.keep_count(64 * 3, 1 / 64) == 3            # divisible case of Eq. 11
+    assert oracle.keep_count(64 * 3 + 1, 1 / 64) == 4
+    assert oracle.keep_count(100, 0.0) == 1                  # a layer always sends one neighborhood ...
+    assert oracle.keep_count(100, 0.0, clamp_min1=False) == 0  # ... unless the clamp is off
+    assert oracle.keep_count(100, 1.0) == 100
+    assert oracle.keep_count(100, 7.5) == 100
+    assert oracle.keep_count(7, 0.5) == 4
+    # the ratio is a binary32 number; the product is taken in binary64
+    assert oracle.keep_count(10, 0.1) == math.ceil(10 * float(np.float32(0.1)))
+    assert oracle.keep_count(1 << 20, 0.001) == math.ceil((1 << 20) * float(np.float32(0.001)))
+
+
+def test_select_1x1_alpha1_is_library_topk(oracle):
+    rng = np.random.default_rng(8)
+    v = rng.standard_normal(5000).astype(np.float32)
+    assert np.unique(np.abs(v)).size == v.size
+    _, f32, _ = oracle.nsi(v, (50, 100, 1, 1), 1.0)
+    for k in (1, 17, 500, 4999, 5000):
+        sel, thr = oracle.select(f32, k)
+        ref = torch.topk(torch.from_numpy(np.abs(v)), k).indices.numpy()
+        assert sel.tolist() == sorted(ref.tolist())
+        part = np.argpartition(-np.abs(v), k - 1)[:k]
+        assert sel.tolist() == sorted(part.tolist())
+        assert thr == np.abs(v)[sel].min()
+
+
+def test_select_brute_force_small(oracle):
+    rng = np.random.default_rng(9)
+    for trial in range(40):
+        K = int(rng.integers(1, 11))
+        # few distinct values => many ties
+        nsi = rng.integers(0, 4, size=K).astype(np.float32) * np.float32(0.5)
+        for k in range(0, K + 1):
+            sel, _ = oracle.select(nsi, k)
+            best, best_sets = None, []
+            for comb in itertools.combinations(range(K), k):
+                s = float(sum(nsi[list(comb)]))
+                if best is None or s > best + 1e-12:
+                    best, best_sets = s, [comb]
+                elif abs(s - best) <= 1e-12:
+                    best_sets.append(comb)
+            assert tuple(sel.tolist()) == min(best_sets)  # lexicographically smallest maximiser
+
+
+def test_select_pure_ties_take_lowest_indices(oracle):
+    nsi = np.full(100, 0.75, dtype=np.float32)
+    sel, thr = oracle.select(nsi, 13)
+    assert sel.tolist() == list(range(13)) and thr == 0.75
+
+
+# ---------------------------------------------------------------------------------------------
+# payload, accumulator update, conservation
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("shape", [(7, 11, 3, 3), (12, 9, 1, 9), (1, 50, 1, 9), (64, 45, 3, 3), (9, 9, 3, 3)])
+def test_compress_layer_invariants(oracle, shape):
+    rows, cols, nh, nw = shape
+    rng = np.random.default_rng(rows + cols)
+    g = rng.standard_normal(rows * cols).astype(np.float32)
+    r = (rng.standard_normal(rows * cols) * 0.1).astype(np.float32)
+    res = oracle.compress_layer(g, r, shape, 0.3, 0.5)
+    K = oracle.tile_count(*shape)
+    assert res.k == math.ceil(K * float(np.float32(0.3))) == res.idx.size
+    assert (np.diff(res.idx) > 0).all() and res.val.size == res.k * nh * nw
+    # every tile above the threshold is kept, none below
+    kept = np.zeros(K, bool)
+    kept[res.idx] = True
+    assert (res.nsi_f32[kept] >= res.threshold).all() and (res.nsi_f32[~kept] <= res.threshold).all()
+    # sent + residual == accumulated input, elementwise; residual is zero exactly on sent tiles
+    sent = np.zeros(rows * cols, dtype=np.float32)
+    oracle.decompress_into(sent, shape, res.idx, res.val, 1.0)
+    assert (sent + res.residual == res.v).all()
+    TC = -(-cols // nw)
+    tile_of = (np.arange(rows)[:, None] // nh) * TC + (np.arange(cols)[None, :] // nw)
+    on_sent = kept[tile_of.reshape(-1)]
+    assert (res.residual[on_sent] == 0).all() and not np.signbit(res.residual[on_sent]).any()
+    np.testing.assert_array_equal(res.residual[~on_sent], res.v[~on_sent])
+    np.testing.assert_array_equal(sent[on_sent], res.v[on_sent])
+    # padded payload slots of clipped tiles are +0
+    vals = res.val.reshape(res.k, nh, nw)
+    for s, t in enumerate(res.idx.tolist()):
+        tr, tc = divmod(t, TC)
+        hh, ww = min(nh, rows - tr * nh), min(nw, cols - tc * nw)
+        block = res.v.reshape(rows, cols)[tr * nh:tr * nh + hh, tc * nw:tc * nw + ww]
+        np.testing.assert_array_equal(vals[s, :hh, :ww], block)
+        pad = vals[s].copy()
+        pad[:hh, :ww] = 1.0
+        assert ((pad == 1.0) | ((pad == 0.0) & ~np.signbit(pad))).all()
+
+
+def test_multi_iteration_conservation(oracle):
+    """Eq. 12: over T iterations, everything sent plus the final accumulator equals the sum
+    of all gradients (up to binary32 rounding of the running adds)."""
+    shape = (30, 27, 3, 3)
+    rng = np.random.default_rng(10)
+    r = np.zeros(30 * 27, dtype=np.float32)
+    total = np.zeros(30 * 27, dtype=np.float64)
+    sent_total = np.zeros(30 * 27, dtype=np.float64)
+    for _ in range(12):
+        g = rng.standard_normal(30 * 27).astype(np.float32)
+        total += g
+        res = oracle.compress_layer(g, r, shape, 0.1, 0.5)
+        s = np.zeros_like(r)
+        oracle.decompress_into(s, shape, res.idx, res.val, 1.0)
+        sent_total += s
+        r = res.residual
+    np.testing.assert_allclose(sent_total + r, total, atol=12 * 2.0 ** -22, rtol=0)
+
+
+# ---------------------------------------------------------------------------------------------
+# aggregation (Eq. 12 third line / Sync)
+# ---------------------------------------------------------------------------------------------
+
+def test_decompress_special_cases(oracle):
+    shape = (10, 10, 3, 3)
+    rng = np.random.default_rng(11)
+    g = rng.standard_normal(100).astype(np.float32)
+    res = oracle.compress_layer(g, np.zeros(100, np.float32), shape, 0.25, 0.5)
+    dense = np.zeros(100, np.float32)
+    oracle.decompress_into(dense, shape, res.idx, res.val, 1.0)
+    sent = res.v - res.residual
+    np.testing.assert_array_equal(dense, sent)                      # one worker: dense == sent
+    oracle.decompress_into(dense, shape, res.idx, res.val, 1.0)
+    np.testing.assert_array_equal(dense, 2 * sent)                  # two identical workers
+    before = dense.copy()
+    oracle.decompress_into(dense, shape, np.zeros(0, np.int32), np.zeros(0, np.float32), 1.0)
+    np.testing.assert_array_equal(dense, before)                    # empty payload
+    d2 = np.ones(100, np.float32)
+    oracle.decompress_into(d2, shape, res.idx, res.val, 0.25)
+    np.testing.assert_array_equal(d2, np.float32(1) + np.float32(0.25) * sent)
+
+
+# ---------------------------------------------------------------------------------------------
+# layer-wise ratio rule (Eq. 3-5)
+# ---------------------------------------------------------------------------------------------
+
+def test_update_ratios_against_numpy_sort(oracle):
+    rng = np.random.default_rng(12)
+    sizes = [64, 1000, 9, 4096, 1]
+    scales = [1.0, 0.1, 5.0, 0.5, 0.0]
+    w = [(rng.standard_normal(n) * s).astype(np.float32) for n, s in zip(sizes, scales)]
+    for rho in (0.001, 0.02, 0.5, 1.0):
+        ratios, surv, n_keep = oracle.update_ratios(w, rho)
+        G = sum(sizes)
+        assert n_keep == math.ceil(float(np.float32(rho)) * G) == surv.sum()   # sum_l c_l = ceil(rho G)
+        flat = np.abs(np.concatenate(w))
+        order = np.argsort(-flat.astype(np.float64), kind="stable")[:n_keep]     # stable: ties -> lower index
+        owner = np.searchsorted(np.cumsum(sizes), order, side="right")
+        expect = np.bincount(owner, minlength=len(sizes))
+        np.testing.assert_array_equal(surv, expect)
+        np.testing.assert_array_equal(ratios, (expect / np.array(sizes)).astype(np.float32))
+
+
+def test_update_ratios_uniform_and_scaled_layer(oracle):
+    rng = np.random.default_rng(13)
+    w = [rng.standard_normal(20000).astype(np.float32) for _ in range(5)]
+    ratios, _, _ = oracle.update_ratios(w, 0.02)
+    np.testing.assert_allclose(ratios, 0.02, rtol=0.25)              # identical distributions => rho_l ~ rho
+    w2 = [x.copy() for x in w]
+    w2[2] *= np.float32(1000.0)
+    r2, surv2, n_keep = oracle.update_ratios(w2, 0.02)
+    assert n_keep == 2000 and r2[2] > 0.09 and all(r2[i] < ratios[i] for i in (0, 1, 3, 4))
+
+
+def test_update_ratios_ties_go_to_lower_flat_index(oracle):
+    w = [np.ones(10, np.float32), -np.ones(10, np.float32), np.ones(10, np.float32)]
+    ratios, surv, n_keep = oracle.update_ratios(w, 0.5)
+    assert n_keep == 15 and surv.tolist() == [10, 5, 0]
+    np.testing.assert_array_equal(ratios, np.array([1.0, 0.5, 0.0], np.float32))
