@@ -1,0 +1,216 @@
+/*
+ * rsdgc.h -- C ABI of the B200 (sm_100a) RS-DGC gradient-compression library.
+ *
+ * The library implements the per-iteration compression step of RS-DGC (arxiv 2312.17530):
+ * local gradient accumulation (Eq. 12), the Neighborhood Statistical Indicator of every
+ * gradient neighborhood (Eq. 8-10), the per-layer keep count (Eq. 11), the choice of the
+ * top neighborhoods of each layer (Algorithm 1, second half), the payload of kept values
+ * plus neighborhood indices (Sec. III-C), the same-device aggregation of several workers'
+ * payloads (Eq. 12 third line / Eq. 2 "Sync"), and the layer-wise dynamic compression
+ * ratio from the weights (Eq. 3-5, Algorithm 1 first half).
+ *
+ * Conventions
+ *  - Every function returns an int: RSDGC_OK (0) or a negative rsdgc_error.  Nothing
+ *    throws, aborts or prints.  Argument errors are reported synchronously; conditions that
+ *    are only known on the device (non-finite indicator, payload capacity exceeded) are
+ *    recorded in a device status word read by rsdgc_get_status().
+ *  - "dev" pointers are device memory of the plan's device, owned by the caller; "host"
+ *    pointers are host memory.  The library allocates only the plan (a host struct plus
+ *    small device tables).  No call reads device memory on the host except
+ *    rsdgc_get_status() and rsdgc_compress_host(), which synchronise the stream.
+ *  - `stream` is a CUDA stream handle (cudaStream_t passed as void*; NULL = default
+ *    stream).  All device work is enqueued on it and is asynchronous.  A plan holds
+ *    per-layer scratch tables, so at most one call per plan may be in flight at a time:
+ *    issue all calls that share a plan on one stream (or order them yourself).
+ *  - Layout: a layer l is a row-major rows x cols matrix partitioned into nh x nw
+ *    neighborhoods ("tiles"; edge tiles are clipped).  TC = ceil(cols/nw), TR =
+ *    ceil(rows/nh), K_l = TR*TC, tile index k = tile_row*TC + tile_col (layer-local,
+ *    int32).  All layers of one quantity (gradients, accumulator/"residual", weights,
+ *    dense output) live in one flat arena; layer l starts at element elem_offset_l
+ *    (a multiple of 64 elements) given by rsdgc_plan_layer_info().  Padding elements
+ *    between layers are never read or written.  Indicator keys live in a flat array of
+ *    total_tiles_padded entries, layer l starting at tile_offset_l.
+ *  - Payload: idx_dev[idx_offset_l + s] is the s-th kept tile of layer l (ascending),
+ *    val_dev[val_offset_l + s*nh*nw + a*nw + b] its element (a, b) (+0 where the tile is
+ *    clipped), with idx_offset_l = sum_{l'<l} k_l' and val_offset_l = sum_{l'<l}
+ *    k_l' * nh_l' * nw_l'; counts_dev[l] = k_l.
+ */
+#ifndef RSDGC_H_
+#define RSDGC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct rsdgc_plan rsdgc_plan; /* opaque, library-owned */
+
+typedef enum { RSDGC_F32 = 0, RSDGC_BF16 = 1 } rsdgc_dtype;
+
+typedef enum {
+    RSDGC_OK = 0,
+    RSDGC_ERR_INVALID = -1,   /* null pointer, non-positive size, value out of range      */
+    RSDGC_ERR_ALIGNMENT = -2, /* a device pointer is not 16-byte aligned                  */
+    RSDGC_ERR_CAPACITY = -3,  /* a size exceeds what the library supports                 */
+    RSDGC_ERR_CUDA = -4,      /* a CUDA runtime call failed (see rsdgc_last_cuda_error)   */
+    RSDGC_ERR_NOMEM = -5      /* host or device allocation of the plan failed             */
+} rsdgc_error;
+
+/* plan flags */
+#define RSDGC_KEEP_AT_LEAST_ONE 1u /* k_l = max(1, ceil(K_l * ratio_l)): every layer sends >= 1 tile */
+
+/* bits of rsdgc_status.flags */
+#define RSDGC_STATUS_NONFINITE 1u         /* some indicator was NaN/Inf (ranked first as +Inf)  */
+#define RSDGC_STATUS_PAYLOAD_OVERFLOW 2u  /* idx/val capacity too small; excess tiles not sent   */
+
+typedef struct {
+    int64_t rows, cols; /* row-major 2-D view of the layer (Sec. III-C)            */
+    int32_t nh, nw;     /* neighborhood shape (the paper's p x p patch, Eq. 7)     */
+} rsdgc_layer_desc;
+
+typedef struct {
+    int32_t n_layers;
+    int32_t grad_dtype;          /* rsdgc_dtype of the gradient arena                       */
+    int64_t arena_elems;         /* length of every element arena, padding included         */
+    int64_t total_elems;         /* sum of rows*cols                                        */
+    int64_t total_tiles;         /* sum of K_l                                              */
+    int64_t total_tiles_padded;  /* length of the key / indicator array                     */
+    int64_t workspace_bytes;     /* size of the workspace rsdgc_compress() needs            */
+    int32_t max_slot;            /* max over layers of nh*nw                                */
+    int32_t reserved;
+} rsdgc_info;
+
+typedef struct {
+    int64_t elem_offset; /* start of the layer in the element arenas              */
+    int64_t tile_offset; /* start of the layer in the key / indicator array       */
+    int64_t rows, cols;
+    int32_t nh, nw;
+    int64_t n_tiles;     /* K_l                                                   */
+} rsdgc_layer_info;
+
+typedef struct {
+    uint32_t flags;        /* RSDGC_STATUS_* bits since the last rsdgc_get_status()            */
+    uint32_t reserved;
+    int64_t nonfinite;     /* number of non-finite indicators seen                             */
+    int64_t idx_needed;    /* payload size the last rsdgc_compress() wanted (tiles)            */
+    int64_t val_needed;    /* payload size the last rsdgc_compress() wanted (values)           */
+} rsdgc_status;
+
+/*
+ * Builds the plan for a set of layers (Algorithm 1's loop over l = 1..L with the
+ * neighborhoods of Eq. 7): arena offsets, tile counts, the work lists the kernels walk and
+ * the per-layer device tables.  `alpha` is the hyper-parameter of Eq. 8 (0 <= alpha <= 1).
+ * `flags`: RSDGC_KEEP_AT_LEAST_ONE or 0.  `device` is the CUDA device ordinal.  On success
+ * *out owns host memory and a few MB of device memory until rsdgc_plan_destroy().
+ * Errors: INVALID (null, n_layers < 1, rows/cols/nh/nw < 1, alpha outside [0,1] or NaN,
+ * unknown dtype), CAPACITY (a layer with more than 2^31-1 tiles or nh*nw > 4096),
+ * CUDA / NOMEM.
+ */
+int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_layers, int32_t grad_dtype,
+                      float alpha, uint32_t flags, int32_t device, rsdgc_plan **out);
+
+/* Frees the plan; the caller must make sure no work that uses it is still in flight. */
+int rsdgc_plan_destroy(rsdgc_plan *plan);
+
+/* Sizes derived from the plan (host only). */
+int rsdgc_plan_info(const rsdgc_plan *plan, rsdgc_info *out_host);
+int rsdgc_plan_layer_info(const rsdgc_plan *plan, int32_t layer, rsdgc_layer_info *out_host);
+
+/* Upper bound of the payload sizes (in tiles and in values) when every layer's ratio is at
+ * most max_ratio: sum_l min(K_l, ceil(K_l*max_ratio) + 1) and the same weighted by nh*nw. */
+int rsdgc_plan_payload_bound(const rsdgc_plan *plan, float max_ratio, int64_t *idx_capacity_host,
+                             int64_t *val_capacity_host);
+
+/* Diagnostic: copies the work list of the accumulate+NSI kernel (5 int32 per item: layer,
+ * first tile row, tile rows, first tile col, tile cols; the items of a layer partition its
+ * tile grid), the first item of every CTA of that kernel (cta_capacity entries at most,
+ * the last entry is the item count) and, per layer, how many CTAs touch it.  Any pointer
+ * may be NULL.  Returns the number of items (or a negative rsdgc_error).  Host only. */
+int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,
+                            int32_t *cta_begin_host, int64_t cta_capacity, int32_t *n_flush_host);
+
+/*
+ * Layer-wise dynamic compression ratio (Eq. 3-5; Algorithm 1, per-epoch part): importance
+ * |w| (Eq. 3), one ranking over all layers of the plan, the ceil(global_keep * G) largest
+ * survive (Eq. 4; equal magnitudes: lower arena position first), ratios_dev[l] =
+ * survivors_l / G_l in binary32 (Eq. 5).  Implemented as a three-level radix selection on
+ * the magnitude bits: no sort, three reads of the weights.
+ * weights_dev: binary32 arena with the plan's layer offsets (read only).
+ * ratios_dev: out, n_layers floats.  global_keep in [0, 1].
+ * Errors: INVALID, ALIGNMENT, CUDA.
+ */
+int rsdgc_update_ratios(rsdgc_plan *plan, const float *weights_dev, float global_keep,
+                        float *ratios_dev, void *stream);
+
+/*
+ * One worker's per-iteration compression (Algorithm 1, per-iteration part; Eq. 8-12):
+ *   v = g + r, written in place over the residual arena           (Eq. 12, second line)
+ *   NSI of every tile of v in binary32                            (Eq. 8-10)
+ *   k_l = ceil(K_l * ratios_dev[l]) clipped to [0 or 1, K_l]      (Eq. 11)
+ *   the k_l tiles of largest NSI per layer, ties to the lower tile index, found by a
+ *   three-level radix selection on the NSI bit patterns           (Algorithm 1 ranking)
+ *   payload idx/val/counts as described at the top of this file   (Sec. III-C)
+ *   residual entries of sent tiles set to +0                      (Eq. 12)
+ * grads_dev: gradient arena, binary32 or bfloat16 as the plan says (read only).
+ * residual_dev: binary32 arena, in: accumulator r, out: r' (what was not sent).
+ * ratios_dev: n_layers floats; values <= 0 give k_l = 0 (or 1 with KEEP_AT_LEAST_ONE),
+ *   values >= 1 keep every tile.
+ * idx_dev/val_dev: payload buffers of idx_capacity tiles / val_capacity values; if the
+ *   payload does not fit, the tiles that do not fit are neither written nor removed from
+ *   the residual and RSDGC_STATUS_PAYLOAD_OVERFLOW is raised.  counts_dev: out, n_layers.
+ * nsi_dev: optional (may be NULL) out array of total_tiles_padded floats receiving the
+ *   indicator of every tile (layer l at tile_offset_l).
+ * workspace_dev: workspace_bytes bytes, 16-byte aligned; may be NULL when nsi_dev is given.
+ * Errors: INVALID, ALIGNMENT, CUDA.
+ */
+int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *residual_dev,
+                   const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity,
+                   float *val_dev, int64_t val_capacity, int32_t *counts_dev, float *nsi_dev,
+                   void *workspace_dev, void *stream);
+
+/*
+ * Same step with the gradient and the payload in HOST memory: copies grads_host into
+ * grads_dev (a caller-owned staging arena), runs rsdgc_compress(), waits, and copies
+ * counts and exactly the used part of idx/val back to the host buffers (which must hold
+ * idx_capacity / val_capacity entries).  Pinned host memory makes the copies asynchronous
+ * to the CPU but is not required.  *idx_used_host / *val_used_host receive the payload
+ * sizes.  The accumulator stays on the device.  Synchronises the stream.
+ */
+int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_dev,
+                        float *residual_dev, const float *ratios_dev, int32_t *idx_dev,
+                        int64_t idx_capacity, float *val_dev, int64_t val_capacity,
+                        int32_t *counts_dev, void *workspace_dev, int32_t *idx_host,
+                        float *val_host, int32_t *counts_host, int64_t *idx_used_host,
+                        int64_t *val_used_host, void *stream);
+
+/*
+ * Aggregation of n_workers payloads into a dense gradient on the same device (Eq. 12,
+ * third line: sum over workers of sparse(v); Eq. 2 "Sync"):
+ *   dense[i] = dense[i] + scale * sent_w[i]   for w = 0 .. n_workers-1 in that order,
+ * product then sum, each rounded to binary32 (scale = 1 gives the paper's plain sum).
+ * idx_dev_host / val_dev_host / counts_dev_host: HOST arrays of n_workers DEVICE pointers
+ * to payloads produced by rsdgc_compress() with this plan (or an identical one).
+ * dense_dev: binary32 arena, in/out.  Tile indices outside a layer are skipped.
+ * Errors: INVALID, ALIGNMENT, CUDA.
+ */
+int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,
+                                const int32_t *const *idx_dev_host,
+                                const float *const *val_dev_host,
+                                const int32_t *const *counts_dev_host, float scale,
+                                float *dense_dev, void *stream);
+
+/* Waits for the stream, copies the device status word to *out_host and clears it. */
+int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *out_host);
+
+/* Number of kernels this library has launched in this process (all plans). */
+int64_t rsdgc_launch_count(void);
+
+/* Text for an rsdgc_error; the cudaError_t of the last RSDGC_ERR_CUDA of this thread. */
+const char *rsdgc_strerror(int code);
+int rsdgc_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RSDGC_H_ */

@@ -1,0 +1,202 @@
+"""ctypes binding of the RS-DGC CUDA library (``include/rsdgc.h``).
+
+Argument marshalling only: every step of the compression path runs in the library's
+kernels.  PyTorch tensors supply device memory and the current CUDA stream.  There is no
+CPU fallback: if the shared library is missing, :func:`lib` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence, Tuple
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "librsdgc_b200.so")
+
+RSDGC_F32, RSDGC_BF16 = 0, 1
+KEEP_AT_LEAST_ONE = 1
+STATUS_NONFINITE, STATUS_PAYLOAD_OVERFLOW = 1, 2
+OK, ERR_INVALID, ERR_ALIGNMENT, ERR_CAPACITY, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
+
+EXPORTS = [
+    "rsdgc_plan_create", "rsdgc_plan_destroy", "rsdgc_plan_info", "rsdgc_plan_layer_info",
+    "rsdgc_plan_payload_bound", "rsdgc_plan_worklist", "rsdgc_update_ratios", "rsdgc_compress",
+    "rsdgc_compress_host", "rsdgc_decompress_accumulate", "rsdgc_get_status", "rsdgc_launch_count",
+    "rsdgc_strerror", "rsdgc_last_cuda_error",
+]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [("rows", C.c_int64), ("cols", C.c_int64), ("nh", C.c_int32), ("nw", C.c_int32)]
+
+
+class Info(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("grad_dtype", C.c_int32), ("arena_elems", C.c_int64),
+                ("total_elems", C.c_int64), ("total_tiles", C.c_int64), ("total_tiles_padded", C.c_int64),
+                ("workspace_bytes", C.c_int64), ("max_slot", C.c_int32), ("reserved", C.c_int32)]
+
+
+class LayerInfo(C.Structure):
+    _fields_ = [("elem_offset", C.c_int64), ("tile_offset", C.c_int64), ("rows", C.c_int64),
+                ("cols", C.c_int64), ("nh", C.c_int32), ("nw", C.c_int32), ("n_tiles", C.c_int64)]
+
+
+class Status(C.Structure):
+    _fields_ = [("flags", C.c_uint32), ("reserved", C.c_uint32), ("nonfinite", C.c_int64),
+                ("idx_needed", C.c_int64), ("val_needed", C.c_int64)]
+
+
+class RsdgcError(RuntimeError):
+    def __init__(self, code: int, what: str):
+        self.code = code
+        msg = lib().rsdgc_strerror(code).decode()
+        if code == ERR_CUDA:
+            msg += " (cudaError %d)" % lib().rsdgc_last_cuda_error()
+        super().__init__("%s: %s [%d]" % (what, msg, code))
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C library; raises if it has not been built (no fallback path exists)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("CUDA library %s is missing: build it with "
+                               "`python -m paper_2312_17530_b200.build`" % LIB_PATH)
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64, f32, u32 = C.c_void_p, C.c_int32, C.c_int64, C.c_float, C.c_uint32
+        L.rsdgc_plan_create.argtypes = [C.POINTER(LayerDesc), i32, i32, f32, u32, i32, C.POINTER(vp)]
+        L.rsdgc_plan_destroy.argtypes = [vp]
+        L.rsdgc_plan_info.argtypes = [vp, C.POINTER(Info)]
+        L.rsdgc_plan_layer_info.argtypes = [vp, i32, C.POINTER(LayerInfo)]
+        L.rsdgc_plan_payload_bound.argtypes = [vp, f32, C.POINTER(i64), C.POINTER(i64)]
+        L.rsdgc_plan_worklist.argtypes = [vp, vp, i64, vp, i64, vp]
+        L.rsdgc_plan_worklist.restype = i64
+        L.rsdgc_update_ratios.argtypes = [vp, vp, f32, vp, vp]
+        L.rsdgc_compress.argtypes = [vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
+        L.rsdgc_compress_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, vp,
+                                          C.POINTER(i64), C.POINTER(i64), vp]
+        L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
+        L.rsdgc_get_status.argtypes = [vp, vp, C.POINTER(Status)]
+        L.rsdgc_launch_count.argtypes = []
+        L.rsdgc_launch_count.restype = i64
+        L.rsdgc_strerror.argtypes = [C.c_int]
+        L.rsdgc_strerror.restype = C.c_char_p
+        L.rsdgc_last_cuda_error.argtypes = []
+        for name in EXPORTS:
+            fn = getattr(L, name)
+            if fn.restype is C.c_int:  # default restype: all the int-returning entry points
+                fn.restype = C.c_int
+        _lib = L
+    return _lib
+
+
+def _check(code: int, what: str) -> None:
+    if code != OK:
+        raise RsdgcError(code, what)
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    import torch
+
+    return torch.cuda.current_stream().cuda_stream
+
+
+class Plan:
+    """Owns an ``rsdgc_plan``.  ``layers``: sequence of (rows, cols, nh, nw).  ``device`` < 0
+    gives a host-only plan (sizes and offsets only; usable without a GPU)."""
+
+    def __init__(self, layers: Sequence[Tuple[int, int, int, int]], grad_dtype: int = RSDGC_F32,
+                 alpha: float = 0.5, flags: int = KEEP_AT_LEAST_ONE, device: int = 0):
+        arr = (LayerDesc * max(1, len(layers)))()
+        for i, (r, c, nh, nw) in enumerate(layers):
+            arr[i] = LayerDesc(int(r), int(c), int(nh), int(nw))
+        h = C.c_void_p()
+        self._h = None
+        _check(lib().rsdgc_plan_create(arr, len(layers), grad_dtype, alpha, flags, device, C.byref(h)),
+               "rsdgc_plan_create")
+        self._h = h
+        self.device = device
+        self.n_layers = len(layers)
+        self.grad_dtype = grad_dtype
+        info = Info()
+        _check(lib().rsdgc_plan_info(self._h, C.byref(info)), "rsdgc_plan_info")
+        self.info = info
+        self.layers: List[LayerInfo] = []
+        for l in range(self.n_layers):
+            li = LayerInfo()
+            _check(lib().rsdgc_plan_layer_info(self._h, l, C.byref(li)), "rsdgc_plan_layer_info")
+            self.layers.append(li)
+
+    def close(self) -> None:
+        if self._h is not None:
+            lib().rsdgc_plan_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ---- sizes --------------------------------------------------------------------------
+    def payload_bound(self, max_ratio: float) -> Tuple[int, int]:
+        a, b = C.c_int64(), C.c_int64()
+        _check(lib().rsdgc_plan_payload_bound(self._h, max_ratio, C.byref(a), C.byref(b)),
+               "rsdgc_plan_payload_bound")
+        return a.value, b.value
+
+    def worklist(self):
+        """(items [n,5] int32, cta_begin int32, n_flush int32) of the accumulate+NSI kernel."""
+        import numpy as np
+
+        n = lib().rsdgc_plan_worklist(self._h, None, 0, None, 0, None)
+        items = np.zeros((n, 5), dtype=np.int32)
+        cta = np.zeros(4096, dtype=np.int32) - 1
+        nf = np.zeros(self.n_layers, dtype=np.int32)
+        lib().rsdgc_plan_worklist(self._h, items.ctypes.data, n, cta.ctypes.data, cta.size, nf.ctypes.data)
+        return items, cta[cta >= 0], nf
+
+    # ---- device calls (torch tensors on the plan's device) -------------------------------
+    def update_ratios(self, weights, global_keep: float, ratios) -> None:
+        _check(lib().rsdgc_update_ratios(self._h, _ptr(weights), global_keep, _ptr(ratios), _stream()),
+               "rsdgc_update_ratios")
+
+    def compress(self, grads, residual, ratios, idx, val, counts, nsi=None, workspace=None) -> None:
+        _check(lib().rsdgc_compress(self._h, _ptr(grads), _ptr(residual), _ptr(ratios), _ptr(idx), idx.numel(),
+                                    _ptr(val), val.numel(), _ptr(counts), _ptr(nsi), _ptr(workspace), _stream()),
+               "rsdgc_compress")
+
+    def compress_host(self, grads_host, grads_dev, residual, ratios, idx, val, counts, workspace,
+                      idx_host, val_host, counts_host) -> Tuple[int, int]:
+        ni, nv = C.c_int64(), C.c_int64()
+        _check(lib().rsdgc_compress_host(self._h, _ptr(grads_host), _ptr(grads_dev), _ptr(residual), _ptr(ratios),
+                                         _ptr(idx), idx.numel(), _ptr(val), val.numel(), _ptr(counts),
+                                         _ptr(workspace), _ptr(idx_host), _ptr(val_host), _ptr(counts_host),
+                                         C.byref(ni), C.byref(nv), _stream()), "rsdgc_compress_host")
+        return ni.value, nv.value
+
+    def decompress_accumulate(self, payloads, dense, scale: float = 1.0) -> None:
+        """``payloads``: sequence of (idx, val, counts) device tensors, one per worker."""
+        n = len(payloads)
+        A = C.c_void_p * max(1, n)
+        ia, va, ca = A(), A(), A()
+        for w, (i, v, c) in enumerate(payloads):
+            ia[w], va[w], ca[w] = i.data_ptr(), v.data_ptr(), c.data_ptr()
+        _check(lib().rsdgc_decompress_accumulate(self._h, n, ia, va, ca, scale, _ptr(dense), _stream()),
+               "rsdgc_decompress_accumulate")
+
+    def status(self) -> Status:
+        st = Status()
+        _check(lib().rsdgc_get_status(self._h, _stream(), C.byref(st)), "rsdgc_get_status")
+        return st
+
+
+def launch_count() -> int:
+    return int(lib().rsdgc_launch_count())

@@ -1,0 +1,81 @@
+// Block-level helpers used by several kernels (256-thread CTAs).
+#pragma once
+
+#include "rsdgc_internal.cuh"
+
+namespace rsdgc {
+
+// Exclusive prefix sum of one value per thread over the CTA, in thread order.
+// `warp_tot` points to kThreads/32 words of shared memory.  Every thread receives the CTA
+// total in *total.  Contains two barriers; all threads must call it.
+template <typename T>
+__device__ __forceinline__ T block_exclusive_scan(T x, T *warp_tot, T *total)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    T incl = x;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        T y = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= d) incl += y;
+    }
+    if (lane == 31) warp_tot[warp] = incl;
+    __syncthreads();
+    T offset = 0, sum = 0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) {
+        T t = warp_tot[w];
+        if (w < warp) offset += t;
+        sum += t;
+    }
+    __syncthreads();
+    *total = sum;
+    return offset + incl - x;
+}
+
+// Walks a histogram in shared memory from its highest bin downwards and finds the bin in
+// which the running count reaches `need` (need >= 1): out[0] = bin, out[1] = how many
+// entries of that bin are still needed (need minus the count of all higher bins).
+// If the histogram holds fewer than `need` entries, bin 0 is returned with what is missing.
+// `out` and `warp_tot` are shared memory; all threads must call; ends with a barrier.
+template <int NBINS>
+__device__ __forceinline__ void find_bin_from_top(const unsigned int *h, unsigned long long need,
+                                                  unsigned long long *out, unsigned long long *warp_tot)
+{
+    constexpr int PER = NBINS / kThreads;
+    static_assert(NBINS % kThreads == 0, "histogram size must be a multiple of the CTA size");
+    unsigned long long local = 0;
+#pragma unroll
+    for (int j = 0; j < PER; ++j) local += h[NBINS - 1 - (threadIdx.x * PER + j)];
+    unsigned long long total;
+    unsigned long long excl = block_exclusive_scan<unsigned long long>(local, warp_tot, &total);
+    if (threadIdx.x == 0 && total < need) {
+        out[0] = 0;
+        out[1] = need - (total - h[0]);
+    }
+    if (excl < need && need <= excl + local) {
+        unsigned long long run = excl;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int b = NBINS - 1 - (threadIdx.x * PER + j);
+            const unsigned long long c = h[b];
+            if (run < need && need <= run + c) {
+                out[0] = (unsigned long long)b;
+                out[1] = need - run;
+            }
+            run += c;
+        }
+    }
+    __syncthreads();
+}
+
+// Number of tiles to keep, k = ceil(K * ratio) (Eq. 11) limited to [0 or 1, K]; the product
+// is taken in binary64 on the binary32 ratio.
+__device__ __forceinline__ int keep_count(int K, float ratio, unsigned int flags)
+{
+    const double x = ceil((double)K * (double)ratio);
+    int k = (x > 0.0) ? ((x >= (double)K) ? K : (int)x) : 0;
+    if ((flags & RSDGC_KEEP_AT_LEAST_ONE) && k < 1) k = 1;
+    return k < K ? k : K;
+}
+
+}  // namespace rsdgc

@@ -1,0 +1,495 @@
+// Host side of the RS-DGC library: plan tables, argument checks, the C entry points.
+#include <atomic>
+#include <cmath>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "rsdgc_internal.cuh"
+
+using namespace rsdgc;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+std::atomic<long long> g_launches{0};
+
+int cuda_fail(cudaError_t e)
+{
+    g_last_cuda_error = (int)e;
+    return RSDGC_ERR_CUDA;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t err = cudaSuccess;
+    explicit DeviceGuard(int dev)
+    {
+        err = cudaGetDevice(&prev);
+        if (err == cudaSuccess && prev != dev) {
+            err = cudaSetDevice(dev);
+            switched = (err == cudaSuccess);
+        }
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+inline int64_t ceil_div64(int64_t a, int64_t b) { return (a + b - 1) / b; }
+inline int64_t round_up64(int64_t a, int64_t b) { return ceil_div64(a, b) * b; }
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+template <typename T>
+cudaError_t upload(T **dst, const std::vector<T> &src)
+{
+    size_t bytes = (src.empty() ? 1 : src.size()) * sizeof(T);
+    cudaError_t e = cudaMalloc((void **)dst, bytes);
+    if (e != cudaSuccess) return e;
+    if (!src.empty()) e = cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice);
+    return e;
+}
+
+template <typename T>
+cudaError_t alloc_zero(T **dst, size_t count)
+{
+    size_t bytes = (count ? count : 1) * sizeof(T);
+    cudaError_t e = cudaMalloc((void **)dst, bytes);
+    if (e != cudaSuccess) return e;
+    return cudaMemset(*dst, 0, bytes);
+}
+
+void free_device_tables(rsdgc_plan *p)
+{
+    cudaFree(p->d_layers);
+    cudaFree(p->d_items);
+    cudaFree(p->d_cta_begin);
+    cudaFree(p->d_chunks);
+    cudaFree(p->d_echunks);
+    cudaFree(p->d_state);
+    cudaFree(p->d_hist);
+    cudaFree(p->d_chunk_cnt);
+    cudaFree(p->d_survivors);
+    cudaFree(p->d_rstate);
+    cudaFree(p->d_status);
+}
+
+}  // namespace
+
+namespace rsdgc {
+
+void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+// Splits every layer into work items for the accumulate+NSI kernel and into key / element
+// chunks for the selection passes, and assigns contiguous item ranges of equal cost to the
+// CTAs of the accumulate+NSI kernel.
+int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers)
+{
+    p->layers.clear();
+    p->items.clear();
+    p->chunks.clear();
+    p->echunks.clear();
+    int64_t elem_off = 0, tile_off = 0, total_elems = 0, total_tiles = 0;
+    int max_slot = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const rsdgc_layer_desc &d = descs[l];
+        if (d.rows < 1 || d.cols < 1 || d.nh < 1 || d.nw < 1) return RSDGC_ERR_INVALID;
+        if ((int64_t)d.nh * d.nw > kMaxSlot) return RSDGC_ERR_CAPACITY;
+        if (d.rows > INT32_MAX || d.cols > INT32_MAX) return RSDGC_ERR_CAPACITY;
+        if (d.rows * d.cols > (int64_t)INT32_MAX) return RSDGC_ERR_CAPACITY;
+        LayerDev L{};
+        L.elem_off = elem_off;
+        L.tile_off = tile_off;
+        L.rows = d.rows;
+        L.cols = d.cols;
+        L.nh = d.nh;
+        L.nw = d.nw;
+        L.TR = (int32_t)ceil_div64(d.rows, d.nh);
+        L.TC = (int32_t)ceil_div64(d.cols, d.nw);
+        L.K = L.TR * L.TC;
+        L.slot = d.nh * d.nw;
+        if (L.slot > max_slot) max_slot = L.slot;
+
+        // --- accumulate+NSI items: rectangles of tiles holding at most kItemElems elements
+        const int64_t band = (int64_t)d.nh * d.cols;  // one full-width row of tiles
+        if (band <= kItemElems) {
+            int64_t ntr_max = kItemElems / band;
+            int64_t n_items = ceil_div64(L.TR, ntr_max);
+            int64_t ntr = ceil_div64(L.TR, n_items);
+            // multiples of 4 tile rows keep every item start 4-element aligned (128-bit loads)
+            if (round_up64(ntr, 4) <= ntr_max) ntr = round_up64(ntr, 4);
+            for (int64_t tr0 = 0; tr0 < L.TR; tr0 += ntr) {
+                Item it{l, (int32_t)tr0, (int32_t)std::min<int64_t>(ntr, L.TR - tr0), 0, L.TC};
+                p->items.push_back(it);
+            }
+        } else {
+            int64_t ntc_max = kItemElems / L.slot;
+            int64_t n_items = ceil_div64(L.TC, ntc_max);
+            int64_t ntc = ceil_div64(L.TC, n_items);
+            if (round_up64(ntc, 4) <= ntc_max) ntc = round_up64(ntc, 4);
+            for (int64_t tr = 0; tr < L.TR; ++tr)
+                for (int64_t tc0 = 0; tc0 < L.TC; tc0 += ntc) {
+                    Item it{l, (int32_t)tr, 1, (int32_t)tc0, (int32_t)std::min<int64_t>(ntc, L.TC - tc0)};
+                    p->items.push_back(it);
+                }
+        }
+
+        // --- key chunks and element chunks
+        L.first_chunk = (int32_t)p->chunks.size();
+        L.n_chunks = (int32_t)ceil_div64(L.K, kChunkKeys);
+        for (int32_t c = 0; c < L.n_chunks; ++c) {
+            int32_t start = c * kChunkKeys;
+            p->chunks.push_back(Chunk{l, start, std::min<int32_t>(kChunkKeys, L.K - start)});
+        }
+        L.first_echunk = (int32_t)p->echunks.size();
+        const int64_t n = d.rows * d.cols;
+        for (int64_t s = 0; s < n; s += kChunkKeys)
+            p->echunks.push_back(EChunk{s, l, (int32_t)std::min<int64_t>(kChunkKeys, n - s)});
+
+        p->layers.push_back(L);
+        total_elems += n;
+        total_tiles += L.K;
+        elem_off += round_up64(n, kArenaAlign);
+        tile_off += round_up64(L.K, kArenaAlign);
+    }
+    if (p->items.size() > (size_t)INT32_MAX || p->echunks.size() > (size_t)INT32_MAX) return RSDGC_ERR_CAPACITY;
+
+    // --- static partition of the items over the CTAs of the accumulate+NSI kernel
+    const int G = p->grid1;
+    const size_t n_items = p->items.size();
+    std::vector<double> cum(n_items + 1, 0.0);
+    for (size_t i = 0; i < n_items; ++i) {
+        const Item &it = p->items[i];
+        const LayerDev &L = p->layers[it.layer];
+        int64_t r0 = (int64_t)it.tr0 * L.nh, r1 = std::min<int64_t>(L.rows, r0 + (int64_t)it.ntr * L.nh);
+        int64_t c0 = (int64_t)it.tc0 * L.nw, c1 = std::min<int64_t>(L.cols, c0 + (int64_t)it.ntc * L.nw);
+        cum[i + 1] = cum[i] + (double)((r1 - r0) * (c1 - c0)) + 512.0;  // + fixed cost per item
+    }
+    p->cta_begin.assign(G + 1, (int32_t)n_items);
+    std::vector<int32_t> owner(n_items);
+    for (size_t i = 0; i < n_items; ++i) {
+        int g = (int)std::floor(cum[i] * G / cum[n_items]);
+        if (g >= G) g = G - 1;
+        owner[i] = g;
+    }
+    {
+        size_t i = 0;
+        for (int g = 0; g <= G; ++g) {
+            while (i < n_items && owner[i] < g) ++i;
+            p->cta_begin[g] = (int32_t)i;
+        }
+    }
+    for (auto &L : p->layers) L.n_flush1 = 0;
+    for (size_t i = 0; i < n_items; ++i) {
+        bool first = (i == 0) || p->items[i - 1].layer != p->items[i].layer || owner[i - 1] != owner[i];
+        if (first) p->layers[p->items[i].layer].n_flush1 += 1;
+    }
+
+    rsdgc_info &I = p->info;
+    I.n_layers = n_layers;
+    I.grad_dtype = p->dtype;
+    I.arena_elems = elem_off;
+    I.total_elems = total_elems;
+    I.total_tiles = total_tiles;
+    I.total_tiles_padded = tile_off;
+    I.workspace_bytes = tile_off * (int64_t)sizeof(uint32_t);
+    I.max_slot = max_slot;
+    I.reserved = 0;
+    return RSDGC_OK;
+}
+
+}  // namespace rsdgc
+
+// ------------------------------------------------------------------------------------------
+// C entry points
+// ------------------------------------------------------------------------------------------
+
+extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_layers, int32_t grad_dtype,
+                                 float alpha, uint32_t flags, int32_t device, rsdgc_plan **out)
+{
+    if (!layers_host || !out || n_layers < 1) return RSDGC_ERR_INVALID;
+    *out = nullptr;
+    if (n_layers > kMaxLayers) return RSDGC_ERR_CAPACITY;
+    if (grad_dtype != RSDGC_F32 && grad_dtype != RSDGC_BF16) return RSDGC_ERR_INVALID;
+    if (!(alpha >= 0.0f && alpha <= 1.0f)) return RSDGC_ERR_INVALID;
+    if (flags & ~RSDGC_KEEP_AT_LEAST_ONE) return RSDGC_ERR_INVALID;
+
+    rsdgc_plan *p = new (std::nothrow) rsdgc_plan();
+    if (!p) return RSDGC_ERR_NOMEM;
+    p->device = device;
+    p->n_layers = n_layers;
+    p->dtype = grad_dtype;
+    p->alpha = alpha;
+    p->flags = flags;
+
+    if (device >= 0) {
+        int n_sm = 0;
+        cudaError_t e = cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device);
+        if (e != cudaSuccess) {
+            delete p;
+            return cuda_fail(e);
+        }
+        p->n_sm = n_sm;
+    }
+    p->grid1 = p->n_sm * 4;
+
+    int rc;
+    try {
+        rc = build_plan_tables(p, layers_host, n_layers);
+    } catch (const std::bad_alloc &) {
+        rc = RSDGC_ERR_NOMEM;
+    }
+    if (rc != RSDGC_OK) {
+        delete p;
+        return rc;
+    }
+
+    if (device >= 0) {
+        DeviceGuard guard(device);
+        cudaError_t e = guard.err;
+        if (e == cudaSuccess) e = upload(&p->d_layers, p->layers);
+        if (e == cudaSuccess) e = upload(&p->d_items, p->items);
+        if (e == cudaSuccess) e = upload(&p->d_cta_begin, p->cta_begin);
+        if (e == cudaSuccess) e = upload(&p->d_chunks, p->chunks);
+        if (e == cudaSuccess) e = upload(&p->d_echunks, p->echunks);
+        if (e == cudaSuccess) e = alloc_zero(&p->d_state, (size_t)n_layers);
+        if (e == cudaSuccess) e = alloc_zero(&p->d_hist, (size_t)n_layers * kHistStride);
+        if (e == cudaSuccess) e = alloc_zero(&p->d_chunk_cnt, p->chunks.size());
+        if (e == cudaSuccess) e = alloc_zero(&p->d_survivors, (size_t)n_layers);
+        if (e == cudaSuccess) e = alloc_zero(&p->d_rstate, 1);
+        if (e == cudaSuccess) e = alloc_zero(&p->d_status, 1);
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) {
+            free_device_tables(p);
+            delete p;
+            return e == cudaErrorMemoryAllocation ? RSDGC_ERR_NOMEM : cuda_fail(e);
+        }
+    }
+    *out = p;
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_plan_destroy(rsdgc_plan *plan)
+{
+    if (!plan) return RSDGC_ERR_INVALID;
+    if (plan->device >= 0) {
+        DeviceGuard guard(plan->device);
+        free_device_tables(plan);
+    }
+    delete plan;
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_plan_info(const rsdgc_plan *plan, rsdgc_info *out_host)
+{
+    if (!plan || !out_host) return RSDGC_ERR_INVALID;
+    *out_host = plan->info;
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_plan_layer_info(const rsdgc_plan *plan, int32_t layer, rsdgc_layer_info *out_host)
+{
+    if (!plan || !out_host || layer < 0 || layer >= plan->n_layers) return RSDGC_ERR_INVALID;
+    const LayerDev &L = plan->layers[layer];
+    out_host->elem_offset = L.elem_off;
+    out_host->tile_offset = L.tile_off;
+    out_host->rows = L.rows;
+    out_host->cols = L.cols;
+    out_host->nh = L.nh;
+    out_host->nw = L.nw;
+    out_host->n_tiles = L.K;
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_plan_payload_bound(const rsdgc_plan *plan, float max_ratio, int64_t *idx_capacity_host,
+                                        int64_t *val_capacity_host)
+{
+    if (!plan || !idx_capacity_host || !val_capacity_host || !(max_ratio >= 0.0f)) return RSDGC_ERR_INVALID;
+    int64_t ni = 0, nv = 0;
+    for (const LayerDev &L : plan->layers) {
+        double x = std::ceil((double)L.K * (double)max_ratio) + 1.0;
+        int64_t k = (x >= (double)L.K) ? (int64_t)L.K : (int64_t)x;
+        ni += k;
+        nv += k * L.slot;
+    }
+    *idx_capacity_host = ni;
+    *val_capacity_host = nv;
+    return RSDGC_OK;
+}
+
+// Diagnostic: copies the accumulate+NSI work list (5 int32 per item: layer, tr0, ntr, tc0,
+// ntc) and the per-CTA item ranges; used by the host-logic tests.  Returns the item count.
+extern "C" int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,
+                                       int32_t *cta_begin_host, int64_t cta_capacity, int32_t *n_flush_host)
+{
+    if (!plan) return RSDGC_ERR_INVALID;
+    int64_t n = (int64_t)plan->items.size();
+    if (items_host)
+        for (int64_t i = 0; i < n && i < items_capacity; ++i) {
+            const Item &it = plan->items[i];
+            int32_t *o = items_host + 5 * i;
+            o[0] = it.layer, o[1] = it.tr0, o[2] = it.ntr, o[3] = it.tc0, o[4] = it.ntc;
+        }
+    if (cta_begin_host)
+        for (int64_t g = 0; g < (int64_t)plan->cta_begin.size() && g < cta_capacity; ++g)
+            cta_begin_host[g] = plan->cta_begin[g];
+    if (n_flush_host)
+        for (int l = 0; l < plan->n_layers; ++l) n_flush_host[l] = plan->layers[l].n_flush1;
+    return n;
+}
+
+namespace {
+
+int check_plan_device(const rsdgc_plan *plan)
+{
+    if (!plan) return RSDGC_ERR_INVALID;
+    if (plan->device < 0) return RSDGC_ERR_INVALID;  // host-only plan: sizing queries only
+    return RSDGC_OK;
+}
+
+}  // namespace
+
+extern "C" int rsdgc_update_ratios(rsdgc_plan *plan, const float *weights_dev, float global_keep,
+                                   float *ratios_dev, void *stream)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (!weights_dev || !ratios_dev || !(global_keep >= 0.0f && global_keep <= 1.0f)) return RSDGC_ERR_INVALID;
+    if (!aligned16(weights_dev)) return RSDGC_ERR_ALIGNMENT;
+    // n_keep = ceil(rho * G), product in binary64 of the binary32 ratio (Eq. 4 read as "keep")
+    const double G = (double)plan->info.total_elems;
+    double x = std::ceil((double)global_keep * G);
+    long long n_keep = x <= 0.0 ? 0 : (x >= G ? plan->info.total_elems : (long long)x);
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaError_t e = launch_update_ratios(plan, weights_dev, n_keep, ratios_dev, (cudaStream_t)stream);
+    return e == cudaSuccess ? RSDGC_OK : cuda_fail(e);
+}
+
+extern "C" int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *residual_dev,
+                              const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, float *val_dev,
+                              int64_t val_capacity, int32_t *counts_dev, float *nsi_dev, void *workspace_dev,
+                              void *stream)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (!grads_dev || !residual_dev || !ratios_dev || !counts_dev) return RSDGC_ERR_INVALID;
+    if (idx_capacity < 0 || val_capacity < 0) return RSDGC_ERR_INVALID;
+    if ((idx_capacity > 0 && !idx_dev) || (val_capacity > 0 && !val_dev)) return RSDGC_ERR_INVALID;
+    if (!nsi_dev && !workspace_dev) return RSDGC_ERR_INVALID;
+    if (!aligned16(grads_dev) || !aligned16(residual_dev) || !aligned16(idx_dev) || !aligned16(val_dev) ||
+        !aligned16(nsi_dev) || !aligned16(workspace_dev))
+        return RSDGC_ERR_ALIGNMENT;
+    uint32_t *keys = nsi_dev ? reinterpret_cast<uint32_t *>(nsi_dev) : reinterpret_cast<uint32_t *>(workspace_dev);
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaError_t e = launch_compress(plan, grads_dev, residual_dev, ratios_dev, idx_dev, idx_capacity, val_dev,
+                                    val_capacity, counts_dev, keys, (cudaStream_t)stream);
+    return e == cudaSuccess ? RSDGC_OK : cuda_fail(e);
+}
+
+extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_dev, float *residual_dev,
+                                   const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, float *val_dev,
+                                   int64_t val_capacity, int32_t *counts_dev, void *workspace_dev,
+                                   int32_t *idx_host, float *val_host, int32_t *counts_host,
+                                   int64_t *idx_used_host, int64_t *val_used_host, void *stream)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (!grads_host || !grads_dev || !counts_host || !idx_used_host || !val_used_host) return RSDGC_ERR_INVALID;
+    if ((idx_capacity > 0 && !idx_host) || (val_capacity > 0 && !val_host)) return RSDGC_ERR_INVALID;
+    cudaStream_t s = (cudaStream_t)stream;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    const size_t esz = plan->dtype == RSDGC_BF16 ? 2 : 4;
+    cudaError_t e = cudaMemcpyAsync(grads_dev, grads_host, (size_t)plan->info.arena_elems * esz,
+                                    cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    rc = rsdgc_compress(plan, grads_dev, residual_dev, ratios_dev, idx_dev, idx_capacity, val_dev, val_capacity,
+                        counts_dev, nullptr, workspace_dev, stream);
+    if (rc) return rc;
+    e = cudaMemcpyAsync(counts_host, counts_dev, (size_t)plan->n_layers * sizeof(int32_t), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    int64_t ni = 0, nv = 0;
+    for (int l = 0; l < plan->n_layers; ++l) {
+        ni += counts_host[l];
+        nv += (int64_t)counts_host[l] * plan->layers[l].slot;
+    }
+    if (ni > idx_capacity) ni = idx_capacity;
+    if (nv > val_capacity) nv = val_capacity;
+    if (ni > 0) e = cudaMemcpyAsync(idx_host, idx_dev, (size_t)ni * sizeof(int32_t), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess && nv > 0)
+        e = cudaMemcpyAsync(val_host, val_dev, (size_t)nv * sizeof(float), cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    *idx_used_host = ni;
+    *val_used_host = nv;
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
+                                           const float *const *val_dev_host,
+                                           const int32_t *const *counts_dev_host, float scale, float *dense_dev,
+                                           void *stream)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (n_workers < 0 || !dense_dev) return RSDGC_ERR_INVALID;
+    if (n_workers > 0 && (!idx_dev_host || !val_dev_host || !counts_dev_host)) return RSDGC_ERR_INVALID;
+    if (!aligned16(dense_dev)) return RSDGC_ERR_ALIGNMENT;
+    for (int w = 0; w < n_workers; ++w) {
+        if (!idx_dev_host[w] || !val_dev_host[w] || !counts_dev_host[w]) return RSDGC_ERR_INVALID;
+        if (!aligned16(idx_dev_host[w]) || !aligned16(val_dev_host[w])) return RSDGC_ERR_ALIGNMENT;
+    }
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    // one launch per worker, in worker order: within a worker no two entries touch the same
+    // element, across workers the stream order fixes the order of the binary32 additions
+    for (int w = 0; w < n_workers; ++w) {
+        cudaError_t e = launch_decompress(plan, idx_dev_host[w], val_dev_host[w], counts_dev_host[w], scale,
+                                          dense_dev, (cudaStream_t)stream);
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *out_host)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (!out_host) return RSDGC_ERR_INVALID;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaStream_t s = (cudaStream_t)stream;
+    StatusDev h{};
+    cudaError_t e = cudaMemcpyAsync(&h, plan->d_status, sizeof h, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(plan->d_status, 0, sizeof(StatusDev), s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return cuda_fail(e);
+    out_host->flags = h.flags;
+    out_host->reserved = 0;
+    out_host->nonfinite = (int64_t)h.nonfinite;
+    out_host->idx_needed = h.idx_needed;
+    out_host->val_needed = h.val_needed;
+    return RSDGC_OK;
+}
+
+extern "C" int64_t rsdgc_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+extern "C" const char *rsdgc_strerror(int code)
+{
+    switch (code) {
+        case RSDGC_OK: return "ok";
+        case RSDGC_ERR_INVALID: return "invalid argument";
+        case RSDGC_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+        case RSDGC_ERR_CAPACITY: return "size beyond what the library supports";
+        case RSDGC_ERR_CUDA: return "CUDA runtime error";
+        case RSDGC_ERR_NOMEM: return "out of memory";
+        default: return "unknown error";
+    }
+}
+
+extern "C" int rsdgc_last_cuda_error(void) { return g_last_cuda_error; }

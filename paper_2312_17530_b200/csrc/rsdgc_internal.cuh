@@ -1,0 +1,131 @@
+// Internal declarations shared by the host code and the kernels of the RS-DGC library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "rsdgc.h"
+
+namespace rsdgc {
+
+// ---- compile-time geometry -------------------------------------------------------------
+constexpr int kThreads = 256;        // threads per CTA, every kernel
+constexpr int kItemElems = 6144;     // elements of one accumulate+NSI work item (24 KB of smem)
+constexpr int kL1Bits = 11;          // radix level 1: key bits 30..20 (8 exponent + 3 mantissa)
+constexpr int kL1Bins = 1 << kL1Bits;
+constexpr int kL1Shift = 20;
+constexpr int kL2Bins = 1024;        // level 2: key bits 19..10
+constexpr int kL2Shift = 10;
+constexpr int kL3Bins = 1024;        // level 3: key bits 9..0
+constexpr int kHistStride = kL1Bins; // words of histogram per layer
+constexpr int kChunkKeys = 16384;    // keys (or weights) per CTA in the key passes
+constexpr int kMaxLayers = 2048;
+constexpr int kMaxSlot = 4096;
+constexpr int kArenaAlign = 64;      // elements; also the alignment of tile offsets
+constexpr uint32_t kTakeNone = 0xFFFFFFFFu;  // prefix / threshold marker: keep nothing
+
+// ---- tables ----------------------------------------------------------------------------
+struct LayerDev {
+    int64_t elem_off;   // start in the element arenas
+    int64_t tile_off;   // start in the key array
+    int64_t rows, cols;
+    int32_t nh, nw;
+    int32_t TR, TC;     // tile grid; K = TR * TC
+    int32_t K, slot;    // tiles, values per tile (nh * nw)
+    int32_t first_chunk, n_chunks;    // key chunks of this layer
+    int32_t n_flush1;                 // CTAs of the accumulate+NSI kernel that touch the layer
+    int32_t first_echunk;             // first element chunk (ratio rule)
+};
+
+// Work item of the accumulate+NSI kernel: tile rows [tr0, tr0+ntr) x tile cols [tc0, tc0+ntc).
+struct Item {
+    int32_t layer, tr0, ntr, tc0, ntc;
+};
+
+// Key chunk: keys [start, start + n) of a layer (layer-local tile indices).
+struct Chunk {
+    int32_t layer, start, n;
+};
+
+// Element chunk: elements [start, start + n) of a layer (layer-local flat positions).
+struct EChunk {
+    int64_t start;
+    int32_t layer, n;
+};
+
+// Per-layer selection state carried from kernel to kernel (device memory, plan-owned).
+struct LayerState {
+    unsigned int ticket[4];  // arrival counters of the four phases; each resets itself
+    int32_t k;               // tiles to keep (Eq. 11)
+    uint32_t prefix;         // key bits resolved so far, or kTakeNone
+    int32_t remaining;       // tiles still to take among keys that carry `prefix`
+    uint32_t T;              // threshold key
+    int32_t e;               // keys equal to T to take, lowest tile index first
+    int32_t pad;
+    int64_t idx_off, val_off;  // payload offsets of the layer
+};
+
+struct RatioState {
+    unsigned int ticket;
+    uint32_t prefix;
+    long long remaining;
+    long long n_keep;
+};
+
+struct StatusDev {
+    unsigned int flags, pad;
+    unsigned long long nonfinite;
+    long long idx_needed, val_needed;
+};
+
+}  // namespace rsdgc
+
+struct rsdgc_plan {
+    int device = -1;  // < 0: host-only plan (sizing queries only)
+    int n_layers = 0;
+    int dtype = 0;
+    float alpha = 0.5f;
+    uint32_t flags = 0;
+    int n_sm = 148;
+    int grid1 = 0;  // CTAs of the accumulate+NSI kernel
+
+    std::vector<rsdgc::LayerDev> layers;
+    std::vector<rsdgc::Item> items;
+    std::vector<int32_t> cta_begin;  // grid1 + 1 item indices
+    std::vector<rsdgc::Chunk> chunks;
+    std::vector<rsdgc::EChunk> echunks;
+
+    rsdgc_info info{};
+
+    // device tables
+    rsdgc::LayerDev *d_layers = nullptr;
+    rsdgc::Item *d_items = nullptr;
+    int32_t *d_cta_begin = nullptr;
+    rsdgc::Chunk *d_chunks = nullptr;
+    rsdgc::EChunk *d_echunks = nullptr;
+    rsdgc::LayerState *d_state = nullptr;
+    uint32_t *d_hist = nullptr;        // n_layers * kHistStride
+    uint2 *d_chunk_cnt = nullptr;      // per key chunk: (#key > T, #key == T), then exclusive bases
+    long long *d_survivors = nullptr;  // ratio rule: per-layer survivor counts
+    rsdgc::RatioState *d_rstate = nullptr;
+    rsdgc::StatusDev *d_status = nullptr;
+};
+
+namespace rsdgc {
+
+// host: builds every table of the plan from the layer descriptors (no CUDA calls)
+int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *layers, int n_layers);
+
+// launches (defined in the .cu files); each returns a cudaError_t
+cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, const float *ratios,
+                            int32_t *idx, int64_t idx_cap, float *val, int64_t val_cap,
+                            int32_t *counts, uint32_t *keys, cudaStream_t s);
+cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long n_keep,
+                                 float *ratios, cudaStream_t s);
+cudaError_t launch_decompress(rsdgc_plan *p, const int32_t *idx, const float *val,
+                              const int32_t *counts, float scale, float *dense, cudaStream_t s);
+void count_launch(int n);
+
+}  // namespace rsdgc

@@ -1,0 +1,158 @@
+"""Helpers of the GPU parity tests: arena marshalling, one GPU compress call through the
+C ABI, and the comparison rules between the CUDA library and the CPU oracle.
+
+Rules (tolerances are the ones the task fixes for this path):
+  R1  |NSI_gpu - NSI_ref| <= 1e-5 * |NSI_ref| + FLT_MIN, NSI_ref in binary64.
+  R2  counts equal k_l; the kept set has exactly k_l strictly ascending tiles; every tile whose
+      NSI_ref is above T(1 + 2e-5) is kept and none below T(1 - 2e-5) is; if the kept set
+      equals the oracle's, idx / val / residual are bit-exact against the oracle; if it differs
+      (only possible inside the band), they are bit-exact against the oracle's pack of the
+      GPU's set.
+  R3  |dense_gpu - dense_ref| <= 1e-6 * sum_w |scale * sent_w| per element.
+"""
+from __future__ import annotations
+
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from paper_2312_17530_b200 import binding
+
+TAU = 1e-5
+FLT_MIN = float(np.finfo(np.float32).tiny)
+CANARY = np.float32(-7.25)
+
+
+def to_arena(plan: binding.Plan, per_layer: Sequence[np.ndarray], dtype=np.float32, fill=CANARY) -> np.ndarray:
+    """Flat arena with the plan's layer offsets; padding holds a canary value."""
+    if dtype == np.uint16:
+        a = np.full(plan.info.arena_elems, 0xC0E8, dtype=np.uint16)  # bfloat16(-7.25)
+    else:
+        a = np.full(plan.info.arena_elems, fill, dtype=dtype)
+    for li, x in zip(plan.layers, per_layer):
+        x = np.asarray(x).reshape(-1)
+        assert x.size == li.rows * li.cols
+        a[li.elem_offset:li.elem_offset + x.size] = x
+    return a
+
+
+def from_arena(plan: binding.Plan, arena: np.ndarray) -> List[np.ndarray]:
+    return [arena[li.elem_offset:li.elem_offset + li.rows * li.cols] for li in plan.layers]
+
+
+def padding_mask(plan: binding.Plan) -> np.ndarray:
+    m = np.ones(plan.info.arena_elems, dtype=bool)
+    for li in plan.layers:
+        m[li.elem_offset:li.elem_offset + li.rows * li.cols] = False
+    return m
+
+
+def dev(x: np.ndarray, device="cuda:0") -> torch.Tensor:
+    t = torch.from_numpy(np.ascontiguousarray(x))
+    if x.dtype == np.uint16:
+        t = t.view(torch.bfloat16)
+    return t.to(device)
+
+
+class GpuCompress:
+    """One worker's buffers on the device plus a call of rsdgc_compress()."""
+
+    def __init__(self, plan: binding.Plan, max_ratio: float = 1.0, device="cuda:0", with_nsi: bool = True):
+        self.plan, self.device = plan, device
+        ni, nv = plan.payload_bound(max_ratio)
+        self.idx = torch.full((max(ni, 4),), -1, dtype=torch.int32, device=device)
+        self.val = torch.full((max(nv, 4),), float(CANARY), dtype=torch.float32, device=device)
+        self.counts = torch.full((plan.n_layers,), -1, dtype=torch.int32, device=device)
+        self.nsi = torch.full((plan.info.total_tiles_padded,), float(CANARY), dtype=torch.float32,
+                              device=device) if with_nsi else None
+        self.workspace = None if with_nsi else torch.empty(max(plan.info.workspace_bytes, 16), dtype=torch.uint8,
+                                                           device=device)
+
+    def run(self, grads: torch.Tensor, residual: torch.Tensor, ratios: torch.Tensor):
+        self.plan.compress(grads, residual, ratios, self.idx, self.val, self.counts, nsi=self.nsi,
+                           workspace=self.workspace)
+        torch.cuda.synchronize()
+        return self.plan.status()
+
+    def payload(self):
+        return self.idx, self.val, self.counts
+
+
+def check_layer(oracle, li, shape, g, r, ratio, alpha, clamp, gpu_nsi, gpu_count, gpu_idx, gpu_val, gpu_res,
+                strict_keys: bool = True, what: str = ""):
+    """Applies R1 and R2 to one layer; returns the oracle's LayerResult."""
+    ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp)
+    K = ref.nsi_f32.size
+    # R1
+    err = np.abs(gpu_nsi.astype(np.float64) - ref.nsi_ref)
+    finite = np.isfinite(ref.nsi_ref)
+    assert (err[finite] <= TAU * np.abs(ref.nsi_ref[finite]) + FLT_MIN).all(), what + ": NSI beyond 1e-5 relative"
+    assert (gpu_nsi[ref.nsi_ref == 0] == 0).all() and not np.signbit(gpu_nsi[finite]).any()
+    if strict_keys:  # same binary32 operations in the same order on both sides
+        np.testing.assert_array_equal(gpu_nsi.view(np.uint32), ref.nsi_f32.view(np.uint32), err_msg=what)
+    # R2
+    assert gpu_count == ref.k, "%s: count %d != k %d" % (what, gpu_count, ref.k)
+    assert gpu_idx.size == ref.k
+    if ref.k:
+        assert (np.diff(gpu_idx) > 0).all() and gpu_idx[0] >= 0 and gpu_idx[-1] < K, what + ": idx not ascending"
+        T = ref.threshold
+        kept = np.zeros(K, dtype=bool)
+        kept[gpu_idx] = True
+        if np.isfinite(T):
+            must = ref.nsi_ref > T * (1 + 2 * TAU)
+            must_not = ref.nsi_ref < T * (1 - 2 * TAU)
+            assert kept[must].all(), what + ": a tile clearly above the threshold is missing"
+            assert not kept[must_not].any(), what + ": a tile clearly below the threshold was kept"
+    if not np.array_equal(gpu_idx, ref.idx):
+        ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp, forced_sel=gpu_idx)
+    np.testing.assert_array_equal(gpu_idx, ref.idx, err_msg=what)
+    np.testing.assert_array_equal(gpu_val.view(np.uint32), ref.val.view(np.uint32), err_msg=what + " val")
+    np.testing.assert_array_equal(gpu_res.view(np.uint32), ref.residual.view(np.uint32), err_msg=what + " residual")
+    return ref
+
+
+def compress_and_check(oracle, plan: binding.Plan, shapes, grads: Sequence[np.ndarray],
+                       residuals: Sequence[np.ndarray], ratios: Sequence[float], alpha: float, clamp: bool = True,
+                       gc: Optional[GpuCompress] = None, strict_keys: bool = True, what: str = "",
+                       max_ratio: float = 1.0):
+    """Runs one GPU compress and checks every layer against the oracle.  Returns
+    (new residuals per layer, oracle results per layer, GpuCompress)."""
+    g_is_bf16 = grads[0].dtype == np.uint16
+    g_arena = to_arena(plan, grads, np.uint16 if g_is_bf16 else np.float32)
+    r_arena = to_arena(plan, residuals)
+    gc = gc or GpuCompress(plan, max_ratio=max_ratio)
+    d_g, d_r = dev(g_arena), dev(r_arena)
+    d_ratios = torch.tensor(np.asarray(ratios, dtype=np.float32), device=gc.device)
+    st = gc.run(d_g, d_r, d_ratios)
+    assert st.flags == 0, "%s: status flags %d" % (what, st.flags)
+    # inputs untouched, padding untouched
+    g_back = d_g.view(torch.int16).cpu().numpy().view(np.uint16) if g_is_bf16 else d_g.cpu().numpy()
+    np.testing.assert_array_equal(g_back, g_arena)
+    res_arena = d_r.cpu().numpy()
+    pad = padding_mask(plan)
+    assert (res_arena[pad] == CANARY).all(), what + ": padding of the residual arena was written"
+    counts = gc.counts.cpu().numpy()
+    idx, val, nsi = gc.idx.cpu().numpy(), gc.val.cpu().numpy(), gc.nsi.cpu().numpy()
+    assert st.idx_needed == counts.sum()
+    io = vo = 0
+    refs, new_res = [], []
+    for l, (li, shape) in enumerate(zip(plan.layers, shapes)):
+        k, slot = int(counts[l]), shape[2] * shape[3]
+        ref = check_layer(oracle, li, shape, grads[l], residuals[l], float(np.float32(ratios[l])), alpha, clamp,
+                          nsi[li.tile_offset:li.tile_offset + li.n_tiles], k, idx[io:io + k],
+                          val[vo:vo + k * slot], res_arena[li.elem_offset:li.elem_offset + li.rows * li.cols],
+                          strict_keys=strict_keys, what="%s layer %d %r" % (what, l, tuple(shape)))
+        io, vo = io + k, vo + k * slot
+        refs.append(ref)
+        new_res.append(ref.residual)
+    assert st.val_needed == vo
+    assert (idx[io:] == -1).all() and (val[vo:] == CANARY).all(), what + ": payload written past its end"
+    return new_res, refs, gc
+
+
+def check_decompress(dense_gpu: np.ndarray, dense_ref: np.ndarray, abs_sent_sum: np.ndarray, exact: bool = True):
+    """R3 (and bit-exactness, which holds because workers are added in order on both sides)."""
+    assert (np.abs(dense_gpu.astype(np.float64) - dense_ref) <= 1e-6 * abs_sent_sum + 1e-45).all()
+    if exact:
+        np.testing.assert_array_equal(dense_gpu.view(np.uint32), dense_ref.view(np.uint32))

@@ -1,0 +1,240 @@
+"""GPU parity: the CUDA library (through the C ABI) against the CPU oracle, element by element,
+on seeded inputs: the 512x512 single layer, a zoo of small / ragged / degenerate layers, the
+ResNet-18-shaped set over 10 iterations with the ratio rule, aggregation of several workers."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2312_17530_b200 import binding, synth
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    binding.lib()  # raises if the CUDA library has not been built: no fallback
+
+
+# ---------------------------------------------------------------------------------------------
+# config 1: one 512x512 layer, clustered outliers, zero residual, 3x3 tiles, keep 1/64
+# ---------------------------------------------------------------------------------------------
+
+def test_single_layer_512(oracle):
+    shapes = [(512, 512, 3, 3)]
+    g = [synth.clustered_matrix(512, 512, seed=0)]
+    r = [np.zeros(512 * 512, np.float32)]
+    plan = binding.Plan(shapes, alpha=0.5)
+    assert plan.layers[0].n_tiles == 171 * 171
+    _, refs, gc = parity.compress_and_check(oracle, plan, shapes, g, r, [1 / 64], 0.5, what="512x512")
+    assert refs[0].k == 457
+    # the boosted 8x8 patches dominate the selection
+    assert np.abs(refs[0].val).mean() > 5e-3
+
+
+# ---------------------------------------------------------------------------------------------
+# small, ragged and degenerate layers
+# ---------------------------------------------------------------------------------------------
+
+ZOO = [
+    (7, 11, 3, 3), (1, 1, 3, 3), (3, 3, 3, 3), (4, 4, 3, 3), (1, 5, 1, 9), (1, 64, 1, 9), (64, 9, 1, 9),
+    (4096, 45, 3, 3), (2, 20000, 3, 3), (100, 6145, 2, 5), (5000, 7, 1, 7), (1, 100003, 1, 9),
+    (130, 130, 64, 64), (30, 30, 1, 1), (192, 49, 1, 49), (257, 1026, 3, 3), (999, 2049, 3, 3),
+    (13, 8190, 4, 6), (70000, 9, 1, 9), (1000, 512, 3, 3),
+]
+
+
+@pytest.mark.parametrize("alpha", [0.5, 0.0, 1.0, 0.25])
+def test_layer_zoo(oracle, alpha):
+    rng = np.random.default_rng(int(alpha * 100) + 1)
+    shapes = ZOO
+    g = [(rng.standard_normal(r * c) * 10 ** rng.uniform(-4, 0)).astype(np.float32) for r, c, _, _ in shapes]
+    res = [(rng.standard_normal(r * c) * 10 ** rng.uniform(-5, -1)).astype(np.float32) for r, c, _, _ in shapes]
+    ratios = rng.choice([0.001, 0.01, 1 / 64, 0.1, 0.3, 1.0, 0.0], size=len(shapes)).astype(np.float32)
+    plan = binding.Plan(shapes, alpha=alpha)
+    new_res, refs, gc = parity.compress_and_check(oracle, plan, shapes, g, res, ratios, alpha, what="zoo")
+    # second iteration on the carried residual, same buffers
+    g2 = [(rng.standard_normal(r * c) * 1e-2).astype(np.float32) for r, c, _, _ in shapes]
+    gc.idx.fill_(-1)
+    gc.val.fill_(float(parity.CANARY))
+    parity.compress_and_check(oracle, plan, shapes, g2, new_res, ratios, alpha, gc=gc, what="zoo it2")
+
+
+def test_degenerate_layers(oracle):
+    rng = np.random.default_rng(5)
+    shapes = [(60, 60, 3, 3), (60, 60, 3, 3), (1, 900, 1, 9), (33, 33, 3, 3), (1, 7, 1, 9), (300, 300, 3, 3)]
+    g = [np.zeros(3600, np.float32),                                    # all-zero layer: all NSI equal 0
+         np.full(3600, 0.125, np.float32),                              # constant: all NSI equal, pure ties
+         np.tile(np.arange(9, dtype=np.float32), 100),                  # identical tiles
+         rng.standard_normal(33 * 33).astype(np.float32),
+         rng.standard_normal(7).astype(np.float32),                    # a single clipped tile
+         np.repeat(rng.integers(0, 3, 100 * 100), 9).reshape(100, 100, 3, 3).transpose(0, 2, 1, 3)
+         .reshape(-1).astype(np.float32)]                               # three distinct NSI values: many ties
+    res = [np.zeros(x.size, np.float32) for x in g]
+    for ratios, clamp in (([0.1, 0.1, 0.05, 1.0, 0.5, 0.4], True), ([0.0] * 6, True), ([0.0] * 6, False),
+                          ([1.0] * 6, True), ([0.5, 1e-9, 2.0, -1.0, 0.0, 0.33], False)):
+        plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE if clamp else 0)
+        _, refs, _ = parity.compress_and_check(oracle, plan, shapes, g, res, ratios, 0.5, clamp=clamp, what="degenerate")
+        if ratios[0] == 0.1:
+            k = oracle.keep_count(400, 0.1)                             # pure ties: the first k tiles
+            assert refs[0].idx.tolist() == list(range(k)) and refs[1].idx.tolist() == list(range(k))
+        if not clamp and ratios[0] == 0.0:
+            assert sum(r.k for r in refs) == 0
+
+
+def test_nonfinite_inputs_are_flagged_and_deterministic(oracle):
+    shapes = [(30, 30, 3, 3), (1, 90, 1, 9)]
+    rng = np.random.default_rng(6)
+    g = [rng.standard_normal(900).astype(np.float32), rng.standard_normal(90).astype(np.float32)]
+    g[0][[5, 400]] = [np.inf, np.nan]
+    g[1][17] = -np.inf
+    plan = binding.Plan(shapes, alpha=0.5)
+    outs = []
+    for _ in range(2):
+        gc = parity.GpuCompress(plan)
+        d_g = parity.dev(parity.to_arena(plan, g))
+        d_r = parity.dev(parity.to_arena(plan, [np.zeros(900, np.float32), np.zeros(90, np.float32)]))
+        st = gc.run(d_g, d_r, torch.tensor([0.05, 0.2], device="cuda:0"))
+        assert st.flags == binding.STATUS_NONFINITE and st.nonfinite == 3
+        outs.append((gc.idx.cpu().numpy().copy(), gc.nsi.cpu().numpy().view(np.uint32).copy()))
+    np.testing.assert_array_equal(outs[0][0], outs[1][0])
+    np.testing.assert_array_equal(outs[0][1], outs[1][1])
+    ref0 = oracle.compress_layer(g[0], np.zeros(900, np.float32), shapes[0], 0.05, 0.5)
+    assert ref0.nonfinite == 2
+    np.testing.assert_array_equal(outs[0][0][:ref0.k], ref0.idx)      # non-finite tiles rank first
+
+
+def test_payload_overflow_is_reported_and_nothing_is_lost(oracle):
+    shapes = [(90, 90, 3, 3), (60, 60, 3, 3)]
+    rng = np.random.default_rng(7)
+    g = [rng.standard_normal(8100).astype(np.float32), rng.standard_normal(3600).astype(np.float32)]
+    plan = binding.Plan(shapes, alpha=0.5)
+    gc = parity.GpuCompress(plan, max_ratio=0.01)           # room for about 1 % of the tiles only
+    cap = gc.idx.numel()
+    k0, k1 = oracle.keep_count(900, 0.1), oracle.keep_count(400, 0.1)
+    assert cap < k0
+    d_g = parity.dev(parity.to_arena(plan, g))
+    r0 = parity.to_arena(plan, [np.zeros(8100, np.float32), np.zeros(3600, np.float32)])
+    d_r = parity.dev(r0)
+    st = gc.run(d_g, d_r, torch.tensor([0.1, 0.1], device="cuda:0"))
+    assert st.flags == binding.STATUS_PAYLOAD_OVERFLOW
+    assert st.idx_needed == k0 + k1 and st.val_needed == 9 * (k0 + k1)
+    counts = gc.counts.cpu().numpy()
+    assert counts.tolist() == [k0, k1]
+    # tiles that fit were sent and zeroed; all others still sit in the residual: sent + residual == v
+    idx, val = gc.idx.cpu().numpy(), gc.val.cpu().numpy()
+    res = parity.from_arena(plan, d_r.cpu().numpy())
+    sent = np.zeros(8100, np.float32)
+    oracle.decompress_into(sent, shapes[0], idx[:cap], val[:cap * 9], 1.0)
+    assert (sent + res[0] == g[0]).all() and (res[1] == g[1]).all()
+
+
+# ---------------------------------------------------------------------------------------------
+# config 2: ResNet-18-shaped set, 10 iterations, residual carried, ratios from the weights
+# ---------------------------------------------------------------------------------------------
+
+def test_resnet18_ten_iterations_with_dynamic_ratios(oracle):
+    tensors = synth.resnet18_tensors()
+    shapes = synth.layer_shapes(tensors)
+    plan = binding.Plan(shapes, alpha=0.5)
+    weights = synth.synthetic_weights(tensors, (2,))
+    # ratio rule (Eq. 3-5) on the GPU against the oracle's full sort
+    d_w = parity.dev(parity.to_arena(plan, weights))
+    d_ratios = torch.full((plan.n_layers,), -1.0, device="cuda:0")
+    plan.update_ratios(d_w, 1 / 50, d_ratios)
+    torch.cuda.synchronize()
+    ratios_ref, surv, n_keep = oracle.update_ratios(weights, 1 / 50)
+    np.testing.assert_array_equal(d_ratios.cpu().numpy(), ratios_ref)
+    assert n_keep == surv.sum() and (ratios_ref == 1.0).any() and (ratios_ref == 0.0).any()
+    total = sum(int(np.ceil(k * float(r))) for k, r in zip([li.n_tiles for li in plan.layers], ratios_ref))
+    assert 30 < plan.info.total_tiles / total < 70                      # about 50x fewer neighborhoods
+
+    scales = synth.log_uniform_scales(len(tensors), (2,))
+    res = [np.zeros(synth.numel(s), np.float32) for _, s in tensors]
+    gc = parity.GpuCompress(plan, max_ratio=1.0)
+    for it in range(10):
+        g = synth.laplace_layers(tensors, (2, it), scales)
+        gc.idx.fill_(-1)
+        gc.val.fill_(float(parity.CANARY))
+        res, refs, _ = parity.compress_and_check(oracle, plan, shapes, g, res, ratios_ref, 0.5, gc=gc,
+                                                 what="resnet18 it%d" % it)
+
+
+# ---------------------------------------------------------------------------------------------
+# aggregation of several workers (Eq. 12 third line) on a mid-sized layer set
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("scale", [1.0, 0.25])
+def test_decompress_accumulate_four_workers(oracle, scale):
+    tensors = synth.vgg19_tensors()[:12] + [("fc.weight", (1000, 513)), ("fc.bias", (1000,))]
+    shapes = synth.layer_shapes(tensors)
+    plan = binding.Plan(shapes, alpha=0.5)
+    sig = synth.log_uniform_scales(len(tensors), (3,))
+    grads = synth.multi_worker_gradients(tensors, 4, (3,), sig)
+    ratios = np.full(len(shapes), 1 / 16, np.float32)
+    zeros = [np.zeros(synth.numel(s), np.float32) for _, s in tensors]
+    payloads, refs_all = [], []
+    for w in range(4):
+        _, refs, gc = parity.compress_and_check(oracle, plan, shapes, grads[w], zeros, ratios, 0.5,
+                                                what="worker %d" % w, max_ratio=1 / 16)
+        payloads.append(gc.payload())
+        refs_all.append(oracle.CompressResult(layers=refs))
+    rng = np.random.default_rng(8)
+    dense0 = [(rng.standard_normal(synth.numel(s)) * 1e-3).astype(np.float32) for _, s in tensors]
+    d_dense = parity.dev(parity.to_arena(plan, dense0))
+    plan.decompress_accumulate(payloads, d_dense, scale)
+    torch.cuda.synchronize()
+    dense_ref = [d.copy() for d in dense0]
+    oracle.decompress_accumulate(shapes, dense_ref, refs_all, scale)
+    out = d_dense.cpu().numpy()
+    assert (out[parity.padding_mask(plan)] == parity.CANARY).all()
+    collisions = 0
+    for l, (got, ref) in enumerate(zip(parity.from_arena(plan, out), dense_ref)):
+        abs_sum = np.zeros(ref.size)
+        hit = np.zeros(ref.size, np.int32)
+        for w in range(4):
+            s = np.zeros(ref.size, np.float32)
+            oracle.decompress_into(s, shapes[l], refs_all[w].layers[l].idx, refs_all[w].layers[l].val, scale)
+            abs_sum += np.abs(s)
+            hit += (s != 0)
+        collisions += int((hit > 1).sum())
+        parity.check_decompress(got, ref, abs_sum)
+    assert collisions > 1000                                   # the workers' selections do overlap
+    # empty payload: nothing changes
+    before = d_dense.clone()
+    zc = torch.zeros(plan.n_layers, dtype=torch.int32, device="cuda:0")
+    plan.decompress_accumulate([(payloads[0][0], payloads[0][1], zc)], d_dense, 1.0)
+    plan.decompress_accumulate([], d_dense, 1.0)
+    torch.cuda.synchronize()
+    assert torch.equal(before, d_dense)
+
+
+def test_bf16_gradients(oracle):
+    shapes = [(300, 515, 3, 3), (128, 64 * 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3)]
+    rng = np.random.default_rng(9)
+    g = [synth.f32_to_bf16_bits((rng.standard_normal(r * c) * 1e-2).astype(np.float32)) for r, c, _, _ in shapes]
+    res = [(rng.standard_normal(r * c) * 1e-3).astype(np.float32) for r, c, _, _ in shapes]
+    plan = binding.Plan(shapes, grad_dtype=binding.RSDGC_BF16, alpha=0.5)
+    parity.compress_and_check(oracle, plan, shapes, g, res, [0.02, 0.1, 0.5, 0.01], 0.5, what="bf16")
+
+
+def test_repeated_runs_are_bit_identical(oracle):
+    tensors = synth.resnet18_tensors()
+    shapes = synth.layer_shapes(tensors)
+    plan = binding.Plan(shapes, alpha=0.5)
+    g = synth.laplace_layers(tensors, (4, 0), synth.log_uniform_scales(len(tensors), (4,)))
+    g_arena = parity.to_arena(plan, g)
+    ratios = torch.full((len(shapes),), 0.02, device="cuda:0")
+    outs = []
+    for rep in range(3):
+        gc = parity.GpuCompress(plan, max_ratio=0.02)
+        d_r = parity.dev(parity.to_arena(plan, [np.zeros(x.size, np.float32) for x in g]))
+        st = gc.run(parity.dev(g_arena), d_r, ratios)
+        assert st.flags == 0
+        outs.append([t.cpu().numpy().copy() for t in (gc.idx, gc.val, gc.counts, gc.nsi, d_r)])
+    for a, b in zip(outs[0], outs[1]):
+        np.testing.assert_array_equal(a.view(np.uint32), b.view(np.uint32))
+    for a, b in zip(outs[0], outs[2]):
+        np.testing.assert_array_equal(a.view(np.uint32), b.view(np.uint32))

@@ -1,0 +1,101 @@
+"""Host-side logic of the CUDA library, checked without a GPU: the shared library loads and
+exports every symbol the header declares, and host-only plans (device < 0) give consistent
+sizes, offsets and work lists."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+from paper_2312_17530_b200 import binding, synth
+from paper_2312_17530_b200.build import build_library
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build_library()
+    return binding.lib()
+
+
+def test_library_exports_every_declared_symbol(lib):
+    header = open(os.path.join(ROOT, "include", "rsdgc.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(rsdgc_[a-z_0-9]+)\s*\(", header))
+    assert declared == set(binding.EXPORTS)
+    for name in declared:
+        assert getattr(lib, name) is not None
+    assert lib.rsdgc_strerror(0) == b"ok" and lib.rsdgc_strerror(-2) != lib.rsdgc_strerror(-1)
+    assert lib.rsdgc_launch_count() == 0
+
+
+def test_plan_create_rejects_bad_arguments(lib):
+    ok = [(8, 8, 3, 3)]
+    for layers, kw in [([], {}), ([(0, 8, 3, 3)], {}), ([(8, 8, 0, 3)], {}), (ok, {"alpha": 1.5}),
+                       (ok, {"alpha": float("nan")}), (ok, {"grad_dtype": 7}), (ok, {"flags": 8})]:
+        with pytest.raises(binding.RsdgcError) as e:
+            binding.Plan(layers, device=-1, **kw)
+        assert e.value.code == binding.ERR_INVALID
+    for layers in ([(8, 8, 65, 65)], [(1 << 20, 1 << 20, 3, 3)], [(4, 4, 3, 3)] * 3000):
+        with pytest.raises(binding.RsdgcError) as e:
+            binding.Plan(layers, device=-1)
+        assert e.value.code == binding.ERR_CAPACITY
+    # a host-only plan cannot launch anything
+    p = binding.Plan(ok, device=-1)
+    assert lib.rsdgc_compress(p._h, 16, 16, 16, 16, 1, 16, 1, 16, None, 16, None) == binding.ERR_INVALID
+
+
+@pytest.mark.parametrize("net", ["resnet18", "resnet50", "vgg19", "odd"])
+def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net):
+    if net == "odd":
+        shapes = [(7, 11, 3, 3), (1, 5, 1, 9), (4096, 45, 3, 3), (3, 20000, 3, 3), (100, 6145, 2, 5),
+                  (5000, 7, 1, 7), (1, 100000, 1, 9), (64, 64, 64, 64), (9, 9, 1, 1)]
+    else:
+        shapes = synth.layer_shapes(getattr(synth, net + "_tensors")())
+    p = binding.Plan(shapes, device=-1)
+    assert p.info.n_layers == len(shapes)
+    assert p.info.total_elems == sum(r * c for r, c, _, _ in shapes)
+    tiles = [(-(-r // nh)) * (-(-c // nw)) for r, c, nh, nw in shapes]
+    assert p.info.total_tiles == sum(tiles)
+    eo = to = 0
+    for l, (li, (r, c, nh, nw)) in enumerate(zip(p.layers, shapes)):
+        assert (li.elem_offset, li.tile_offset, li.n_tiles) == (eo, to, tiles[l])
+        assert li.elem_offset % 64 == 0 and li.tile_offset % 64 == 0
+        eo += -(-r * c // 64) * 64
+        to += -(-tiles[l] // 64) * 64
+    assert p.info.arena_elems == eo and p.info.total_tiles_padded == to
+    assert p.info.workspace_bytes == 4 * to
+
+    items, cta, nflush = p.worklist()
+    assert cta[0] == 0 and cta[-1] == len(items) and (np.diff(cta) >= 0).all() and len(cta) == 148 * 4 + 1
+    assert (np.diff(items[:, 0]) >= 0).all()          # layers in order
+    owner = np.searchsorted(cta, np.arange(len(items)), side="right") - 1
+    for l, (r, c, nh, nw) in enumerate(shapes):
+        TR, TC = -(-r // nh), -(-c // nw)
+        cover = np.zeros((TR, TC), dtype=np.int32)
+        sel = items[items[:, 0] == l]
+        for _, tr0, ntr, tc0, ntc in sel.tolist():
+            assert ntr >= 1 and ntc >= 1 and tr0 + ntr <= TR and tc0 + ntc <= TC
+            rows = min(r, (tr0 + ntr) * nh) - tr0 * nh
+            cols = min(c, (tc0 + ntc) * nw) - tc0 * nw
+            assert rows * cols <= 6144
+            assert ntr == 1 or (tc0 == 0 and ntc == TC)   # several tile rows only at full width
+            cover[tr0:tr0 + ntr, tc0:tc0 + ntc] += 1
+        assert (cover == 1).all()
+        assert nflush[l] == len(set(owner[items[:, 0] == l].tolist()))
+    # the static partition is balanced: no CTA holds much more than the mean cost
+    cost = np.zeros(len(cta) - 1)
+    for i, (l, tr0, ntr, tc0, ntc) in enumerate(items.tolist()):
+        r, c, nh, nw = shapes[l]
+        cost[owner[i]] += (min(r, (tr0 + ntr) * nh) - tr0 * nh) * (min(c, (tc0 + ntc) * nw) - tc0 * nw) + 512
+    assert cost.max() <= cost.sum() / len(cost) + 6144 + 512 + 1
+
+
+def test_payload_bound(lib):
+    shapes = [(512, 512, 3, 3), (1, 64, 1, 9)]
+    p = binding.Plan(shapes, device=-1)
+    ni, nv = p.payload_bound(1 / 64)
+    assert ni == (457 + 1) + 2 and nv == 9 * ni
+    ni, nv = p.payload_bound(1.0)
+    assert ni == 29241 + 8
