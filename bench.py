@@ -1,0 +1,360 @@
+#!/usr/bin/env python
+"""Benchmark of the RS-DGC compression path on B200.
+
+Workload: the VGG-19-shaped gradient set (38 tensors, 139,754,605 fp32 elements per worker),
+4 simulated workers per GPU, uniform keep ratio 1/64, alpha 0.5.  One step = every worker's
+rsdgc_compress() (accumulate, NSI, threshold select, pack, residual update) followed by one
+rsdgc_decompress_accumulate() of the 4 payloads into a dense buffer on the same GPU.  The
+per-epoch ratio rule (rsdgc_update_ratios) is timed separately and reported in "extra".
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl b200|reference]
+
+With N > 1 launch through torch.distributed.run (one rank per GPU); every rank runs the same
+step on its own workers (weak scaling, no data-path collective); rank 0 prints ONE JSON line.
+--impl reference times the CPU oracle (the deliberately slow checker) on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "gradient GB/s compressed (NSI+select+pack)"
+UNIT = "GB/s"
+N_WORKERS = 4
+KEEP_RATIO = 1.0 / 64.0
+ALPHA = 0.5
+WORKLOAD = ("VGG-19-shaped gradient set (38 tensors, 139754605 fp32 elements per worker), %d workers per GPU, "
+            "keep 1/64 of the neighborhoods per layer, alpha 0.5; step = %d x compress + 1 x "
+            "decompress_accumulate" % (N_WORKERS, N_WORKERS))
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    return 6650.0, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """nvidia-smi sampling of SM clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = os.path.join("/tmp", "rsdgc_clocks_%d_%d.csv" % (os.getpid(), gpu_index))
+
+    def start(self):
+        try:
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=self.out, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            tok = [t.strip() for t in line.split(",")]
+            if len(tok) < 9:
+                continue
+            try:
+                sm.append(float(tok[1]))
+                smax.append(float(tok[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, tok[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def vgg_inputs(rank: int, n_workers: int = N_WORKERS):
+    """(tensors, shapes, per-worker per-layer gradients) for this rank's workers."""
+    from paper_2312_17530_b200 import dist, synth
+
+    tensors = synth.vgg19_tensors()
+    shapes = synth.layer_shapes(tensors)
+    sig = synth.log_uniform_scales(len(tensors), (3,))
+    ids = dist.worker_ids(rank, N_WORKERS)
+    # one shared component per rank's group of workers; worker ids key the independent parts
+    grads = synth.multi_worker_gradients(tensors, n_workers, (3, rank), sig)
+    return tensors, shapes, grads, ids
+
+
+def run_reference(args):
+    """The CPU oracle as it stands, timed on the host cores: one step = the oracle's compress
+    of one worker's full VGG-19-shaped gradient (bounded sample of the 4-worker step)."""
+    from paper_2312_17530_b200 import dist
+
+    rank, _, world = dist.env_world()
+    if rank != 0:
+        return 0
+    import oracle
+
+    oracle.build()
+    tensors, shapes, grads, _ = vgg_inputs(0, 1)
+    g = grads[0]
+    n = sum(x.size for x in g)
+    res = [np.zeros(x.size, np.float32) for x in g]
+    ratios = [KEEP_RATIO] * len(shapes)
+    times = []
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        out = oracle.compress(shapes, g, res, ratios, ALPHA)
+        dt = time.perf_counter() - t0
+        res = [l.residual for l in out.layers]
+        if it >= args.warmup:
+            times.append(dt)
+    total = sum(times)
+    value = 4.0 * n * len(times) / total / 1e9
+    sample = "oracle compress of 1 worker's full VGG-19-shaped gradient (139754605 elements) per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                         "host_cores": os.cpu_count()},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def cpu_baseline(shapes, g):
+    """The oracle on one worker's full gradient, one thread, on this host."""
+    import oracle
+
+    oracle.build()
+    n = sum(x.size for x in g)
+    res = [np.zeros(x.size, np.float32) for x in g]
+    t0 = time.perf_counter()
+    oracle.compress(shapes, g, res, [KEEP_RATIO] * len(shapes), ALPHA)
+    dt = time.perf_counter() - t0
+    return {"value": 4.0 * n / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "1 of the %d workers of one step (139754605 elements), 1 iteration, %.1f s" % (N_WORKERS, dt),
+            "host_cores": os.cpu_count(), "us_per_model_iteration": dt * 1e6}
+
+
+def run_b200(args):
+    import torch
+
+    from paper_2312_17530_b200 import binding, dist
+
+    rank, local_rank, world = dist.init("nccl")
+    if world != args.gpus:
+        raise SystemExit("--gpus %d but WORLD_SIZE is %d: launch with torch.distributed.run" % (args.gpus, world))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    binding.lib()  # raises if the CUDA library has not been built; there is no other path
+
+    tensors, shapes, grads, _ = vgg_inputs(rank)
+    plan = binding.Plan(shapes, alpha=ALPHA, device=local_rank)
+    n = plan.info.total_elems
+    arena = plan.info.arena_elems
+    ni, nv = plan.payload_bound(KEEP_RATIO)
+
+    def to_arena(per_layer, pin=False):
+        a = torch.zeros(arena, dtype=torch.float32, pin_memory=pin)
+        an = a.numpy()
+        for li, x in zip(plan.layers, per_layer):
+            an[li.elem_offset:li.elem_offset + x.size] = x
+        return a
+
+    host_g = [to_arena(grads[w], pin=True) for w in range(N_WORKERS)]
+    d_g = [h.to(device, non_blocking=True) for h in host_g]
+    d_r = [torch.zeros(arena, dtype=torch.float32, device=device) for _ in range(N_WORKERS)]
+    d_idx = [torch.zeros(ni, dtype=torch.int32, device=device) for _ in range(N_WORKERS)]
+    d_val = [torch.zeros(nv, dtype=torch.float32, device=device) for _ in range(N_WORKERS)]
+    d_cnt = [torch.zeros(plan.n_layers, dtype=torch.int32, device=device) for _ in range(N_WORKERS)]
+    d_ws = torch.empty(plan.info.workspace_bytes, dtype=torch.uint8, device=device)
+    d_ratios = torch.full((plan.n_layers,), KEEP_RATIO, dtype=torch.float32, device=device)
+    d_dense = torch.zeros(arena, dtype=torch.float32, device=device)
+    torch.cuda.synchronize()
+
+    def step():
+        for w in range(N_WORKERS):
+            plan.compress(d_g[w], d_r[w], d_ratios, d_idx[w], d_val[w], d_cnt[w], workspace=d_ws)
+        plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
+
+    # ---- device-resident timing: W warm-up steps, then exactly K steps between two events
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    assert plan.status().flags == 0
+    plan.profile_enable(True)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev_dec = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    dist.barrier()
+    torch.cuda.synchronize()
+    launches0 = binding.launch_count()
+    ev0.record()
+    for s in range(args.steps):
+        for w in range(N_WORKERS):
+            plan.compress(d_g[w], d_r[w], d_ratios, d_idx[w], d_val[w], d_cnt[w], workspace=d_ws)
+        ev_dec[s][0].record()
+        plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
+        ev_dec[s][1].record()
+    ev1.record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    launches = binding.launch_count() - launches0
+    clocks = sampler.stop()
+    elapsed_s = ev0.elapsed_time(ev1) / 1e3
+    kernel_ms, n_calls = plan.profile_read()
+    plan.profile_enable(False)
+    dec_ms = sum(a.elapsed_time(b) for a, b in ev_dec) / args.steps
+    st = plan.status()
+    assert st.flags == 0, "status flags %d after the timed region" % st.flags
+
+    grad_bytes_step = 4.0 * n * N_WORKERS
+    value_bps, t_max = dist.aggregate_throughput(grad_bytes_step * args.steps, elapsed_s)
+    value = value_bps / 1e9
+
+    # ---- end to end: host buffers in, payload out, through rsdgc_compress_host()
+    h_idx = torch.zeros(ni, dtype=torch.int32, pin_memory=True)
+    h_val = torch.zeros(nv, dtype=torch.float32, pin_memory=True)
+    h_cnt = torch.zeros(plan.n_layers, dtype=torch.int32, pin_memory=True)
+    d_stage = torch.empty(arena, dtype=torch.float32, device=device)
+    e2e_steps = max(1, min(args.steps, 5))
+    d2h = 0
+
+    def e2e_step():
+        nonlocal d2h
+        d2h = 0
+        for w in range(N_WORKERS):
+            a, b = plan.compress_host(host_g[w], d_stage, d_r[w], d_ratios, d_idx[w], d_val[w], d_cnt[w], d_ws,
+                                      h_idx, h_val, h_cnt)
+            d2h += 4 * a + 4 * b + 4 * plan.n_layers
+        plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
+
+    e2e_step()
+    dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    ev0.record()
+    for _ in range(e2e_steps):
+        e2e_step()
+    ev1.record()
+    torch.cuda.synchronize()
+    e2e_wall = time.perf_counter() - t0
+    e2e_s = max(ev0.elapsed_time(ev1) / 1e3, e2e_wall)  # host-side waits are part of this path
+    e2e_bps, _ = dist.aggregate_throughput(grad_bytes_step * e2e_steps, e2e_s)
+
+    # ---- separately timed: ratio rule (per epoch), dense zero fill
+    extra = {}
+    if rank == 0:
+        d_w = d_g[0]  # any fp32 arena of the right layout serves as "weights" for timing
+        d_rat2 = torch.empty(plan.n_layers, dtype=torch.float32, device=device)
+        plan.update_ratios(d_w, 1.0 / 50.0, d_rat2)
+        torch.cuda.synchronize()
+        ev0.record()
+        for _ in range(3):
+            plan.update_ratios(d_w, 1.0 / 50.0, d_rat2)
+        ev1.record()
+        torch.cuda.synchronize()
+        extra["update_ratios_us"] = ev0.elapsed_time(ev1) / 3 * 1e3
+        ev0.record()
+        for _ in range(3):
+            d_dense.zero_()
+        ev1.record()
+        torch.cuda.synchronize()
+        extra["dense_zero_fill_us"] = ev0.elapsed_time(ev1) / 3 * 1e3
+
+    if rank == 0:
+        peak, peak_src = measured_peaks()
+        k1_s = kernel_ms[0] / 1e3 / max(n_calls, 1)
+        compress_s = sum(kernel_ms) / 1e3 / max(n_calls, 1)
+        alg_bytes = 12.0 * n  # read g, read r, write v: 12 B per element for fp32 gradients
+        achieved = alg_bytes / k1_s / 1e9
+        per_kernel_us = {name: 1e3 * ms / max(n_calls, 1) for name, ms in zip(binding.COMPRESS_KERNELS, kernel_ms)}
+        extra.update({
+            "us_per_model_iteration": compress_s * 1e6,
+            "layers_per_s": plan.n_layers / compress_s,
+            "compress_kernels_us": per_kernel_us,
+            "compress_roofline_frac": alg_bytes / compress_s / 1e9 / peak,
+            "compress_roofline_frac_of_nominal_8TBs": alg_bytes / compress_s / 1e9 / 8000.0,
+            "decompress_accumulate_us": dec_ms * 1e3,
+            "payload_bytes_per_worker": int(4 * st.idx_needed + 4 * st.val_needed),
+            "compression_ratio_bytes": 4.0 * n / (4 * st.idx_needed + 4 * st.val_needed),
+            "e2e_steps": e2e_steps,
+        })
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * t_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "l2": "inputs larger than L2 (4 x 1.1 GB streamed per step)",
+                       "parallelism": "dp%d (independent replicas, no collective)" % args.gpus},
+            "clocks": clocks,
+            "e2e": {"value": e2e_bps / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(4 * arena * N_WORKERS),
+                    "d2h_bytes_per_step": int(d2h)},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "hbm", "kernel": "k1_accumulate_nsi", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "traffic": K1_TRAFFIC_BYTES,
+                         "peak_source": peak_src, "algorithmic_bytes": alg_bytes, "launch_us": k1_s * 1e6},
+            "extra": extra,
+        }
+        if args.gpus == 1 and not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(shapes, grads[0])
+        print(json.dumps(line))
+    dist.barrier()
+    dist.finalize()
+    return 0
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum of one k1_accumulate_nsi launch on this workload
+# from an ncu capture; None until a capture of the current kernel exists (see profiles/).
+K1_TRAFFIC_BYTES = None
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "b200":
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_b200(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

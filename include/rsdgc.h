@@ -200,6 +200,19 @@ int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,
                                 const int32_t *const *counts_dev_host, float scale,
                                 float *dense_dev, void *stream);
 
+/*
+ * Optional per-kernel timing of rsdgc_compress().  While enabled, every rsdgc_compress() on
+ * this plan records CUDA events on its stream before its first kernel and after each of its
+ * RSDGC_N_COMPRESS_KERNELS kernels (accumulate+NSI, refine level 2, refine level 3, count,
+ * pack).  rsdgc_profile_read() waits for the recorded events, adds the elapsed milliseconds
+ * of every kernel over all recorded calls into ms_per_kernel_host[RSDGC_N_COMPRESS_KERNELS],
+ * stores the number of calls and forgets them.  Off by default; not for use during stream
+ * capture.
+ */
+#define RSDGC_N_COMPRESS_KERNELS 5
+int rsdgc_profile_enable(rsdgc_plan *plan, int32_t enable);
+int rsdgc_profile_read(rsdgc_plan *plan, double *ms_per_kernel_host, int64_t *n_calls_host);
+
 /* Waits for the stream, copies the device status word to *out_host and clears it. */
 int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *out_host);
 

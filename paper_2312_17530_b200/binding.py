@@ -22,8 +22,10 @@ EXPORTS = [
     "rsdgc_plan_create", "rsdgc_plan_destroy", "rsdgc_plan_info", "rsdgc_plan_layer_info",
     "rsdgc_plan_payload_bound", "rsdgc_plan_worklist", "rsdgc_update_ratios", "rsdgc_compress",
     "rsdgc_compress_host", "rsdgc_decompress_accumulate", "rsdgc_get_status", "rsdgc_launch_count",
-    "rsdgc_strerror", "rsdgc_last_cuda_error",
+    "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
 ]
+N_COMPRESS_KERNELS = 5
+COMPRESS_KERNELS = ("accumulate_nsi", "refine2", "refine3", "count", "pack")
 
 
 class LayerDesc(C.Structure):
@@ -80,6 +82,8 @@ def lib():
                                           C.POINTER(i64), C.POINTER(i64), vp]
         L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
         L.rsdgc_get_status.argtypes = [vp, vp, C.POINTER(Status)]
+        L.rsdgc_profile_enable.argtypes = [vp, i32]
+        L.rsdgc_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
         L.rsdgc_launch_count.argtypes = []
         L.rsdgc_launch_count.restype = i64
         L.rsdgc_strerror.argtypes = [C.c_int]
@@ -191,6 +195,16 @@ class Plan:
             ia[w], va[w], ca[w] = i.data_ptr(), v.data_ptr(), c.data_ptr()
         _check(lib().rsdgc_decompress_accumulate(self._h, n, ia, va, ca, scale, _ptr(dense), _stream()),
                "rsdgc_decompress_accumulate")
+
+    def profile_enable(self, on: bool) -> None:
+        _check(lib().rsdgc_profile_enable(self._h, 1 if on else 0), "rsdgc_profile_enable")
+
+    def profile_read(self):
+        """(milliseconds summed per compress kernel, number of compress calls recorded)."""
+        ms = (C.c_double * N_COMPRESS_KERNELS)()
+        n = C.c_int64()
+        _check(lib().rsdgc_profile_read(self._h, ms, C.byref(n)), "rsdgc_profile_read")
+        return list(ms), n.value
 
     def status(self) -> Status:
         st = Status()

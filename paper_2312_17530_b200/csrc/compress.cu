@@ -91,7 +91,7 @@ __device__ __forceinline__ float tile_nsi_fixed(const float *p, int pitch, float
 }
 
 struct K1Shared {
-    float v[kItemElems];
+    float v[2][kItemElems];  // double buffer: tiles of item i are reduced while item i+1 streams in
     unsigned int hist[kL1Bins];
     unsigned long long scan_tmp[kThreads / 32];
     unsigned long long found[2];
@@ -121,9 +121,15 @@ __device__ void k1_flush_layer(K1Shared &sh, int layer, const LayerDev *layers, 
     __syncthreads();
     if (!sh.is_last) return;  // uniform for the CTA
     __threadfence();
-    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) {
-        sh.hist[b] = __ldcg(gh + b);
-        gh[b] = 0;
+    {
+        unsigned int h[kL1Bins / kThreads];
+#pragma unroll
+        for (int j = 0; j < kL1Bins / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + threadIdx.x);
+#pragma unroll
+        for (int j = 0; j < kL1Bins / kThreads; ++j) {
+            sh.hist[j * kThreads + threadIdx.x] = h[j];
+            gh[j * kThreads + threadIdx.x] = 0;
+        }
     }
     __syncthreads();
     const int K = layers[layer].K;
@@ -142,107 +148,181 @@ __device__ void k1_flush_layer(K1Shared &sh, int layer, const LayerDev *layers, 
     __syncthreads();
 }
 
+__device__ __forceinline__ ItemDev load_item(const ItemDev *items, int i)
+{
+    const uint4 *p = reinterpret_cast<const uint4 *>(items + i);
+    union {
+        uint4 q[3];
+        ItemDev d;
+    } u;
+    u.q[0] = __ldg(p);
+    u.q[1] = __ldg(p + 1);
+    u.q[2] = __ldg(p + 2);
+    return u.d;
+}
+
+// Registers that carry one item's g and r from the loads to the add: kVecPerThread 128-bit
+// words each (or 4 * kVecPerThread scalars on the unaligned path).
+struct K1Regs {
+    float4 g[kVecPerThread], r[kVecPerThread];
+};
+
+// Global (arena-relative) and shared-memory position of element e (0 <= e < R * W) of an item
+// whose rows are not contiguous in memory.
+__device__ __forceinline__ void item_pos(const ItemDev &d, int e, long long *g, int *s)
+{
+    const int row = e / d.W, col = e - row * d.W;
+    *g = d.gbase + (long long)row * d.cols + col;
+    *s = e;  // shared memory holds the R x W block densely
+}
+
+template <typename G>
+__device__ __forceinline__ void k1_issue_loads(const ItemDev &d, const G *__restrict__ grads,
+                                               const float *__restrict__ resid, K1Regs &x)
+{
+    const int tid = threadIdx.x;
+    const int n = d.R * d.W;
+    if (d.flags & kItemVec) {
+        const int nvec = (d.flags & kItemFull) ? (n >> 2) : n >> 2;  // W % 4 == 0 when rows are separate
+        const int wv = d.W >> 2;
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const int i = u * kThreads + tid;
+            if (i < nvec) {
+                long long gi;
+                if (d.flags & kItemFull) {
+                    gi = (d.gbase >> 2) + i;
+                } else {
+                    const int row = i / wv, j = i - row * wv;
+                    gi = ((d.gbase + (long long)row * d.cols) >> 2) + j;
+                }
+                x.g[u] = load_grad4(grads, gi);
+                x.r[u] = __ldcs(reinterpret_cast<const float4 *>(resid) + gi);
+            }
+        }
+    } else {
+        float *gs = reinterpret_cast<float *>(x.g), *rs = reinterpret_cast<float *>(x.r);
+#pragma unroll
+        for (int u = 0; u < 4 * kVecPerThread; ++u) {
+            const int e = u * kThreads + tid;
+            if (e < n) {
+                long long gi;
+                int si;
+                if (d.flags & kItemFull) gi = d.gbase + e; else item_pos(d, e, &gi, &si);
+                gs[u] = load_grad1(grads, gi);
+                rs[u] = __ldcs(resid + gi);
+            }
+        }
+    }
+}
+
+// v = g + r (Eq. 12): written in place over the residual and into the shared-memory block.
+__device__ __forceinline__ void k1_add_store(const ItemDev &d, float *__restrict__ resid, float *sv, K1Regs &x)
+{
+    const int tid = threadIdx.x;
+    const int n = d.R * d.W;
+    if (d.flags & kItemVec) {
+        const int nvec = n >> 2;
+        const int wv = d.W >> 2;
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const int i = u * kThreads + tid;
+            if (i < nvec) {
+                long long gi;
+                if (d.flags & kItemFull) {
+                    gi = (d.gbase >> 2) + i;
+                } else {
+                    const int row = i / wv, j = i - row * wv;
+                    gi = ((d.gbase + (long long)row * d.cols) >> 2) + j;
+                }
+                float4 v;
+                v.x = __fadd_rn(x.g[u].x, x.r[u].x);
+                v.y = __fadd_rn(x.g[u].y, x.r[u].y);
+                v.z = __fadd_rn(x.g[u].z, x.r[u].z);
+                v.w = __fadd_rn(x.g[u].w, x.r[u].w);
+                __stcs(reinterpret_cast<float4 *>(resid) + gi, v);
+                reinterpret_cast<float4 *>(sv)[i] = v;
+            }
+        }
+    } else {
+        const float *gs = reinterpret_cast<const float *>(x.g), *rs = reinterpret_cast<const float *>(x.r);
+#pragma unroll
+        for (int u = 0; u < 4 * kVecPerThread; ++u) {
+            const int e = u * kThreads + tid;
+            if (e < n) {
+                long long gi;
+                int si = e;
+                if (d.flags & kItemFull) gi = d.gbase + e; else item_pos(d, e, &gi, &si);
+                const float v = __fadd_rn(gs[u], rs[u]);
+                __stcs(resid + gi, v);
+                sv[si] = v;
+            }
+        }
+    }
+}
+
+// The (at most 3) elements of a contiguous vector-path item beyond its last full 128-bit word.
+template <typename G>
+__device__ __forceinline__ void k1_tail(const ItemDev &d, const G *__restrict__ grads, float *__restrict__ resid,
+                                        float *sv)
+{
+    if ((d.flags & (kItemVec | kItemFull)) == (kItemVec | kItemFull)) {
+        const int n = d.R * d.W;
+        const int e = (n & ~3) + threadIdx.x;
+        if (e < n) {
+            const float v = __fadd_rn(load_grad1(grads, d.gbase + e), resid[d.gbase + e]);
+            resid[d.gbase + e] = v;
+            sv[e] = v;
+        }
+    }
+}
+
 template <typename G>
 __global__ void __launch_bounds__(kThreads)
 k1_accumulate_nsi(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restrict__ keys,
-                  const LayerDev *__restrict__ layers, const Item *__restrict__ items,
+                  const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
                   const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
                   const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha,
                   unsigned int flags)
 {
-    __shared__ K1Shared sh;
+    extern __shared__ __align__(16) unsigned char k1_smem_raw[];
+    K1Shared &sh = *reinterpret_cast<K1Shared *>(k1_smem_raw);
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     if (begin >= end) return;
     const int tid = threadIdx.x;
     for (int b = tid; b < kL1Bins; b += kThreads) sh.hist[b] = 0;
     unsigned int nonfinite = 0;
-    int cur_layer = items[begin].layer;
-    __syncthreads();
+
+    K1Regs x;
+    ItemDev cur = load_item(items, begin);
+    k1_issue_loads(cur, grads, resid, x);
+    int buf = 0;
 
     for (int it = begin; it < end; ++it) {
-        const Item im = items[it];
-        if (im.layer != cur_layer) {
-            k1_flush_layer(sh, cur_layer, layers, hist, state, ratios, counts, flags);
-            cur_layer = im.layer;
-        }
-        const LayerDev L = layers[im.layer];
-        const int nh = L.nh, nw = L.nw;
-        const long long row0 = (long long)im.tr0 * nh;
-        const int R = (int)min((long long)im.ntr * nh, L.rows - row0);     // rows held
-        const long long col0 = (long long)im.tc0 * nw;
-        const int W = (int)min((long long)im.ntc * nw, L.cols - col0);     // cols held = smem pitch
-        const bool full = (W == L.cols);
-        const int nseg = full ? 1 : R;              // contiguous global runs
-        const int seglen = full ? R * W : W;
-        const long long gbase = L.elem_off + row0 * L.cols + col0;
+        const bool has_next = (it + 1 < end);
+        ItemDev nxt = cur;
+        if (has_next) nxt = load_item(items, it + 1);
 
-        // ---- v = g + r : global -> registers -> global (in place) and shared memory
-        const bool vec = ((gbase & 3) == 0) && (nseg == 1 || ((L.cols & 3) == 0 && (W & 3) == 0));
-        if (vec) {
-            const int wv = seglen >> 2;            // 128-bit vectors per run
-            const int nvec = wv * nseg;
-            for (int base = 0; base < nvec; base += kThreads * kVecPerThread) {
-                float4 g[kVecPerThread], r[kVecPerThread];
-                long long gi[kVecPerThread];
-                int si[kVecPerThread];
-#pragma unroll
-                for (int u = 0; u < kVecPerThread; ++u) {
-                    const int i = base + u * kThreads + tid;
-                    if (i < nvec) {
-                        const int seg = (nseg == 1) ? 0 : i / wv;
-                        const int j = i - seg * wv;
-                        gi[u] = ((gbase + (long long)seg * L.cols) >> 2) + j;
-                        si[u] = ((seg * W) >> 2) + j;
-                        g[u] = load_grad4(grads, gi[u]);
-                        r[u] = __ldcs(reinterpret_cast<const float4 *>(resid) + gi[u]);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < kVecPerThread; ++u) {
-                    const int i = base + u * kThreads + tid;
-                    if (i < nvec) {
-                        float4 v;
-                        v.x = __fadd_rn(g[u].x, r[u].x);
-                        v.y = __fadd_rn(g[u].y, r[u].y);
-                        v.z = __fadd_rn(g[u].z, r[u].z);
-                        v.w = __fadd_rn(g[u].w, r[u].w);
-                        reinterpret_cast<float4 *>(resid)[gi[u]] = v;
-                        reinterpret_cast<float4 *>(sh.v)[si[u]] = v;
-                    }
-                }
-            }
-            if (nseg == 1) {  // scalar tail of a run whose length is not a multiple of 4
-                const int i = (wv << 2) + tid;
-                if (i < seglen) {
-                    const float v = __fadd_rn(load_grad1(grads, gbase + i), resid[gbase + i]);
-                    resid[gbase + i] = v;
-                    sh.v[i] = v;
-                }
-            }
-        } else {
-            const int n = nseg * seglen;
-            for (int i = tid; i < n; i += kThreads) {
-                const int seg = (nseg == 1) ? 0 : i / seglen;
-                const int j = i - seg * seglen;
-                const long long gidx = gbase + (long long)seg * L.cols + j;
-                const float v = __fadd_rn(load_grad1(grads, gidx), resid[gidx]);
-                resid[gidx] = v;
-                sh.v[seg * W + j] = v;
-            }
-        }
+        // ---- v = g + r for the current item (its loads were issued one iteration ago)
+        float *sv = sh.v[buf];
+        k1_add_store(cur, resid, sv, x);
+        k1_tail(cur, grads, resid, sv);
+        // ---- next item's g and r start streaming in while this item's tiles are reduced
+        if (has_next) k1_issue_loads(nxt, grads, resid, x);
         __syncthreads();
 
         // ---- NSI of every tile of the item, one thread per tile
+        const int nh = cur.nh, nw = cur.nw, R = cur.R, W = cur.W;
         const int ntr = (R + nh - 1) / nh;
-        const int ntc = im.ntc;
+        const int ntc = cur.ntc;
         const int ntile = ntr * ntc;
-        uint32_t *kout = keys + L.tile_off + (long long)im.tr0 * L.TC + im.tc0;
+        uint32_t *kout = keys + cur.kbase;
         for (int t = tid; t < ntile; t += kThreads) {
             const int ti = (ntr == 1) ? 0 : t / ntc;
             const int tj = t - ti * ntc;
             const int hh = min(nh, R - ti * nh);
             const int ww = min(nw, W - tj * nw);
-            const float *p = sh.v + (ti * nh) * W + tj * nw;
+            const float *p = sv + (ti * nh) * W + tj * nw;
             float nsi;
             if (hh == 3 && ww == 3 && nh == 3 && nw == 3)
                 nsi = tile_nsi_fixed<3, 3>(p, W, alpha);
@@ -255,12 +335,14 @@ k1_accumulate_nsi(const G *__restrict__ grads, float *__restrict__ resid, uint32
                 key = 0x7F800000u;
                 ++nonfinite;
             }
-            kout[(long long)ti * L.TC + tj] = key;
+            kout[(long long)ti * cur.TC + tj] = key;
             atomicAdd(&sh.hist[key >> kL1Shift], 1u);
         }
-        __syncthreads();
+        if (!has_next || nxt.layer != cur.layer)
+            k1_flush_layer(sh, cur.layer, layers, hist, state, ratios, counts, flags);
+        cur = nxt;
+        buf ^= 1;
     }
-    k1_flush_layer(sh, cur_layer, layers, hist, state, ratios, counts, flags);
     if (nonfinite) {
         atomicAdd(&status->nonfinite, (unsigned long long)nonfinite);
         atomicOr(&status->flags, RSDGC_STATUS_NONFINITE);
@@ -270,6 +352,8 @@ k1_accumulate_nsi(const G *__restrict__ grads, float *__restrict__ resid, uint32
 // ------------------------------------------------------------------------------------------
 // K2 / K3: refinement passes over the keys (levels 2 and 3 of the radix selection)
 // ------------------------------------------------------------------------------------------
+
+constexpr int kKeyVecBatch = 8;  // 128-bit key loads in flight per thread in the key passes
 
 struct RefineShared {
     unsigned int hist[kL2Bins];
@@ -298,12 +382,20 @@ k_refine(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     if (prefix != kTakeNone) {
         const uint32_t *kp = keys + layers[c.layer].tile_off + c.start;
         const int nvec = c.n >> 2;
-        for (int i = tid; i < nvec; i += kThreads) {
-            const uint4 q = __ldg(reinterpret_cast<const uint4 *>(kp) + i);
-            if ((q.x >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q.x >> SHIFT_LO) & (kL2Bins - 1)], 1u);
-            if ((q.y >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q.y >> SHIFT_LO) & (kL2Bins - 1)], 1u);
-            if ((q.z >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q.z >> SHIFT_LO) & (kL2Bins - 1)], 1u);
-            if ((q.w >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q.w >> SHIFT_LO) & (kL2Bins - 1)], 1u);
+        for (int base = 0; base < nvec; base += kThreads * kKeyVecBatch) {
+            uint4 q[kKeyVecBatch];  // all loads of a batch are issued before any is consumed
+#pragma unroll
+            for (int u = 0; u < kKeyVecBatch; ++u) {
+                const int i = base + u * kThreads + tid;
+                q[u] = (i < nvec) ? __ldg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(~0u, ~0u, ~0u, ~0u);
+            }
+#pragma unroll
+            for (int u = 0; u < kKeyVecBatch; ++u) {  // the all-ones filler never matches a prefix
+                if ((q[u].x >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].x >> SHIFT_LO) & (kL2Bins - 1)], 1u);
+                if ((q[u].y >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].y >> SHIFT_LO) & (kL2Bins - 1)], 1u);
+                if ((q[u].z >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].z >> SHIFT_LO) & (kL2Bins - 1)], 1u);
+                if ((q[u].w >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].w >> SHIFT_LO) & (kL2Bins - 1)], 1u);
+            }
         }
         const int i = (nvec << 2) + tid;
         if (i < c.n) {
@@ -326,9 +418,15 @@ k_refine(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     __syncthreads();
     if (!sh.is_last) return;
     __threadfence();
-    for (int b = tid; b < kL2Bins; b += kThreads) {
-        sh.hist[b] = __ldcg(gh + b);
-        gh[b] = 0;
+    {
+        unsigned int h[kL2Bins / kThreads];
+#pragma unroll
+        for (int j = 0; j < kL2Bins / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + tid);
+#pragma unroll
+        for (int j = 0; j < kL2Bins / kThreads; ++j) {
+            sh.hist[j * kThreads + tid] = h[j];
+            gh[j * kThreads + tid] = 0;
+        }
     }
     __syncthreads();
     const int remaining = st.remaining;
@@ -379,10 +477,23 @@ k_count(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     {
         const uint32_t *kp = keys + L.tile_off + c.start;
         const int nvec = c.n >> 2;
-        for (int i = tid; i < nvec; i += kThreads) {
-            const uint4 q = __ldg(reinterpret_cast<const uint4 *>(kp) + i);
-            gt += (q.x > T) + (q.y > T) + (q.z > T) + (q.w > T);
-            eq += (q.x == T) + (q.y == T) + (q.z == T) + (q.w == T);
+        for (int base = 0; base < nvec; base += kThreads * kKeyVecBatch) {
+            uint4 q[kKeyVecBatch];
+#pragma unroll
+            for (int u = 0; u < kKeyVecBatch; ++u) {
+                const int i = base + u * kThreads + tid;
+                q[u] = (i < nvec) ? __ldg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
+            }
+            // the zero filler is neither above nor equal to T unless T == 0, in which case it
+            // would count as equal: mask it out explicitly
+#pragma unroll
+            for (int u = 0; u < kKeyVecBatch; ++u) {
+                const int i = base + u * kThreads + tid;
+                if (i < nvec) {
+                    gt += (q[u].x > T) + (q[u].y > T) + (q[u].z > T) + (q[u].w > T);
+                    eq += (q[u].x == T) + (q[u].y == T) + (q[u].z == T) + (q[u].w == T);
+                }
+            }
         }
         const int i = (nvec << 2) + tid;
         if (i < c.n) {
@@ -463,8 +574,12 @@ k_count(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
 // ------------------------------------------------------------------------------------------
 
 constexpr int kKeysPerThread = kChunkKeys / kThreads;  // 64 consecutive keys per thread
+constexpr int kChunkVecs = kChunkKeys / 4;             // 128-bit words of keys per chunk
+constexpr int kCopyBatch = 8;                          // gathered loads in flight per thread
 
 struct PackShared {
+    // one byte per 128-bit word of keys: bit c = key c above T, bit 4 + c = key c equal to T
+    __align__(16) unsigned char code[kChunkVecs];
     unsigned short pos[kChunkKeys];  // position in the chunk of the r-th kept tile
     unsigned long long scan_tmp[kThreads / 32];
 };
@@ -486,36 +601,66 @@ k_pack(const uint32_t *__restrict__ keys, float *__restrict__ resid, const Layer
     // equal keys of this chunk that are still taken: those with layer-wide equal-rank < e
     const long long eq_room = max(0ll, (long long)st.e - (long long)base.y);
 
+    // ---- phase 1: coalesced read of the chunk's keys, 2 bits per key into shared memory
     const uint32_t *kp = keys + L.tile_off + c.start;
-    const int p0 = tid * kKeysPerThread;
-    const int p1 = min(c.n, p0 + kKeysPerThread);
-    unsigned int gt = 0, eq = 0;
-    for (int p = p0; p < p1; p += 4) {  // chunk starts and p0 are multiples of 4
-        if (p + 4 <= c.n) {
-            const uint4 q = __ldg(reinterpret_cast<const uint4 *>(kp + p));
-            gt += (q.x > T) + (q.y > T) + (q.z > T) + (q.w > T);
-            eq += (q.x == T) + (q.y == T) + (q.z == T) + (q.w == T);
-        } else {
-            for (int j = p; j < c.n; ++j) {
-                const uint32_t q = kp[j];
-                gt += (q > T);
-                eq += (q == T);
-            }
+    const int nvec = c.n >> 2;
+    for (int b0 = 0; b0 < kChunkVecs; b0 += kThreads * kKeyVecBatch) {
+        uint4 q[kKeyVecBatch];
+#pragma unroll
+        for (int u = 0; u < kKeyVecBatch; ++u) {
+            const int i = b0 + u * kThreads + tid;
+            q[u] = (i < nvec) ? __ldg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
         }
+#pragma unroll
+        for (int u = 0; u < kKeyVecBatch; ++u) {
+            const int i = b0 + u * kThreads + tid;
+            unsigned int code = 0;
+            if (i < nvec) {
+                code = (q[u].x > T) | ((q[u].y > T) << 1) | ((q[u].z > T) << 2) | ((q[u].w > T) << 3) |
+                       ((q[u].x == T) << 4) | ((q[u].y == T) << 5) | ((q[u].z == T) << 6) | ((q[u].w == T) << 7);
+            } else if (i == nvec) {  // the last, partial word of the chunk
+                for (int j = 0; j < (c.n & 3); ++j) {
+                    const uint32_t k1 = kp[(nvec << 2) + j];
+                    code |= ((k1 > T) << j) | ((k1 == T) << (4 + j));
+                }
+            }
+            sh.code[i] = (unsigned char)code;
+        }
+    }
+    __syncthreads();
+
+    // ---- phase 2: ranks.  Thread t owns keys [64 t, 64 t + 64) = 16 code bytes.
+    const uint4 cw = reinterpret_cast<const uint4 *>(sh.code)[tid];
+    const unsigned int w[4] = {cw.x, cw.y, cw.z, cw.w};
+    unsigned int gt = 0, eq = 0;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        gt += __popc(w[j] & 0x0F0F0F0Fu);
+        eq += __popc(w[j] & 0xF0F0F0F0u);
     }
     unsigned long long total;
     const unsigned long long ex =
         block_exclusive_scan<unsigned long long>(((unsigned long long)eq << 32) | gt, sh.scan_tmp, &total);
     unsigned int gt_before = (unsigned int)(ex & 0xFFFFFFFFull), eq_before = (unsigned int)(ex >> 32);
-    for (int p = p0; p < p1; ++p) {
-        const uint32_t q = __ldg(kp + p);
-        if (q > T) {
-            sh.pos[gt_before + (unsigned int)min((long long)eq_before, eq_room)] = (unsigned short)p;
-            ++gt_before;
-        } else if (q == T) {
-            if ((long long)eq_before < eq_room)
-                sh.pos[gt_before + eq_before] = (unsigned short)p;
-            ++eq_before;
+    if (gt | eq) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+#pragma unroll
+            for (int b = 0; b < 4; ++b) {
+                const unsigned int byte = (w[j] >> (8 * b)) & 0xFFu;
+                if (byte == 0) continue;
+                const int p0 = tid * kKeysPerThread + (j * 4 + b) * 4;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    if (byte & (1u << k)) {
+                        sh.pos[gt_before + (unsigned int)min((long long)eq_before, eq_room)] = (unsigned short)(p0 + k);
+                        ++gt_before;
+                    } else if (byte & (16u << k)) {
+                        if ((long long)eq_before < eq_room) sh.pos[gt_before + eq_before] = (unsigned short)(p0 + k);
+                        ++eq_before;
+                    }
+                }
+            }
         }
     }
     __syncthreads();
@@ -524,51 +669,108 @@ k_pack(const uint32_t *__restrict__ keys, float *__restrict__ resid, const Layer
     // rank in the layer of this chunk's first kept tile
     const long long rank0 = (long long)base.x + min((long long)base.y, (long long)st.e);
 
+    // ---- phase 3: gather the kept tiles out of the residual, zero them there, write the payload
     const int slot = L.slot;
-    const long long n_copy = (long long)n_kept * slot;
-    for (long long j = tid; j < n_copy; j += kThreads) {
-        const int r = (int)(j / slot);
-        const int el = (int)(j - (long long)r * slot);
-        const int tile = c.start + sh.pos[r];
-        const long long s = st.idx_off + rank0 + r;           // payload slot (tiles)
-        const long long vbase = st.val_off + (rank0 + r) * slot;
-        if (s >= idx_cap || vbase + slot > val_cap) continue;  // does not fit: not sent
-        const int tr = tile / L.TC, tc = tile - tr * L.TC;
-        const int a = el / L.nw, b = el - a * L.nw;
-        const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
-        float x = 0.0f;
-        if (i < L.rows && jj < L.cols) {
-            const long long g = L.elem_off + i * L.cols + jj;
-            x = resid[g];
-            resid[g] = 0.0f;
+    const int n_copy = n_kept * slot;  // at most 16384 * 4096
+    for (int j0 = 0; j0 < n_copy; j0 += kThreads * kCopyBatch) {
+        long long ga[kCopyBatch], vo[kCopyBatch];
+        float xv[kCopyBatch];
+#pragma unroll
+        for (int u = 0; u < kCopyBatch; ++u) {
+            const int j = j0 + u * kThreads + tid;
+            ga[u] = -1;
+            vo[u] = -1;
+            if (j < n_copy) {
+                const int r = j / slot, el = j - r * slot;
+                const int tile = c.start + sh.pos[r];
+                const long long s = st.idx_off + rank0 + r;              // payload slot (tiles)
+                const long long vbase = st.val_off + (rank0 + r) * slot;
+                if (s < idx_cap && vbase + slot <= val_cap) {            // else: does not fit, not sent
+                    const int tr = tile / L.TC, tc = tile - tr * L.TC;
+                    const int a = el / L.nw, b = el - a * L.nw;
+                    const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
+                    if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+                    vo[u] = vbase + el;
+                    if (el == 0) idx[s] = tile;
+                }
+            }
         }
-        val[vbase + el] = x;
-        if (el == 0) idx[s] = tile;
+#pragma unroll
+        for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? __ldcs(resid + ga[u]) : 0.0f;
+#pragma unroll
+        for (int u = 0; u < kCopyBatch; ++u) {
+            if (ga[u] >= 0) resid[ga[u]] = 0.0f;
+            if (vo[u] >= 0) val[vo[u]] = xv[u];
+        }
     }
 }
 
 // ------------------------------------------------------------------------------------------
+
+// Resident CTAs per SM of the accumulate+NSI kernel on the current device.
+int k1_ctas_per_sm(int dtype)
+{
+    int n = 0;
+    const size_t smem = sizeof(K1Shared);
+    cudaError_t e = cudaFuncSetAttribute(k1_accumulate_nsi<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(k1_accumulate_nsi<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e == cudaSuccess)
+        e = (dtype == RSDGC_BF16)
+                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_accumulate_nsi<__nv_bfloat16>, kThreads, smem)
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_accumulate_nsi<float>, kThreads, smem);
+    if (e != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        n = 2;
+    }
+    return n;
+}
+
+// Next event of the plan's pool (created on demand), recorded on the stream.
+static cudaError_t record_event(rsdgc_plan *p, cudaStream_t s)
+{
+    if (p->events_used == p->events.size()) {
+        cudaEvent_t ev;
+        cudaError_t e = cudaEventCreate(&ev);
+        if (e != cudaSuccess) return e;
+        p->events.push_back(ev);
+    }
+    return cudaEventRecord(p->events[p->events_used++], s);
+}
 
 cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, const float *ratios, int32_t *idx,
                             int64_t idx_cap, float *val, int64_t val_cap, int32_t *counts, uint32_t *keys,
                             cudaStream_t s)
 {
     const int n_chunks = (int)p->chunks.size();
+    const bool prof = p->profile;
+    cudaError_t e = cudaSuccess;
+#define RSDGC_MARK()                                   \
+    if (prof && e == cudaSuccess) e = record_event(p, s)
+    RSDGC_MARK();
     if (p->dtype == RSDGC_BF16)
-        k1_accumulate_nsi<__nv_bfloat16><<<p->grid1, kThreads, 0, s>>>(
+        k1_accumulate_nsi<__nv_bfloat16><<<p->grid1, kThreads, sizeof(K1Shared), s>>>(
             reinterpret_cast<const __nv_bfloat16 *>(grads), resid, keys, p->d_layers, p->d_items, p->d_cta_begin,
             p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
     else
-        k1_accumulate_nsi<float><<<p->grid1, kThreads, 0, s>>>(
+        k1_accumulate_nsi<float><<<p->grid1, kThreads, sizeof(K1Shared), s>>>(
             reinterpret_cast<const float *>(grads), resid, keys, p->d_layers, p->d_items, p->d_cta_begin,
             p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
+    RSDGC_MARK();
     k_refine<2><<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
+    RSDGC_MARK();
     k_refine<3><<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
+    RSDGC_MARK();
     k_count<<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt,
                                           p->n_layers, idx_cap, val_cap, p->d_status);
+    RSDGC_MARK();
     k_pack<<<n_chunks, kThreads, 0, s>>>(keys, resid, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, idx,
                                          idx_cap, val, val_cap);
+    RSDGC_MARK();
+#undef RSDGC_MARK
     count_launch(5);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 

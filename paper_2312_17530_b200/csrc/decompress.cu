@@ -42,32 +42,56 @@ k_decompress(const int32_t *__restrict__ idx, const float *__restrict__ val,
     __syncthreads();
     const long long total = val_off[n_layers];
 
-    for (long long j = (long long)blockIdx.x * kThreads + tid; j < total; j += (long long)gridDim.x * kThreads) {
-        int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (val_off[mid] <= j) lo = mid; else hi = mid;
+    constexpr int B = 4;  // independent entries per thread: index loads, then dense loads, then stores
+    const long long stride = (long long)gridDim.x * kThreads;
+    for (long long j0 = (long long)blockIdx.x * kThreads + tid; j0 < total; j0 += stride * B) {
+        long long ga[B];
+        float pv[B], dv[B];
+        int tile[B], lay[B], el[B];
+#pragma unroll
+        for (int u = 0; u < B; ++u) {
+            const long long j = j0 + u * stride;
+            ga[u] = -1;
+            tile[u] = -1;
+            if (j < total) {
+                int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (val_off[mid] <= j) lo = mid; else hi = mid;
+                }
+                const int slot = layers[lo].slot;
+                const long long jl = j - val_off[lo];
+                const long long s = jl / slot;
+                lay[u] = lo;
+                el[u] = (int)(jl - s * slot);
+                tile[u] = __ldg(idx + idx_off[lo] + s);
+                pv[u] = __ldg(val + j);
+            }
         }
-        const LayerDev &L = layers[lo];
-        const long long jl = j - val_off[lo];
-        const long long s = jl / L.slot;
-        const int el = (int)(jl - s * L.slot);
-        const int tile = idx[idx_off[lo] + s];
-        if (tile < 0 || tile >= L.K) continue;
-        const int tr = tile / L.TC, tc = tile - tr * L.TC;
-        const int a = el / L.nw, b = el - a * L.nw;
-        const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
-        if (i < L.rows && jj < L.cols) {
-            const long long g = L.elem_off + i * L.cols + jj;
-            dense[g] = __fadd_rn(dense[g], __fmul_rn(scale, val[j]));
+#pragma unroll
+        for (int u = 0; u < B; ++u) {
+            if (tile[u] >= 0) {
+                const LayerDev &L = layers[lay[u]];
+                if (tile[u] < L.K) {
+                    const int tr = tile[u] / L.TC, tc = tile[u] - tr * L.TC;
+                    const int a = el[u] / L.nw, b = el[u] - a * L.nw;
+                    const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
+                    if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+                }
+            }
         }
+#pragma unroll
+        for (int u = 0; u < B; ++u) dv[u] = (ga[u] >= 0) ? dense[ga[u]] : 0.0f;
+#pragma unroll
+        for (int u = 0; u < B; ++u)
+            if (ga[u] >= 0) dense[ga[u]] = __fadd_rn(dv[u], __fmul_rn(scale, pv[u]));
     }
 }
 
 cudaError_t launch_decompress(rsdgc_plan *p, const int32_t *idx, const float *val, const int32_t *counts,
                               float scale, float *dense, cudaStream_t s)
 {
-    k_decompress<<<p->n_sm * 4, kThreads, 0, s>>>(idx, val, counts, p->d_layers, p->n_layers, scale, dense);
+    k_decompress<<<p->n_sm * 8, kThreads, 0, s>>>(idx, val, counts, p->d_layers, p->n_layers, scale, dense);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -74,6 +74,8 @@ void free_device_tables(rsdgc_plan *p)
     cudaFree(p->d_survivors);
     cudaFree(p->d_rstate);
     cudaFree(p->d_status);
+    for (cudaEvent_t ev : p->events) cudaEventDestroy(ev);
+    p->events.clear();
 }
 
 }  // namespace
@@ -96,7 +98,7 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
     for (int l = 0; l < n_layers; ++l) {
         const rsdgc_layer_desc &d = descs[l];
         if (d.rows < 1 || d.cols < 1 || d.nh < 1 || d.nw < 1) return RSDGC_ERR_INVALID;
-        if ((int64_t)d.nh * d.nw > kMaxSlot) return RSDGC_ERR_CAPACITY;
+        if ((int64_t)d.nh * d.nw > kMaxSlot || d.nh > INT16_MAX || d.nw > INT16_MAX) return RSDGC_ERR_CAPACITY;
         if (d.rows > INT32_MAX || d.cols > INT32_MAX) return RSDGC_ERR_CAPACITY;
         if (d.rows * d.cols > (int64_t)INT32_MAX) return RSDGC_ERR_CAPACITY;
         LayerDev L{};
@@ -120,6 +122,7 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
             int64_t ntr = ceil_div64(L.TR, n_items);
             // multiples of 4 tile rows keep every item start 4-element aligned (128-bit loads)
             if (round_up64(ntr, 4) <= ntr_max) ntr = round_up64(ntr, 4);
+            else if (ntr_max >= 4) ntr = ntr_max & ~(int64_t)3;
             for (int64_t tr0 = 0; tr0 < L.TR; tr0 += ntr) {
                 Item it{l, (int32_t)tr0, (int32_t)std::min<int64_t>(ntr, L.TR - tr0), 0, L.TC};
                 p->items.push_back(it);
@@ -129,6 +132,7 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
             int64_t n_items = ceil_div64(L.TC, ntc_max);
             int64_t ntc = ceil_div64(L.TC, n_items);
             if (round_up64(ntc, 4) <= ntc_max) ntc = round_up64(ntc, 4);
+            else if (ntc_max >= 4) ntc = ntc_max & ~(int64_t)3;
             for (int64_t tr = 0; tr < L.TR; ++tr)
                 for (int64_t tc0 = 0; tc0 < L.TC; tc0 += ntc) {
                     Item it{l, (int32_t)tr, 1, (int32_t)tc0, (int32_t)std::min<int64_t>(ntc, L.TC - tc0)};
@@ -187,6 +191,29 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
         if (first) p->layers[p->items[i].layer].n_flush1 += 1;
     }
 
+    // --- device form of the items
+    p->items_dev.resize(n_items);
+    for (size_t i = 0; i < n_items; ++i) {
+        const Item &it = p->items[i];
+        const LayerDev &L = p->layers[it.layer];
+        ItemDev d{};
+        const int64_t row0 = (int64_t)it.tr0 * L.nh, col0 = (int64_t)it.tc0 * L.nw;
+        d.R = (int32_t)std::min<int64_t>((int64_t)it.ntr * L.nh, L.rows - row0);
+        d.W = (int32_t)std::min<int64_t>((int64_t)it.ntc * L.nw, L.cols - col0);
+        d.gbase = L.elem_off + row0 * L.cols + col0;
+        d.kbase = L.tile_off + (int64_t)it.tr0 * L.TC + it.tc0;
+        d.cols = (int32_t)L.cols;
+        d.ntc = it.ntc;
+        d.TC = L.TC;
+        d.nh = (int16_t)L.nh;
+        d.nw = (int16_t)L.nw;
+        d.layer = it.layer;
+        const bool full = (d.W == L.cols) || d.R == 1;  // one contiguous run
+        const bool vec = (d.gbase % 4 == 0) && (full || (L.cols % 4 == 0 && d.W % 4 == 0));
+        d.flags = (full ? kItemFull : 0) | (vec ? kItemVec : 0);
+        p->items_dev[i] = d;
+    }
+
     rsdgc_info &I = p->info;
     I.n_layers = n_layers;
     I.grad_dtype = p->dtype;
@@ -232,8 +259,12 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
             return cuda_fail(e);
         }
         p->n_sm = n_sm;
+        DeviceGuard guard(device);
+        // one CTA per resident slot: the static partition assumes all CTAs run concurrently
+        p->grid1 = n_sm * k1_ctas_per_sm(grad_dtype);
+    } else {
+        p->grid1 = p->n_sm * 2;
     }
-    p->grid1 = p->n_sm * 4;
 
     int rc;
     try {
@@ -250,7 +281,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         DeviceGuard guard(device);
         cudaError_t e = guard.err;
         if (e == cudaSuccess) e = upload(&p->d_layers, p->layers);
-        if (e == cudaSuccess) e = upload(&p->d_items, p->items);
+        if (e == cudaSuccess) e = upload(&p->d_items, p->items_dev);
         if (e == cudaSuccess) e = upload(&p->d_cta_begin, p->cta_begin);
         if (e == cudaSuccess) e = upload(&p->d_chunks, p->chunks);
         if (e == cudaSuccess) e = upload(&p->d_echunks, p->echunks);
@@ -474,6 +505,39 @@ extern "C" int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *ou
     out_host->nonfinite = (int64_t)h.nonfinite;
     out_host->idx_needed = h.idx_needed;
     out_host->val_needed = h.val_needed;
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_profile_enable(rsdgc_plan *plan, int32_t enable)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    plan->profile = enable != 0;
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_profile_read(rsdgc_plan *plan, double *ms_per_kernel_host, int64_t *n_calls_host)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (!ms_per_kernel_host || !n_calls_host) return RSDGC_ERR_INVALID;
+    constexpr size_t per_call = RSDGC_N_COMPRESS_KERNELS + 1;
+    const size_t n_calls = plan->events_used / per_call;
+    for (int k = 0; k < RSDGC_N_COMPRESS_KERNELS; ++k) ms_per_kernel_host[k] = 0.0;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    for (size_t c = 0; c < n_calls; ++c) {
+        const cudaEvent_t *ev = plan->events.data() + c * per_call;
+        cudaError_t e = cudaEventSynchronize(ev[per_call - 1]);
+        for (int k = 0; k < RSDGC_N_COMPRESS_KERNELS && e == cudaSuccess; ++k) {
+            float ms = 0.0f;
+            e = cudaEventElapsedTime(&ms, ev[k], ev[k + 1]);
+            ms_per_kernel_host[k] += ms;
+        }
+        if (e != cudaSuccess) return cuda_fail(e);
+    }
+    *n_calls_host = (int64_t)n_calls;
+    plan->events_used = 0;
     return RSDGC_OK;
 }
 

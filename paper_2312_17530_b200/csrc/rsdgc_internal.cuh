@@ -44,6 +44,22 @@ struct Item {
     int32_t layer, tr0, ntr, tc0, ntc;
 };
 
+// The same item resolved for the device: everything the accumulate+NSI kernel needs, so that
+// one 48-byte load per item replaces the chain item -> layer table -> data.
+struct __align__(16) ItemDev {
+    long long gbase;  // arena index of the first element held
+    long long kbase;  // key-array index of the first tile
+    int32_t R, W;     // rows and columns held; W is the row pitch in shared memory
+    int32_t cols;     // row stride in global memory
+    int32_t ntc;      // tile columns in the item
+    int32_t TC;       // tile columns of the layer = key stride between tile rows
+    int16_t nh, nw;
+    int32_t layer;
+    int32_t flags;    // kItemFull: rows are contiguous in memory; kItemVec: 128-bit path usable
+};
+static_assert(sizeof(ItemDev) == 48, "ItemDev is loaded as three 16-byte words");
+constexpr int kItemFull = 1, kItemVec = 2;
+
 // Key chunk: keys [start, start + n) of a layer (layer-local tile indices).
 struct Chunk {
     int32_t layer, start, n;
@@ -93,6 +109,7 @@ struct rsdgc_plan {
 
     std::vector<rsdgc::LayerDev> layers;
     std::vector<rsdgc::Item> items;
+    std::vector<rsdgc::ItemDev> items_dev;
     std::vector<int32_t> cta_begin;  // grid1 + 1 item indices
     std::vector<rsdgc::Chunk> chunks;
     std::vector<rsdgc::EChunk> echunks;
@@ -101,7 +118,7 @@ struct rsdgc_plan {
 
     // device tables
     rsdgc::LayerDev *d_layers = nullptr;
-    rsdgc::Item *d_items = nullptr;
+    rsdgc::ItemDev *d_items = nullptr;
     int32_t *d_cta_begin = nullptr;
     rsdgc::Chunk *d_chunks = nullptr;
     rsdgc::EChunk *d_echunks = nullptr;
@@ -111,6 +128,11 @@ struct rsdgc_plan {
     long long *d_survivors = nullptr;  // ratio rule: per-layer survivor counts
     rsdgc::RatioState *d_rstate = nullptr;
     rsdgc::StatusDev *d_status = nullptr;
+
+    // optional per-kernel timing of compress calls
+    bool profile = false;
+    std::vector<cudaEvent_t> events;  // pool; (RSDGC_N_COMPRESS_KERNELS + 1) per recorded call
+    size_t events_used = 0;
 };
 
 namespace rsdgc {
@@ -127,5 +149,6 @@ cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long 
 cudaError_t launch_decompress(rsdgc_plan *p, const int32_t *idx, const float *val,
                               const int32_t *counts, float scale, float *dense, cudaStream_t s);
 void count_launch(int n);
+int k1_ctas_per_sm(int dtype);
 
 }  // namespace rsdgc

@@ -68,7 +68,7 @@ def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net):
     assert p.info.workspace_bytes == 4 * to
 
     items, cta, nflush = p.worklist()
-    assert cta[0] == 0 and cta[-1] == len(items) and (np.diff(cta) >= 0).all() and len(cta) == 148 * 4 + 1
+    assert cta[0] == 0 and cta[-1] == len(items) and (np.diff(cta) >= 0).all() and len(cta) == 148 * 2 + 1
     assert (np.diff(items[:, 0]) >= 0).all()          # layers in order
     owner = np.searchsorted(cta, np.arange(len(items)), side="right") - 1
     for l, (r, c, nh, nw) in enumerate(shapes):
