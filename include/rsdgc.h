@@ -59,10 +59,12 @@ typedef enum {
 
 /* plan flags */
 #define RSDGC_KEEP_AT_LEAST_ONE 1u /* k_l = max(1, ceil(K_l * ratio_l)): every layer sends >= 1 tile */
+#define RSDGC_NO_BULK_COPY 2u      /* first pass: register-staged kernel for every item           */
 
 /* bits of rsdgc_status.flags */
 #define RSDGC_STATUS_NONFINITE 1u         /* some indicator was NaN/Inf (ranked first as +Inf)  */
 #define RSDGC_STATUS_PAYLOAD_OVERFLOW 2u  /* idx/val capacity too small; excess tiles not sent   */
+#define RSDGC_STATUS_TIMEOUT 4u           /* a bounded on-chip wait gave up; results are invalid  */
 
 typedef struct {
     int64_t rows, cols; /* row-major 2-D view of the layer (Sec. III-C)            */
@@ -101,7 +103,7 @@ typedef struct {
  * Builds the plan for a set of layers (Algorithm 1's loop over l = 1..L with the
  * neighborhoods of Eq. 7): arena offsets, tile counts, the work lists the kernels walk and
  * the per-layer device tables.  `alpha` is the hyper-parameter of Eq. 8 (0 <= alpha <= 1).
- * `flags`: RSDGC_KEEP_AT_LEAST_ONE or 0.  `device` is the CUDA device ordinal.  On success
+ * `flags`: an OR of RSDGC_KEEP_AT_LEAST_ONE and RSDGC_NO_BULK_COPY, or 0.  `device` is the CUDA device ordinal.  On success
  * *out owns host memory and a few MB of device memory until rsdgc_plan_destroy().
  * Errors: INVALID (null, n_layers < 1, rows/cols/nh/nw < 1, alpha outside [0,1] or NaN,
  * unknown dtype), CAPACITY (a layer with more than 2^31-1 tiles or nh*nw > 4096),
@@ -122,13 +124,14 @@ int rsdgc_plan_layer_info(const rsdgc_plan *plan, int32_t layer, rsdgc_layer_inf
 int rsdgc_plan_payload_bound(const rsdgc_plan *plan, float max_ratio, int64_t *idx_capacity_host,
                              int64_t *val_capacity_host);
 
-/* Diagnostic: copies the work list of the accumulate+NSI kernel (5 int32 per item: layer,
- * first tile row, tile rows, first tile col, tile cols; the items of a layer partition its
- * tile grid), the first item of every CTA of that kernel (cta_capacity entries at most,
- * the last entry is the item count) and, per layer, how many CTAs touch it.  Any pointer
+/* Diagnostic: copies the work list of the accumulate+NSI pass, 7 int32 per item: layer,
+ * first tile row, tile rows, first tile col, tile cols (the items of a layer partition its
+ * tile grid), the kernel that takes the item (0 = bulk-copy kernel, 1 = register-staged
+ * kernel) and the CTA of that kernel that owns it; grids_host[0..1] receive the two kernels'
+ * grid sizes and n_flush_host[l] how many (kernel, CTA) pairs touch layer l.  Any pointer
  * may be NULL.  Returns the number of items (or a negative rsdgc_error).  Host only. */
 int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,
-                            int32_t *cta_begin_host, int64_t cta_capacity, int32_t *n_flush_host);
+                            int32_t *grids_host, int32_t *n_flush_host);
 
 /*
  * Layer-wise dynamic compression ratio (Eq. 3-5; Algorithm 1, per-epoch part): importance

@@ -68,7 +68,9 @@ void rsdgc_oracle_accumulate_bf16(const uint16_t *g, const float *r, float *v, i
  *   NSI    = alpha * mean_p + (1 - alpha) * std_p      (Eq. 8)
  * nsi_ref: binary64 from the binary32 inputs.
  * nsi_f32: binary32, elements visited row-major inside the tile, plain running
- *          sums, mean first and squared deviations in a second sweep.
+ *          sums, mean first and squared deviations in a second sweep; the factor
+ *          1/p^2 of Eq. 9-10 is formed once (1/n rounded to binary32) and each of
+ *          the three sums is multiplied by it, as the equations are written.
  * A non-finite nsi_f32 is replaced by +infinity (so it ranks first, deterministically)
  * and counted in the return value.
  */
@@ -111,9 +113,9 @@ int64_t rsdgc_oracle_nsi(const float *v, int64_t rows, int64_t cols, int32_t nh,
                     sa = sa + fabsf(x);
                     sv = sv + x;
                 }
-            const float fn = (float)cnt;
-            const float a = sa / fn;
-            const float m = sv / fn;
+            const float inv_n = 1.0f / (float)cnt;
+            const float a = sa * inv_n;
+            const float m = sv * inv_n;
             float sq = 0.0f;
             for (int64_t i = i0; i < i1; ++i)
                 for (int64_t j = j0; j < j1; ++j) {
@@ -121,7 +123,7 @@ int64_t rsdgc_oracle_nsi(const float *v, int64_t rows, int64_t cols, int32_t nh,
                     float dd = d * d;
                     sq = sq + dd;
                 }
-            const float s = sqrtf(sq / fn);
+            const float s = sqrtf(sq * inv_n);
             const float t1 = alpha * a;
             const float t2 = (1.0f - alpha) * s;
             float nsi = t1 + t2;

@@ -15,7 +15,8 @@ LIB_PATH = os.path.join(_HERE, "librsdgc_b200.so")
 
 RSDGC_F32, RSDGC_BF16 = 0, 1
 KEEP_AT_LEAST_ONE = 1
-STATUS_NONFINITE, STATUS_PAYLOAD_OVERFLOW = 1, 2
+NO_BULK_COPY = 2
+STATUS_NONFINITE, STATUS_PAYLOAD_OVERFLOW, STATUS_TIMEOUT = 1, 2, 4
 OK, ERR_INVALID, ERR_ALIGNMENT, ERR_CAPACITY, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
 
 EXPORTS = [
@@ -74,7 +75,7 @@ def lib():
         L.rsdgc_plan_info.argtypes = [vp, C.POINTER(Info)]
         L.rsdgc_plan_layer_info.argtypes = [vp, i32, C.POINTER(LayerInfo)]
         L.rsdgc_plan_payload_bound.argtypes = [vp, f32, C.POINTER(i64), C.POINTER(i64)]
-        L.rsdgc_plan_worklist.argtypes = [vp, vp, i64, vp, i64, vp]
+        L.rsdgc_plan_worklist.argtypes = [vp, vp, i64, vp, vp]
         L.rsdgc_plan_worklist.restype = i64
         L.rsdgc_update_ratios.argtypes = [vp, vp, f32, vp, vp]
         L.rsdgc_compress.argtypes = [vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
@@ -157,15 +158,15 @@ class Plan:
         return a.value, b.value
 
     def worklist(self):
-        """(items [n,5] int32, cta_begin int32, n_flush int32) of the accumulate+NSI kernel."""
+        """(items [n,7] int32: layer, tr0, ntr, tc0, ntc, kernel, cta; grids [2]; n_flush [L])."""
         import numpy as np
 
-        n = lib().rsdgc_plan_worklist(self._h, None, 0, None, 0, None)
-        items = np.zeros((n, 5), dtype=np.int32)
-        cta = np.zeros(4096, dtype=np.int32) - 1
+        n = lib().rsdgc_plan_worklist(self._h, None, 0, None, None)
+        items = np.zeros((n, 7), dtype=np.int32)
+        grids = np.zeros(2, dtype=np.int32)
         nf = np.zeros(self.n_layers, dtype=np.int32)
-        lib().rsdgc_plan_worklist(self._h, items.ctypes.data, n, cta.ctypes.data, cta.size, nf.ctypes.data)
-        return items, cta[cta >= 0], nf
+        lib().rsdgc_plan_worklist(self._h, items.ctypes.data, n, grids.ctypes.data, nf.ctypes.data)
+        return items, grids, nf
 
     # ---- device calls (torch tensors on the plan's device) -------------------------------
     def update_ratios(self, weights, global_keep: float, ratios) -> None:

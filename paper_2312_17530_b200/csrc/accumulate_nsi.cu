@@ -1,0 +1,805 @@
+// First pass of rsdgc_compress(): v = g + r in place (Eq. 12), the NSI key of every tile
+// (Eq. 8-10), and the level-1 histogram of the keys per layer.
+//
+// Two kernels share the work list:
+//  * k1_bulk: one persistent 512-thread CTA per SM.  The g and r blocks of an item are brought
+//    into shared memory by the bulk-copy engine (cp.async.bulk + mbarrier) two items ahead
+//    of their use, v is formed in shared memory and written back with a bulk store, and the
+//    tiles are reduced from shared memory.  Bytes in flight do not occupy registers.
+//    It takes every item whose rows are 16-byte aligned in memory (all the usual shapes).
+//  * k1_reg: 256-thread CTAs that stage an item in registers (128-bit loads where possible,
+//    scalar otherwise).  It takes the remaining items (odd pitches, unaligned starts).
+//
+// Ordering between CTAs comes only from kernel boundaries and from "last arriver finishes the
+// job" tickets; the only waits are on a CTA's own mbarriers and every such wait is bounded.
+#include <cfloat>
+#include <cuda_bf16.h>
+
+#include "device_utils.cuh"
+
+namespace rsdgc {
+
+// ------------------------------------------------------------------------------------------
+// NSI of one tile
+// ------------------------------------------------------------------------------------------
+
+// NSI of one tile held in shared memory (Eq. 8-10) in binary32: elements visited row-major,
+// plain running sums, mean first and squared deviations in a second sweep; the three
+// "(1/n) sum" of Eq. 9-10 multiply the sum by inv_n = 1/n (rounded once).  Every operation is
+// an explicitly rounded single operation (no fused multiply-add).
+__device__ float tile_nsi_generic(const float *p, int pitch, int hh, int ww, float alpha)
+{
+    float sa = 0.0f, sv = 0.0f;
+    for (int a = 0; a < hh; ++a)
+        for (int b = 0; b < ww; ++b) {
+            const float x = p[a * pitch + b];
+            sa = __fadd_rn(sa, fabsf(x));
+            sv = __fadd_rn(sv, x);
+        }
+    const float inv_n = __fdiv_rn(1.0f, (float)(hh * ww));
+    const float mean_abs = __fmul_rn(sa, inv_n);
+    const float m = __fmul_rn(sv, inv_n);
+    float sq = 0.0f;
+    for (int a = 0; a < hh; ++a)
+        for (int b = 0; b < ww; ++b) {
+            const float d = __fsub_rn(p[a * pitch + b], m);
+            sq = __fadd_rn(sq, __fmul_rn(d, d));
+        }
+    const float s = __fsqrt_rn(__fmul_rn(sq, inv_n));
+    return __fadd_rn(__fmul_rn(alpha, mean_abs), __fmul_rn(__fsub_rn(1.0f, alpha), s));
+}
+
+template <int HH, int WW>
+__device__ __forceinline__ float tile_nsi_fixed(const float *p, int pitch, float alpha)
+{
+    float x[HH * WW];
+#pragma unroll
+    for (int a = 0; a < HH; ++a)
+#pragma unroll
+        for (int b = 0; b < WW; ++b) x[a * WW + b] = p[a * pitch + b];
+    float sa = 0.0f, sv = 0.0f;
+#pragma unroll
+    for (int i = 0; i < HH * WW; ++i) {
+        sa = __fadd_rn(sa, fabsf(x[i]));
+        sv = __fadd_rn(sv, x[i]);
+    }
+    const float inv_n = __fdiv_rn(1.0f, (float)(HH * WW));  // folded at compile time
+    const float mean_abs = __fmul_rn(sa, inv_n);
+    const float m = __fmul_rn(sv, inv_n);
+    float sq = 0.0f;
+#pragma unroll
+    for (int i = 0; i < HH * WW; ++i) {
+        const float d = __fsub_rn(x[i], m);
+        sq = __fadd_rn(sq, __fmul_rn(d, d));
+    }
+    const float s = __fsqrt_rn(__fmul_rn(sq, inv_n));
+    return __fadd_rn(__fmul_rn(alpha, mean_abs), __fmul_rn(__fsub_rn(1.0f, alpha), s));
+}
+
+#ifndef RSDGC_PAIR_MODE
+#define RSDGC_PAIR_MODE 0
+#endif
+
+// Packed binary32x2 arithmetic of sm_100 with explicit round-to-nearest (never fused).
+__device__ __forceinline__ float2 add2_rn(float2 a, float2 b)
+{
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+__device__ __forceinline__ float2 mul2_rn(float2 a, float2 b)
+{
+    unsigned long long ra, rb, rd;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
+    float2 d;
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
+    return d;
+}
+
+// Two full HH x WW tiles at once (component x = tile A, y = tile B): each component goes
+// through exactly the operations of tile_nsi_generic, in the same order, with the same
+// per-operation rounding; the two independent chains hide each other's latency.
+template <int HH, int WW>
+__device__ __forceinline__ float2 tile_pair_nsi(const float *pa, const float *pb, int pitch, float alpha)
+{
+    float2 x[HH * WW];
+#pragma unroll
+    for (int a = 0; a < HH; ++a)
+#pragma unroll
+        for (int b = 0; b < WW; ++b) x[a * WW + b] = make_float2(pa[a * pitch + b], pb[a * pitch + b]);
+    const float inv_n = __fdiv_rn(1.0f, (float)(HH * WW));  // folded at compile time
+    const float one_minus = __fsub_rn(1.0f, alpha);
+#if RSDGC_PAIR_MODE == 2
+    float2 sa = make_float2(0.0f, 0.0f), sv = make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int i = 0; i < HH * WW; ++i) {
+        sa = add2_rn(sa, make_float2(fabsf(x[i].x), fabsf(x[i].y)));
+        sv = add2_rn(sv, x[i]);
+    }
+    const float2 inv2 = make_float2(inv_n, inv_n);
+    const float2 mean_abs = mul2_rn(sa, inv2);
+    const float2 m = mul2_rn(sv, inv2);
+    const float2 neg_m = make_float2(-m.x, -m.y);  // x - m == x + (-m) in IEEE arithmetic
+    float2 sq = make_float2(0.0f, 0.0f);
+#pragma unroll
+    for (int i = 0; i < HH * WW; ++i) {
+        const float2 d = add2_rn(x[i], neg_m);
+        sq = add2_rn(sq, mul2_rn(d, d));
+    }
+    const float2 var = mul2_rn(sq, inv2);
+    const float2 s = make_float2(__fsqrt_rn(var.x), __fsqrt_rn(var.y));
+    return add2_rn(mul2_rn(make_float2(alpha, alpha), mean_abs), mul2_rn(make_float2(one_minus, one_minus), s));
+#else
+    float sa0 = 0.0f, sv0 = 0.0f, sa1 = 0.0f, sv1 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < HH * WW; ++i) {
+        sa0 = __fadd_rn(sa0, fabsf(x[i].x));
+        sa1 = __fadd_rn(sa1, fabsf(x[i].y));
+        sv0 = __fadd_rn(sv0, x[i].x);
+        sv1 = __fadd_rn(sv1, x[i].y);
+    }
+    const float a0 = __fmul_rn(sa0, inv_n), a1 = __fmul_rn(sa1, inv_n);
+    const float m0 = __fmul_rn(sv0, inv_n), m1 = __fmul_rn(sv1, inv_n);
+    float sq0 = 0.0f, sq1 = 0.0f;
+#pragma unroll
+    for (int i = 0; i < HH * WW; ++i) {
+        const float d0 = __fsub_rn(x[i].x, m0), d1 = __fsub_rn(x[i].y, m1);
+        sq0 = __fadd_rn(sq0, __fmul_rn(d0, d0));
+        sq1 = __fadd_rn(sq1, __fmul_rn(d1, d1));
+    }
+    const float s0 = __fsqrt_rn(__fmul_rn(sq0, inv_n)), s1 = __fsqrt_rn(__fmul_rn(sq1, inv_n));
+    return make_float2(__fadd_rn(__fmul_rn(alpha, a0), __fmul_rn(one_minus, s0)),
+                       __fadd_rn(__fmul_rn(alpha, a1), __fmul_rn(one_minus, s1)));
+#endif
+}
+
+// Key of one indicator value; counts it in the CTA's level-1 histogram.
+__device__ __forceinline__ void emit_key(float nsi, uint32_t *dst, unsigned int *hist_smem, unsigned int &nonfinite)
+{
+    uint32_t key = __float_as_uint(nsi);
+    if (!(nsi <= FLT_MAX)) {  // NaN or infinity: ranks first, deterministically
+        key = 0x7F800000u;
+        ++nonfinite;
+    }
+    *dst = key;
+    atomicAdd(&hist_smem[key >> kL1Shift], 1u);
+}
+
+// Keys of all tiles of one item from its v block in shared memory (row pitch d.P).
+// Returns the number of non-finite indicators this thread saw.
+template <int NTHREADS>
+__device__ __forceinline__ unsigned int item_tile_keys(const ItemDev &d, const float *sv, uint32_t *__restrict__ keys,
+                                                       unsigned int *hist_smem, float alpha)
+{
+    const int nh = d.nh, nw = d.nw, R = d.R, W = d.W, P = d.P;
+    const int ntr = (R + nh - 1) / nh;
+    const int ntc = d.ntc;
+    const int ntile = ntr * ntc;
+    uint32_t *kout = keys + d.kbase;
+    unsigned int nonfinite = 0;
+    const bool noclip = (d.flags & kItemNoClip) != 0;
+    if (RSDGC_PAIR_MODE != 0 && noclip && ((nh == 3 && nw == 3) || (nh == 1 && nw == 9))) {
+        // two tiles per thread and step: t and t + NTHREADS
+        for (int t = threadIdx.x; t < ntile; t += 2 * NTHREADS) {
+            const int t2 = t + NTHREADS;
+            const bool two = t2 < ntile;
+            const int ti = (ntr == 1) ? 0 : fast_div(t, d.inv_ntc), tj = t - ti * ntc;
+            const int tb = two ? t2 : t;
+            const int ti2 = (ntr == 1) ? 0 : fast_div(tb, d.inv_ntc), tj2 = tb - ti2 * ntc;
+            const float *pa = sv + (ti * nh) * P + tj * nw;
+            const float *pb = sv + (ti2 * nh) * P + tj2 * nw;
+            const float2 nsi = (nh == 3) ? tile_pair_nsi<3, 3>(pa, pb, P, alpha) : tile_pair_nsi<1, 9>(pa, pb, P, alpha);
+            emit_key(nsi.x, kout + ti * d.TC + tj, hist_smem, nonfinite);
+            if (two) emit_key(nsi.y, kout + ti2 * d.TC + tj2, hist_smem, nonfinite);
+        }
+    } else {
+        for (int t = threadIdx.x; t < ntile; t += NTHREADS) {
+            const int ti = (ntr == 1) ? 0 : fast_div(t, d.inv_ntc);
+            const int tj = t - ti * ntc;
+            const int hh = min(nh, R - ti * nh);
+            const int ww = min(nw, W - tj * nw);
+            const float *pt = sv + (ti * nh) * P + tj * nw;
+            const float nsi = (hh == 3 && ww == 3) ? tile_nsi_fixed<3, 3>(pt, P, alpha)
+                              : (hh == 1 && ww == 9) ? tile_nsi_fixed<1, 9>(pt, P, alpha)
+                                                     : tile_nsi_generic(pt, P, hh, ww, alpha);
+            emit_key(nsi, kout + ti * d.TC + tj, hist_smem, nonfinite);
+        }
+    }
+    return nonfinite;
+}
+
+// ------------------------------------------------------------------------------------------
+// level-1 histogram flush and the first step of the per-layer selection
+// ------------------------------------------------------------------------------------------
+
+struct FlushShared {
+    unsigned long long scan_tmp[32];
+    unsigned long long found[2];
+    int is_last;
+};
+
+// Adds this CTA's level-1 histogram to the layer's global histogram; the last CTA to do so
+// for the layer computes k_l (Eq. 11) and resolves the first 11 key bits of the threshold.
+// Called by all threads of the CTA.
+template <int NTHREADS>
+__device__ void k1_flush_layer(unsigned int *hist_smem, FlushShared &fs, int layer, const LayerDev *layers,
+                               unsigned int *hist, LayerState *state, const float *ratios, int32_t *counts,
+                               unsigned int flags)
+{
+    __syncthreads();
+    unsigned int *gh = hist + (size_t)layer * kHistStride;
+    for (int b = threadIdx.x; b < kL1Bins; b += NTHREADS) {
+        const unsigned int c = hist_smem[b];
+        if (c) {
+            atomicAdd(gh + b, c);
+            hist_smem[b] = 0;
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned int t = atomicAdd(&state[layer].ticket[0], 1u);
+        fs.is_last = (t + 1u == (unsigned int)layers[layer].n_flush1);
+    }
+    __syncthreads();
+    if (!fs.is_last) return;  // uniform for the CTA
+    __threadfence();
+    {
+        unsigned int h[kL1Bins / NTHREADS];
+#pragma unroll
+        for (int j = 0; j < kL1Bins / NTHREADS; ++j) h[j] = __ldcg(gh + j * NTHREADS + threadIdx.x);
+#pragma unroll
+        for (int j = 0; j < kL1Bins / NTHREADS; ++j) {
+            hist_smem[j * NTHREADS + threadIdx.x] = h[j];
+            gh[j * NTHREADS + threadIdx.x] = 0;
+        }
+    }
+    __syncthreads();
+    const int K = layers[layer].K;
+    const int k = keep_count(K, ratios[layer], flags);
+    if (k > 0) find_bin_from_top<kL1Bins, NTHREADS>(hist_smem, (unsigned long long)k, fs.found, fs.scan_tmp);
+    if (threadIdx.x == 0) {
+        LayerState &st = state[layer];
+        st.k = k;
+        st.prefix = k > 0 ? (uint32_t)fs.found[0] : kTakeNone;
+        st.remaining = k > 0 ? (int32_t)fs.found[1] : 0;
+        st.ticket[0] = 0;
+        counts[layer] = k;
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < kL1Bins; b += NTHREADS) hist_smem[b] = 0;
+    __syncthreads();
+}
+
+// ------------------------------------------------------------------------------------------
+// gradient element access (binary32 or bfloat16 widened exactly)
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ float4 load_grad4(const float *g, long long i4)
+{
+    return __ldcs(reinterpret_cast<const float4 *>(g) + i4);
+}
+__device__ __forceinline__ float4 bf16x4_to_f32(uint2 u)
+{
+    float4 f;
+    f.x = __uint_as_float(u.x << 16);
+    f.y = __uint_as_float(u.x & 0xFFFF0000u);
+    f.z = __uint_as_float(u.y << 16);
+    f.w = __uint_as_float(u.y & 0xFFFF0000u);
+    return f;
+}
+__device__ __forceinline__ float4 load_grad4(const __nv_bfloat16 *g, long long i4)
+{
+    return bf16x4_to_f32(__ldcs(reinterpret_cast<const uint2 *>(g) + i4));
+}
+__device__ __forceinline__ float load_grad1(const float *g, long long i) { return __ldcs(g + i); }
+__device__ __forceinline__ float load_grad1(const __nv_bfloat16 *g, long long i)
+{
+    return __uint_as_float(((unsigned int)__ldcs(reinterpret_cast<const unsigned short *>(g) + i)) << 16);
+}
+__device__ __forceinline__ float4 smem_grad4(const float *g, int i4) { return reinterpret_cast<const float4 *>(g)[i4]; }
+__device__ __forceinline__ float4 smem_grad4(const __nv_bfloat16 *g, int i4)
+{
+    return bf16x4_to_f32(reinterpret_cast<const uint2 *>(g)[i4]);
+}
+
+__device__ __forceinline__ ItemDev load_item(const ItemDev *items, int i)
+{
+    const uint4 *p = reinterpret_cast<const uint4 *>(items + i);
+    union {
+        uint4 q[4];
+        ItemDev d;
+    } u;
+    u.q[0] = __ldg(p);
+    u.q[1] = __ldg(p + 1);
+    u.q[2] = __ldg(p + 2);
+    u.q[3] = __ldg(p + 3);
+    return u.d;
+}
+
+// The elements of a contiguous item beyond its last full group of `gran` elements (gran = 4
+// or 8): plain loads and stores, results also placed in the shared-memory block.
+template <typename G>
+__device__ __forceinline__ void k1_tail(const ItemDev &d, int gran, const G *__restrict__ grads,
+                                        float *__restrict__ resid, float *sv)
+{
+    const int n = d.R * d.W;
+    const int e = (n / gran) * gran + threadIdx.x;
+    if (e < n) {
+        const float v = __fadd_rn(load_grad1(grads, d.gbase + e), resid[d.gbase + e]);
+        resid[d.gbase + e] = v;
+        sv[e] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// k1_reg: register-staged variant (any alignment)
+// ------------------------------------------------------------------------------------------
+
+constexpr int kVecPerThread = (kItemElems + 4 * kThreads - 1) / (4 * kThreads);  // 128-bit loads of g and of r per thread
+
+struct K1RegShared {
+    float v[2][kItemElems];  // double buffer: tiles of item i are reduced while item i+1 streams in
+    unsigned int hist[kL1Bins];
+    FlushShared fs;
+};
+
+struct K1Regs {
+    float4 g[kVecPerThread], r[kVecPerThread];
+};
+
+// Where each of a thread's kVecPerThread vector slots falls inside an item whose rows are
+// separate in memory.  Slot u of thread t is vector i = u * kThreads + t of the shared-memory
+// block (row pitch P / 4 vectors): row = i / (P/4), j = i % (P/4).  All items of a layer share
+// P and the row stride, so the map is recomputed only when those change.
+struct K1Map {
+    int rel[kVecPerThread];           // row * (cols / 4) + j: vector offset from the item's start
+    unsigned int rowj[kVecPerThread]; // row << 16 | j
+    int P = -1, cols = -1;
+};
+
+__device__ __forceinline__ void k1_update_map(const ItemDev &d, K1Map &m)
+{
+    if (d.P == m.P && d.cols == m.cols) return;
+    m.P = d.P;
+    m.cols = d.cols;
+    const int pv = d.P >> 2;
+#pragma unroll
+    for (int u = 0; u < kVecPerThread; ++u) {
+        const int i = u * kThreads + threadIdx.x;
+        const int row = fast_div(i, d.inv_pv), j = i - row * pv;
+        m.rel[u] = row * (d.cols >> 2) + j;
+        m.rowj[u] = ((unsigned int)row << 16) | (unsigned int)j;
+    }
+}
+
+// Arena index of element e (0 <= e < R * P) of an item whose rows are not contiguous; the
+// caller checks that the column lies inside the item.
+__device__ __forceinline__ long long item_elem_index(const ItemDev &d, int e, bool *valid)
+{
+    const int row = fast_div(e, d.inv_p), col = e - row * d.P;
+    *valid = col < d.W;
+    return d.gbase + (long long)row * d.cols + col;
+}
+
+template <typename G>
+__device__ __forceinline__ void k1_issue_loads(const ItemDev &d, const G *__restrict__ grads,
+                                               const float *__restrict__ resid, K1Regs &x, K1Map &m)
+{
+    const int tid = threadIdx.x;
+    if (d.flags & kItemVec) {
+        const long long base4 = d.gbase >> 2;
+        if (d.flags & kItemFull) {
+            const int nvec = (d.R * d.W) >> 2;
+#pragma unroll
+            for (int u = 0; u < kVecPerThread; ++u) {
+                const int i = u * kThreads + tid;
+                if (i < nvec) {
+                    x.g[u] = load_grad4(grads, base4 + i);
+                    x.r[u] = __ldcs(reinterpret_cast<const float4 *>(resid) + base4 + i);
+                }
+            }
+        } else {
+            k1_update_map(d, m);
+            const unsigned int wv = (unsigned int)d.W >> 2, R = (unsigned int)d.R;
+#pragma unroll
+            for (int u = 0; u < kVecPerThread; ++u) {
+                if ((m.rowj[u] >> 16) < R && (m.rowj[u] & 0xFFFFu) < wv) {
+                    x.g[u] = load_grad4(grads, base4 + m.rel[u]);
+                    x.r[u] = __ldcs(reinterpret_cast<const float4 *>(resid) + base4 + m.rel[u]);
+                }
+            }
+        }
+    } else {
+        float *gs = reinterpret_cast<float *>(x.g), *rs = reinterpret_cast<float *>(x.r);
+        const int n = d.R * d.P;
+#pragma unroll
+        for (int u = 0; u < 4 * kVecPerThread; ++u) {
+            const int e = u * kThreads + tid;
+            if (e < n) {
+                bool valid = true;
+                const long long gi = (d.flags & kItemFull) ? d.gbase + e : item_elem_index(d, e, &valid);
+                if (valid) {
+                    gs[u] = load_grad1(grads, gi);
+                    rs[u] = __ldcs(resid + gi);
+                }
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void k1_add_store(const ItemDev &d, float *__restrict__ resid, float *sv, K1Regs &x,
+                                             K1Map &m)
+{
+    const int tid = threadIdx.x;
+    if (d.flags & kItemVec) {
+        const long long base4 = d.gbase >> 2;
+        const bool full = (d.flags & kItemFull) != 0;
+        if (!full) k1_update_map(d, m);
+        const int nvec = (d.R * d.W) >> 2;
+        const unsigned int wv = (unsigned int)d.W >> 2, R = (unsigned int)d.R;
+#pragma unroll
+        for (int u = 0; u < kVecPerThread; ++u) {
+            const int i = u * kThreads + tid;
+            const bool valid = full ? (i < nvec) : ((m.rowj[u] >> 16) < R && (m.rowj[u] & 0xFFFFu) < wv);
+            if (valid) {
+                const long long gi = base4 + (full ? i : m.rel[u]);
+                float4 v;
+                v.x = __fadd_rn(x.g[u].x, x.r[u].x);
+                v.y = __fadd_rn(x.g[u].y, x.r[u].y);
+                v.z = __fadd_rn(x.g[u].z, x.r[u].z);
+                v.w = __fadd_rn(x.g[u].w, x.r[u].w);
+                __stcs(reinterpret_cast<float4 *>(resid) + gi, v);
+                reinterpret_cast<float4 *>(sv)[i] = v;
+            }
+        }
+    } else {
+        const float *gs = reinterpret_cast<const float *>(x.g), *rs = reinterpret_cast<const float *>(x.r);
+        const int n = d.R * d.P;
+#pragma unroll
+        for (int u = 0; u < 4 * kVecPerThread; ++u) {
+            const int e = u * kThreads + tid;
+            if (e < n) {
+                bool valid = true;
+                const long long gi = (d.flags & kItemFull) ? d.gbase + e : item_elem_index(d, e, &valid);
+                if (valid) {
+                    const float v = __fadd_rn(gs[u], rs[u]);
+                    __stcs(resid + gi, v);
+                    sv[e] = v;
+                }
+            }
+        }
+    }
+}
+
+template <typename G>
+__global__ void __launch_bounds__(kThreads)
+k1_reg(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restrict__ keys,
+       const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
+       const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
+       const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags)
+{
+    extern __shared__ __align__(16) unsigned char k1_smem_raw[];
+    K1RegShared &sh = *reinterpret_cast<K1RegShared *>(k1_smem_raw);
+    const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
+    if (begin >= end) return;
+    const int tid = threadIdx.x;
+    for (int b = tid; b < kL1Bins; b += kThreads) sh.hist[b] = 0;
+    unsigned int nonfinite = 0;
+
+    K1Regs x;
+    K1Map map;
+    ItemDev cur = load_item(items, begin);
+    k1_issue_loads(cur, grads, resid, x, map);
+    int buf = 0;
+
+    for (int it = begin; it < end; ++it) {
+        const bool has_next = (it + 1 < end);
+        ItemDev nxt = cur;
+        if (has_next) nxt = load_item(items, it + 1);
+        // v = g + r for the current item (its loads were issued one iteration ago)
+        float *sv = sh.v[buf];
+        k1_add_store(cur, resid, sv, x, map);
+        if ((cur.flags & (kItemVec | kItemFull)) == (kItemVec | kItemFull)) k1_tail(cur, 4, grads, resid, sv);
+        // the next item's g and r stream in while this item's tiles are reduced
+        if (has_next) k1_issue_loads(nxt, grads, resid, x, map);
+        __syncthreads();
+        nonfinite += item_tile_keys<kThreads>(cur, sv, keys, sh.hist, alpha);
+        if (!has_next || nxt.layer != cur.layer)
+            k1_flush_layer<kThreads>(sh.hist, sh.fs, cur.layer, layers, hist, state, ratios, counts, flags);
+        cur = nxt;
+        buf ^= 1;
+    }
+    if (nonfinite) {
+        atomicAdd(&status->nonfinite, (unsigned long long)nonfinite);
+        atomicOr(&status->flags, RSDGC_STATUS_NONFINITE);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// k1_bulk: bulk-copy (TMA) pipelined variant
+// ------------------------------------------------------------------------------------------
+
+#ifndef RSDGC_BULK_STAGES
+#define RSDGC_BULK_STAGES 2
+#endif
+#ifndef RSDGC_BULK_CTAS
+#define RSDGC_BULK_CTAS 3
+#endif
+#ifndef RSDGC_BULK_THREADS
+#define RSDGC_BULK_THREADS 256
+#endif
+constexpr int kBulkThreads = RSDGC_BULK_THREADS;
+constexpr int kBulkCtasPerSm = RSDGC_BULK_CTAS;
+constexpr int kStages = RSDGC_BULK_STAGES;  // shared-memory stages; loads run kStages - 1 items ahead
+constexpr int kLookahead = kStages - 1;
+constexpr unsigned int kSpinLimit = 1u << 22;  // bounded mbarrier waits
+
+struct K1BulkShared {
+    __align__(128) float r[kStages][kItemElems];  // residual block; becomes v in place
+    __align__(128) float g[kStages][kItemElems];  // gradient block (binary32 or bfloat16 packed)
+    unsigned int hist[kL1Bins];
+    __align__(8) unsigned long long full[kStages];  // mbarriers: stage loaded
+    FlushShared fs;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(unsigned long long *bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(unsigned long long *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait; returns false if the barrier did not complete within the limit.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, uint32_t parity)
+{
+    for (unsigned int i = 0; i < kSpinLimit; ++i)
+        if (mbar_try_wait(bar, parity)) return true;
+    return false;
+}
+__device__ __forceinline__ void bulk_load(void *dst_smem, const void *src_gmem, uint32_t bytes, unsigned long long *bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                     smem_u32(dst_smem)),
+                 "l"(__cvta_generic_to_global(src_gmem)), "r"(bytes), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *dst_gmem, const void *src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(__cvta_generic_to_global(dst_gmem)),
+                 "r"(smem_u32(src_smem)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_all()
+{
+    asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Elements of the shared-memory block covered by bulk copies: R rows of pitch P for separate
+// rows (the columns W..P of a narrower last chunk hold stale values that are never stored),
+// the largest multiple of the 16-byte granule for a contiguous run (the rest goes through
+// k1_tail).
+template <typename G>
+__device__ __forceinline__ int bulk_elems(const ItemDev &d)
+{
+    constexpr int gran = (sizeof(G) == 2) ? 8 : 4;
+    return (d.flags & kItemFull) ? ((d.R * d.W) / gran) * gran : d.R * d.P;
+}
+
+// One thread: arm the stage's barrier and start the copies of g and r for an item.
+template <typename G>
+__device__ __forceinline__ void bulk_issue_item(const ItemDev &d, const G *grads, const float *resid, float *sr,
+                                                G *sg, unsigned long long *bar)
+{
+    if (d.flags & kItemFull) {
+        const int n = bulk_elems<G>(d);
+        if (n > 0) {
+            mbar_arrive_expect_tx(bar, (uint32_t)(n * (sizeof(float) + sizeof(G))));
+            bulk_load(sr, resid + d.gbase, (uint32_t)(n * sizeof(float)), bar);
+            bulk_load(sg, grads + d.gbase, (uint32_t)(n * sizeof(G)), bar);
+        } else {
+            mbar_arrive_expect_tx(bar, 0);
+        }
+    } else {
+        mbar_arrive_expect_tx(bar, (uint32_t)(d.R * d.W * (sizeof(float) + sizeof(G))));
+        for (int row = 0; row < d.R; ++row) {
+            const long long gi = d.gbase + (long long)row * d.cols;
+            bulk_load(sr + row * d.P, resid + gi, (uint32_t)(d.W * sizeof(float)), bar);
+            bulk_load(sg + row * d.P, grads + gi, (uint32_t)(d.W * sizeof(G)), bar);
+        }
+    }
+}
+
+template <typename G>
+__global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm)
+k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restrict__ keys,
+        const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
+        const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
+        const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags)
+{
+    extern __shared__ __align__(128) unsigned char k1_smem_raw[];
+    K1BulkShared &sh = *reinterpret_cast<K1BulkShared *>(k1_smem_raw);
+    const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
+    if (begin >= end) return;
+    const int tid = threadIdx.x;
+    for (int b = tid; b < kL1Bins; b += kBulkThreads) sh.hist[b] = 0;
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) mbar_init(&sh.full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    __syncthreads();
+    // prologue: the first kLookahead items start loading
+    if (tid == 0) {
+        for (int j = 0; j < kLookahead && begin + j < end; ++j) {
+            const ItemDev d = load_item(items, begin + j);
+            bulk_issue_item<G>(d, grads, resid, sh.r[j % kStages], reinterpret_cast<G *>(sh.g[j % kStages]),
+                               &sh.full[j % kStages]);
+        }
+    }
+    unsigned int nonfinite = 0;
+    bool timed_out = false;
+    ItemDev cur = load_item(items, begin);
+    // the producer thread keeps the descriptor of the next item to load one iteration ahead
+    ItemDev ahead = cur;
+    if (tid == 0 && begin + kLookahead < end) ahead = load_item(items, begin + kLookahead);
+
+    for (int it = begin; it < end; ++it) {
+        const int rel = it - begin;
+        const int stage = rel % kStages;
+        const bool has_next = (it + 1 < end);
+        ItemDev nxt = cur;
+        if (has_next) nxt = load_item(items, it + 1);
+
+        // ---- wait for this item's blocks (bounded), form v in place
+        float *sr = sh.r[stage];
+        const G *sg = reinterpret_cast<const G *>(sh.g[stage]);
+        if (!mbar_wait_bounded(&sh.full[stage], (uint32_t)((rel / kStages) & 1))) timed_out = true;
+        const int nb = bulk_elems<G>(cur);
+        const int nvec = nb >> 2;
+        for (int i = tid; i < nvec; i += kBulkThreads) {
+            const float4 g = smem_grad4(sg, i);
+            float4 r = reinterpret_cast<const float4 *>(sr)[i];
+            r.x = __fadd_rn(g.x, r.x);
+            r.y = __fadd_rn(g.y, r.y);
+            r.z = __fadd_rn(g.z, r.z);
+            r.w = __fadd_rn(g.w, r.w);
+            reinterpret_cast<float4 *>(sr)[i] = r;
+        }
+        fence_async_smem();  // the bulk store below reads what the threads just wrote
+        if (cur.flags & kItemFull) k1_tail(cur, (sizeof(G) == 2) ? 8 : 4, grads, resid, sr);
+        __syncthreads();
+        if (tid == 0) {
+            if (cur.flags & kItemFull) {
+                if (nb > 0) bulk_store(resid + cur.gbase, sr, (uint32_t)(nb * sizeof(float)));
+            } else {
+                for (int row = 0; row < cur.R; ++row)
+                    bulk_store(resid + cur.gbase + (long long)row * cur.cols, sr + row * cur.P,
+                               (uint32_t)(cur.W * sizeof(float)));
+            }
+            bulk_commit();
+            // ---- producer: item it + kLookahead goes into the stage item it - 1 used.  Every
+            // thread finished that item's tiles before the barrier above, and its bulk store
+            // has finished reading shared memory once only the store just committed is pending.
+            if (it + kLookahead < end) {
+                bulk_wait_read<1>();
+                const int ps = (rel + kLookahead) % kStages;
+                bulk_issue_item<G>(ahead, grads, resid, sh.r[ps], reinterpret_cast<G *>(sh.g[ps]), &sh.full[ps]);
+                if (it + 1 + kLookahead < end) ahead = load_item(items, it + 1 + kLookahead);
+            }
+        }
+
+        // ---- NSI of every tile of the item
+        nonfinite += item_tile_keys<kBulkThreads>(cur, sr, keys, sh.hist, alpha);
+        if (!has_next || nxt.layer != cur.layer)
+            k1_flush_layer<kBulkThreads>(sh.hist, sh.fs, cur.layer, layers, hist, state, ratios, counts, flags);
+        cur = nxt;
+    }
+    if (tid == 0) bulk_wait_all<0>();  // all stores of this CTA have landed before it exits
+    if (nonfinite) {
+        atomicAdd(&status->nonfinite, (unsigned long long)nonfinite);
+        atomicOr(&status->flags, RSDGC_STATUS_NONFINITE);
+    }
+    if (timed_out) atomicOr(&status->flags, RSDGC_STATUS_TIMEOUT);
+}
+
+// ------------------------------------------------------------------------------------------
+
+static cudaError_t configure_once()
+{
+    static cudaError_t result = [] {
+        cudaError_t e = cudaFuncSetAttribute(k1_reg<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)sizeof(K1RegShared));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k1_reg<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(K1RegShared));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k1_bulk<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(K1BulkShared));
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(k1_bulk<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)sizeof(K1BulkShared));
+        return e;
+    }();
+    return result;
+}
+
+int k1_bulk_ctas_per_sm() { return kBulkCtasPerSm; }
+
+// Resident CTAs per SM of the register-staged kernel on the current device.
+int k1_reg_ctas_per_sm(int dtype)
+{
+    int n = 0;
+    cudaError_t e = configure_once();
+    if (e == cudaSuccess)
+        e = (dtype == RSDGC_BF16)
+                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_reg<__nv_bfloat16>, kThreads, sizeof(K1RegShared))
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_reg<float>, kThreads, sizeof(K1RegShared));
+    if (e != cudaSuccess || n < 1) {
+        (void)cudaGetLastError();
+        n = 2;
+    }
+    return n;
+}
+
+int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, const float *ratios, int32_t *counts,
+                          uint32_t *keys, cudaStream_t s)
+{
+    int launches = 0;
+    if (configure_once() != cudaSuccess) return 0;
+    if (p->n_items_bulk > 0) {
+        if (p->dtype == RSDGC_BF16)
+            k1_bulk<__nv_bfloat16><<<p->grid_bulk, kBulkThreads, sizeof(K1BulkShared), s>>>(
+                reinterpret_cast<const __nv_bfloat16 *>(grads), resid, keys, p->d_layers, p->d_items,
+                p->d_cta_begin_bulk, p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
+        else
+            k1_bulk<float><<<p->grid_bulk, kBulkThreads, sizeof(K1BulkShared), s>>>(
+                reinterpret_cast<const float *>(grads), resid, keys, p->d_layers, p->d_items, p->d_cta_begin_bulk,
+                p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
+        ++launches;
+    }
+    if (p->n_items_reg > 0) {
+        const ItemDev *items = p->d_items + p->n_items_bulk;
+        if (p->dtype == RSDGC_BF16)
+            k1_reg<__nv_bfloat16><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
+                reinterpret_cast<const __nv_bfloat16 *>(grads), resid, keys, p->d_layers, items, p->d_cta_begin_reg,
+                p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
+        else
+            k1_reg<float><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
+                reinterpret_cast<const float *>(grads), resid, keys, p->d_layers, items, p->d_cta_begin_reg,
+                p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
+        ++launches;
+    }
+    count_launch(launches);
+    return launches;
+}
+
+}  // namespace rsdgc

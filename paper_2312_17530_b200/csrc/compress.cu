@@ -1,353 +1,14 @@
-// Kernels of rsdgc_compress(): accumulate + NSI (+ level-1 histogram), two refinement
-// passes of the per-layer radix selection, the per-chunk count/scan and the pack.
+// Kernels of rsdgc_compress() after the accumulate+NSI pass: two refinement passes of the
+// per-layer radix selection, the per-chunk count/scan and the pack.
 //
 // Ordering between CTAs comes only from kernel boundaries and from "last arriver finishes
 // the job" tickets (an atomic counter per layer and phase); no thread ever waits on another
 // CTA.  The per-layer histograms and tickets are reset by the CTA that consumes them, so the
 // plan's tables are all-zero again when a compress call has run to completion.
-#include <cfloat>
-#include <cuda_bf16.h>
 
 #include "device_utils.cuh"
 
 namespace rsdgc {
-
-// ------------------------------------------------------------------------------------------
-// K1: v = g + r in place, NSI key of every tile, level-1 histogram of the keys
-// ------------------------------------------------------------------------------------------
-
-constexpr int kVecPerThread = 6;  // 128-bit loads of g and of r in flight per thread
-
-__device__ __forceinline__ float4 load_grad4(const float *g, long long i4)
-{
-    return __ldcs(reinterpret_cast<const float4 *>(g) + i4);
-}
-__device__ __forceinline__ float4 load_grad4(const __nv_bfloat16 *g, long long i4)
-{
-    const uint2 u = __ldcs(reinterpret_cast<const uint2 *>(g) + i4);
-    float4 f;
-    f.x = __uint_as_float(u.x << 16);
-    f.y = __uint_as_float(u.x & 0xFFFF0000u);
-    f.z = __uint_as_float(u.y << 16);
-    f.w = __uint_as_float(u.y & 0xFFFF0000u);
-    return f;
-}
-__device__ __forceinline__ float load_grad1(const float *g, long long i) { return __ldcs(g + i); }
-__device__ __forceinline__ float load_grad1(const __nv_bfloat16 *g, long long i)
-{
-    return __uint_as_float(((unsigned int)__ldcs(reinterpret_cast<const unsigned short *>(g) + i)) << 16);
-}
-
-// NSI of one tile held in shared memory (Eq. 8-10), binary32, elements visited row-major,
-// plain running sums, mean first and squared deviations in a second sweep; every operation
-// is an explicitly rounded single operation (no fused multiply-add).
-__device__ __forceinline__ float tile_nsi(const float *p, int pitch, int hh, int ww, float alpha)
-{
-    float sa = 0.0f, sv = 0.0f;
-    for (int a = 0; a < hh; ++a)
-        for (int b = 0; b < ww; ++b) {
-            const float x = p[a * pitch + b];
-            sa = __fadd_rn(sa, fabsf(x));
-            sv = __fadd_rn(sv, x);
-        }
-    const float fn = (float)(hh * ww);
-    const float mean_abs = __fdiv_rn(sa, fn);
-    const float m = __fdiv_rn(sv, fn);
-    float sq = 0.0f;
-    for (int a = 0; a < hh; ++a)
-        for (int b = 0; b < ww; ++b) {
-            const float d = __fsub_rn(p[a * pitch + b], m);
-            sq = __fadd_rn(sq, __fmul_rn(d, d));
-        }
-    const float s = __fsqrt_rn(__fdiv_rn(sq, fn));
-    return __fadd_rn(__fmul_rn(alpha, mean_abs), __fmul_rn(__fsub_rn(1.0f, alpha), s));
-}
-
-template <int HH, int WW>
-__device__ __forceinline__ float tile_nsi_fixed(const float *p, int pitch, float alpha)
-{
-    float x[HH * WW];
-#pragma unroll
-    for (int a = 0; a < HH; ++a)
-#pragma unroll
-        for (int b = 0; b < WW; ++b) x[a * WW + b] = p[a * pitch + b];
-    float sa = 0.0f, sv = 0.0f;
-#pragma unroll
-    for (int i = 0; i < HH * WW; ++i) {
-        sa = __fadd_rn(sa, fabsf(x[i]));
-        sv = __fadd_rn(sv, x[i]);
-    }
-    const float fn = (float)(HH * WW);
-    const float mean_abs = __fdiv_rn(sa, fn);
-    const float m = __fdiv_rn(sv, fn);
-    float sq = 0.0f;
-#pragma unroll
-    for (int i = 0; i < HH * WW; ++i) {
-        const float d = __fsub_rn(x[i], m);
-        sq = __fadd_rn(sq, __fmul_rn(d, d));
-    }
-    const float s = __fsqrt_rn(__fdiv_rn(sq, fn));
-    return __fadd_rn(__fmul_rn(alpha, mean_abs), __fmul_rn(__fsub_rn(1.0f, alpha), s));
-}
-
-struct K1Shared {
-    float v[2][kItemElems];  // double buffer: tiles of item i are reduced while item i+1 streams in
-    unsigned int hist[kL1Bins];
-    unsigned long long scan_tmp[kThreads / 32];
-    unsigned long long found[2];
-    int is_last;
-};
-
-// Adds this CTA's level-1 histogram to the layer's global histogram; the last CTA to do so
-// for the layer computes k_l (Eq. 11) and resolves the first 11 key bits of the threshold.
-__device__ void k1_flush_layer(K1Shared &sh, int layer, const LayerDev *layers, unsigned int *hist,
-                               LayerState *state, const float *ratios, int32_t *counts, unsigned int flags)
-{
-    __syncthreads();
-    unsigned int *gh = hist + (size_t)layer * kHistStride;
-    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) {
-        const unsigned int c = sh.hist[b];
-        if (c) {
-            atomicAdd(gh + b, c);
-            sh.hist[b] = 0;
-        }
-    }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int t = atomicAdd(&state[layer].ticket[0], 1u);
-        sh.is_last = (t + 1u == (unsigned int)layers[layer].n_flush1);
-    }
-    __syncthreads();
-    if (!sh.is_last) return;  // uniform for the CTA
-    __threadfence();
-    {
-        unsigned int h[kL1Bins / kThreads];
-#pragma unroll
-        for (int j = 0; j < kL1Bins / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + threadIdx.x);
-#pragma unroll
-        for (int j = 0; j < kL1Bins / kThreads; ++j) {
-            sh.hist[j * kThreads + threadIdx.x] = h[j];
-            gh[j * kThreads + threadIdx.x] = 0;
-        }
-    }
-    __syncthreads();
-    const int K = layers[layer].K;
-    const int k = keep_count(K, ratios[layer], flags);
-    if (k > 0) find_bin_from_top<kL1Bins>(sh.hist, (unsigned long long)k, sh.found, sh.scan_tmp);
-    if (threadIdx.x == 0) {
-        LayerState &st = state[layer];
-        st.k = k;
-        st.prefix = k > 0 ? (uint32_t)sh.found[0] : kTakeNone;
-        st.remaining = k > 0 ? (int32_t)sh.found[1] : 0;
-        st.ticket[0] = 0;
-        counts[layer] = k;
-    }
-    __syncthreads();
-    for (int b = threadIdx.x; b < kL1Bins; b += kThreads) sh.hist[b] = 0;
-    __syncthreads();
-}
-
-__device__ __forceinline__ ItemDev load_item(const ItemDev *items, int i)
-{
-    const uint4 *p = reinterpret_cast<const uint4 *>(items + i);
-    union {
-        uint4 q[3];
-        ItemDev d;
-    } u;
-    u.q[0] = __ldg(p);
-    u.q[1] = __ldg(p + 1);
-    u.q[2] = __ldg(p + 2);
-    return u.d;
-}
-
-// Registers that carry one item's g and r from the loads to the add: kVecPerThread 128-bit
-// words each (or 4 * kVecPerThread scalars on the unaligned path).
-struct K1Regs {
-    float4 g[kVecPerThread], r[kVecPerThread];
-};
-
-// Global (arena-relative) and shared-memory position of element e (0 <= e < R * W) of an item
-// whose rows are not contiguous in memory.
-__device__ __forceinline__ void item_pos(const ItemDev &d, int e, long long *g, int *s)
-{
-    const int row = e / d.W, col = e - row * d.W;
-    *g = d.gbase + (long long)row * d.cols + col;
-    *s = e;  // shared memory holds the R x W block densely
-}
-
-template <typename G>
-__device__ __forceinline__ void k1_issue_loads(const ItemDev &d, const G *__restrict__ grads,
-                                               const float *__restrict__ resid, K1Regs &x)
-{
-    const int tid = threadIdx.x;
-    const int n = d.R * d.W;
-    if (d.flags & kItemVec) {
-        const int nvec = (d.flags & kItemFull) ? (n >> 2) : n >> 2;  // W % 4 == 0 when rows are separate
-        const int wv = d.W >> 2;
-#pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u) {
-            const int i = u * kThreads + tid;
-            if (i < nvec) {
-                long long gi;
-                if (d.flags & kItemFull) {
-                    gi = (d.gbase >> 2) + i;
-                } else {
-                    const int row = i / wv, j = i - row * wv;
-                    gi = ((d.gbase + (long long)row * d.cols) >> 2) + j;
-                }
-                x.g[u] = load_grad4(grads, gi);
-                x.r[u] = __ldcs(reinterpret_cast<const float4 *>(resid) + gi);
-            }
-        }
-    } else {
-        float *gs = reinterpret_cast<float *>(x.g), *rs = reinterpret_cast<float *>(x.r);
-#pragma unroll
-        for (int u = 0; u < 4 * kVecPerThread; ++u) {
-            const int e = u * kThreads + tid;
-            if (e < n) {
-                long long gi;
-                int si;
-                if (d.flags & kItemFull) gi = d.gbase + e; else item_pos(d, e, &gi, &si);
-                gs[u] = load_grad1(grads, gi);
-                rs[u] = __ldcs(resid + gi);
-            }
-        }
-    }
-}
-
-// v = g + r (Eq. 12): written in place over the residual and into the shared-memory block.
-__device__ __forceinline__ void k1_add_store(const ItemDev &d, float *__restrict__ resid, float *sv, K1Regs &x)
-{
-    const int tid = threadIdx.x;
-    const int n = d.R * d.W;
-    if (d.flags & kItemVec) {
-        const int nvec = n >> 2;
-        const int wv = d.W >> 2;
-#pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u) {
-            const int i = u * kThreads + tid;
-            if (i < nvec) {
-                long long gi;
-                if (d.flags & kItemFull) {
-                    gi = (d.gbase >> 2) + i;
-                } else {
-                    const int row = i / wv, j = i - row * wv;
-                    gi = ((d.gbase + (long long)row * d.cols) >> 2) + j;
-                }
-                float4 v;
-                v.x = __fadd_rn(x.g[u].x, x.r[u].x);
-                v.y = __fadd_rn(x.g[u].y, x.r[u].y);
-                v.z = __fadd_rn(x.g[u].z, x.r[u].z);
-                v.w = __fadd_rn(x.g[u].w, x.r[u].w);
-                __stcs(reinterpret_cast<float4 *>(resid) + gi, v);
-                reinterpret_cast<float4 *>(sv)[i] = v;
-            }
-        }
-    } else {
-        const float *gs = reinterpret_cast<const float *>(x.g), *rs = reinterpret_cast<const float *>(x.r);
-#pragma unroll
-        for (int u = 0; u < 4 * kVecPerThread; ++u) {
-            const int e = u * kThreads + tid;
-            if (e < n) {
-                long long gi;
-                int si = e;
-                if (d.flags & kItemFull) gi = d.gbase + e; else item_pos(d, e, &gi, &si);
-                const float v = __fadd_rn(gs[u], rs[u]);
-                __stcs(resid + gi, v);
-                sv[si] = v;
-            }
-        }
-    }
-}
-
-// The (at most 3) elements of a contiguous vector-path item beyond its last full 128-bit word.
-template <typename G>
-__device__ __forceinline__ void k1_tail(const ItemDev &d, const G *__restrict__ grads, float *__restrict__ resid,
-                                        float *sv)
-{
-    if ((d.flags & (kItemVec | kItemFull)) == (kItemVec | kItemFull)) {
-        const int n = d.R * d.W;
-        const int e = (n & ~3) + threadIdx.x;
-        if (e < n) {
-            const float v = __fadd_rn(load_grad1(grads, d.gbase + e), resid[d.gbase + e]);
-            resid[d.gbase + e] = v;
-            sv[e] = v;
-        }
-    }
-}
-
-template <typename G>
-__global__ void __launch_bounds__(kThreads)
-k1_accumulate_nsi(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restrict__ keys,
-                  const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
-                  const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
-                  const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha,
-                  unsigned int flags)
-{
-    extern __shared__ __align__(16) unsigned char k1_smem_raw[];
-    K1Shared &sh = *reinterpret_cast<K1Shared *>(k1_smem_raw);
-    const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
-    if (begin >= end) return;
-    const int tid = threadIdx.x;
-    for (int b = tid; b < kL1Bins; b += kThreads) sh.hist[b] = 0;
-    unsigned int nonfinite = 0;
-
-    K1Regs x;
-    ItemDev cur = load_item(items, begin);
-    k1_issue_loads(cur, grads, resid, x);
-    int buf = 0;
-
-    for (int it = begin; it < end; ++it) {
-        const bool has_next = (it + 1 < end);
-        ItemDev nxt = cur;
-        if (has_next) nxt = load_item(items, it + 1);
-
-        // ---- v = g + r for the current item (its loads were issued one iteration ago)
-        float *sv = sh.v[buf];
-        k1_add_store(cur, resid, sv, x);
-        k1_tail(cur, grads, resid, sv);
-        // ---- next item's g and r start streaming in while this item's tiles are reduced
-        if (has_next) k1_issue_loads(nxt, grads, resid, x);
-        __syncthreads();
-
-        // ---- NSI of every tile of the item, one thread per tile
-        const int nh = cur.nh, nw = cur.nw, R = cur.R, W = cur.W;
-        const int ntr = (R + nh - 1) / nh;
-        const int ntc = cur.ntc;
-        const int ntile = ntr * ntc;
-        uint32_t *kout = keys + cur.kbase;
-        for (int t = tid; t < ntile; t += kThreads) {
-            const int ti = (ntr == 1) ? 0 : t / ntc;
-            const int tj = t - ti * ntc;
-            const int hh = min(nh, R - ti * nh);
-            const int ww = min(nw, W - tj * nw);
-            const float *p = sv + (ti * nh) * W + tj * nw;
-            float nsi;
-            if (hh == 3 && ww == 3 && nh == 3 && nw == 3)
-                nsi = tile_nsi_fixed<3, 3>(p, W, alpha);
-            else if (hh == 1 && ww == 9 && nw == 9)
-                nsi = tile_nsi_fixed<1, 9>(p, W, alpha);
-            else
-                nsi = tile_nsi(p, W, hh, ww, alpha);
-            uint32_t key = __float_as_uint(nsi);
-            if (!(nsi <= FLT_MAX)) {  // NaN or infinity: ranks first, deterministically
-                key = 0x7F800000u;
-                ++nonfinite;
-            }
-            kout[(long long)ti * cur.TC + tj] = key;
-            atomicAdd(&sh.hist[key >> kL1Shift], 1u);
-        }
-        if (!has_next || nxt.layer != cur.layer)
-            k1_flush_layer(sh, cur.layer, layers, hist, state, ratios, counts, flags);
-        cur = nxt;
-        buf ^= 1;
-    }
-    if (nonfinite) {
-        atomicAdd(&status->nonfinite, (unsigned long long)nonfinite);
-        atomicOr(&status->flags, RSDGC_STATUS_NONFINITE);
-    }
-}
 
 // ------------------------------------------------------------------------------------------
 // K2 / K3: refinement passes over the keys (levels 2 and 3 of the radix selection)
@@ -362,7 +23,7 @@ struct RefineShared {
     int is_last;
 };
 
-// LEVEL 2: among keys whose bits 30..20 equal the layer's prefix, histogram bits 19..10.
+// LEVEL 2: among keys whose bits 30..21 equal the layer's prefix, histogram bits 20..10.
 // LEVEL 3: among keys whose bits 30..10 equal the prefix, histogram bits 9..0; the last CTA
 // of the layer then knows the threshold key T and how many keys equal to T are taken.
 template <int LEVEL>
@@ -373,11 +34,13 @@ k_refine(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     __shared__ RefineShared sh;
     constexpr int SHIFT_HI = (LEVEL == 2) ? kL1Shift : kL2Shift;
     constexpr int SHIFT_LO = (LEVEL == 2) ? kL2Shift : 0;
+    constexpr int NBITS = (LEVEL == 2) ? kL2Bits : kL3Bits;
+    constexpr int NBINS = 1 << NBITS;
     const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x;
     LayerState &st = state[c.layer];
     const uint32_t prefix = st.prefix;
-    for (int b = tid; b < kL2Bins; b += kThreads) sh.hist[b] = 0;
+    for (int b = tid; b < NBINS; b += kThreads) sh.hist[b] = 0;
     __syncthreads();
     if (prefix != kTakeNone) {
         const uint32_t *kp = keys + layers[c.layer].tile_off + c.start;
@@ -391,21 +54,21 @@ k_refine(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
             }
 #pragma unroll
             for (int u = 0; u < kKeyVecBatch; ++u) {  // the all-ones filler never matches a prefix
-                if ((q[u].x >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].x >> SHIFT_LO) & (kL2Bins - 1)], 1u);
-                if ((q[u].y >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].y >> SHIFT_LO) & (kL2Bins - 1)], 1u);
-                if ((q[u].z >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].z >> SHIFT_LO) & (kL2Bins - 1)], 1u);
-                if ((q[u].w >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].w >> SHIFT_LO) & (kL2Bins - 1)], 1u);
+                if ((q[u].x >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].x >> SHIFT_LO) & (NBINS - 1)], 1u);
+                if ((q[u].y >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].y >> SHIFT_LO) & (NBINS - 1)], 1u);
+                if ((q[u].z >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].z >> SHIFT_LO) & (NBINS - 1)], 1u);
+                if ((q[u].w >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].w >> SHIFT_LO) & (NBINS - 1)], 1u);
             }
         }
         const int i = (nvec << 2) + tid;
         if (i < c.n) {
             const uint32_t q = kp[i];
-            if ((q >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q >> SHIFT_LO) & (kL2Bins - 1)], 1u);
+            if ((q >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q >> SHIFT_LO) & (NBINS - 1)], 1u);
         }
     }
     __syncthreads();
     unsigned int *gh = hist + (size_t)c.layer * kHistStride;
-    for (int b = tid; b < kL2Bins; b += kThreads) {
+    for (int b = tid; b < NBINS; b += kThreads) {
         const unsigned int n = sh.hist[b];
         if (n) atomicAdd(gh + b, n);
     }
@@ -419,11 +82,11 @@ k_refine(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     if (!sh.is_last) return;
     __threadfence();
     {
-        unsigned int h[kL2Bins / kThreads];
+        unsigned int h[NBINS / kThreads];
 #pragma unroll
-        for (int j = 0; j < kL2Bins / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + tid);
+        for (int j = 0; j < NBINS / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + tid);
 #pragma unroll
-        for (int j = 0; j < kL2Bins / kThreads; ++j) {
+        for (int j = 0; j < NBINS / kThreads; ++j) {
             sh.hist[j * kThreads + tid] = h[j];
             gh[j * kThreads + tid] = 0;
         }
@@ -431,11 +94,11 @@ k_refine(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     __syncthreads();
     const int remaining = st.remaining;
     if (prefix != kTakeNone)
-        find_bin_from_top<kL2Bins>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
+        find_bin_from_top<NBINS>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
     if (tid == 0) {
         st.ticket[LEVEL - 1] = 0;
         if (prefix != kTakeNone) {
-            const uint32_t next = (prefix << 10) | (uint32_t)sh.found[0];
+            const uint32_t next = (prefix << NBITS) | (uint32_t)sh.found[0];
             if (LEVEL == 2) {
                 st.prefix = next;
                 st.remaining = (int32_t)sh.found[1];
@@ -707,26 +370,6 @@ k_pack(const uint32_t *__restrict__ keys, float *__restrict__ resid, const Layer
 
 // ------------------------------------------------------------------------------------------
 
-// Resident CTAs per SM of the accumulate+NSI kernel on the current device.
-int k1_ctas_per_sm(int dtype)
-{
-    int n = 0;
-    const size_t smem = sizeof(K1Shared);
-    cudaError_t e = cudaFuncSetAttribute(k1_accumulate_nsi<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)smem);
-    if (e == cudaSuccess)
-        e = cudaFuncSetAttribute(k1_accumulate_nsi<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-    if (e == cudaSuccess)
-        e = (dtype == RSDGC_BF16)
-                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_accumulate_nsi<__nv_bfloat16>, kThreads, smem)
-                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_accumulate_nsi<float>, kThreads, smem);
-    if (e != cudaSuccess || n < 1) {
-        (void)cudaGetLastError();
-        n = 2;
-    }
-    return n;
-}
-
 // Next event of the plan's pool (created on demand), recorded on the stream.
 static cudaError_t record_event(rsdgc_plan *p, cudaStream_t s)
 {
@@ -749,14 +392,7 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, cons
 #define RSDGC_MARK()                                   \
     if (prof && e == cudaSuccess) e = record_event(p, s)
     RSDGC_MARK();
-    if (p->dtype == RSDGC_BF16)
-        k1_accumulate_nsi<__nv_bfloat16><<<p->grid1, kThreads, sizeof(K1Shared), s>>>(
-            reinterpret_cast<const __nv_bfloat16 *>(grads), resid, keys, p->d_layers, p->d_items, p->d_cta_begin,
-            p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
-    else
-        k1_accumulate_nsi<float><<<p->grid1, kThreads, sizeof(K1Shared), s>>>(
-            reinterpret_cast<const float *>(grads), resid, keys, p->d_layers, p->d_items, p->d_cta_begin,
-            p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
+    launch_accumulate_nsi(p, grads, resid, ratios, counts, keys, s);
     RSDGC_MARK();
     k_refine<2><<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
     RSDGC_MARK();
@@ -769,7 +405,7 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, cons
                                          idx_cap, val, val_cap);
     RSDGC_MARK();
 #undef RSDGC_MARK
-    count_launch(5);
+    count_launch(4);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

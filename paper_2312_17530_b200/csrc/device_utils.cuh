@@ -6,9 +6,9 @@
 namespace rsdgc {
 
 // Exclusive prefix sum of one value per thread over the CTA, in thread order.
-// `warp_tot` points to kThreads/32 words of shared memory.  Every thread receives the CTA
+// `warp_tot` points to NTHREADS/32 words of shared memory.  Every thread receives the CTA
 // total in *total.  Contains two barriers; all threads must call it.
-template <typename T>
+template <typename T, int NTHREADS = kThreads>
 __device__ __forceinline__ T block_exclusive_scan(T x, T *warp_tot, T *total)
 {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -22,7 +22,7 @@ __device__ __forceinline__ T block_exclusive_scan(T x, T *warp_tot, T *total)
     __syncthreads();
     T offset = 0, sum = 0;
 #pragma unroll
-    for (int w = 0; w < kThreads / 32; ++w) {
+    for (int w = 0; w < NTHREADS / 32; ++w) {
         T t = warp_tot[w];
         if (w < warp) offset += t;
         sum += t;
@@ -37,17 +37,17 @@ __device__ __forceinline__ T block_exclusive_scan(T x, T *warp_tot, T *total)
 // entries of that bin are still needed (need minus the count of all higher bins).
 // If the histogram holds fewer than `need` entries, bin 0 is returned with what is missing.
 // `out` and `warp_tot` are shared memory; all threads must call; ends with a barrier.
-template <int NBINS>
+template <int NBINS, int NTHREADS = kThreads>
 __device__ __forceinline__ void find_bin_from_top(const unsigned int *h, unsigned long long need,
                                                   unsigned long long *out, unsigned long long *warp_tot)
 {
-    constexpr int PER = NBINS / kThreads;
-    static_assert(NBINS % kThreads == 0, "histogram size must be a multiple of the CTA size");
+    constexpr int PER = NBINS / NTHREADS;
+    static_assert(NBINS % NTHREADS == 0, "histogram size must be a multiple of the CTA size");
     unsigned long long local = 0;
 #pragma unroll
     for (int j = 0; j < PER; ++j) local += h[NBINS - 1 - (threadIdx.x * PER + j)];
     unsigned long long total;
-    unsigned long long excl = block_exclusive_scan<unsigned long long>(local, warp_tot, &total);
+    unsigned long long excl = block_exclusive_scan<unsigned long long, NTHREADS>(local, warp_tot, &total);
     if (threadIdx.x == 0 && total < need) {
         out[0] = 0;
         out[1] = need - (total - h[0]);
@@ -66,6 +66,13 @@ __device__ __forceinline__ void find_bin_from_top(const unsigned int *h, unsigne
         }
     }
     __syncthreads();
+}
+
+// floor(x / d) for x < 8192 and d <= 8192 by a multiply-high with inv = ceil(2^32 / d)
+// (inv = 0 encodes d = 1).
+__device__ __forceinline__ int fast_div(int x, unsigned int inv)
+{
+    return inv ? (int)__umulhi((unsigned int)x, inv) : x;
 }
 
 // Number of tiles to keep, k = ceil(K * ratio) (Eq. 11) limited to [0 or 1, K]; the product

@@ -65,7 +65,8 @@ void free_device_tables(rsdgc_plan *p)
 {
     cudaFree(p->d_layers);
     cudaFree(p->d_items);
-    cudaFree(p->d_cta_begin);
+    cudaFree(p->d_cta_begin_bulk);
+    cudaFree(p->d_cta_begin_reg);
     cudaFree(p->d_chunks);
     cudaFree(p->d_echunks);
     cudaFree(p->d_state);
@@ -93,6 +94,7 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
     p->items.clear();
     p->chunks.clear();
     p->echunks.clear();
+    std::vector<int64_t> chunk_w(n_layers, 0);  // columns of a regular (not last) column chunk
     int64_t elem_off = 0, tile_off = 0, total_elems = 0, total_tiles = 0;
     int max_slot = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -120,9 +122,10 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
             int64_t ntr_max = kItemElems / band;
             int64_t n_items = ceil_div64(L.TR, ntr_max);
             int64_t ntr = ceil_div64(L.TR, n_items);
-            // multiples of 4 tile rows keep every item start 4-element aligned (128-bit loads)
-            if (round_up64(ntr, 4) <= ntr_max) ntr = round_up64(ntr, 4);
-            else if (ntr_max >= 4) ntr = ntr_max & ~(int64_t)3;
+            // multiples of 8 tile rows keep every item start 16-byte aligned in both arenas
+            // (8 bfloat16 or 4 binary32 elements): 128-bit loads and bulk copies
+            if (round_up64(ntr, 8) <= ntr_max) ntr = round_up64(ntr, 8);
+            else if (ntr_max >= 8) ntr = ntr_max & ~(int64_t)7;
             for (int64_t tr0 = 0; tr0 < L.TR; tr0 += ntr) {
                 Item it{l, (int32_t)tr0, (int32_t)std::min<int64_t>(ntr, L.TR - tr0), 0, L.TC};
                 p->items.push_back(it);
@@ -131,8 +134,9 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
             int64_t ntc_max = kItemElems / L.slot;
             int64_t n_items = ceil_div64(L.TC, ntc_max);
             int64_t ntc = ceil_div64(L.TC, n_items);
-            if (round_up64(ntc, 4) <= ntc_max) ntc = round_up64(ntc, 4);
-            else if (ntc_max >= 4) ntc = ntc_max & ~(int64_t)3;
+            if (round_up64(ntc, 8) <= ntc_max) ntc = round_up64(ntc, 8);
+            else if (ntc_max >= 8) ntc = ntc_max & ~(int64_t)7;
+            chunk_w[l] = std::min<int64_t>(ntc * d.nw, d.cols);
             for (int64_t tr = 0; tr < L.TR; ++tr)
                 for (int64_t tc0 = 0; tc0 < L.TC; tc0 += ntc) {
                     Item it{l, (int32_t)tr, 1, (int32_t)tc0, (int32_t)std::min<int64_t>(ntc, L.TC - tc0)};
@@ -160,39 +164,14 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
     }
     if (p->items.size() > (size_t)INT32_MAX || p->echunks.size() > (size_t)INT32_MAX) return RSDGC_ERR_CAPACITY;
 
-    // --- static partition of the items over the CTAs of the accumulate+NSI kernel
-    const int G = p->grid1;
+    // --- device form of the items; choice of kernel per item
     const size_t n_items = p->items.size();
-    std::vector<double> cum(n_items + 1, 0.0);
-    for (size_t i = 0; i < n_items; ++i) {
-        const Item &it = p->items[i];
-        const LayerDev &L = p->layers[it.layer];
-        int64_t r0 = (int64_t)it.tr0 * L.nh, r1 = std::min<int64_t>(L.rows, r0 + (int64_t)it.ntr * L.nh);
-        int64_t c0 = (int64_t)it.tc0 * L.nw, c1 = std::min<int64_t>(L.cols, c0 + (int64_t)it.ntc * L.nw);
-        cum[i + 1] = cum[i] + (double)((r1 - r0) * (c1 - c0)) + 512.0;  // + fixed cost per item
-    }
-    p->cta_begin.assign(G + 1, (int32_t)n_items);
-    std::vector<int32_t> owner(n_items);
-    for (size_t i = 0; i < n_items; ++i) {
-        int g = (int)std::floor(cum[i] * G / cum[n_items]);
-        if (g >= G) g = G - 1;
-        owner[i] = g;
-    }
-    {
-        size_t i = 0;
-        for (int g = 0; g <= G; ++g) {
-            while (i < n_items && owner[i] < g) ++i;
-            p->cta_begin[g] = (int32_t)i;
-        }
-    }
-    for (auto &L : p->layers) L.n_flush1 = 0;
-    for (size_t i = 0; i < n_items; ++i) {
-        bool first = (i == 0) || p->items[i - 1].layer != p->items[i].layer || owner[i - 1] != owner[i];
-        if (first) p->layers[p->items[i].layer].n_flush1 += 1;
-    }
-
-    // --- device form of the items
-    p->items_dev.resize(n_items);
+    auto magic = [](int64_t d) -> uint32_t { return d <= 1 ? 0u : (uint32_t)(((1ll << 32) + d - 1) / d); };
+    const int64_t gran = (p->dtype == RSDGC_BF16) ? 8 : 4;  // elements per 16 bytes of the gradient arena
+    std::vector<ItemDev> all(n_items);
+    p->item_path.assign(n_items, 0);
+    p->item_cta.assign(n_items, 0);
+    std::vector<double> cost(n_items);
     for (size_t i = 0; i < n_items; ++i) {
         const Item &it = p->items[i];
         const LayerDev &L = p->layers[it.layer];
@@ -210,8 +189,53 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
         d.layer = it.layer;
         const bool full = (d.W == L.cols) || d.R == 1;  // one contiguous run
         const bool vec = (d.gbase % 4 == 0) && (full || (L.cols % 4 == 0 && d.W % 4 == 0));
-        d.flags = (full ? kItemFull : 0) | (vec ? kItemVec : 0);
-        p->items_dev[i] = d;
+        const bool bulk = !(p->flags & RSDGC_NO_BULK_COPY) && (d.gbase % gran == 0) &&
+                          (full || (L.cols % gran == 0 && d.W % gran == 0));
+        const bool noclip = (d.R % L.nh == 0) && (d.W % L.nw == 0);
+        d.flags = (full ? kItemFull : 0) | (vec ? kItemVec : 0) | (bulk ? kItemBulk : 0) | (noclip ? kItemNoClip : 0);
+        // shared-memory pitch: the width of the layer's regular column chunk, so that every item
+        // of a layer maps threads to elements the same way (the last chunk of a row is narrower)
+        d.P = full ? d.W : (int32_t)chunk_w[it.layer];
+        d.inv_ntc = magic(d.ntc);
+        d.inv_p = magic(d.P);
+        d.inv_pv = magic(d.P / 4);
+        all[i] = d;
+        p->item_path[i] = bulk ? 0 : 1;
+        cost[i] = (double)d.R * d.W + 512.0;  // elements + a fixed cost per item
+    }
+
+    // --- each kernel's items in layer order, split into contiguous ranges of equal cost, one
+    // range per CTA (all CTAs of a kernel are resident at once)
+    p->items_dev.clear();
+    p->grid_bulk = p->n_sm * k1_bulk_ctas_per_sm();
+    p->grid_reg = p->n_sm * p->reg_ctas_per_sm;
+    for (auto &L : p->layers) L.n_flush1 = 0;
+    for (int path = 0; path < 2; ++path) {
+        std::vector<size_t> mine;
+        for (size_t i = 0; i < n_items; ++i)
+            if (p->item_path[i] == path) mine.push_back(i);
+        const int G = path == 0 ? p->grid_bulk : p->grid_reg;
+        std::vector<int32_t> &cta_begin = path == 0 ? p->cta_begin_bulk : p->cta_begin_reg;
+        (path == 0 ? p->n_items_bulk : p->n_items_reg) = (int)mine.size();
+        double total = 0.0;
+        for (size_t i : mine) total += cost[i];
+        cta_begin.assign(G + 1, (int32_t)mine.size());
+        double cum = 0.0;
+        size_t next_cta = 0;
+        int prev_layer = -1, prev_cta = -1;
+        for (size_t j = 0; j < mine.size(); ++j) {
+            int g = total > 0.0 ? (int)std::floor(cum * G / total) : 0;
+            if (g >= G) g = G - 1;
+            while (next_cta <= (size_t)g) cta_begin[next_cta++] = (int32_t)j;
+            const size_t i = mine[j];
+            p->item_cta[i] = g;
+            if (all[i].layer != prev_layer || g != prev_cta) p->layers[all[i].layer].n_flush1 += 1;
+            prev_layer = all[i].layer;
+            prev_cta = g;
+            cum += cost[i];
+            p->items_dev.push_back(all[i]);
+        }
+        while (next_cta <= (size_t)G) cta_begin[next_cta++] = (int32_t)mine.size();
     }
 
     rsdgc_info &I = p->info;
@@ -241,7 +265,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
     if (n_layers > kMaxLayers) return RSDGC_ERR_CAPACITY;
     if (grad_dtype != RSDGC_F32 && grad_dtype != RSDGC_BF16) return RSDGC_ERR_INVALID;
     if (!(alpha >= 0.0f && alpha <= 1.0f)) return RSDGC_ERR_INVALID;
-    if (flags & ~RSDGC_KEEP_AT_LEAST_ONE) return RSDGC_ERR_INVALID;
+    if (flags & ~(RSDGC_KEEP_AT_LEAST_ONE | RSDGC_NO_BULK_COPY)) return RSDGC_ERR_INVALID;
 
     rsdgc_plan *p = new (std::nothrow) rsdgc_plan();
     if (!p) return RSDGC_ERR_NOMEM;
@@ -260,10 +284,8 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         }
         p->n_sm = n_sm;
         DeviceGuard guard(device);
-        // one CTA per resident slot: the static partition assumes all CTAs run concurrently
-        p->grid1 = n_sm * k1_ctas_per_sm(grad_dtype);
-    } else {
-        p->grid1 = p->n_sm * 2;
+        // one CTA per resident slot: the static partitions assume all CTAs run concurrently
+        p->reg_ctas_per_sm = k1_reg_ctas_per_sm(grad_dtype);
     }
 
     int rc;
@@ -282,7 +304,8 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         cudaError_t e = guard.err;
         if (e == cudaSuccess) e = upload(&p->d_layers, p->layers);
         if (e == cudaSuccess) e = upload(&p->d_items, p->items_dev);
-        if (e == cudaSuccess) e = upload(&p->d_cta_begin, p->cta_begin);
+        if (e == cudaSuccess) e = upload(&p->d_cta_begin_bulk, p->cta_begin_bulk);
+        if (e == cudaSuccess) e = upload(&p->d_cta_begin_reg, p->cta_begin_reg);
         if (e == cudaSuccess) e = upload(&p->d_chunks, p->chunks);
         if (e == cudaSuccess) e = upload(&p->d_echunks, p->echunks);
         if (e == cudaSuccess) e = alloc_zero(&p->d_state, (size_t)n_layers);
@@ -350,22 +373,21 @@ extern "C" int rsdgc_plan_payload_bound(const rsdgc_plan *plan, float max_ratio,
     return RSDGC_OK;
 }
 
-// Diagnostic: copies the accumulate+NSI work list (5 int32 per item: layer, tr0, ntr, tc0,
-// ntc) and the per-CTA item ranges; used by the host-logic tests.  Returns the item count.
+// Diagnostic: the accumulate+NSI work list (7 int32 per item: layer, tr0, ntr, tc0, ntc, kernel,
+// CTA), the two grid sizes and the per-layer flush counts; used by the host-logic tests.
 extern "C" int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,
-                                       int32_t *cta_begin_host, int64_t cta_capacity, int32_t *n_flush_host)
+                                       int32_t *grids_host, int32_t *n_flush_host)
 {
     if (!plan) return RSDGC_ERR_INVALID;
     int64_t n = (int64_t)plan->items.size();
     if (items_host)
         for (int64_t i = 0; i < n && i < items_capacity; ++i) {
             const Item &it = plan->items[i];
-            int32_t *o = items_host + 5 * i;
+            int32_t *o = items_host + 7 * i;
             o[0] = it.layer, o[1] = it.tr0, o[2] = it.ntr, o[3] = it.tc0, o[4] = it.ntc;
+            o[5] = plan->item_path[i], o[6] = plan->item_cta[i];
         }
-    if (cta_begin_host)
-        for (int64_t g = 0; g < (int64_t)plan->cta_begin.size() && g < cta_capacity; ++g)
-            cta_begin_host[g] = plan->cta_begin[g];
+    if (grids_host) grids_host[0] = plan->grid_bulk, grids_host[1] = plan->grid_reg;
     if (n_flush_host)
         for (int l = 0; l < plan->n_layers; ++l) n_flush_host[l] = plan->layers[l].n_flush1;
     return n;

@@ -11,7 +11,7 @@
 namespace rsdgc {
 
 struct RatioShared {
-    unsigned int hist[kL1Bins];
+    unsigned int hist[kHistStride];
     unsigned long long scan_tmp[kThreads / 32];
     unsigned long long found[2];
     int is_last;
@@ -24,7 +24,7 @@ k_ratio_level(const float *__restrict__ weights, const LayerDev *__restrict__ la
               RatioState *rs, long long *survivors, float *ratios, long long n_keep)
 {
     __shared__ RatioShared sh;
-    constexpr int NBINS = (LEVEL == 1) ? kL1Bins : kL2Bins;
+    constexpr int NBINS = (LEVEL == 1) ? kL1Bins : (LEVEL == 2 ? kL2Bins : kL3Bins);
     constexpr int SHIFT_HI = (LEVEL == 1) ? 31 : (LEVEL == 2 ? kL1Shift : kL2Shift);
     constexpr int SHIFT_LO = (LEVEL == 1) ? kL1Shift : (LEVEL == 2 ? kL2Shift : 0);
     const int tid = threadIdx.x;
@@ -79,7 +79,7 @@ k_ratio_level(const float *__restrict__ weights, const LayerDev *__restrict__ la
     }
     // find the bin from the top with 64-bit running sums: bins are owned top-down by thread
     // order in find_bin_from_top, so redo it here on 64-bit per-bin totals kept in registers
-    __shared__ unsigned long long gh64[NBINS];
+    __shared__ unsigned long long gh64[NBINS];  // per-bin totals over all layers
 #pragma unroll
     for (int j = 0; j < NBINS / kThreads; ++j) gh64[j * kThreads + tid] = gsum[j];
     __syncthreads();
@@ -149,7 +149,7 @@ k_ratio_level(const float *__restrict__ weights, const LayerDev *__restrict__ la
             rs->remaining = rem_next;
             rs->n_keep = n_keep;
         } else if (LEVEL == 2) {
-            if (active) rs->prefix = (prefix << 10) | (uint32_t)bin;
+            if (active) rs->prefix = (prefix << kL2Bits) | (uint32_t)bin;
             rs->remaining = rem_next;
         }
     }

@@ -12,14 +12,19 @@ namespace rsdgc {
 
 // ---- compile-time geometry -------------------------------------------------------------
 constexpr int kThreads = 256;        // threads per CTA, every kernel
-constexpr int kItemElems = 6144;     // elements of one accumulate+NSI work item (24 KB of smem)
-constexpr int kL1Bits = 11;          // radix level 1: key bits 30..20 (8 exponent + 3 mantissa)
+#ifndef RSDGC_ITEM_ELEMS
+#define RSDGC_ITEM_ELEMS 4400
+#endif
+constexpr int kItemElems = RSDGC_ITEM_ELEMS;  // elements of one accumulate+NSI work item
+constexpr int kL1Bits = 10;          // radix level 1: key bits 30..21 (8 exponent + 2 mantissa)
 constexpr int kL1Bins = 1 << kL1Bits;
-constexpr int kL1Shift = 20;
-constexpr int kL2Bins = 1024;        // level 2: key bits 19..10
+constexpr int kL1Shift = 21;
+constexpr int kL2Bits = 11;          // level 2: key bits 20..10
+constexpr int kL2Bins = 1 << kL2Bits;
 constexpr int kL2Shift = 10;
-constexpr int kL3Bins = 1024;        // level 3: key bits 9..0
-constexpr int kHistStride = kL1Bins; // words of histogram per layer
+constexpr int kL3Bits = 10;          // level 3: key bits 9..0
+constexpr int kL3Bins = 1 << kL3Bits;
+constexpr int kHistStride = kL2Bins; // words of histogram per layer (the largest level)
 constexpr int kChunkKeys = 16384;    // keys (or weights) per CTA in the key passes
 constexpr int kMaxLayers = 2048;
 constexpr int kMaxSlot = 4096;
@@ -44,21 +49,28 @@ struct Item {
     int32_t layer, tr0, ntr, tc0, ntc;
 };
 
-// The same item resolved for the device: everything the accumulate+NSI kernel needs, so that
-// one 48-byte load per item replaces the chain item -> layer table -> data.
+// The same item resolved for the device: everything the accumulate+NSI kernels need, so that
+// one 64-byte load per item replaces the chain item -> layer table -> data.
 struct __align__(16) ItemDev {
     long long gbase;  // arena index of the first element held
     long long kbase;  // key-array index of the first tile
-    int32_t R, W;     // rows and columns held; W is the row pitch in shared memory
+    int32_t R, W;     // rows and columns held
     int32_t cols;     // row stride in global memory
     int32_t ntc;      // tile columns in the item
     int32_t TC;       // tile columns of the layer = key stride between tile rows
     int16_t nh, nw;
     int32_t layer;
-    int32_t flags;    // kItemFull: rows are contiguous in memory; kItemVec: 128-bit path usable
+    int32_t flags;    // kItem* bits
+    uint32_t inv_ntc; // ceil(2^32 / d) for d = ntc, P, P / 4 (0 when d = 1): see fast_div()
+    uint32_t inv_p;
+    uint32_t inv_pv;
+    int32_t P;        // row pitch of the block in shared memory (elements, >= W)
 };
-static_assert(sizeof(ItemDev) == 48, "ItemDev is loaded as three 16-byte words");
-constexpr int kItemFull = 1, kItemVec = 2;
+static_assert(sizeof(ItemDev) == 64, "ItemDev is loaded as four 16-byte words");
+constexpr int kItemFull = 1;    // the rows held are one contiguous run in memory
+constexpr int kItemVec = 2;     // every row starts on a 16-byte boundary of the binary32 arenas
+constexpr int kItemBulk = 4;    // eligible for the bulk-copy kernel (16-byte rule for g as well)
+constexpr int kItemNoClip = 8;  // no tile of the item is clipped by the layer's edge
 
 // Key chunk: keys [start, start + n) of a layer (layer-local tile indices).
 struct Chunk {
@@ -105,12 +117,15 @@ struct rsdgc_plan {
     float alpha = 0.5f;
     uint32_t flags = 0;
     int n_sm = 148;
-    int grid1 = 0;  // CTAs of the accumulate+NSI kernel
+    int reg_ctas_per_sm = 2;
+    int grid_bulk = 0, grid_reg = 0;        // CTAs of the two accumulate+NSI kernels
+    int n_items_bulk = 0, n_items_reg = 0;  // items_dev = [bulk items..., register items...]
 
     std::vector<rsdgc::LayerDev> layers;
     std::vector<rsdgc::Item> items;
     std::vector<rsdgc::ItemDev> items_dev;
-    std::vector<int32_t> cta_begin;  // grid1 + 1 item indices
+    std::vector<int32_t> item_path, item_cta;          // per host item: kernel (0 bulk, 1 reg) and CTA
+    std::vector<int32_t> cta_begin_bulk, cta_begin_reg;  // grid + 1 indices into each kernel's item list
     std::vector<rsdgc::Chunk> chunks;
     std::vector<rsdgc::EChunk> echunks;
 
@@ -119,7 +134,7 @@ struct rsdgc_plan {
     // device tables
     rsdgc::LayerDev *d_layers = nullptr;
     rsdgc::ItemDev *d_items = nullptr;
-    int32_t *d_cta_begin = nullptr;
+    int32_t *d_cta_begin_bulk = nullptr, *d_cta_begin_reg = nullptr;
     rsdgc::Chunk *d_chunks = nullptr;
     rsdgc::EChunk *d_echunks = nullptr;
     rsdgc::LayerState *d_state = nullptr;
@@ -149,6 +164,9 @@ cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long 
 cudaError_t launch_decompress(rsdgc_plan *p, const int32_t *idx, const float *val,
                               const int32_t *counts, float scale, float *dense, cudaStream_t s);
 void count_launch(int n);
-int k1_ctas_per_sm(int dtype);
+int k1_reg_ctas_per_sm(int dtype);
+int k1_bulk_ctas_per_sm();
+int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, const float *ratios, int32_t *counts,
+                          uint32_t *keys, cudaStream_t s);
 
 }  // namespace rsdgc

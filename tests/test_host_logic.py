@@ -49,7 +49,7 @@ def test_plan_create_rejects_bad_arguments(lib):
 @pytest.mark.parametrize("net", ["resnet18", "resnet50", "vgg19", "odd"])
 def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net):
     if net == "odd":
-        shapes = [(7, 11, 3, 3), (1, 5, 1, 9), (4096, 45, 3, 3), (3, 20000, 3, 3), (100, 6145, 2, 5),
+        shapes = [(7, 11, 3, 3), (1, 5, 1, 9), (4096, 45, 3, 3), (3, 20000, 3, 3), (100, 4401, 2, 5),
                   (5000, 7, 1, 7), (1, 100000, 1, 9), (64, 64, 64, 64), (9, 9, 1, 1)]
     else:
         shapes = synth.layer_shapes(getattr(synth, net + "_tensors")())
@@ -67,29 +67,42 @@ def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net):
     assert p.info.arena_elems == eo and p.info.total_tiles_padded == to
     assert p.info.workspace_bytes == 4 * to
 
-    items, cta, nflush = p.worklist()
-    assert cta[0] == 0 and cta[-1] == len(items) and (np.diff(cta) >= 0).all() and len(cta) == 148 * 2 + 1
+    items, grids, nflush = p.worklist()
+    assert grids.tolist() == [148 * 3, 148 * 2]
     assert (np.diff(items[:, 0]) >= 0).all()          # layers in order
-    owner = np.searchsorted(cta, np.arange(len(items)), side="right") - 1
     for l, (r, c, nh, nw) in enumerate(shapes):
         TR, TC = -(-r // nh), -(-c // nw)
         cover = np.zeros((TR, TC), dtype=np.int32)
         sel = items[items[:, 0] == l]
-        for _, tr0, ntr, tc0, ntc in sel.tolist():
+        for _, tr0, ntr, tc0, ntc, path, cta in sel.tolist():
             assert ntr >= 1 and ntc >= 1 and tr0 + ntr <= TR and tc0 + ntc <= TC
             rows = min(r, (tr0 + ntr) * nh) - tr0 * nh
             cols = min(c, (tc0 + ntc) * nw) - tc0 * nw
-            assert rows * cols <= 6144
+            assert rows * cols <= 4400
             assert ntr == 1 or (tc0 == 0 and ntc == TC)   # several tile rows only at full width
+            assert path in (0, 1) and 0 <= cta < grids[path]
+            # the bulk-copy kernel only takes items whose rows start on 16-byte boundaries
+            start = p.layers[l].elem_offset + tr0 * nh * c + tc0 * nw
+            contiguous = cols == c or rows == 1
+            aligned = start % 4 == 0 and (contiguous or (c % 4 == 0 and cols % 4 == 0))
+            assert (path == 0) == aligned
             cover[tr0:tr0 + ntr, tc0:tc0 + ntc] += 1
         assert (cover == 1).all()
-        assert nflush[l] == len(set(owner[items[:, 0] == l].tolist()))
-    # the static partition is balanced: no CTA holds much more than the mean cost
-    cost = np.zeros(len(cta) - 1)
-    for i, (l, tr0, ntr, tc0, ntc) in enumerate(items.tolist()):
-        r, c, nh, nw = shapes[l]
-        cost[owner[i]] += (min(r, (tr0 + ntr) * nh) - tr0 * nh) * (min(c, (tc0 + ntc) * nw) - tc0 * nw) + 512
-    assert cost.max() <= cost.sum() / len(cost) + 6144 + 512 + 1
+        assert nflush[l] == len(set((pa, ct) for *_, pa, ct in sel.tolist()))
+    # within a kernel the CTA of consecutive items never decreases, and the static partition is
+    # balanced: no CTA holds much more than the mean cost
+    for path in (0, 1):
+        sel = items[items[:, 5] == path]
+        if not len(sel):
+            continue
+        assert (np.diff(sel[:, 6]) >= 0).all()
+        cost = np.zeros(grids[path])
+        for l, tr0, ntr, tc0, ntc, _, cta in sel.tolist():
+            r, c, nh, nw = shapes[l]
+            cost[cta] += (min(r, (tr0 + ntr) * nh) - tr0 * nh) * (min(c, (tc0 + ntc) * nw) - tc0 * nw) + 512
+        assert cost.max() <= cost.sum() / len(cost) + 4400 + 512 + 1
+    if net != "odd":
+        assert (items[:, 5] == 0).mean() > 0.99       # the usual shapes go to the bulk-copy kernel
 
 
 def test_payload_bound(lib):
