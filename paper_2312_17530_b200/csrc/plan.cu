@@ -202,6 +202,8 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
         all[i] = d;
         p->item_path[i] = bulk ? 0 : 1;
         cost[i] = (double)d.R * d.W + 512.0;  // elements + a fixed cost per item
+        // the first item of a layer pays for the previous layer's histogram flush in its CTA
+        if (i > 0 && p->items[i - 1].layer != it.layer) cost[i] += 6000.0;
     }
 
     // --- each kernel's items in layer order, split into contiguous ranges of equal cost, one
