@@ -645,8 +645,8 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__rest
         const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
         const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags)
 {
-    extern __shared__ __align__(128) unsigned char k1_smem_raw[];
-    K1BulkShared &sh = *reinterpret_cast<K1BulkShared *>(k1_smem_raw);
+    extern __shared__ __align__(128) unsigned char k1_bulk_smem_raw[];
+    K1BulkShared &sh = *reinterpret_cast<K1BulkShared *>(k1_bulk_smem_raw);
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     if (begin >= end) return;
     const int tid = threadIdx.x;
