@@ -147,6 +147,37 @@ int rsdgc_update_ratios(rsdgc_plan *plan, const float *weights_dev, float global
                         float *ratios_dev, void *stream);
 
 /*
+ * The ratio rule of rsdgc_update_ratios() for callers that must not allocate device memory.
+ * (The paper has no counterpart: it describes the rule, Eq. 3-5, not how memory is managed.)
+ *
+ * Who cannot allocate: code that runs while a stream capture is open on its thread (cudaMalloc
+ * is not allowed there), runtimes that hand all device memory to their own pool at start-up
+ * and forbid driver allocations afterwards, and loops that cannot afford the device-wide
+ * synchronisation an allocation or a free may imply.  rsdgc_plan_create() allocates, so such
+ * callers cannot use a plan; this entry point needs none.  The caller passes the weights and
+ * the output; every byte of scratch (per-layer histograms, counters) lives in one fixed array
+ * inside the library: about 513 KB of device memory on every GPU that loads the library, kept
+ * until the process exits.
+ *
+ * weights_dev: binary32 weights; layer l occupies layer_sizes_host[l] elements starting at
+ *   element layer_offsets_host[l] (a multiple of 4).  ratios_dev: out, n_layers floats.  The
+ *   result equals rsdgc_update_ratios() on a plan with the same layers and offsets.
+ * Limits: 1 <= n_layers <= RSDGC_NOALLOC_MAX_LAYERS, each layer below 2^31 elements; beyond
+ *   them the call returns RSDGC_ERR_CAPACITY and does nothing.  Other errors: INVALID,
+ *   ALIGNMENT, CUDA.
+ * The first call on a device looks up the device address of the scratch array (one runtime
+ * query, with that device current; later calls reuse it): make that first call before any
+ * stream capture begins.  No call allocates or frees memory.
+ * All calls on a device share the scratch array, and it keeps what the previous call left in
+ * it, so each call starts by clearing it on `stream`.  Two calls whose work overlaps on the
+ * GPU (different streams, or different threads) race on it and give wrong ratios: order them.
+ */
+#define RSDGC_NOALLOC_MAX_LAYERS 64
+int rsdgc_update_ratios_noalloc(const float *weights_dev, const int64_t *layer_offsets_host,
+                                const int64_t *layer_sizes_host, int32_t n_layers, float global_keep,
+                                float *ratios_dev, void *stream);
+
+/*
  * One worker's per-iteration compression (Algorithm 1, per-iteration part; Eq. 8-12):
  *   v = g + r, written in place over the residual arena           (Eq. 12, second line)
  *   NSI of every tile of v in binary32                            (Eq. 8-10)

@@ -24,7 +24,9 @@ EXPORTS = [
     "rsdgc_plan_payload_bound", "rsdgc_plan_worklist", "rsdgc_update_ratios", "rsdgc_compress",
     "rsdgc_compress_host", "rsdgc_decompress_accumulate", "rsdgc_get_status", "rsdgc_launch_count",
     "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
+    "rsdgc_update_ratios_noalloc",
 ]
+NOALLOC_MAX_LAYERS = 64
 N_COMPRESS_KERNELS = 5
 COMPRESS_KERNELS = ("accumulate_nsi", "refine2", "refine3", "count", "pack")
 
@@ -85,6 +87,7 @@ def lib():
         L.rsdgc_get_status.argtypes = [vp, vp, C.POINTER(Status)]
         L.rsdgc_profile_enable.argtypes = [vp, i32]
         L.rsdgc_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
+        L.rsdgc_update_ratios_noalloc.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), i32, f32, vp, vp]
         L.rsdgc_launch_count.argtypes = []
         L.rsdgc_launch_count.restype = i64
         L.rsdgc_strerror.argtypes = [C.c_int]
@@ -211,6 +214,17 @@ class Plan:
         st = Status()
         _check(lib().rsdgc_get_status(self._h, _stream(), C.byref(st)), "rsdgc_get_status")
         return st
+
+
+def update_ratios_noalloc(weights, layer_offsets: Sequence[int], layer_sizes: Sequence[int], global_keep: float,
+                          ratios) -> None:
+    """rsdgc_update_ratios_noalloc(): the ratio rule without a plan and without any allocation
+    (scratch is a fixed array inside the library; at most NOALLOC_MAX_LAYERS layers)."""
+    n = len(layer_offsets)
+    offs = (C.c_int64 * max(1, n))(*[int(x) for x in layer_offsets])
+    sizes = (C.c_int64 * max(1, n))(*[int(x) for x in layer_sizes])
+    _check(lib().rsdgc_update_ratios_noalloc(_ptr(weights), offs, sizes, n, global_keep, _ptr(ratios), _stream()),
+           "rsdgc_update_ratios_noalloc")
 
 
 def launch_count() -> int:

@@ -84,6 +84,7 @@ void free_device_tables(rsdgc_plan *p)
 namespace rsdgc {
 
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+void set_last_cuda_error(int e) { g_last_cuda_error = e; }
 
 // Splits every layer into work items for the accumulate+NSI kernel and into key / element
 // chunks for the selection passes, and assigns contiguous item ranges of equal cost to the

@@ -2,6 +2,8 @@
 // allocate device memory.  Same computation as rsdgc_update_ratios() (three-level radix
 // selection on the weight magnitudes), but it needs no plan: the layer table travels in the
 // kernel parameters and every byte of scratch lives in one file-scope device array.
+#include <climits>
+#include <cmath>
 #include <mutex>
 
 #include "device_utils.cuh"
@@ -213,8 +215,6 @@ static cudaError_t noalloc_scratch_ptr(NoAllocScratch **out)
 
 using namespace rsdgc;
 
-extern thread_local int rsdgc_tls_last_cuda_error;
-
 extern "C" int rsdgc_update_ratios_noalloc(const float *weights_dev, const int64_t *layer_offsets_host,
                                            const int64_t *layer_sizes_host, int32_t n_layers, float global_keep,
                                            float *ratios_dev, void *stream)
@@ -256,7 +256,7 @@ extern "C" int rsdgc_update_ratios_noalloc(const float *weights_dev, const int64
         e = cudaGetLastError();
     }
     if (e != cudaSuccess) {
-        rsdgc_tls_last_cuda_error = (int)e;
+        set_last_cuda_error((int)e);
         return RSDGC_ERR_CUDA;
     }
     return RSDGC_OK;

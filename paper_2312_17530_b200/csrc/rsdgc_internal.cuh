@@ -164,6 +164,7 @@ cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long 
 cudaError_t launch_decompress(rsdgc_plan *p, const int32_t *idx, const float *val,
                               const int32_t *counts, float scale, float *dense, cudaStream_t s);
 void count_launch(int n);
+void set_last_cuda_error(int e);
 int k1_reg_ctas_per_sm(int dtype);
 int k1_bulk_ctas_per_sm();
 int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, const float *ratios, int32_t *counts,
