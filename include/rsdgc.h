@@ -237,13 +237,13 @@ int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,
 /*
  * Optional per-kernel timing of rsdgc_compress().  While enabled, every rsdgc_compress() on
  * this plan records CUDA events on its stream before its first kernel and after each of its
- * RSDGC_N_COMPRESS_KERNELS kernels (accumulate+NSI, refine level 2, refine level 3, count,
- * pack).  rsdgc_profile_read() waits for the recorded events, adds the elapsed milliseconds
+ * RSDGC_N_COMPRESS_KERNELS stages (accumulate+NSI, refine level 2, refine level 3, count,
+ * mark, gather).  rsdgc_profile_read() waits for the recorded events, adds the elapsed milliseconds
  * of every kernel over all recorded calls into ms_per_kernel_host[RSDGC_N_COMPRESS_KERNELS],
  * stores the number of calls and forgets them.  Off by default; not for use during stream
  * capture.
  */
-#define RSDGC_N_COMPRESS_KERNELS 5
+#define RSDGC_N_COMPRESS_KERNELS 6
 int rsdgc_profile_enable(rsdgc_plan *plan, int32_t enable);
 int rsdgc_profile_read(rsdgc_plan *plan, double *ms_per_kernel_host, int64_t *n_calls_host);
 

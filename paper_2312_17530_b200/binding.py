@@ -27,8 +27,8 @@ EXPORTS = [
     "rsdgc_update_ratios_noalloc",
 ]
 NOALLOC_MAX_LAYERS = 64
-N_COMPRESS_KERNELS = 5
-COMPRESS_KERNELS = ("accumulate_nsi", "refine2", "refine3", "count", "pack")
+N_COMPRESS_KERNELS = 6
+COMPRESS_KERNELS = ("accumulate_nsi", "refine2", "refine3", "count", "mark", "gather")
 
 
 class LayerDesc(C.Structure):

@@ -1,5 +1,5 @@
 // Kernels of rsdgc_compress() after the accumulate+NSI pass: two refinement passes of the
-// per-layer radix selection, the per-chunk count/scan and the pack.
+// per-layer radix selection, the per-chunk count/scan, the payload indices and the gather.
 //
 // Ordering between CTAs comes only from kernel boundaries and from "last arriver finishes
 // the job" tickets (an atomic counter per layer and phase); no thread ever waits on another
@@ -231,41 +231,38 @@ k_count(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
 }
 
 // ------------------------------------------------------------------------------------------
-// K5: pack.  A tile is kept if its key is above T, or equals T and fewer than e equal keys
+// K5: mark.  A tile is kept if its key is above T, or equals T and fewer than e equal keys
 // precede it in the layer.  Its payload slot is its rank among the kept tiles of the layer
-// (ascending tile index).  Kept tiles are copied out of the residual and zeroed there.
+// (ascending tile index).  This kernel writes the tile indices of the payload; the values are
+// moved by k_gather, whose work is spread evenly whatever the spatial pattern of the kept tiles.
 // ------------------------------------------------------------------------------------------
 
 constexpr int kKeysPerThread = kChunkKeys / kThreads;  // 64 consecutive keys per thread
 constexpr int kChunkVecs = kChunkKeys / 4;             // 128-bit words of keys per chunk
-constexpr int kCopyBatch = 8;                          // gathered loads in flight per thread
 
-struct PackShared {
+struct MarkShared {
     // one byte per 128-bit word of keys: bit c = key c above T, bit 4 + c = key c equal to T
     __align__(16) unsigned char code[kChunkVecs];
-    unsigned short pos[kChunkKeys];  // position in the chunk of the r-th kept tile
     unsigned long long scan_tmp[kThreads / 32];
 };
 
 __global__ void __launch_bounds__(kThreads)
-k_pack(const uint32_t *__restrict__ keys, float *__restrict__ resid, const LayerDev *__restrict__ layers,
-       const Chunk *__restrict__ chunks, const LayerState *__restrict__ state,
-       const uint2 *__restrict__ chunk_cnt, int32_t *__restrict__ idx, long long idx_cap,
-       float *__restrict__ val, long long val_cap)
+k_mark(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers, const Chunk *__restrict__ chunks,
+       const LayerState *__restrict__ state, const uint2 *__restrict__ chunk_cnt, int32_t *__restrict__ idx,
+       long long idx_cap)
 {
-    __shared__ PackShared sh;
+    __shared__ MarkShared sh;
     const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x;
     const LayerState st = state[c.layer];
     if (st.k == 0) return;
-    const LayerDev L = layers[c.layer];
     const uint32_t T = st.T;
     const uint2 base = chunk_cnt[blockIdx.x];  // tiles above T / equal to T in earlier chunks
     // equal keys of this chunk that are still taken: those with layer-wide equal-rank < e
     const long long eq_room = max(0ll, (long long)st.e - (long long)base.y);
 
     // ---- phase 1: coalesced read of the chunk's keys, 2 bits per key into shared memory
-    const uint32_t *kp = keys + L.tile_off + c.start;
+    const uint32_t *kp = keys + layers[c.layer].tile_off + c.start;
     const int nvec = c.n >> 2;
     for (int b0 = 0; b0 < kChunkVecs; b0 += kThreads * kKeyVecBatch) {
         uint4 q[kKeyVecBatch];
@@ -305,57 +302,96 @@ k_pack(const uint32_t *__restrict__ keys, float *__restrict__ resid, const Layer
     const unsigned long long ex =
         block_exclusive_scan<unsigned long long>(((unsigned long long)eq << 32) | gt, sh.scan_tmp, &total);
     unsigned int gt_before = (unsigned int)(ex & 0xFFFFFFFFull), eq_before = (unsigned int)(ex >> 32);
-    if (gt | eq) {
+    if ((gt | eq) == 0) return;
+    // payload position of this chunk's first kept tile
+    const long long slot0 = st.idx_off + (long long)base.x + min((long long)base.y, (long long)st.e);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
+    for (int j = 0; j < 4; ++j) {
 #pragma unroll
-            for (int b = 0; b < 4; ++b) {
-                const unsigned int byte = (w[j] >> (8 * b)) & 0xFFu;
-                if (byte == 0) continue;
-                const int p0 = tid * kKeysPerThread + (j * 4 + b) * 4;
+        for (int b = 0; b < 4; ++b) {
+            const unsigned int byte = (w[j] >> (8 * b)) & 0xFFu;
+            if (byte == 0) continue;
+            const int p0 = c.start + tid * kKeysPerThread + (j * 4 + b) * 4;
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    if (byte & (1u << k)) {
-                        sh.pos[gt_before + (unsigned int)min((long long)eq_before, eq_room)] = (unsigned short)(p0 + k);
-                        ++gt_before;
-                    } else if (byte & (16u << k)) {
-                        if ((long long)eq_before < eq_room) sh.pos[gt_before + eq_before] = (unsigned short)(p0 + k);
-                        ++eq_before;
-                    }
+            for (int k = 0; k < 4; ++k) {
+                long long s = -1;
+                if (byte & (1u << k)) {
+                    s = slot0 + gt_before + min((long long)eq_before, eq_room);
+                    ++gt_before;
+                } else if (byte & (16u << k)) {
+                    if ((long long)eq_before < eq_room) s = slot0 + gt_before + eq_before;
+                    ++eq_before;
                 }
+                if (s >= 0 && s < idx_cap) idx[s] = p0 + k;
             }
         }
     }
-    __syncthreads();
-    const unsigned int tot_gt = (unsigned int)(total & 0xFFFFFFFFull), tot_eq = (unsigned int)(total >> 32);
-    const int n_kept = (int)(tot_gt + (unsigned int)min((long long)tot_eq, eq_room));
-    // rank in the layer of this chunk's first kept tile
-    const long long rank0 = (long long)base.x + min((long long)base.y, (long long)st.e);
+}
 
-    // ---- phase 3: gather the kept tiles out of the residual, zero them there, write the payload
-    const int slot = L.slot;
-    const int n_copy = n_kept * slot;  // at most 16384 * 4096
-    for (int j0 = 0; j0 < n_copy; j0 += kThreads * kCopyBatch) {
+// ------------------------------------------------------------------------------------------
+// K6: gather.  Payload value j of the whole call belongs to layer l (val_off_l <= j <
+// val_off_l + k_l * slot_l), payload slot s = (j - val_off_l) / slot_l, element el of the tile
+// idx[idx_off_l + s].  The value is moved from the residual to val and the residual entry
+// becomes +0 (Eq. 12: what is sent leaves the accumulator).  Grid-stride with kCopyBatch
+// independent entries in flight per thread.
+// ------------------------------------------------------------------------------------------
+
+constexpr int kCopyBatch = 8;
+
+__global__ void __launch_bounds__(kThreads)
+k_gather(float *__restrict__ resid, const LayerDev *__restrict__ layers, const LayerState *__restrict__ state,
+         int n_layers, const int32_t *__restrict__ idx, long long idx_cap, float *__restrict__ val, long long val_cap)
+{
+    __shared__ long long val_off[kMaxLayers + 1];
+    __shared__ long long idx_off[kMaxLayers];
+    const int tid = threadIdx.x;
+    for (int l = tid; l < n_layers; l += kThreads) {
+        val_off[l] = state[l].val_off;
+        idx_off[l] = state[l].idx_off;
+    }
+    if (tid == 0) {
+        const LayerState &last = state[n_layers - 1];
+        val_off[n_layers] = last.val_off + (long long)last.k * layers[n_layers - 1].slot;
+    }
+    __syncthreads();
+    const long long total = val_off[n_layers];
+    const long long stride = (long long)gridDim.x * kThreads;
+    for (long long j0 = (long long)blockIdx.x * kThreads + tid; j0 < total; j0 += stride * kCopyBatch) {
         long long ga[kCopyBatch], vo[kCopyBatch];
+        int tile[kCopyBatch], lay[kCopyBatch], el[kCopyBatch];
         float xv[kCopyBatch];
 #pragma unroll
         for (int u = 0; u < kCopyBatch; ++u) {
-            const int j = j0 + u * kThreads + tid;
+            const long long j = j0 + u * stride;
             ga[u] = -1;
             vo[u] = -1;
-            if (j < n_copy) {
-                const int r = j / slot, el = j - r * slot;
-                const int tile = c.start + sh.pos[r];
-                const long long s = st.idx_off + rank0 + r;              // payload slot (tiles)
-                const long long vbase = st.val_off + (rank0 + r) * slot;
-                if (s < idx_cap && vbase + slot <= val_cap) {            // else: does not fit, not sent
-                    const int tr = tile / L.TC, tc = tile - tr * L.TC;
-                    const int a = el / L.nw, b = el - a * L.nw;
-                    const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
-                    if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
-                    vo[u] = vbase + el;
-                    if (el == 0) idx[s] = tile;
+            tile[u] = -1;
+            if (j < total) {
+                int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
+                while (hi - lo > 1) {
+                    const int mid = (lo + hi) >> 1;
+                    if (val_off[mid] <= j) lo = mid; else hi = mid;
                 }
+                const int slot = layers[lo].slot;
+                const long long jl = j - val_off[lo];
+                const long long s = jl / slot;
+                lay[u] = lo;
+                el[u] = (int)(jl - s * slot);
+                // tiles that do not fit the payload buffers are not sent and stay in the residual
+                if (idx_off[lo] + s < idx_cap && val_off[lo] + (s + 1) * slot <= val_cap) {
+                    tile[u] = __ldg(idx + idx_off[lo] + s);
+                    vo[u] = j;
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kCopyBatch; ++u) {
+            if (tile[u] >= 0) {
+                const LayerDev &L = layers[lay[u]];
+                const int tr = tile[u] / L.TC, tc = tile[u] - tr * L.TC;
+                const int a = el[u] / L.nw, b = el[u] - a * L.nw;
+                const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
+                if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
             }
         }
 #pragma unroll
@@ -401,11 +437,13 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, cons
     k_count<<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt,
                                           p->n_layers, idx_cap, val_cap, p->d_status);
     RSDGC_MARK();
-    k_pack<<<n_chunks, kThreads, 0, s>>>(keys, resid, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, idx,
-                                         idx_cap, val, val_cap);
+    k_mark<<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, idx, idx_cap);
+    RSDGC_MARK();
+    k_gather<<<p->n_sm * 8, kThreads, 0, s>>>(resid, p->d_layers, p->d_state, p->n_layers, idx, idx_cap, val,
+                                              val_cap);
     RSDGC_MARK();
 #undef RSDGC_MARK
-    count_launch(4);
+    count_launch(5);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
