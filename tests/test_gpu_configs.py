@@ -1,0 +1,148 @@
+"""GPU parity on the full-size workloads: the VGG-19-shaped set with 4 workers and their
+aggregation (the configuration the benchmark times), the ResNet-50-shaped set over 100 iterations
+with drifting scales and refreshed ratios, and the single-matrix sweep from 1M to 1B elements in
+binary32 and bfloat16.  Sizes the oracle can sort are compared element by element; above that,
+sampled tiles go through the oracle and the rest is checked by exact properties."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2312_17530_b200 import binding, synth
+
+import parity
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    binding.lib()
+
+
+# ---------------------------------------------------------------------------------------------
+# config 3: VGG-19-shaped set, 4 workers, keep 1/64, aggregation into one dense buffer
+# ---------------------------------------------------------------------------------------------
+
+def test_vgg19_four_workers_full_size(oracle):
+    tensors = synth.vgg19_tensors()
+    shapes = synth.layer_shapes(tensors)
+    plan = binding.Plan(shapes, alpha=0.5)
+    assert plan.info.total_elems == 139_754_605
+    sig = synth.log_uniform_scales(len(tensors), (3,))
+    grads = synth.multi_worker_gradients(tensors, 4, (3, 0), sig)        # the benchmark's rank-0 inputs
+    ratios = np.full(len(shapes), 1 / 64, np.float32)
+    zeros = [np.zeros(synth.numel(s), np.float32) for _, s in tensors]
+    payloads, refs_all = [], []
+    for w in range(4):
+        _, refs, gc = parity.compress_and_check(oracle, plan, shapes, grads[w], zeros, ratios, 0.5,
+                                                what="vgg worker %d" % w, max_ratio=1 / 64)
+        payloads.append(gc.payload())
+        refs_all.append(oracle.CompressResult(layers=refs))
+        n_bytes = 4 * sum(r.idx.size + r.val.size for r in refs)
+        assert 50 < 4 * plan.info.total_elems / n_bytes < 60                # "more than 50x" in bytes
+    d_dense = torch.zeros(plan.info.arena_elems, device="cuda:0")
+    plan.decompress_accumulate(payloads, d_dense, 1.0)
+    torch.cuda.synchronize()
+    dense_ref = [np.zeros(synth.numel(s), np.float32) for _, s in tensors]
+    oracle.decompress_accumulate(shapes, dense_ref, refs_all, 1.0)
+    for got, ref in zip(parity.from_arena(plan, d_dense.cpu().numpy()), dense_ref):
+        np.testing.assert_array_equal(got.view(np.uint32), ref.view(np.uint32))
+    # the workers' selections overlap (shared gradient component): the scatter-add does collide
+    fc6_tiles = np.concatenate([refs_all[w].layers[32].idx for w in range(4)])
+    assert int((np.bincount(fc6_tiles) > 1).sum()) > 1000
+
+
+# ---------------------------------------------------------------------------------------------
+# config 4: ResNet-50-shaped set, 100 iterations, scales drift, ratios refreshed every 10
+# ---------------------------------------------------------------------------------------------
+
+def test_resnet50_hundred_iterations(oracle):
+    tensors = synth.resnet50_tensors()
+    shapes = synth.layer_shapes(tensors)
+    L = len(tensors)
+    plan = binding.Plan(shapes, alpha=0.5)
+    base_w = synth.synthetic_weights(tensors, (4,))
+    b0 = synth.log_uniform_scales(L, (4,))
+    g_walk = synth.random_walk(L, 100, (4, 1), 0.1)
+    w_walk = synth.random_walk(L, 100, (4, 2), 0.05)
+    res = [np.zeros(synth.numel(s), np.float32) for _, s in tensors]
+    gc = parity.GpuCompress(plan, max_ratio=1.0)
+    d_ratios = torch.zeros(L, device="cuda:0")
+    ratios_ref = ratios_first = None
+    for it in range(100):
+        if it % 10 == 0:
+            w = [bw * np.float32(np.exp(w_walk[it, l])) for l, bw in enumerate(base_w)]
+            plan.update_ratios(parity.dev(parity.to_arena(plan, w)), 1 / 50, d_ratios)
+            torch.cuda.synchronize()
+            ratios_new, surv, n_keep = oracle.update_ratios(w, 1 / 50)
+            np.testing.assert_array_equal(d_ratios.cpu().numpy(), ratios_new)
+            if ratios_first is None:
+                ratios_first = ratios_new
+            elif it == 50:
+                assert not np.array_equal(ratios_new, ratios_first)      # the rule does track the drift
+            ratios_ref = ratios_new
+        g = synth.laplace_layers(tensors, (4, it), b0 * np.exp(g_walk[it]))
+        gc.idx.fill_(-1)
+        gc.val.fill_(float(parity.CANARY))
+        res, refs, _ = parity.compress_and_check(oracle, plan, shapes, g, res, ratios_ref, 0.5, gc=gc,
+                                                 what="resnet50 it%d" % it)
+
+
+# ---------------------------------------------------------------------------------------------
+# config 5: single matrices, 1M .. 1B elements, binary32 and bfloat16, keep 1/10, 1/100, 1/1000
+# ---------------------------------------------------------------------------------------------
+
+def _sweep_inputs(rows, cols, bf16):
+    x = synth.clustered_matrix(rows, cols, seed=5)
+    return synth.f32_to_bf16_bits(x) if bf16 else x
+
+
+def _run_single(plan, g, ratio):
+    gc = parity.GpuCompress(plan, max_ratio=ratio)
+    d_g = parity.dev(parity.to_arena(plan, [g], np.uint16 if g.dtype == np.uint16 else np.float32))
+    d_r = torch.zeros(plan.info.arena_elems, device="cuda:0")            # a real buffer, still read
+    st = gc.run(d_g, d_r, torch.tensor([ratio], dtype=torch.float32, device="cuda:0"))
+    assert st.flags == 0
+    return gc, d_r
+
+
+@pytest.mark.parametrize("rows,cols", [(1024, 1024), (4096, 4096), (2450, 400), (7840, 1280)])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_sweep_small_full_oracle(oracle, rows, cols, bf16):
+    shapes = [(rows, cols, 3, 3)]
+    g = _sweep_inputs(rows, cols, bf16)
+    plan = binding.Plan(shapes, grad_dtype=binding.RSDGC_BF16 if bf16 else binding.RSDGC_F32, alpha=0.5)
+    zeros = [np.zeros(rows * cols, np.float32)]
+    for ratio in synth.SWEEP_RATIOS:
+        parity.compress_and_check(oracle, plan, shapes, [g], zeros, [ratio], 0.5, max_ratio=ratio,
+                                  what="sweep %dx%d bf16=%s 1/%d" % (rows, cols, bf16, round(1 / ratio)))
+
+
+@pytest.mark.parametrize("rows,cols,bf16,ratio", [(8192, 8192, False, 1 / 100), (25088, 4096, False, 1 / 1000)])
+def test_sweep_medium_full_oracle(oracle, rows, cols, bf16, ratio):
+    shapes = [(rows, cols, 3, 3)]
+    g = _sweep_inputs(rows, cols, bf16)
+    plan = binding.Plan(shapes, grad_dtype=binding.RSDGC_BF16 if bf16 else binding.RSDGC_F32, alpha=0.5)
+    parity.compress_and_check(oracle, plan, shapes, [g], [np.zeros(rows * cols, np.float32)], [ratio], 0.5,
+                              max_ratio=ratio, what="sweep %dx%d" % (rows, cols))
+
+
+@pytest.mark.parametrize("rows,cols,bf16,ratio", [(8192, 8192, True, 1 / 10), (16384, 16384, False, 1 / 10),
+                                                  (32768, 32768, True, 1 / 100), (78400, 12800, False, 1 / 1000)])
+def test_sweep_large_sampled(oracle, rows, cols, bf16, ratio):
+    shape = (rows, cols, 3, 3)
+    g = _sweep_inputs(rows, cols, bf16)
+    plan = binding.Plan([shape], grad_dtype=binding.RSDGC_BF16 if bf16 else binding.RSDGC_F32, alpha=0.5)
+    gc, d_r = _run_single(plan, g, ratio)
+    k = int(gc.counts.cpu().numpy()[0])
+    li = plan.layers[0]
+    nsi = gc.nsi.cpu().numpy()[:li.n_tiles]
+    idx = gc.idx.cpu().numpy()[:k]
+    val = gc.val.cpu().numpy()[:k * 9]
+    res = d_r.cpu().numpy()[:rows * cols]
+    del gc, d_r
+    torch.cuda.empty_cache()
+    parity.check_single_layer_sampled(oracle, shape, g, np.zeros(rows * cols, np.float32), float(np.float32(ratio)),
+                                      0.5, nsi, k, idx, val, res,
+                                      what="sweep %dx%d bf16=%s 1/%d" % (rows, cols, bf16, round(1 / ratio)))
