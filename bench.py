@@ -99,11 +99,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def vgg_inputs(rank: int, n_workers: int = N_WORKERS):
+def vgg_inputs(rank: int, n_workers: int = N_WORKERS, only_fc6: bool = False):
     """(tensors, shapes, per-worker per-layer gradients) for this rank's workers."""
     from paper_2312_17530_b200 import dist, synth
 
     tensors = synth.vgg19_tensors()
+    if only_fc6:  # the largest layer alone: the small case used for ncu captures
+        tensors = [t for t in tensors if t[0] == "fc6.weight"]
     shapes = synth.layer_shapes(tensors)
     sig = synth.log_uniform_scales(len(tensors), (3,))
     ids = dist.worker_ids(rank, N_WORKERS)
@@ -180,7 +182,10 @@ def run_b200(args):
     device = torch.device("cuda", local_rank)
     binding.lib()  # raises if the CUDA library has not been built; there is no other path
 
-    tensors, shapes, grads, _ = vgg_inputs(rank)
+    global N_WORKERS
+    if args.workload == "fc6":
+        N_WORKERS = 1
+    tensors, shapes, grads, _ = vgg_inputs(rank, N_WORKERS, only_fc6=(args.workload == "fc6"))
     plan = binding.Plan(shapes, alpha=ALPHA, device=local_rank)
     n = plan.info.total_elems
     arena = plan.info.arena_elems
@@ -250,7 +255,7 @@ def run_b200(args):
     h_val = torch.zeros(nv, dtype=torch.float32, pin_memory=True)
     h_cnt = torch.zeros(plan.n_layers, dtype=torch.int32, pin_memory=True)
     d_stage = torch.empty(arena, dtype=torch.float32, device=device)
-    e2e_steps = max(1, min(args.steps, 5))
+    e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 5))
     d2h = 0
 
     def e2e_step():
@@ -262,18 +267,20 @@ def run_b200(args):
             d2h += 4 * a + 4 * b + 4 * plan.n_layers
         plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
 
-    e2e_step()
-    dist.barrier()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    ev0.record()
-    for _ in range(e2e_steps):
+    e2e_bps = 0.0
+    if e2e_steps:
         e2e_step()
-    ev1.record()
-    torch.cuda.synchronize()
-    e2e_wall = time.perf_counter() - t0
-    e2e_s = max(ev0.elapsed_time(ev1) / 1e3, e2e_wall)  # host-side waits are part of this path
-    e2e_bps, _ = dist.aggregate_throughput(grad_bytes_step * e2e_steps, e2e_s)
+        dist.barrier()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ev0.record()
+        for _ in range(e2e_steps):
+            e2e_step()
+        ev1.record()
+        torch.cuda.synchronize()
+        e2e_wall = time.perf_counter() - t0
+        e2e_s = max(ev0.elapsed_time(ev1) / 1e3, e2e_wall)  # host-side waits are part of this path
+        e2e_bps, _ = dist.aggregate_throughput(grad_bytes_step * e2e_steps, e2e_s)
 
     # ---- separately timed: ratio rule (per epoch), dense zero fill
     extra = {}
@@ -317,14 +324,16 @@ def run_b200(args):
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": 1e3 * t_max / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "l2": "inputs larger than L2 (4 x 1.1 GB streamed per step)",
+            "config": {"workload": WORKLOAD if args.workload == "vgg19" else
+                       "fc6 25088x4096 alone, 1 worker (small case for profiler captures, not the benchmark)",
+                       "l2": "inputs larger than L2 (4 x 1.1 GB streamed per step)",
                        "parallelism": "dp%d (independent replicas, no collective)" % args.gpus},
             "clocks": clocks,
             "e2e": {"value": e2e_bps / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(4 * arena * N_WORKERS),
                     "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": int(launches),
-            "roofline": {"bound": "hbm", "kernel": "k1_accumulate_nsi", "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "traffic": K1_TRAFFIC_BYTES,
+            "roofline": {"bound": "hbm", "kernel": "k1_bulk", "achieved": achieved, "peak": peak,
+                         "unit": "GB/s", "frac": achieved / peak, "traffic": K1_TRAFFIC_BYTES if args.workload == "vgg19" else None,
                          "peak_source": peak_src, "algorithmic_bytes": alg_bytes, "launch_us": k1_s * 1e6},
             "extra": extra,
         }
@@ -336,9 +345,11 @@ def run_b200(args):
     return 0
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one k1_accumulate_nsi launch on this workload
-# from an ncu capture; None until a capture of the current kernel exists (see profiles/).
-K1_TRAFFIC_BYTES = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one k1_bulk launch on the benchmark workload:
+# 12.03 B/element measured by ncu on the fc6 layer alone (1236.05 MB for 102,760,448 elements,
+# profiles/k1_bulk_fc6_25088x4096.md), scaled to the 139,754,605 elements of one launch here
+# (traffic is proportional to the elements streamed).  Set to None when k1_bulk changes.
+K1_TRAFFIC_BYTES = int(1236.05e6 * 139754605 / 102760448)
 
 
 def main():
@@ -348,6 +359,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--workload", choices=["vgg19", "fc6"], default="vgg19",
+                    help="vgg19: the benchmark; fc6: its largest layer alone, for profiler captures")
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "b200":
         args.warmup = 3
