@@ -224,8 +224,9 @@ int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_de
  *   dense[i] = dense[i] + scale * sent_w[i]   for w = 0 .. n_workers-1 in that order,
  * product then sum, each rounded to binary32 (scale = 1 gives the paper's plain sum).
  * idx_dev_host / val_dev_host / counts_dev_host: HOST arrays of n_workers DEVICE pointers
- * to payloads produced by rsdgc_compress() with this plan (or an identical one).
- * dense_dev: binary32 arena, in/out.  Tile indices outside a layer are skipped.
+ * to payloads produced by rsdgc_compress() with this plan (or an identical one): the tile
+ * indices of a layer must be ascending.  dense_dev: binary32 arena, in/out.  Entries whose tile
+ * index breaks that order or lies outside the layer are skipped.
  * Errors: INVALID, ALIGNMENT, CUDA.
  */
 int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,

@@ -1,98 +1,146 @@
-// Kernel of rsdgc_decompress_accumulate(): scatter-add of one worker's payload into the dense
-// gradient arena (Eq. 12 third line / Eq. 2 Sync).  One launch per worker; inside a launch
-// every dense element is touched by at most one thread, so plain read-modify-write is enough
-// and the order of the binary32 additions across workers is the launch order.
+// Kernel of rsdgc_decompress_accumulate(): scatter-add of several workers' payloads into the
+// dense gradient arena (Eq. 12 third line / Eq. 2 Sync).
+//
+// One launch handles up to kMaxWorkersPerLaunch workers.  A CTA owns one chunk of 16384
+// consecutive tile indices of one layer.  Every worker's index list is ascending inside a
+// layer (rsdgc_compress() writes it that way), so the entries of a worker that fall into the
+// chunk are one contiguous run, found with a 32-way search by one warp per worker.  The CTA
+// then applies the workers one after the other, with a barrier in between: every element of the
+// dense arena is only ever touched by the CTA that owns its tile, in worker order, with plain
+// read-modify-write, so the binary32 sums are reproducible (no atomics) although all workers
+// are processed by one launch.
 #include "device_utils.cuh"
 
 namespace rsdgc {
 
-__global__ void __launch_bounds__(kThreads)
-k_decompress(const int32_t *__restrict__ idx, const float *__restrict__ val,
-             const int32_t *__restrict__ counts, const LayerDev *__restrict__ layers, int n_layers,
-             float scale, float *__restrict__ dense)
+constexpr int kMaxWorkersPerLaunch = 16;
+constexpr int kScatterBatch = 4;  // independent entries in flight per thread
+
+struct WorkerPayloads {
+    const int32_t *idx[kMaxWorkersPerLaunch];
+    const float *val[kMaxWorkersPerLaunch];
+    const int32_t *counts[kMaxWorkersPerLaunch];
+    int n_workers;
+};
+
+struct DecompressShared {
+    long long idx_off[kMaxWorkersPerLaunch];  // payload offsets of the chunk's layer, per worker
+    long long val_off[kMaxWorkersPerLaunch];
+    int lo[kMaxWorkersPerLaunch], hi[kMaxWorkersPerLaunch];  // the worker's entries inside the chunk
+};
+
+// First position in a[0, n) whose value is >= key (a ascending); all 32 lanes of the warp take
+// part and return the same result.  Each step probes 32 positions, shrinking the range 33-fold.
+__device__ __forceinline__ int warp_lower_bound(const int32_t *a, int n, int key)
 {
-    // exclusive prefix sums over the layers of k_l * slot_l (values) and k_l (tiles)
-    __shared__ long long val_off[kMaxLayers + 1];
-    __shared__ long long idx_off[kMaxLayers + 1];
-    __shared__ unsigned long long scan_tmp[kThreads / 32];
-    const int tid = threadIdx.x;
-    unsigned long long carry_v = 0, carry_i = 0;
-    for (int base = 0; base < n_layers; base += kThreads) {
-        const int l = base + tid;
-        long long k = 0, kv = 0;
-        if (l < n_layers) {
-            k = counts[l];
-            if (k < 0) k = 0;
-            kv = k * layers[l].slot;
-        }
-        unsigned long long tv, ti;
-        const unsigned long long ev = block_exclusive_scan<unsigned long long>((unsigned long long)kv, scan_tmp, &tv);
-        const unsigned long long ei = block_exclusive_scan<unsigned long long>((unsigned long long)k, scan_tmp, &ti);
-        if (l < n_layers) {
-            val_off[l] = (long long)(carry_v + ev);
-            idx_off[l] = (long long)(carry_i + ei);
-        }
-        carry_v += tv;
-        carry_i += ti;
+    const int lane = threadIdx.x & 31;
+    int lo = 0, hi = n;  // answer in [lo, hi]
+    while (hi - lo > 0) {
+        const int span = hi - lo;
+        const int step = (span + 32) / 33;  // >= 1
+        const int pos = lo + (lane + 1) * step - 1;  // probe positions lo+step-1, lo+2step-1, ...
+        const bool below = (pos < hi) ? (__ldg(a + pos) < key) : false;  // a[pos] < key
+        const unsigned int m = __ballot_sync(0xFFFFFFFFu, below);
+        const int nb = __popc(m);  // ascending array: the lanes with a[pos] < key are a prefix
+        const int new_lo = lo + nb * step;
+        const int new_hi = (nb < 32) ? min(hi, lo + (nb + 1) * step - 1) : hi;
+        lo = min(new_lo, hi);
+        hi = max(new_hi, lo);
     }
-    if (tid == 0) {
-        val_off[n_layers] = (long long)carry_v;
-        idx_off[n_layers] = (long long)carry_i;
+    return lo;
+}
+
+__global__ void __launch_bounds__(kThreads)
+k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restrict__ layers,
+             const Chunk *__restrict__ chunks, float scale, float *__restrict__ dense)
+{
+    __shared__ DecompressShared sh;
+    const Chunk c = chunks[blockIdx.x];
+    const LayerDev L = layers[c.layer];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int W = wp.n_workers;
+
+    // ---- per worker (one warp each, round-robin): payload offsets of this layer = sums of the
+    // counts of the preceding layers, and the run of entries that falls into the chunk
+    for (int w = warp; w < W; w += kThreads / 32) {
+        long long si = 0, sv = 0;
+        for (int l = lane; l < c.layer; l += 32) {
+            long long k = wp.counts[w][l];
+            if (k < 0) k = 0;
+            si += k;
+            sv += k * layers[l].slot;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            si += __shfl_xor_sync(0xFFFFFFFFu, si, d);
+            sv += __shfl_xor_sync(0xFFFFFFFFu, sv, d);
+        }
+        int k = wp.counts[w][c.layer];
+        if (k < 0) k = 0;
+        const int32_t *a = wp.idx[w] + si;
+        const int lo = warp_lower_bound(a, k, c.start);
+        const int hi = lo + warp_lower_bound(a + lo, k - lo, c.start + c.n);
+        if (lane == 0) {
+            sh.idx_off[w] = si;
+            sh.val_off[w] = sv;
+            sh.lo[w] = lo;
+            sh.hi[w] = hi;
+        }
     }
     __syncthreads();
-    const long long total = val_off[n_layers];
 
-    constexpr int B = 4;  // independent entries per thread: index loads, then dense loads, then stores
-    const long long stride = (long long)gridDim.x * kThreads;
-    for (long long j0 = (long long)blockIdx.x * kThreads + tid; j0 < total; j0 += stride * B) {
-        long long ga[B];
-        float pv[B], dv[B];
-        int tile[B], lay[B], el[B];
+    const int slot = L.slot;
+    for (int w = 0; w < W; ++w) {
+        const int lo = sh.lo[w];
+        const int n_copy = (sh.hi[w] - lo) * slot;
+        const int32_t *idx = wp.idx[w] + sh.idx_off[w] + lo;
+        const float *val = wp.val[w] + sh.val_off[w] + (long long)lo * slot;
+        for (int j0 = 0; j0 < n_copy; j0 += kThreads * kScatterBatch) {
+            long long ga[kScatterBatch];
+            float pv[kScatterBatch], dv[kScatterBatch];
 #pragma unroll
-        for (int u = 0; u < B; ++u) {
-            const long long j = j0 + u * stride;
-            ga[u] = -1;
-            tile[u] = -1;
-            if (j < total) {
-                int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (val_off[mid] <= j) lo = mid; else hi = mid;
-                }
-                const int slot = layers[lo].slot;
-                const long long jl = j - val_off[lo];
-                const long long s = jl / slot;
-                lay[u] = lo;
-                el[u] = (int)(jl - s * slot);
-                tile[u] = __ldg(idx + idx_off[lo] + s);
-                pv[u] = __ldg(val + j);
-            }
-        }
-#pragma unroll
-        for (int u = 0; u < B; ++u) {
-            if (tile[u] >= 0) {
-                const LayerDev &L = layers[lay[u]];
-                if (tile[u] < L.K) {
-                    const int tr = tile[u] / L.TC, tc = tile[u] - tr * L.TC;
-                    const int a = el[u] / L.nw, b = el[u] - a * L.nw;
-                    const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
-                    if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+            for (int u = 0; u < kScatterBatch; ++u) {
+                const int j = j0 + u * kThreads + tid;
+                ga[u] = -1;
+                if (j < n_copy) {
+                    const int r = j / slot, el = j - r * slot;
+                    const int tile = __ldg(idx + r);
+                    pv[u] = __ldg(val + j);
+                    if (tile >= c.start && tile < c.start + c.n) {  // always true for ascending lists
+                        const int tr = tile / L.TC, tc = tile - tr * L.TC;
+                        const int a = el / L.nw, b = el - a * L.nw;
+                        const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
+                        if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+                    }
                 }
             }
+#pragma unroll
+            for (int u = 0; u < kScatterBatch; ++u) dv[u] = (ga[u] >= 0) ? dense[ga[u]] : 0.0f;
+#pragma unroll
+            for (int u = 0; u < kScatterBatch; ++u)
+                if (ga[u] >= 0) dense[ga[u]] = __fadd_rn(dv[u], __fmul_rn(scale, pv[u]));
         }
-#pragma unroll
-        for (int u = 0; u < B; ++u) dv[u] = (ga[u] >= 0) ? dense[ga[u]] : 0.0f;
-#pragma unroll
-        for (int u = 0; u < B; ++u)
-            if (ga[u] >= 0) dense[ga[u]] = __fadd_rn(dv[u], __fmul_rn(scale, pv[u]));
+        __syncthreads();  // the next worker may touch the same elements
     }
 }
 
-cudaError_t launch_decompress(rsdgc_plan *p, const int32_t *idx, const float *val, const int32_t *counts,
-                              float scale, float *dense, cudaStream_t s)
+// Applies workers [0, n_workers) in order; groups of kMaxWorkersPerLaunch go into one launch
+// each, and the stream orders the groups.
+cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const float *const *val,
+                              const int32_t *const *counts, float scale, float *dense, cudaStream_t s)
 {
-    k_decompress<<<p->n_sm * 8, kThreads, 0, s>>>(idx, val, counts, p->d_layers, p->n_layers, scale, dense);
-    count_launch(1);
+    const int n_chunks = (int)p->chunks.size();
+    for (int w0 = 0; w0 < n_workers; w0 += kMaxWorkersPerLaunch) {
+        WorkerPayloads wp{};
+        wp.n_workers = n_workers - w0 < kMaxWorkersPerLaunch ? n_workers - w0 : kMaxWorkersPerLaunch;
+        for (int w = 0; w < wp.n_workers; ++w) {
+            wp.idx[w] = idx[w0 + w];
+            wp.val[w] = val[w0 + w];
+            wp.counts[w] = counts[w0 + w];
+        }
+        k_decompress<<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense);
+        count_launch(1);
+    }
     return cudaGetLastError();
 }
 

@@ -502,10 +502,9 @@ extern "C" int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers, 
     }
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
-    // one launch per worker, in worker order: within a worker no two entries touch the same
-    // element, across workers the stream order fixes the order of the binary32 additions
-    for (int w = 0; w < n_workers; ++w) {
-        cudaError_t e = launch_decompress(plan, idx_dev_host[w], val_dev_host[w], counts_dev_host[w], scale,
+    // every dense element is updated by one CTA, worker after worker: reproducible binary32 sums
+    if (n_workers > 0) {
+        cudaError_t e = launch_decompress(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, scale,
                                           dense_dev, (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_fail(e);
     }
