@@ -127,8 +127,8 @@ struct CountShared {
 
 __global__ void __launch_bounds__(kThreads)
 k_count(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
-        const Chunk *__restrict__ chunks, LayerState *state, uint2 *chunk_cnt, int n_layers,
-        long long idx_cap, long long val_cap, StatusDev *status)
+        const Chunk *__restrict__ chunks, LayerState *state, uint2 *chunk_cnt, unsigned char *__restrict__ codes,
+        int n_layers, long long idx_cap, long long val_cap, StatusDev *status)
 {
     __shared__ CountShared sh;
     const Chunk c = chunks[blockIdx.x];
@@ -138,31 +138,37 @@ k_count(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     const uint32_t T = st.T;
     unsigned int gt = 0, eq = 0;
     {
+        // one code byte per 128-bit word of keys (bit c: key c above T, bit 4 + c: key c equal
+        // to T) is left for k_mark, which then needs no second look at the keys
         const uint32_t *kp = keys + L.tile_off + c.start;
+        unsigned char *cp = codes + ((L.tile_off + c.start) >> 2);
         const int nvec = c.n >> 2;
-        for (int base = 0; base < nvec; base += kThreads * kKeyVecBatch) {
+        const int nvec_all = (c.n + 3) >> 2;
+        for (int base = 0; base < nvec_all; base += kThreads * kKeyVecBatch) {
             uint4 q[kKeyVecBatch];
 #pragma unroll
             for (int u = 0; u < kKeyVecBatch; ++u) {
                 const int i = base + u * kThreads + tid;
                 q[u] = (i < nvec) ? __ldg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
             }
-            // the zero filler is neither above nor equal to T unless T == 0, in which case it
-            // would count as equal: mask it out explicitly
 #pragma unroll
             for (int u = 0; u < kKeyVecBatch; ++u) {
                 const int i = base + u * kThreads + tid;
+                if (i >= nvec_all) continue;
+                unsigned int code = 0;
                 if (i < nvec) {
-                    gt += (q[u].x > T) + (q[u].y > T) + (q[u].z > T) + (q[u].w > T);
-                    eq += (q[u].x == T) + (q[u].y == T) + (q[u].z == T) + (q[u].w == T);
+                    code = (q[u].x > T) | ((q[u].y > T) << 1) | ((q[u].z > T) << 2) | ((q[u].w > T) << 3) |
+                           ((q[u].x == T) << 4) | ((q[u].y == T) << 5) | ((q[u].z == T) << 6) | ((q[u].w == T) << 7);
+                } else {  // the last, partial word of the chunk
+                    for (int j = 0; j < (c.n & 3); ++j) {
+                        const uint32_t k1 = kp[(nvec << 2) + j];
+                        code |= ((k1 > T) << j) | ((k1 == T) << (4 + j));
+                    }
                 }
+                cp[i] = (unsigned char)code;
+                gt += __popc(code & 0x0Fu);
+                eq += __popc(code & 0xF0u);
             }
-        }
-        const int i = (nvec << 2) + tid;
-        if (i < c.n) {
-            const uint32_t q = kp[i];
-            gt += (q > T);
-            eq += (q == T);
         }
     }
 #pragma unroll
@@ -238,60 +244,43 @@ k_count(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
 // ------------------------------------------------------------------------------------------
 
 constexpr int kKeysPerThread = kChunkKeys / kThreads;  // 64 consecutive keys per thread
-constexpr int kChunkVecs = kChunkKeys / 4;             // 128-bit words of keys per chunk
 
 struct MarkShared {
-    // one byte per 128-bit word of keys: bit c = key c above T, bit 4 + c = key c equal to T
-    __align__(16) unsigned char code[kChunkVecs];
     unsigned long long scan_tmp[kThreads / 32];
 };
 
 __global__ void __launch_bounds__(kThreads)
-k_mark(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers, const Chunk *__restrict__ chunks,
-       const LayerState *__restrict__ state, const uint2 *__restrict__ chunk_cnt, int32_t *__restrict__ idx,
-       long long idx_cap)
+k_mark(const unsigned char *__restrict__ codes, const LayerDev *__restrict__ layers,
+       const Chunk *__restrict__ chunks, const LayerState *__restrict__ state,
+       const uint2 *__restrict__ chunk_cnt, int32_t *__restrict__ idx, long long idx_cap)
 {
     __shared__ MarkShared sh;
     const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x;
     const LayerState st = state[c.layer];
     if (st.k == 0) return;
-    const uint32_t T = st.T;
     const uint2 base = chunk_cnt[blockIdx.x];  // tiles above T / equal to T in earlier chunks
     // equal keys of this chunk that are still taken: those with layer-wide equal-rank < e
     const long long eq_room = max(0ll, (long long)st.e - (long long)base.y);
 
-    // ---- phase 1: coalesced read of the chunk's keys, 2 bits per key into shared memory
-    const uint32_t *kp = keys + layers[c.layer].tile_off + c.start;
-    const int nvec = c.n >> 2;
-    for (int b0 = 0; b0 < kChunkVecs; b0 += kThreads * kKeyVecBatch) {
-        uint4 q[kKeyVecBatch];
+    // ---- the code bytes k_count left: thread t owns keys [64 t, 64 t + 64) = 16 bytes; bytes
+    // beyond the chunk's last word belong to whatever follows in the array and are masked off
+    const unsigned char *cp = codes + ((layers[c.layer].tile_off + c.start) >> 2);
+    const int nvec_all = (c.n + 3) >> 2;
+    unsigned int w[4] = {0u, 0u, 0u, 0u};
+    if (tid * 16 < nvec_all) {
+        const uint4 cw = __ldg(reinterpret_cast<const uint4 *>(cp) + tid);
+        w[0] = cw.x, w[1] = cw.y, w[2] = cw.z, w[3] = cw.w;
+        const int valid = nvec_all - tid * 16;  // code bytes of this thread that are inside the chunk
+        if (valid < 16) {
 #pragma unroll
-        for (int u = 0; u < kKeyVecBatch; ++u) {
-            const int i = b0 + u * kThreads + tid;
-            q[u] = (i < nvec) ? __ldg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
-        }
-#pragma unroll
-        for (int u = 0; u < kKeyVecBatch; ++u) {
-            const int i = b0 + u * kThreads + tid;
-            unsigned int code = 0;
-            if (i < nvec) {
-                code = (q[u].x > T) | ((q[u].y > T) << 1) | ((q[u].z > T) << 2) | ((q[u].w > T) << 3) |
-                       ((q[u].x == T) << 4) | ((q[u].y == T) << 5) | ((q[u].z == T) << 6) | ((q[u].w == T) << 7);
-            } else if (i == nvec) {  // the last, partial word of the chunk
-                for (int j = 0; j < (c.n & 3); ++j) {
-                    const uint32_t k1 = kp[(nvec << 2) + j];
-                    code |= ((k1 > T) << j) | ((k1 == T) << (4 + j));
-                }
+            for (int j = 0; j < 4; ++j) {
+                const int vb = valid - 4 * j;  // valid bytes of word j
+                if (vb <= 0) w[j] = 0;
+                else if (vb < 4) w[j] &= (1u << (8 * vb)) - 1u;
             }
-            sh.code[i] = (unsigned char)code;
         }
     }
-    __syncthreads();
-
-    // ---- phase 2: ranks.  Thread t owns keys [64 t, 64 t + 64) = 16 code bytes.
-    const uint4 cw = reinterpret_cast<const uint4 *>(sh.code)[tid];
-    const unsigned int w[4] = {cw.x, cw.y, cw.z, cw.w};
     unsigned int gt = 0, eq = 0;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
@@ -434,10 +423,11 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, cons
     RSDGC_MARK();
     k_refine<3><<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
     RSDGC_MARK();
-    k_count<<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt,
+    k_count<<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, p->d_codes,
                                           p->n_layers, idx_cap, val_cap, p->d_status);
     RSDGC_MARK();
-    k_mark<<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, idx, idx_cap);
+    k_mark<<<n_chunks, kThreads, 0, s>>>(p->d_codes, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, idx,
+                                         idx_cap);
     RSDGC_MARK();
     k_gather<<<p->n_sm * 8, kThreads, 0, s>>>(resid, p->d_layers, p->d_state, p->n_layers, idx, idx_cap, val,
                                               val_cap);

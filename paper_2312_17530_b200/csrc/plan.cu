@@ -72,6 +72,7 @@ void free_device_tables(rsdgc_plan *p)
     cudaFree(p->d_state);
     cudaFree(p->d_hist);
     cudaFree(p->d_chunk_cnt);
+    cudaFree(p->d_codes);
     cudaFree(p->d_survivors);
     cudaFree(p->d_rstate);
     cudaFree(p->d_status);
@@ -314,6 +315,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         if (e == cudaSuccess) e = alloc_zero(&p->d_state, (size_t)n_layers);
         if (e == cudaSuccess) e = alloc_zero(&p->d_hist, (size_t)n_layers * kHistStride);
         if (e == cudaSuccess) e = alloc_zero(&p->d_chunk_cnt, p->chunks.size());
+        if (e == cudaSuccess) e = alloc_zero(&p->d_codes, (size_t)p->info.total_tiles_padded / 4 + kChunkKeys / 4 + 16);
         if (e == cudaSuccess) e = alloc_zero(&p->d_survivors, (size_t)n_layers);
         if (e == cudaSuccess) e = alloc_zero(&p->d_rstate, 1);
         if (e == cudaSuccess) e = alloc_zero(&p->d_status, 1);

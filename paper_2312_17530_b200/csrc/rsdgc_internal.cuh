@@ -139,6 +139,7 @@ struct rsdgc_plan {
     rsdgc::EChunk *d_echunks = nullptr;
     rsdgc::LayerState *d_state = nullptr;
     uint32_t *d_hist = nullptr;        // n_layers * kHistStride
+    unsigned char *d_codes = nullptr;  // one byte per 4 tiles: above / equal flags left by k_count for k_mark
     uint2 *d_chunk_cnt = nullptr;      // per key chunk: (#key > T, #key == T), then exclusive bases
     long long *d_survivors = nullptr;  // ratio rule: per-layer survivor counts
     rsdgc::RatioState *d_rstate = nullptr;
