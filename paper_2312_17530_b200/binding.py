@@ -200,8 +200,9 @@ class Plan:
         _check(lib().rsdgc_decompress_accumulate(self._h, n, ia, va, ca, scale, _ptr(dense), _stream()),
                "rsdgc_decompress_accumulate")
 
-    def profile_enable(self, on: bool) -> None:
-        _check(lib().rsdgc_profile_enable(self._h, 1 if on else 0), "rsdgc_profile_enable")
+    def profile_enable(self, level: int) -> None:
+        """0 off; 1 events around the first pass only; 2 events around every kernel."""
+        _check(lib().rsdgc_profile_enable(self._h, int(level)), "rsdgc_profile_enable")
 
     def profile_read(self):
         """(milliseconds summed per compress kernel, number of compress calls recorded)."""

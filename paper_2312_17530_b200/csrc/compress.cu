@@ -39,8 +39,10 @@ k_refine(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x;
     LayerState &st = state[c.layer];
-    const uint32_t prefix = st.prefix;
     for (int b = tid; b < NBINS; b += kThreads) sh.hist[b] = 0;
+    grid_dependency_wait();
+    grid_dependency_launch_next();
+    const uint32_t prefix = st.prefix;
     __syncthreads();
     if (prefix != kTakeNone) {
         const uint32_t *kp = keys + layers[c.layer].tile_off + c.start;
@@ -135,6 +137,8 @@ k_count(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     LayerState &st = state[c.layer];
     const LayerDev &L = layers[c.layer];
+    grid_dependency_wait();
+    grid_dependency_launch_next();
     const uint32_t T = st.T;
     unsigned int gt = 0, eq = 0;
     {
@@ -257,6 +261,8 @@ k_mark(const unsigned char *__restrict__ codes, const LayerDev *__restrict__ lay
     __shared__ MarkShared sh;
     const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x;
+    grid_dependency_wait();
+    grid_dependency_launch_next();
     const LayerState st = state[c.layer];
     if (st.k == 0) return;
     const uint2 base = chunk_cnt[blockIdx.x];  // tiles above T / equal to T in earlier chunks
@@ -334,6 +340,7 @@ k_gather(float *__restrict__ resid, const LayerDev *__restrict__ layers, const L
     __shared__ long long val_off[kMaxLayers + 1];
     __shared__ long long idx_off[kMaxLayers];
     const int tid = threadIdx.x;
+    grid_dependency_wait();
     for (int l = tid; l < n_layers; l += kThreads) {
         val_off[l] = state[l].val_off;
         idx_off[l] = state[l].idx_off;
@@ -407,31 +414,56 @@ static cudaError_t record_event(rsdgc_plan *p, cudaStream_t s)
     return cudaEventRecord(p->events[p->events_used++], s);
 }
 
+// Launch with the programmatic-stream-serialization attribute: the kernel may be scheduled
+// while its predecessor drains; it calls grid_dependency_wait() before touching that kernel's
+// results.
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_chained(void (*kernel)(KArgs...), int grid, cudaStream_t s, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, const float *ratios, int32_t *idx,
                             int64_t idx_cap, float *val, int64_t val_cap, int32_t *counts, uint32_t *keys,
                             cudaStream_t s)
 {
     const int n_chunks = (int)p->chunks.size();
-    const bool prof = p->profile;
+    const int prof = p->profile;
     cudaError_t e = cudaSuccess;
-#define RSDGC_MARK()                                   \
-    if (prof && e == cudaSuccess) e = record_event(p, s)
-    RSDGC_MARK();
+#define RSDGC_MARK(level)                              \
+    if (prof >= (level) && e == cudaSuccess) e = record_event(p, s)
+    if (prof) p->profile_recorded = prof;
+    RSDGC_MARK(1);
     launch_accumulate_nsi(p, grads, resid, ratios, counts, keys, s);
-    RSDGC_MARK();
-    k_refine<2><<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
-    RSDGC_MARK();
-    k_refine<3><<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
-    RSDGC_MARK();
-    k_count<<<n_chunks, kThreads, 0, s>>>(keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, p->d_codes,
-                                          p->n_layers, idx_cap, val_cap, p->d_status);
-    RSDGC_MARK();
-    k_mark<<<n_chunks, kThreads, 0, s>>>(p->d_codes, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, idx,
-                                         idx_cap);
-    RSDGC_MARK();
-    k_gather<<<p->n_sm * 8, kThreads, 0, s>>>(resid, p->d_layers, p->d_state, p->n_layers, idx, idx_cap, val,
-                                              val_cap);
-    RSDGC_MARK();
+    RSDGC_MARK(1);
+    if (e == cudaSuccess)
+        e = launch_chained(k_refine<2>, n_chunks, s, keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
+    RSDGC_MARK(2);
+    if (e == cudaSuccess)
+        e = launch_chained(k_refine<3>, n_chunks, s, keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
+    RSDGC_MARK(2);
+    if (e == cudaSuccess)
+        e = launch_chained(k_count, n_chunks, s, keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt,
+                           p->d_codes, p->n_layers, (long long)idx_cap, (long long)val_cap, p->d_status);
+    RSDGC_MARK(2);
+    if (e == cudaSuccess)
+        e = launch_chained(k_mark, n_chunks, s, p->d_codes, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, idx,
+                           (long long)idx_cap);
+    RSDGC_MARK(2);
+    if (e == cudaSuccess)
+        e = launch_chained(k_gather, p->n_sm * 8, s, resid, p->d_layers, p->d_state, p->n_layers, idx,
+                           (long long)idx_cap, val, (long long)val_cap);
+    RSDGC_MARK(2);
 #undef RSDGC_MARK
     count_launch(5);
     if (e != cudaSuccess) return e;

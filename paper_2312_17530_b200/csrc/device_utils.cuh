@@ -68,6 +68,18 @@ __device__ __forceinline__ void find_bin_from_top(const unsigned int *h, unsigne
     __syncthreads();
 }
 
+// Programmatic dependent launch: a kernel launched with the "programmatic stream
+// serialization" attribute may start while its predecessor in the stream is still draining.
+// grid_dependency_wait() returns once the predecessor has completed and its writes are visible;
+// everything before it may only touch data that no earlier kernel of the same call writes
+// (plan tables, shared memory).  grid_dependency_launch_next() lets the successor start; it is
+// called after the wait so that completion stays transitive along the chain of kernels.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dependency_launch_next()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 // floor(x / d) for x < 8192 and d <= 8192 by a multiply-high with inv = ceil(2^32 / d)
 // (inv = 0 encodes d = 1).
 __device__ __forceinline__ int fast_div(int x, unsigned int inv)

@@ -534,11 +534,14 @@ extern "C" int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *ou
     return RSDGC_OK;
 }
 
-extern "C" int rsdgc_profile_enable(rsdgc_plan *plan, int32_t enable)
+extern "C" int rsdgc_profile_enable(rsdgc_plan *plan, int32_t level)
 {
     int rc = check_plan_device(plan);
     if (rc) return rc;
-    plan->profile = enable != 0;
+    if (level < 0 || level > 2) return RSDGC_ERR_INVALID;
+    if (plan->events_used && level != plan->profile_recorded && level != 0)
+        return RSDGC_ERR_INVALID;  // read the recorded calls before switching level
+    plan->profile = level;
     return RSDGC_OK;
 }
 
@@ -547,7 +550,8 @@ extern "C" int rsdgc_profile_read(rsdgc_plan *plan, double *ms_per_kernel_host, 
     int rc = check_plan_device(plan);
     if (rc) return rc;
     if (!ms_per_kernel_host || !n_calls_host) return RSDGC_ERR_INVALID;
-    constexpr size_t per_call = RSDGC_N_COMPRESS_KERNELS + 1;
+    const size_t stages = plan->profile_recorded == 2 ? RSDGC_N_COMPRESS_KERNELS : 1;
+    const size_t per_call = stages + 1;
     const size_t n_calls = plan->events_used / per_call;
     for (int k = 0; k < RSDGC_N_COMPRESS_KERNELS; ++k) ms_per_kernel_host[k] = 0.0;
     DeviceGuard guard(plan->device);
@@ -555,7 +559,7 @@ extern "C" int rsdgc_profile_read(rsdgc_plan *plan, double *ms_per_kernel_host, 
     for (size_t c = 0; c < n_calls; ++c) {
         const cudaEvent_t *ev = plan->events.data() + c * per_call;
         cudaError_t e = cudaEventSynchronize(ev[per_call - 1]);
-        for (int k = 0; k < RSDGC_N_COMPRESS_KERNELS && e == cudaSuccess; ++k) {
+        for (size_t k = 0; k < stages && e == cudaSuccess; ++k) {
             float ms = 0.0f;
             e = cudaEventElapsedTime(&ms, ev[k], ev[k + 1]);
             ms_per_kernel_host[k] += ms;

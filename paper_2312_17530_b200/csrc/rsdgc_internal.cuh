@@ -146,8 +146,9 @@ struct rsdgc_plan {
     rsdgc::StatusDev *d_status = nullptr;
 
     // optional per-kernel timing of compress calls
-    bool profile = false;
-    std::vector<cudaEvent_t> events;  // pool; (RSDGC_N_COMPRESS_KERNELS + 1) per recorded call
+    int profile = 0;                  // 0 off, 1 first pass only, 2 every stage
+    int profile_recorded = 0;         // level of the calls recorded since the last read
+    std::vector<cudaEvent_t> events;  // pool; 2 (level 1) or RSDGC_N_COMPRESS_KERNELS + 1 (level 2) per call
     size_t events_used = 0;
 };
 
