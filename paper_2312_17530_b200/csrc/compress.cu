@@ -351,26 +351,36 @@ k_gather(float *__restrict__ resid, const LayerDev *__restrict__ layers, const L
     }
     __syncthreads();
     const long long total = val_off[n_layers];
-    const long long stride = (long long)gridDim.x * kThreads;
-    for (long long j0 = (long long)blockIdx.x * kThreads + tid; j0 < total; j0 += stride * kCopyBatch) {
+    // a CTA takes blocks of kThreads * kCopyBatch consecutive payload values: almost always one
+    // layer per block, so the layer search is done once per block, not once per value
+    constexpr long long kBlock = (long long)kThreads * kCopyBatch;
+    auto find_layer = [&](long long j) {
+        int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (val_off[mid] <= j) lo = mid; else hi = mid;
+        }
+        return lo;
+    };
+    for (long long jb = (long long)blockIdx.x * kBlock; jb < total; jb += (long long)gridDim.x * kBlock) {
+        const long long jend = min(total, jb + kBlock) - 1;
+        const int l_first = find_layer(jb);
+        const bool one_layer = val_off[l_first + 1] > jend;
         long long ga[kCopyBatch], vo[kCopyBatch];
         int tile[kCopyBatch], lay[kCopyBatch], el[kCopyBatch];
         float xv[kCopyBatch];
 #pragma unroll
         for (int u = 0; u < kCopyBatch; ++u) {
-            const long long j = j0 + u * stride;
+            const long long j = jb + u * kThreads + tid;
             ga[u] = -1;
             vo[u] = -1;
             tile[u] = -1;
             if (j < total) {
-                int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (val_off[mid] <= j) lo = mid; else hi = mid;
-                }
+                const int lo = one_layer ? l_first : find_layer(j);
                 const int slot = layers[lo].slot;
                 const long long jl = j - val_off[lo];
-                const long long s = jl / slot;
+                // 32-bit division whenever the layer's payload is below 2^31 values (the usual case)
+                const long long s = (jl < 0x7FFFFFFFll) ? (long long)((int)jl / slot) : jl / slot;
                 lay[u] = lo;
                 el[u] = (int)(jl - s * slot);
                 // tiles that do not fit the payload buffers are not sent and stay in the residual
