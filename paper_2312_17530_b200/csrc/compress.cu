@@ -331,7 +331,10 @@ k_mark(const unsigned char *__restrict__ codes, const LayerDev *__restrict__ lay
 // independent entries in flight per thread.
 // ------------------------------------------------------------------------------------------
 
-constexpr int kCopyBatch = 8;
+#ifndef RSDGC_COPY_BATCH
+#define RSDGC_COPY_BATCH 8
+#endif
+constexpr int kCopyBatch = RSDGC_COPY_BATCH;
 
 __global__ void __launch_bounds__(kThreads)
 k_gather(float *__restrict__ resid, const LayerDev *__restrict__ layers, const LayerState *__restrict__ state,
@@ -380,9 +383,17 @@ k_gather(float *__restrict__ resid, const LayerDev *__restrict__ layers, const L
                 const int slot = layers[lo].slot;
                 const long long jl = j - val_off[lo];
                 // 32-bit division whenever the layer's payload is below 2^31 values (the usual case)
-                const long long s = (jl < 0x7FFFFFFFll) ? (long long)((int)jl / slot) : jl / slot;
+                long long s;
+                if (jl < 0x7FFFFFFFll) {
+                    int q, r;
+                    divmod_small((int)jl, slot, &q, &r);
+                    s = q;
+                    el[u] = r;
+                } else {
+                    s = jl / slot;
+                    el[u] = (int)(jl - s * slot);
+                }
                 lay[u] = lo;
-                el[u] = (int)(jl - s * slot);
                 // tiles that do not fit the payload buffers are not sent and stay in the residual
                 if (idx_off[lo] + s < idx_cap && val_off[lo] + (s + 1) * slot <= val_cap) {
                     tile[u] = __ldg(idx + idx_off[lo] + s);
@@ -395,13 +406,14 @@ k_gather(float *__restrict__ resid, const LayerDev *__restrict__ layers, const L
             if (tile[u] >= 0) {
                 const LayerDev &L = layers[lay[u]];
                 const int tr = tile[u] / L.TC, tc = tile[u] - tr * L.TC;
-                const int a = el[u] / L.nw, b = el[u] - a * L.nw;
+                int a, b;
+                divmod_small(el[u], L.nw, &a, &b);
                 const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
                 if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
             }
         }
 #pragma unroll
-        for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? __ldcs(resid + ga[u]) : 0.0f;
+        for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
 #pragma unroll
         for (int u = 0; u < kCopyBatch; ++u) {
             if (ga[u] >= 0) resid[ga[u]] = 0.0f;

@@ -14,7 +14,7 @@
 namespace rsdgc {
 
 constexpr int kMaxWorkersPerLaunch = 16;
-constexpr int kScatterBatch = 4;  // independent entries in flight per thread
+constexpr int kScatterBatch = 8;  // independent entries in flight per thread
 
 struct WorkerPayloads {
     const int32_t *idx[kMaxWorkersPerLaunch];
@@ -103,12 +103,14 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
                 const int j = j0 + u * kThreads + tid;
                 ga[u] = -1;
                 if (j < n_copy) {
-                    const int r = j / slot, el = j - r * slot;
+                    int r, el;
+                    divmod_small(j, slot, &r, &el);
                     const int tile = __ldg(idx + r);
                     pv[u] = __ldg(val + j);
                     if (tile >= c.start && tile < c.start + c.n) {  // always true for ascending lists
                         const int tr = tile / L.TC, tc = tile - tr * L.TC;
-                        const int a = el / L.nw, b = el - a * L.nw;
+                        int a, b;
+                        divmod_small(el, L.nw, &a, &b);
                         const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
                         if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
                     }

@@ -87,6 +87,19 @@ __device__ __forceinline__ int fast_div(int x, unsigned int inv)
     return inv ? (int)__umulhi((unsigned int)x, inv) : x;
 }
 
+// x / d and x % d for 0 <= x < 2^31, d >= 1, with the common divisors (3, 9) as compile-time
+// constants (multiply + shift instead of the generic division sequence).
+__device__ __forceinline__ void divmod_small(int x, int d, int *q, int *r)
+{
+    int qq;
+    if (d == 9) qq = x / 9;
+    else if (d == 3) qq = x / 3;
+    else if (d == 1) qq = x;
+    else qq = x / d;
+    *q = qq;
+    *r = x - qq * d;
+}
+
 // Number of tiles to keep, k = ceil(K * ratio) (Eq. 11) limited to [0 or 1, K]; the product
 // is taken in binary64 on the binary32 ratio.
 __device__ __forceinline__ int keep_count(int K, float ratio, unsigned int flags)
