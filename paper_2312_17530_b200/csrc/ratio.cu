@@ -35,13 +35,26 @@ k_ratio_level(const float *__restrict__ weights, const LayerDev *__restrict__ la
     if (prefix != kTakeNone) {
         const uint32_t *wp = reinterpret_cast<const uint32_t *>(weights) + layers[c.layer].elem_off + c.start;
         const int nvec = c.n >> 2;  // layer starts and chunk starts are multiples of 4 elements
-        for (int i = tid; i < nvec; i += kThreads) {
-            uint4 q = __ldcs(reinterpret_cast<const uint4 *>(wp) + i);
-            q.x &= 0x7FFFFFFFu, q.y &= 0x7FFFFFFFu, q.z &= 0x7FFFFFFFu, q.w &= 0x7FFFFFFFu;
-            if ((q.x >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q.x >> SHIFT_LO) & (NBINS - 1)], 1u);
-            if ((q.y >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q.y >> SHIFT_LO) & (NBINS - 1)], 1u);
-            if ((q.z >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q.z >> SHIFT_LO) & (NBINS - 1)], 1u);
-            if ((q.w >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q.w >> SHIFT_LO) & (NBINS - 1)], 1u);
+        constexpr int BATCH = 8;
+        for (int base = 0; base < nvec; base += kThreads * BATCH) {
+            uint4 q[BATCH];  // all loads of a batch are issued before any is consumed
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                const int i = base + u * kThreads + tid;
+                q[u] = (i < nvec) ? __ldcs(reinterpret_cast<const uint4 *>(wp) + i) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < BATCH; ++u) {
+                const int i = base + u * kThreads + tid;
+                if (i < nvec) {
+                    const uint32_t k0 = q[u].x & 0x7FFFFFFFu, k1 = q[u].y & 0x7FFFFFFFu;
+                    const uint32_t k2 = q[u].z & 0x7FFFFFFFu, k3 = q[u].w & 0x7FFFFFFFu;
+                    if ((k0 >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(k0 >> SHIFT_LO) & (NBINS - 1)], 1u);
+                    if ((k1 >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(k1 >> SHIFT_LO) & (NBINS - 1)], 1u);
+                    if ((k2 >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(k2 >> SHIFT_LO) & (NBINS - 1)], 1u);
+                    if ((k3 >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(k3 >> SHIFT_LO) & (NBINS - 1)], 1u);
+                }
+            }
         }
         const int i = (nvec << 2) + tid;
         if (i < c.n) {
@@ -65,8 +78,7 @@ k_ratio_level(const float *__restrict__ weights, const LayerDev *__restrict__ la
     if (!sh.is_last) return;
     __threadfence();
 
-    // ---- last CTA: histogram summed over the layers (counts of one bin fit 32 bits per
-    // layer; the sum over layers is clamped to 32 bits only if it cannot matter: see below)
+    // ---- last CTA: histogram summed over the layers in 64 bits (Eq. 4 ranks across the whole network)
     const long long remaining = (LEVEL == 1) ? n_keep : rs->remaining;
     const bool active = (LEVEL == 1) ? (n_keep > 0) : (prefix != kTakeNone);
     unsigned long long gsum[NBINS / kThreads];

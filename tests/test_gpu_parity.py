@@ -238,3 +238,54 @@ def test_repeated_runs_are_bit_identical(oracle):
         np.testing.assert_array_equal(a.view(np.uint32), b.view(np.uint32))
     for a, b in zip(outs[0], outs[2]):
         np.testing.assert_array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_compress_and_aggregate_replay_from_a_cuda_graph(oracle):
+    """The whole per-iteration sequence is stream-ordered and reads nothing on the host, so it can
+    be captured once and replayed: three replays on fresh gradients match the oracle."""
+    tensors = synth.resnet18_tensors()[:30]
+    shapes = synth.layer_shapes(tensors)
+    plan = binding.Plan(shapes, alpha=0.5)
+    ratio = 1 / 32
+    ni, nv = plan.payload_bound(ratio)
+    dev = "cuda:0"
+    d_g = torch.zeros(plan.info.arena_elems, device=dev)
+    d_r = torch.zeros(plan.info.arena_elems, device=dev)
+    d_dense = torch.zeros(plan.info.arena_elems, device=dev)
+    idx = torch.zeros(ni, dtype=torch.int32, device=dev)
+    val = torch.zeros(nv, device=dev)
+    cnt = torch.zeros(len(shapes), dtype=torch.int32, device=dev)
+    ws = torch.empty(plan.info.workspace_bytes, dtype=torch.uint8, device=dev)
+    ratios = torch.full((len(shapes),), ratio, device=dev)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        plan.compress(d_g, d_r, ratios, idx, val, cnt, workspace=ws)      # warm-up outside the capture
+        plan.decompress_accumulate([(idx, val, cnt)], d_dense, 1.0)
+    side.synchronize()
+    d_r.zero_()
+    d_dense.zero_()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        plan.compress(d_g, d_r, ratios, idx, val, cnt, workspace=ws)
+        plan.decompress_accumulate([(idx, val, cnt)], d_dense, 1.0)
+    scales = synth.log_uniform_scales(len(tensors), (11,))
+    res = [np.zeros(synth.numel(s), np.float32) for _, s in tensors]
+    dense_ref = [np.zeros(synth.numel(s), np.float32) for _, s in tensors]
+    d_r.zero_()
+    d_dense.zero_()
+    for it in range(3):
+        g = synth.laplace_layers(tensors, (11, it), scales)
+        d_g.copy_(torch.from_numpy(parity.to_arena(plan, g, fill=0.0)))
+        graph.replay()
+        torch.cuda.synchronize()
+        ref = oracle.compress(shapes, g, res, [ratio] * len(shapes), 0.5)
+        oracle.decompress_accumulate(shapes, dense_ref, [ref], 1.0)
+        res = [l.residual for l in ref.layers]
+        k = int(ref.counts.sum())
+        np.testing.assert_array_equal(cnt.cpu().numpy(), ref.counts)
+        np.testing.assert_array_equal(idx.cpu().numpy()[:k], np.concatenate([l.idx for l in ref.layers]))
+        for got, want in zip(parity.from_arena(plan, d_r.cpu().numpy()), res):
+            np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+        for got, want in zip(parity.from_arena(plan, d_dense.cpu().numpy()), dense_ref):
+            np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert plan.status().flags == 0
