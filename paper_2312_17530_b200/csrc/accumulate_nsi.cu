@@ -234,23 +234,26 @@ __device__ void k1_flush_layer(unsigned int *hist_smem, FlushShared &fs, int lay
 {
     __syncthreads();
     unsigned int *gh = hist + (size_t)layer * kHistStride;
-    for (int b = threadIdx.x; b < kL1Bins; b += NTHREADS) {
-        const unsigned int c = hist_smem[b];
-        if (c) {
-            atomicAdd(gh + b, c);
-            hist_smem[b] = 0;
+    const bool sole_owner = layers[layer].n_flush1 == 1;  // the whole layer went through this CTA
+    if (!sole_owner) {
+        for (int b = threadIdx.x; b < kL1Bins; b += NTHREADS) {
+            const unsigned int c = hist_smem[b];
+            if (c) {
+                atomicAdd(gh + b, c);
+                hist_smem[b] = 0;
+            }
         }
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            const unsigned int t = atomicAdd(&state[layer].ticket[0], 1u);
+            fs.is_last = (t + 1u == (unsigned int)layers[layer].n_flush1);
+        }
+        __syncthreads();
+        if (!fs.is_last) return;  // uniform for the CTA
+        __threadfence();
     }
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const unsigned int t = atomicAdd(&state[layer].ticket[0], 1u);
-        fs.is_last = (t + 1u == (unsigned int)layers[layer].n_flush1);
-    }
-    __syncthreads();
-    if (!fs.is_last) return;  // uniform for the CTA
-    __threadfence();
-    {
+    if (!sole_owner) {  // otherwise the shared-memory histogram already is the layer's histogram
         unsigned int h[kL1Bins / NTHREADS];
 #pragma unroll
         for (int j = 0; j < kL1Bins / NTHREADS; ++j) h[j] = __ldcg(gh + j * NTHREADS + threadIdx.x);
@@ -269,7 +272,7 @@ __device__ void k1_flush_layer(unsigned int *hist_smem, FlushShared &fs, int lay
         st.k = k;
         st.prefix = k > 0 ? (uint32_t)fs.found[0] : kTakeNone;
         st.remaining = k > 0 ? (int32_t)fs.found[1] : 0;
-        st.ticket[0] = 0;
+        if (!sole_owner) st.ticket[0] = 0;
         counts[layer] = k;
     }
     __syncthreads();
