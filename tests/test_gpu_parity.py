@@ -289,3 +289,41 @@ def test_compress_and_aggregate_replay_from_a_cuda_graph(oracle):
         for got, want in zip(parity.from_arena(plan, d_dense.cpu().numpy()), dense_ref):
             np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
     assert plan.status().flags == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# the ablation rows of Table I as settings of the same path: "Neighbor" only (alpha = 1), no
+# "Dynamic" (one fixed ratio), and plain Top-k as the 1x1-neighborhood special case
+# ---------------------------------------------------------------------------------------------
+
+def test_topk_special_case_matches_library_topk(oracle):
+    rows, cols = 700, 1031
+    rng = np.random.default_rng(12)
+    g = rng.standard_normal(rows * cols).astype(np.float32)
+    r = (rng.standard_normal(rows * cols) * 0.1).astype(np.float32)
+    shapes = [(rows, cols, 1, 1)]
+    plan = binding.Plan(shapes, alpha=1.0)
+    ratio = 0.01
+    _, refs, gc = parity.compress_and_check(oracle, plan, shapes, [g], [r], [ratio], 1.0, max_ratio=ratio, what="top-k")
+    v = torch.from_numpy(g) + torch.from_numpy(r)
+    k = refs[0].k
+    top = torch.topk(v.abs(), k).indices.numpy()
+    got = gc.idx.cpu().numpy()[:k]
+    av = np.abs(v.numpy())
+    # the kept magnitudes are exactly the k largest; where the k-th magnitude is not tied the index
+    # sets coincide as well
+    np.testing.assert_array_equal(np.sort(av[got]), np.sort(av[top]))
+    if (av == av[top].min()).sum() == 1:
+        np.testing.assert_array_equal(got, np.sort(top))
+    np.testing.assert_array_equal(gc.val.cpu().numpy()[:k], v.numpy()[got])
+
+
+@pytest.mark.parametrize("alpha,shape", [(1.0, (640, 1152, 3, 3)), (0.0, (640, 1152, 3, 3)), (0.5, (192, 49, 1, 49)),
+                                         (0.5, (448, 21, 7, 7)), (1.0, (448, 21, 7, 7))])
+def test_ablation_variants_and_other_neighborhood_shapes(oracle, alpha, shape):
+    rows, cols = shape[0], shape[1]
+    rng = np.random.default_rng(13)
+    g = (rng.standard_normal(rows * cols) * 1e-2).astype(np.float32)
+    r = (rng.standard_normal(rows * cols) * 1e-2).astype(np.float32)
+    plan = binding.Plan([shape], alpha=alpha)
+    parity.compress_and_check(oracle, plan, [shape], [g], [r], [0.001], alpha, what="variant alpha=%g %r" % (alpha, shape))
