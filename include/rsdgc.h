@@ -60,6 +60,7 @@ typedef enum {
 /* plan flags */
 #define RSDGC_KEEP_AT_LEAST_ONE 1u /* k_l = max(1, ceil(K_l * ratio_l)): every layer sends >= 1 tile */
 #define RSDGC_NO_BULK_COPY 2u      /* first pass: register-staged kernel for every item           */
+#define RSDGC_MOMENTUM 4u          /* the plan is used with rsdgc_compress_momentum() (Eq. 12 l.1) */
 
 /* bits of rsdgc_status.flags */
 #define RSDGC_STATUS_NONFINITE 1u         /* some indicator was NaN/Inf (ranked first as +Inf)  */
@@ -103,7 +104,7 @@ typedef struct {
  * Builds the plan for a set of layers (Algorithm 1's loop over l = 1..L with the
  * neighborhoods of Eq. 7): arena offsets, tile counts, the work lists the kernels walk and
  * the per-layer device tables.  `alpha` is the hyper-parameter of Eq. 8 (0 <= alpha <= 1).
- * `flags`: an OR of RSDGC_KEEP_AT_LEAST_ONE and RSDGC_NO_BULK_COPY, or 0.  `device` is the CUDA device ordinal.  On success
+ * `flags`: an OR of RSDGC_KEEP_AT_LEAST_ONE, RSDGC_NO_BULK_COPY and RSDGC_MOMENTUM, or 0.  `device` is the CUDA device ordinal.  On success
  * *out owns host memory and a few MB of device memory until rsdgc_plan_destroy().
  * Errors: INVALID (null, n_layers < 1, rows/cols/nh/nw < 1, alpha outside [0,1] or NaN,
  * unknown dtype), CAPACITY (a layer with more than 2^31-1 tiles or nh*nw > 4096),
@@ -202,6 +203,21 @@ int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *residual_dev,
                    const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity,
                    float *val_dev, int64_t val_capacity, int32_t *counts_dev, float *nsi_dev,
                    void *workspace_dev, void *stream);
+
+/*
+ * The same step with momentum correction ahead of the accumulation (Eq. 12, first and second
+ * line): u = momentum * u + g (product then sum, each rounded to binary32), v = r + u; the
+ * rest is rsdgc_compress().  velocity_dev: binary32 arena with the plan's layout, in: u of the
+ * previous iteration (zeros at the start), out: the new u; it is not masked where tiles are
+ * sent (Eq. 12 does not say so).  The plan must have been created with RSDGC_MOMENTUM, which
+ * sizes the first pass for the third stream (20 instead of 12 bytes per element); such a plan
+ * is not accepted by rsdgc_compress().  momentum in [0, 1]; 0 reproduces rsdgc_compress().
+ * Errors: INVALID, ALIGNMENT, CUDA.
+ */
+int rsdgc_compress_momentum(rsdgc_plan *plan, const void *grads_dev, float *velocity_dev, float momentum,
+                            float *residual_dev, const float *ratios_dev, int32_t *idx_dev,
+                            int64_t idx_capacity, float *val_dev, int64_t val_capacity, int32_t *counts_dev,
+                            float *nsi_dev, void *workspace_dev, void *stream);
 
 /*
  * Same step with the gradient and the payload in HOST memory: copies grads_host into

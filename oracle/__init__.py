@@ -60,6 +60,10 @@ def lib():
         L.rsdgc_oracle_accumulate_f32.argtypes = [p, p, p, i64]
         L.rsdgc_oracle_accumulate_bf16.restype = None
         L.rsdgc_oracle_accumulate_bf16.argtypes = [p, p, p, i64]
+        L.rsdgc_oracle_accumulate_momentum_f32.restype = None
+        L.rsdgc_oracle_accumulate_momentum_f32.argtypes = [p, p, p, p, f32, i64]
+        L.rsdgc_oracle_accumulate_momentum_bf16.restype = None
+        L.rsdgc_oracle_accumulate_momentum_bf16.argtypes = [p, p, p, p, f32, i64]
         L.rsdgc_oracle_nsi.restype = i64
         L.rsdgc_oracle_nsi.argtypes = [p, i64, i64, i32, i32, f32, p, p]
         L.rsdgc_oracle_keep_count.restype = i64
@@ -105,6 +109,22 @@ def accumulate(g: np.ndarray, r: np.ndarray) -> np.ndarray:
         assert g.size == r.size
         lib().rsdgc_oracle_accumulate_f32(_ptr(g), _ptr(r), _ptr(v), r.size)
     return v
+
+
+def accumulate_momentum(g: np.ndarray, u: np.ndarray, r: np.ndarray, m: float):
+    """(u_new, v) with u_new = m*u + g and v = r + u_new (Eq. 12, first and second line)."""
+    r = _f32(r)
+    u_new = _f32(u).copy()
+    v = np.empty_like(r)
+    if g.dtype == np.uint16:  # bfloat16 bit patterns
+        g = np.ascontiguousarray(g).reshape(-1)
+        fn = lib().rsdgc_oracle_accumulate_momentum_bf16
+    else:
+        g = _f32(g)
+        fn = lib().rsdgc_oracle_accumulate_momentum_f32
+    assert g.size == r.size == u_new.size
+    fn(_ptr(g), _ptr(u_new), _ptr(r), _ptr(v), float(np.float32(m)), r.size)
+    return u_new, v
 
 
 def nsi(v: np.ndarray, shape: LayerShape, alpha: float):
@@ -181,6 +201,7 @@ class LayerResult:
     val: np.ndarray          # float32 [k * nh * nw]
     residual: np.ndarray     # float32 [rows * cols], new accumulator
     nonfinite: int = 0
+    velocity: Optional[np.ndarray] = None  # new u when momentum correction is on
 
 
 @dataclass
@@ -193,12 +214,17 @@ class CompressResult:
 
 
 def compress_layer(g: np.ndarray, r: np.ndarray, shape: LayerShape, ratio: float, alpha: float,
-                   clamp_min1: bool = True, forced_sel: Optional[np.ndarray] = None) -> LayerResult:
+                   clamp_min1: bool = True, forced_sel: Optional[np.ndarray] = None,
+                   velocity: Optional[np.ndarray] = None, momentum: float = 0.0) -> LayerResult:
     """One layer of the per-iteration half of Algorithm 1.
 
     ``forced_sel`` replaces the ranking step by a given ascending tile set (used by the
     parity tests when two sets differ only inside the tolerance band at the threshold)."""
-    v = accumulate(g, r)
+    u_new = None
+    if velocity is None:
+        v = accumulate(g, r)
+    else:
+        u_new, v = accumulate_momentum(g, velocity, r, momentum)
     ref, f32, nonfinite = nsi(v, shape, alpha)
     k = keep_count(f32.size, ratio, clamp_min1)
     if forced_sel is None:
@@ -208,7 +234,7 @@ def compress_layer(g: np.ndarray, r: np.ndarray, shape: LayerShape, ratio: float
         thr = float(f32[sel].min()) if sel.size else 0.0
     idx, val, res = pack(v, shape, sel)
     return LayerResult(v=v, nsi_ref=ref, nsi_f32=f32, k=k, sel=sel, threshold=thr, idx=idx, val=val,
-                       residual=res, nonfinite=nonfinite)
+                       residual=res, nonfinite=nonfinite, velocity=u_new)
 
 
 def compress(shapes: Sequence[LayerShape], grads: Sequence[np.ndarray], residuals: Sequence[np.ndarray],

@@ -61,6 +61,30 @@ void rsdgc_oracle_accumulate_bf16(const uint16_t *g, const float *r, float *v, i
     for (int64_t i = 0; i < n; ++i) v[i] = bf16_to_f32(g[i]) + r[i];
 }
 
+/* Momentum correction ahead of the accumulation (Eq. 12, first and second line):
+ * u = m * u_prev + g, v = v_prev + u; product, sum, sum, each rounded to binary32.
+ * u is updated in place; it is not masked where neighborhoods are sent (Eq. 12 has no
+ * such step). */
+void rsdgc_oracle_accumulate_momentum_f32(const float *g, float *u, const float *r, float *v, float m, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        float mu = m * u[i];
+        u[i] = mu + g[i];
+        v[i] = r[i] + u[i];
+    }
+}
+
+/* Same with the incoming gradient stored as bfloat16 (widened exactly first). */
+void rsdgc_oracle_accumulate_momentum_bf16(const uint16_t *g, float *u, const float *r, float *v, float m,
+                                           int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        float mu = m * u[i];
+        u[i] = mu + bf16_to_f32(g[i]);
+        v[i] = r[i] + u[i];
+    }
+}
+
 /*
  * Neighborhood Statistical Indicator of every tile (Eq. 8-10):
  *   mean_p = (1/n) sum |v_i|                           (Eq. 9)

@@ -16,6 +16,7 @@ LIB_PATH = os.path.join(_HERE, "librsdgc_b200.so")
 RSDGC_F32, RSDGC_BF16 = 0, 1
 KEEP_AT_LEAST_ONE = 1
 NO_BULK_COPY = 2
+MOMENTUM = 4
 STATUS_NONFINITE, STATUS_PAYLOAD_OVERFLOW, STATUS_TIMEOUT = 1, 2, 4
 OK, ERR_INVALID, ERR_ALIGNMENT, ERR_CAPACITY, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
 
@@ -24,7 +25,7 @@ EXPORTS = [
     "rsdgc_plan_payload_bound", "rsdgc_plan_worklist", "rsdgc_update_ratios", "rsdgc_compress",
     "rsdgc_compress_host", "rsdgc_decompress_accumulate", "rsdgc_get_status", "rsdgc_launch_count",
     "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
-    "rsdgc_update_ratios_noalloc",
+    "rsdgc_update_ratios_noalloc", "rsdgc_compress_momentum",
 ]
 NOALLOC_MAX_LAYERS = 64
 N_COMPRESS_KERNELS = 6
@@ -81,6 +82,7 @@ def lib():
         L.rsdgc_plan_worklist.restype = i64
         L.rsdgc_update_ratios.argtypes = [vp, vp, f32, vp, vp]
         L.rsdgc_compress.argtypes = [vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
+        L.rsdgc_compress_momentum.argtypes = [vp, vp, vp, f32, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
         L.rsdgc_compress_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, vp,
                                           C.POINTER(i64), C.POINTER(i64), vp]
         L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
@@ -180,6 +182,13 @@ class Plan:
         _check(lib().rsdgc_compress(self._h, _ptr(grads), _ptr(residual), _ptr(ratios), _ptr(idx), idx.numel(),
                                     _ptr(val), val.numel(), _ptr(counts), _ptr(nsi), _ptr(workspace), _stream()),
                "rsdgc_compress")
+
+    def compress_momentum(self, grads, velocity, momentum: float, residual, ratios, idx, val, counts, nsi=None,
+                          workspace=None) -> None:
+        _check(lib().rsdgc_compress_momentum(self._h, _ptr(grads), _ptr(velocity), momentum, _ptr(residual),
+                                             _ptr(ratios), _ptr(idx), idx.numel(), _ptr(val), val.numel(),
+                                             _ptr(counts), _ptr(nsi), _ptr(workspace), _stream()),
+               "rsdgc_compress_momentum")
 
     def compress_host(self, grads_host, grads_dev, residual, ratios, idx, val, counts, workspace,
                       idx_host, val_host, counts_host) -> Tuple[int, int]:

@@ -326,16 +326,37 @@ __device__ __forceinline__ ItemDev load_item(const ItemDev *items, int i)
     return u.d;
 }
 
+// Momentum correction (Eq. 12, first line): u = m * u_prev + g, product then sum, each rounded.
+__device__ __forceinline__ float momentum_step(float m, float u_prev, float g)
+{
+    return __fadd_rn(__fmul_rn(m, u_prev), g);
+}
+__device__ __forceinline__ float4 momentum_step4(float m, float4 u, float4 g)
+{
+    return make_float4(momentum_step(m, u.x, g.x), momentum_step(m, u.y, g.y), momentum_step(m, u.z, g.z),
+                       momentum_step(m, u.w, g.w));
+}
+__device__ __forceinline__ float4 add4_rn(float4 a, float4 b)
+{
+    return make_float4(__fadd_rn(a.x, b.x), __fadd_rn(a.y, b.y), __fadd_rn(a.z, b.z), __fadd_rn(a.w, b.w));
+}
+
 // The elements of a contiguous item beyond its last full group of `gran` elements (gran = 4
-// or 8): plain loads and stores, results also placed in the shared-memory block.
-template <typename G>
+// or 8): plain loads and stores, results also placed in the shared-memory block.  With MOM the
+// velocity u = m * u + g is updated in place and takes the gradient's role in v = r + u.
+template <typename G, bool MOM>
 __device__ __forceinline__ void k1_tail(const ItemDev &d, int gran, const G *__restrict__ grads,
-                                        float *__restrict__ resid, float *sv)
+                                        float *__restrict__ resid, float *sv, float *__restrict__ vel, float mom)
 {
     const int n = d.R * d.W;
     const int e = (n / gran) * gran + threadIdx.x;
     if (e < n) {
-        const float v = __fadd_rn(load_grad1(grads, d.gbase + e), resid[d.gbase + e]);
+        float g = load_grad1(grads, d.gbase + e);
+        if (MOM) {
+            g = momentum_step(mom, vel[d.gbase + e], g);
+            vel[d.gbase + e] = g;
+        }
+        const float v = __fadd_rn(g, resid[d.gbase + e]);
         resid[d.gbase + e] = v;
         sv[e] = v;
     }
@@ -353,8 +374,10 @@ struct K1RegShared {
     FlushShared fs;
 };
 
+template <bool MOM>
 struct K1Regs {
     float4 g[kVecPerThread], r[kVecPerThread];
+    float4 u[MOM ? kVecPerThread : 1];  // velocity (momentum correction), staged like g and r
 };
 
 // Where each of a thread's kVecPerThread vector slots falls inside an item whose rows are
@@ -391,9 +414,10 @@ __device__ __forceinline__ long long item_elem_index(const ItemDev &d, int e, bo
     return d.gbase + (long long)row * d.cols + col;
 }
 
-template <typename G>
+template <typename G, bool MOM>
 __device__ __forceinline__ void k1_issue_loads(const ItemDev &d, const G *__restrict__ grads,
-                                               const float *__restrict__ resid, K1Regs &x, K1Map &m)
+                                               const float *__restrict__ resid, const float *__restrict__ vel,
+                                               K1Regs<MOM> &x, K1Map &m)
 {
     const int tid = threadIdx.x;
     if (d.flags & kItemVec) {
@@ -406,6 +430,7 @@ __device__ __forceinline__ void k1_issue_loads(const ItemDev &d, const G *__rest
                 if (i < nvec) {
                     x.g[u] = load_grad4(grads, base4 + i);
                     x.r[u] = __ldcs(reinterpret_cast<const float4 *>(resid) + base4 + i);
+                    if (MOM) x.u[u] = __ldcs(reinterpret_cast<const float4 *>(vel) + base4 + i);
                 }
             }
         } else {
@@ -416,11 +441,13 @@ __device__ __forceinline__ void k1_issue_loads(const ItemDev &d, const G *__rest
                 if ((m.rowj[u] >> 16) < R && (m.rowj[u] & 0xFFFFu) < wv) {
                     x.g[u] = load_grad4(grads, base4 + m.rel[u]);
                     x.r[u] = __ldcs(reinterpret_cast<const float4 *>(resid) + base4 + m.rel[u]);
+                    if (MOM) x.u[u] = __ldcs(reinterpret_cast<const float4 *>(vel) + base4 + m.rel[u]);
                 }
             }
         }
     } else {
         float *gs = reinterpret_cast<float *>(x.g), *rs = reinterpret_cast<float *>(x.r);
+        float *us = reinterpret_cast<float *>(x.u);
         const int n = d.R * d.P;
 #pragma unroll
         for (int u = 0; u < 4 * kVecPerThread; ++u) {
@@ -431,14 +458,16 @@ __device__ __forceinline__ void k1_issue_loads(const ItemDev &d, const G *__rest
                 if (valid) {
                     gs[u] = load_grad1(grads, gi);
                     rs[u] = __ldcs(resid + gi);
+                    if (MOM) us[u] = __ldcs(vel + gi);
                 }
             }
         }
     }
 }
 
-__device__ __forceinline__ void k1_add_store(const ItemDev &d, float *__restrict__ resid, float *sv, K1Regs &x,
-                                             K1Map &m)
+template <bool MOM>
+__device__ __forceinline__ void k1_add_store(const ItemDev &d, float *__restrict__ resid, float *__restrict__ vel,
+                                             float mom, float *sv, K1Regs<MOM> &x, K1Map &m)
 {
     const int tid = threadIdx.x;
     if (d.flags & kItemVec) {
@@ -453,17 +482,19 @@ __device__ __forceinline__ void k1_add_store(const ItemDev &d, float *__restrict
             const bool valid = full ? (i < nvec) : ((m.rowj[u] >> 16) < R && (m.rowj[u] & 0xFFFFu) < wv);
             if (valid) {
                 const long long gi = base4 + (full ? i : m.rel[u]);
-                float4 v;
-                v.x = __fadd_rn(x.g[u].x, x.r[u].x);
-                v.y = __fadd_rn(x.g[u].y, x.r[u].y);
-                v.z = __fadd_rn(x.g[u].z, x.r[u].z);
-                v.w = __fadd_rn(x.g[u].w, x.r[u].w);
+                float4 g = x.g[u];
+                if (MOM) {
+                    g = momentum_step4(mom, x.u[u], g);
+                    __stcs(reinterpret_cast<float4 *>(vel) + gi, g);
+                }
+                const float4 v = add4_rn(g, x.r[u]);
                 __stcs(reinterpret_cast<float4 *>(resid) + gi, v);
                 reinterpret_cast<float4 *>(sv)[i] = v;
             }
         }
     } else {
         const float *gs = reinterpret_cast<const float *>(x.g), *rs = reinterpret_cast<const float *>(x.r);
+        const float *us = reinterpret_cast<const float *>(x.u);
         const int n = d.R * d.P;
 #pragma unroll
         for (int u = 0; u < 4 * kVecPerThread; ++u) {
@@ -472,7 +503,12 @@ __device__ __forceinline__ void k1_add_store(const ItemDev &d, float *__restrict
                 bool valid = true;
                 const long long gi = (d.flags & kItemFull) ? d.gbase + e : item_elem_index(d, e, &valid);
                 if (valid) {
-                    const float v = __fadd_rn(gs[u], rs[u]);
+                    float g = gs[u];
+                    if (MOM) {
+                        g = momentum_step(mom, us[u], g);
+                        __stcs(vel + gi, g);
+                    }
+                    const float v = __fadd_rn(g, rs[u]);
                     __stcs(resid + gi, v);
                     sv[e] = v;
                 }
@@ -481,10 +517,10 @@ __device__ __forceinline__ void k1_add_store(const ItemDev &d, float *__restrict
     }
 }
 
-template <typename G>
+template <typename G, bool MOM>
 __global__ void __launch_bounds__(kThreads)
-k1_reg(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restrict__ keys,
-       const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
+k1_reg(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict__ vel, float mom,
+       uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
        const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
        const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags)
 {
@@ -496,10 +532,10 @@ k1_reg(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restr
     for (int b = tid; b < kL1Bins; b += kThreads) sh.hist[b] = 0;
     unsigned int nonfinite = 0;
 
-    K1Regs x;
+    K1Regs<MOM> x;
     K1Map map;
     ItemDev cur = load_item(items, begin);
-    k1_issue_loads(cur, grads, resid, x, map);
+    k1_issue_loads<G, MOM>(cur, grads, resid, vel, x, map);
     int buf = 0;
 
     for (int it = begin; it < end; ++it) {
@@ -508,10 +544,11 @@ k1_reg(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restr
         if (has_next) nxt = load_item(items, it + 1);
         // v = g + r for the current item (its loads were issued one iteration ago)
         float *sv = sh.v[buf];
-        k1_add_store(cur, resid, sv, x, map);
-        if ((cur.flags & (kItemVec | kItemFull)) == (kItemVec | kItemFull)) k1_tail(cur, 4, grads, resid, sv);
+        k1_add_store<MOM>(cur, resid, vel, mom, sv, x, map);
+        if ((cur.flags & (kItemVec | kItemFull)) == (kItemVec | kItemFull))
+            k1_tail<G, MOM>(cur, 4, grads, resid, sv, vel, mom);
         // the next item's g and r stream in while this item's tiles are reduced
-        if (has_next) k1_issue_loads(nxt, grads, resid, x, map);
+        if (has_next) k1_issue_loads<G, MOM>(nxt, grads, resid, vel, x, map);
         __syncthreads();
         nonfinite += item_tile_keys<kThreads>(cur, sv, keys, sh.hist, alpha);
         if (!has_next || nxt.layer != cur.layer)
@@ -540,13 +577,16 @@ k1_reg(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restr
 #endif
 constexpr int kBulkThreads = RSDGC_BULK_THREADS;
 constexpr int kBulkCtasPerSm = RSDGC_BULK_CTAS;
+constexpr int kBulkCtasPerSmMomentum = 2;  // a third block per stage: 110 KB of shared memory per CTA
 constexpr int kStages = RSDGC_BULK_STAGES;  // shared-memory stages; loads run kStages - 1 items ahead
 constexpr int kLookahead = kStages - 1;
 constexpr unsigned int kSpinLimit = 1u << 22;  // bounded mbarrier waits
 
+template <bool MOM>
 struct K1BulkShared {
     __align__(128) float r[kStages][kItemElems];  // residual block; becomes v in place
     __align__(128) float g[kStages][kItemElems];  // gradient block (binary32 or bfloat16 packed)
+    __align__(128) float u[MOM ? kStages : 1][MOM ? kItemElems : 4];  // velocity block, updated in place
     unsigned int hist[kL1Bins];
     __align__(8) unsigned long long full[kStages];  // mbarriers: stage loaded
     FlushShared fs;
@@ -617,39 +657,43 @@ __device__ __forceinline__ int bulk_elems(const ItemDev &d)
     return (d.flags & kItemFull) ? ((d.R * d.W) / gran) * gran : d.R * d.P;
 }
 
-// One thread: arm the stage's barrier and start the copies of g and r for an item.
-template <typename G>
-__device__ __forceinline__ void bulk_issue_item(const ItemDev &d, const G *grads, const float *resid, float *sr,
-                                                G *sg, unsigned long long *bar)
+// One thread: arm the stage's barrier and start the copies of g and r (and u) for an item.
+template <typename G, bool MOM>
+__device__ __forceinline__ void bulk_issue_item(const ItemDev &d, const G *grads, const float *resid,
+                                                const float *vel, float *sr, G *sg, float *su,
+                                                unsigned long long *bar)
 {
+    constexpr uint32_t per_elem = sizeof(float) + sizeof(G) + (MOM ? sizeof(float) : 0);
     if (d.flags & kItemFull) {
         const int n = bulk_elems<G>(d);
         if (n > 0) {
-            mbar_arrive_expect_tx(bar, (uint32_t)(n * (sizeof(float) + sizeof(G))));
+            mbar_arrive_expect_tx(bar, (uint32_t)n * per_elem);
             bulk_load(sr, resid + d.gbase, (uint32_t)(n * sizeof(float)), bar);
             bulk_load(sg, grads + d.gbase, (uint32_t)(n * sizeof(G)), bar);
+            if (MOM) bulk_load(su, vel + d.gbase, (uint32_t)(n * sizeof(float)), bar);
         } else {
             mbar_arrive_expect_tx(bar, 0);
         }
     } else {
-        mbar_arrive_expect_tx(bar, (uint32_t)(d.R * d.W * (sizeof(float) + sizeof(G))));
+        mbar_arrive_expect_tx(bar, (uint32_t)(d.R * d.W) * per_elem);
         for (int row = 0; row < d.R; ++row) {
             const long long gi = d.gbase + (long long)row * d.cols;
             bulk_load(sr + row * d.P, resid + gi, (uint32_t)(d.W * sizeof(float)), bar);
             bulk_load(sg + row * d.P, grads + gi, (uint32_t)(d.W * sizeof(G)), bar);
+            if (MOM) bulk_load(su + row * d.P, vel + gi, (uint32_t)(d.W * sizeof(float)), bar);
         }
     }
 }
 
-template <typename G>
-__global__ void __launch_bounds__(kBulkThreads, kBulkCtasPerSm)
-k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__restrict__ keys,
-        const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
+template <typename G, bool MOM>
+__global__ void __launch_bounds__(kBulkThreads, MOM ? kBulkCtasPerSmMomentum : kBulkCtasPerSm)
+k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict__ vel, float mom,
+        uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
         const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
         const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags)
 {
     extern __shared__ __align__(128) unsigned char k1_bulk_smem_raw[];
-    K1BulkShared &sh = *reinterpret_cast<K1BulkShared *>(k1_bulk_smem_raw);
+    K1BulkShared<MOM> &sh = *reinterpret_cast<K1BulkShared<MOM> *>(k1_bulk_smem_raw);
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     if (begin >= end) return;
     const int tid = threadIdx.x;
@@ -664,8 +708,8 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__rest
     if (tid == 0) {
         for (int j = 0; j < kLookahead && begin + j < end; ++j) {
             const ItemDev d = load_item(items, begin + j);
-            bulk_issue_item<G>(d, grads, resid, sh.r[j % kStages], reinterpret_cast<G *>(sh.g[j % kStages]),
-                               &sh.full[j % kStages]);
+            bulk_issue_item<G, MOM>(d, grads, resid, vel, sh.r[j % kStages], reinterpret_cast<G *>(sh.g[j % kStages]),
+                                    sh.u[MOM ? j % kStages : 0], &sh.full[j % kStages]);
         }
     }
     unsigned int nonfinite = 0;
@@ -688,25 +732,30 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__rest
         if (!mbar_wait_bounded(&sh.full[stage], (uint32_t)((rel / kStages) & 1))) timed_out = true;
         const int nb = bulk_elems<G>(cur);
         const int nvec = nb >> 2;
+        float *su = sh.u[MOM ? stage : 0];
         for (int i = tid; i < nvec; i += kBulkThreads) {
-            const float4 g = smem_grad4(sg, i);
-            float4 r = reinterpret_cast<const float4 *>(sr)[i];
-            r.x = __fadd_rn(g.x, r.x);
-            r.y = __fadd_rn(g.y, r.y);
-            r.z = __fadd_rn(g.z, r.z);
-            r.w = __fadd_rn(g.w, r.w);
-            reinterpret_cast<float4 *>(sr)[i] = r;
+            float4 g = smem_grad4(sg, i);
+            if (MOM) {  // u = m * u + g takes the gradient's place (Eq. 12, first line)
+                g = momentum_step4(mom, reinterpret_cast<const float4 *>(su)[i], g);
+                reinterpret_cast<float4 *>(su)[i] = g;
+            }
+            reinterpret_cast<float4 *>(sr)[i] = add4_rn(g, reinterpret_cast<const float4 *>(sr)[i]);
         }
-        fence_async_smem();  // the bulk store below reads what the threads just wrote
-        if (cur.flags & kItemFull) k1_tail(cur, (sizeof(G) == 2) ? 8 : 4, grads, resid, sr);
+        fence_async_smem();  // the bulk stores below read what the threads just wrote
+        if (cur.flags & kItemFull) k1_tail<G, MOM>(cur, (sizeof(G) == 2) ? 8 : 4, grads, resid, sr, vel, mom);
         __syncthreads();
         if (tid == 0) {
             if (cur.flags & kItemFull) {
-                if (nb > 0) bulk_store(resid + cur.gbase, sr, (uint32_t)(nb * sizeof(float)));
+                if (nb > 0) {
+                    bulk_store(resid + cur.gbase, sr, (uint32_t)(nb * sizeof(float)));
+                    if (MOM) bulk_store(vel + cur.gbase, su, (uint32_t)(nb * sizeof(float)));
+                }
             } else {
-                for (int row = 0; row < cur.R; ++row)
-                    bulk_store(resid + cur.gbase + (long long)row * cur.cols, sr + row * cur.P,
-                               (uint32_t)(cur.W * sizeof(float)));
+                for (int row = 0; row < cur.R; ++row) {
+                    const long long gi = cur.gbase + (long long)row * cur.cols;
+                    bulk_store(resid + gi, sr + row * cur.P, (uint32_t)(cur.W * sizeof(float)));
+                    if (MOM) bulk_store(vel + gi, su + row * cur.P, (uint32_t)(cur.W * sizeof(float)));
+                }
             }
             bulk_commit();
             // ---- producer: item it + kLookahead goes into the stage item it - 1 used.  Every
@@ -715,7 +764,8 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__rest
             if (it + kLookahead < end) {
                 bulk_wait_read<1>();
                 const int ps = (rel + kLookahead) % kStages;
-                bulk_issue_item<G>(ahead, grads, resid, sh.r[ps], reinterpret_cast<G *>(sh.g[ps]), &sh.full[ps]);
+                bulk_issue_item<G, MOM>(ahead, grads, resid, vel, sh.r[ps], reinterpret_cast<G *>(sh.g[ps]),
+                                        sh.u[MOM ? ps : 0], &sh.full[ps]);
                 if (it + 1 + kLookahead < end) ahead = load_item(items, it + 1 + kLookahead);
             }
         }
@@ -736,36 +786,44 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, uint32_t *__rest
 
 // ------------------------------------------------------------------------------------------
 
+template <typename K>
+static cudaError_t allow_smem(K kernel, size_t bytes)
+{
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+}
+
 static cudaError_t configure_once()
 {
     static cudaError_t result = [] {
-        cudaError_t e = cudaFuncSetAttribute(k1_reg<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)sizeof(K1RegShared));
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k1_reg<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)sizeof(K1RegShared));
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k1_bulk<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)sizeof(K1BulkShared));
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(k1_bulk<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)sizeof(K1BulkShared));
+        cudaError_t e = allow_smem(k1_reg<float, false>, sizeof(K1RegShared));
+        if (e == cudaSuccess) e = allow_smem(k1_reg<float, true>, sizeof(K1RegShared));
+        if (e == cudaSuccess) e = allow_smem(k1_reg<__nv_bfloat16, false>, sizeof(K1RegShared));
+        if (e == cudaSuccess) e = allow_smem(k1_reg<__nv_bfloat16, true>, sizeof(K1RegShared));
+        if (e == cudaSuccess) e = allow_smem(k1_bulk<float, false>, sizeof(K1BulkShared<false>));
+        if (e == cudaSuccess) e = allow_smem(k1_bulk<float, true>, sizeof(K1BulkShared<true>));
+        if (e == cudaSuccess) e = allow_smem(k1_bulk<__nv_bfloat16, false>, sizeof(K1BulkShared<false>));
+        if (e == cudaSuccess) e = allow_smem(k1_bulk<__nv_bfloat16, true>, sizeof(K1BulkShared<true>));
         return e;
     }();
     return result;
 }
 
-int k1_bulk_ctas_per_sm() { return kBulkCtasPerSm; }
+int k1_bulk_ctas_per_sm(bool momentum) { return momentum ? kBulkCtasPerSmMomentum : kBulkCtasPerSm; }
 
 // Resident CTAs per SM of the register-staged kernel on the current device.
-int k1_reg_ctas_per_sm(int dtype)
+int k1_reg_ctas_per_sm(int dtype, bool momentum)
 {
     int n = 0;
     cudaError_t e = configure_once();
-    if (e == cudaSuccess)
-        e = (dtype == RSDGC_BF16)
-                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_reg<__nv_bfloat16>, kThreads, sizeof(K1RegShared))
-                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_reg<float>, kThreads, sizeof(K1RegShared));
+    const size_t smem = sizeof(K1RegShared);
+    if (e == cudaSuccess) {
+        if (dtype == RSDGC_BF16)
+            e = momentum ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_reg<__nv_bfloat16, true>, kThreads, smem)
+                         : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_reg<__nv_bfloat16, false>, kThreads, smem);
+        else
+            e = momentum ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_reg<float, true>, kThreads, smem)
+                         : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, k1_reg<float, false>, kThreads, smem);
+    }
     if (e != cudaSuccess || n < 1) {
         (void)cudaGetLastError();
         n = 2;
@@ -773,33 +831,37 @@ int k1_reg_ctas_per_sm(int dtype)
     return n;
 }
 
-int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, const float *ratios, int32_t *counts,
-                          uint32_t *keys, cudaStream_t s)
+template <typename G, bool MOM>
+static void launch_k1_typed(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
+                            const float *ratios, int32_t *counts, uint32_t *keys, cudaStream_t s, int *launches)
+{
+    const G *g = reinterpret_cast<const G *>(grads);
+    if (p->n_items_bulk > 0) {
+        k1_bulk<G, MOM><<<p->grid_bulk, kBulkThreads, sizeof(K1BulkShared<MOM>), s>>>(
+            g, resid, vel, mom, keys, p->d_layers, p->d_items, p->d_cta_begin_bulk, p->d_hist, p->d_state, ratios,
+            counts, p->d_status, p->alpha, p->flags);
+        ++*launches;
+    }
+    if (p->n_items_reg > 0) {
+        k1_reg<G, MOM><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
+            g, resid, vel, mom, keys, p->d_layers, p->d_items + p->n_items_bulk, p->d_cta_begin_reg, p->d_hist,
+            p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
+        ++*launches;
+    }
+}
+
+// vel == nullptr: plain accumulation v = g + r; otherwise u = mom * u + g, v = r + u.
+int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
+                          const float *ratios, int32_t *counts, uint32_t *keys, cudaStream_t s)
 {
     int launches = 0;
     if (configure_once() != cudaSuccess) return 0;
-    if (p->n_items_bulk > 0) {
-        if (p->dtype == RSDGC_BF16)
-            k1_bulk<__nv_bfloat16><<<p->grid_bulk, kBulkThreads, sizeof(K1BulkShared), s>>>(
-                reinterpret_cast<const __nv_bfloat16 *>(grads), resid, keys, p->d_layers, p->d_items,
-                p->d_cta_begin_bulk, p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
-        else
-            k1_bulk<float><<<p->grid_bulk, kBulkThreads, sizeof(K1BulkShared), s>>>(
-                reinterpret_cast<const float *>(grads), resid, keys, p->d_layers, p->d_items, p->d_cta_begin_bulk,
-                p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
-        ++launches;
-    }
-    if (p->n_items_reg > 0) {
-        const ItemDev *items = p->d_items + p->n_items_bulk;
-        if (p->dtype == RSDGC_BF16)
-            k1_reg<__nv_bfloat16><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
-                reinterpret_cast<const __nv_bfloat16 *>(grads), resid, keys, p->d_layers, items, p->d_cta_begin_reg,
-                p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
-        else
-            k1_reg<float><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
-                reinterpret_cast<const float *>(grads), resid, keys, p->d_layers, items, p->d_cta_begin_reg,
-                p->d_hist, p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
-        ++launches;
+    if (p->dtype == RSDGC_BF16) {
+        if (vel) launch_k1_typed<__nv_bfloat16, true>(p, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+        else launch_k1_typed<__nv_bfloat16, false>(p, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+    } else {
+        if (vel) launch_k1_typed<float, true>(p, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+        else launch_k1_typed<float, false>(p, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
     }
     count_launch(launches);
     return launches;

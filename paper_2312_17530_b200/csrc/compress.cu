@@ -455,9 +455,9 @@ static cudaError_t launch_chained(void (*kernel)(KArgs...), int grid, cudaStream
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, const float *ratios, int32_t *idx,
-                            int64_t idx_cap, float *val, int64_t val_cap, int32_t *counts, uint32_t *keys,
-                            cudaStream_t s)
+cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
+                            const float *ratios, int32_t *idx, int64_t idx_cap, float *val, int64_t val_cap,
+                            int32_t *counts, uint32_t *keys, cudaStream_t s)
 {
     const int n_chunks = (int)p->chunks.size();
     const int prof = p->profile;
@@ -466,7 +466,7 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, cons
     if (prof >= (level) && e == cudaSuccess) e = record_event(p, s)
     if (prof) p->profile_recorded = prof;
     RSDGC_MARK(1);
-    launch_accumulate_nsi(p, grads, resid, ratios, counts, keys, s);
+    launch_accumulate_nsi(p, grads, resid, vel, mom, ratios, counts, keys, s);
     RSDGC_MARK(1);
     if (e == cudaSuccess)
         e = launch_chained(k_refine<2>, n_chunks, s, keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);

@@ -211,7 +211,7 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
     // --- each kernel's items in layer order, split into contiguous ranges of equal cost, one
     // range per CTA (all CTAs of a kernel are resident at once)
     p->items_dev.clear();
-    p->grid_bulk = p->n_sm * k1_bulk_ctas_per_sm();
+    p->grid_bulk = p->n_sm * k1_bulk_ctas_per_sm((p->flags & RSDGC_MOMENTUM) != 0);
     p->grid_reg = p->n_sm * p->reg_ctas_per_sm;
     for (auto &L : p->layers) L.n_flush1 = 0;
     for (int path = 0; path < 2; ++path) {
@@ -269,7 +269,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
     if (n_layers > kMaxLayers) return RSDGC_ERR_CAPACITY;
     if (grad_dtype != RSDGC_F32 && grad_dtype != RSDGC_BF16) return RSDGC_ERR_INVALID;
     if (!(alpha >= 0.0f && alpha <= 1.0f)) return RSDGC_ERR_INVALID;
-    if (flags & ~(RSDGC_KEEP_AT_LEAST_ONE | RSDGC_NO_BULK_COPY)) return RSDGC_ERR_INVALID;
+    if (flags & ~(RSDGC_KEEP_AT_LEAST_ONE | RSDGC_NO_BULK_COPY | RSDGC_MOMENTUM)) return RSDGC_ERR_INVALID;
 
     rsdgc_plan *p = new (std::nothrow) rsdgc_plan();
     if (!p) return RSDGC_ERR_NOMEM;
@@ -289,7 +289,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         p->n_sm = n_sm;
         DeviceGuard guard(device);
         // one CTA per resident slot: the static partitions assume all CTAs run concurrently
-        p->reg_ctas_per_sm = k1_reg_ctas_per_sm(grad_dtype);
+        p->reg_ctas_per_sm = k1_reg_ctas_per_sm(grad_dtype, (flags & RSDGC_MOMENTUM) != 0);
     }
 
     int rc;
@@ -426,10 +426,11 @@ extern "C" int rsdgc_update_ratios(rsdgc_plan *plan, const float *weights_dev, f
     return e == cudaSuccess ? RSDGC_OK : cuda_fail(e);
 }
 
-extern "C" int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *residual_dev,
-                              const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, float *val_dev,
-                              int64_t val_capacity, int32_t *counts_dev, float *nsi_dev, void *workspace_dev,
-                              void *stream)
+namespace {
+
+int compress_common(rsdgc_plan *plan, const void *grads_dev, float *velocity_dev, float momentum, float *residual_dev,
+                    const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, float *val_dev,
+                    int64_t val_capacity, int32_t *counts_dev, float *nsi_dev, void *workspace_dev, void *stream)
 {
     int rc = check_plan_device(plan);
     if (rc) return rc;
@@ -438,14 +439,37 @@ extern "C" int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *re
     if ((idx_capacity > 0 && !idx_dev) || (val_capacity > 0 && !val_dev)) return RSDGC_ERR_INVALID;
     if (!nsi_dev && !workspace_dev) return RSDGC_ERR_INVALID;
     if (!aligned16(grads_dev) || !aligned16(residual_dev) || !aligned16(idx_dev) || !aligned16(val_dev) ||
-        !aligned16(nsi_dev) || !aligned16(workspace_dev))
+        !aligned16(nsi_dev) || !aligned16(workspace_dev) || !aligned16(velocity_dev))
         return RSDGC_ERR_ALIGNMENT;
     uint32_t *keys = nsi_dev ? reinterpret_cast<uint32_t *>(nsi_dev) : reinterpret_cast<uint32_t *>(workspace_dev);
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
-    cudaError_t e = launch_compress(plan, grads_dev, residual_dev, ratios_dev, idx_dev, idx_capacity, val_dev,
-                                    val_capacity, counts_dev, keys, (cudaStream_t)stream);
+    cudaError_t e = launch_compress(plan, grads_dev, residual_dev, velocity_dev, momentum, ratios_dev, idx_dev,
+                                    idx_capacity, val_dev, val_capacity, counts_dev, keys, (cudaStream_t)stream);
     return e == cudaSuccess ? RSDGC_OK : cuda_fail(e);
+}
+
+}  // namespace
+
+extern "C" int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *residual_dev,
+                              const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, float *val_dev,
+                              int64_t val_capacity, int32_t *counts_dev, float *nsi_dev, void *workspace_dev,
+                              void *stream)
+{
+    if (plan && (plan->flags & RSDGC_MOMENTUM)) return RSDGC_ERR_INVALID;  // use rsdgc_compress_momentum()
+    return compress_common(plan, grads_dev, nullptr, 0.0f, residual_dev, ratios_dev, idx_dev, idx_capacity, val_dev,
+                           val_capacity, counts_dev, nsi_dev, workspace_dev, stream);
+}
+
+extern "C" int rsdgc_compress_momentum(rsdgc_plan *plan, const void *grads_dev, float *velocity_dev, float momentum,
+                                       float *residual_dev, const float *ratios_dev, int32_t *idx_dev,
+                                       int64_t idx_capacity, float *val_dev, int64_t val_capacity,
+                                       int32_t *counts_dev, float *nsi_dev, void *workspace_dev, void *stream)
+{
+    if (!plan || !(plan->flags & RSDGC_MOMENTUM) || !velocity_dev) return RSDGC_ERR_INVALID;
+    if (!(momentum >= 0.0f && momentum <= 1.0f)) return RSDGC_ERR_INVALID;
+    return compress_common(plan, grads_dev, velocity_dev, momentum, residual_dev, ratios_dev, idx_dev, idx_capacity,
+                           val_dev, val_capacity, counts_dev, nsi_dev, workspace_dev, stream);
 }
 
 extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_dev, float *residual_dev,

@@ -158,8 +158,8 @@ namespace rsdgc {
 int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *layers, int n_layers);
 
 // launches (defined in the .cu files); each returns a cudaError_t
-cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, const float *ratios,
-                            int32_t *idx, int64_t idx_cap, float *val, int64_t val_cap,
+cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
+                            const float *ratios, int32_t *idx, int64_t idx_cap, float *val, int64_t val_cap,
                             int32_t *counts, uint32_t *keys, cudaStream_t s);
 cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long n_keep,
                                  float *ratios, cudaStream_t s);
@@ -167,9 +167,9 @@ cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const
                               const int32_t *const *counts, float scale, float *dense, cudaStream_t s);
 void count_launch(int n);
 void set_last_cuda_error(int e);
-int k1_reg_ctas_per_sm(int dtype);
-int k1_bulk_ctas_per_sm();
-int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, const float *ratios, int32_t *counts,
-                          uint32_t *keys, cudaStream_t s);
+int k1_reg_ctas_per_sm(int dtype, bool momentum);
+int k1_bulk_ctas_per_sm(bool momentum);
+int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
+                          const float *ratios, int32_t *counts, uint32_t *keys, cudaStream_t s);
 
 }  // namespace rsdgc

@@ -69,9 +69,14 @@ class GpuCompress:
         self.workspace = None if with_nsi else torch.empty(max(plan.info.workspace_bytes, 16), dtype=torch.uint8,
                                                            device=device)
 
-    def run(self, grads: torch.Tensor, residual: torch.Tensor, ratios: torch.Tensor):
-        self.plan.compress(grads, residual, ratios, self.idx, self.val, self.counts, nsi=self.nsi,
-                           workspace=self.workspace)
+    def run(self, grads: torch.Tensor, residual: torch.Tensor, ratios: torch.Tensor, velocity=None,
+            momentum: float = 0.0):
+        if velocity is None:
+            self.plan.compress(grads, residual, ratios, self.idx, self.val, self.counts, nsi=self.nsi,
+                               workspace=self.workspace)
+        else:
+            self.plan.compress_momentum(grads, velocity, momentum, residual, ratios, self.idx, self.val,
+                                        self.counts, nsi=self.nsi, workspace=self.workspace)
         torch.cuda.synchronize()
         return self.plan.status()
 
@@ -80,9 +85,9 @@ class GpuCompress:
 
 
 def check_layer(oracle, li, shape, g, r, ratio, alpha, clamp, gpu_nsi, gpu_count, gpu_idx, gpu_val, gpu_res,
-                strict_keys: bool = True, what: str = ""):
+                strict_keys: bool = True, what: str = "", velocity=None, momentum: float = 0.0):
     """Applies R1 and R2 to one layer; returns the oracle's LayerResult."""
-    ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp)
+    ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp, velocity=velocity, momentum=momentum)
     K = ref.nsi_f32.size
     # R1
     err = np.abs(gpu_nsi.astype(np.float64) - ref.nsi_ref)
@@ -105,7 +110,8 @@ def check_layer(oracle, li, shape, g, r, ratio, alpha, clamp, gpu_nsi, gpu_count
             assert kept[must].all(), what + ": a tile clearly above the threshold is missing"
             assert not kept[must_not].any(), what + ": a tile clearly below the threshold was kept"
     if not np.array_equal(gpu_idx, ref.idx):
-        ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp, forced_sel=gpu_idx)
+        ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp, forced_sel=gpu_idx,
+                                    velocity=velocity, momentum=momentum)
     np.testing.assert_array_equal(gpu_idx, ref.idx, err_msg=what)
     np.testing.assert_array_equal(gpu_val.view(np.uint32), ref.val.view(np.uint32), err_msg=what + " val")
     np.testing.assert_array_equal(gpu_res.view(np.uint32), ref.residual.view(np.uint32), err_msg=what + " residual")
@@ -115,16 +121,20 @@ def check_layer(oracle, li, shape, g, r, ratio, alpha, clamp, gpu_nsi, gpu_count
 def compress_and_check(oracle, plan: binding.Plan, shapes, grads: Sequence[np.ndarray],
                        residuals: Sequence[np.ndarray], ratios: Sequence[float], alpha: float, clamp: bool = True,
                        gc: Optional[GpuCompress] = None, strict_keys: bool = True, what: str = "",
-                       max_ratio: float = 1.0):
+                       max_ratio: float = 1.0, velocities: Optional[Sequence[np.ndarray]] = None,
+                       momentum: float = 0.0):
     """Runs one GPU compress and checks every layer against the oracle.  Returns
-    (new residuals per layer, oracle results per layer, GpuCompress)."""
+    (new residuals per layer, oracle results per layer, GpuCompress).  With ``velocities`` the
+    momentum-corrected entry point is used and the new velocities are checked bit for bit
+    (they are in the oracle results)."""
     g_is_bf16 = grads[0].dtype == np.uint16
     g_arena = to_arena(plan, grads, np.uint16 if g_is_bf16 else np.float32)
     r_arena = to_arena(plan, residuals)
     gc = gc or GpuCompress(plan, max_ratio=max_ratio)
     d_g, d_r = dev(g_arena), dev(r_arena)
     d_ratios = torch.tensor(np.asarray(ratios, dtype=np.float32), device=gc.device)
-    st = gc.run(d_g, d_r, d_ratios)
+    d_u = dev(to_arena(plan, velocities)) if velocities is not None else None
+    st = gc.run(d_g, d_r, d_ratios, velocity=d_u, momentum=momentum)
     assert st.flags == 0, "%s: status flags %d" % (what, st.flags)
     # inputs untouched, padding untouched
     g_back = d_g.view(torch.int16).cpu().numpy().view(np.uint16) if g_is_bf16 else d_g.cpu().numpy()
@@ -132,6 +142,9 @@ def compress_and_check(oracle, plan: binding.Plan, shapes, grads: Sequence[np.nd
     res_arena = d_r.cpu().numpy()
     pad = padding_mask(plan)
     assert (res_arena[pad] == CANARY).all(), what + ": padding of the residual arena was written"
+    vel_arena = d_u.cpu().numpy() if d_u is not None else None
+    if vel_arena is not None:
+        assert (vel_arena[pad] == CANARY).all(), what + ": padding of the velocity arena was written"
     counts = gc.counts.cpu().numpy()
     idx, val, nsi = gc.idx.cpu().numpy(), gc.val.cpu().numpy(), gc.nsi.cpu().numpy()
     assert st.idx_needed == counts.sum()
@@ -142,7 +155,12 @@ def compress_and_check(oracle, plan: binding.Plan, shapes, grads: Sequence[np.nd
         ref = check_layer(oracle, li, shape, grads[l], residuals[l], float(np.float32(ratios[l])), alpha, clamp,
                           nsi[li.tile_offset:li.tile_offset + li.n_tiles], k, idx[io:io + k],
                           val[vo:vo + k * slot], res_arena[li.elem_offset:li.elem_offset + li.rows * li.cols],
-                          strict_keys=strict_keys, what="%s layer %d %r" % (what, l, tuple(shape)))
+                          strict_keys=strict_keys, what="%s layer %d %r" % (what, l, tuple(shape)),
+                          velocity=None if velocities is None else velocities[l], momentum=momentum)
+        if vel_arena is not None:
+            np.testing.assert_array_equal(
+                vel_arena[li.elem_offset:li.elem_offset + li.rows * li.cols].view(np.uint32),
+                ref.velocity.view(np.uint32), err_msg="%s layer %d velocity" % (what, l))
         io, vo = io + k, vo + k * slot
         refs.append(ref)
         new_res.append(ref.residual)

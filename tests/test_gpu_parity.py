@@ -327,3 +327,38 @@ def test_ablation_variants_and_other_neighborhood_shapes(oracle, alpha, shape):
     r = (rng.standard_normal(rows * cols) * 1e-2).astype(np.float32)
     plan = binding.Plan([shape], alpha=alpha)
     parity.compress_and_check(oracle, plan, [shape], [g], [r], [0.001], alpha, what="variant alpha=%g %r" % (alpha, shape))
+
+
+# ---------------------------------------------------------------------------------------------
+# momentum correction ahead of the accumulation (Eq. 12, first line)
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_momentum_correction_five_iterations(oracle, bf16):
+    shapes = [(300, 1032, 3, 3), (256 * 64, 9, 1, 9), (1, 777, 1, 9), (77, 45, 3, 3), (129, 4401, 3, 3),
+              (2000, 1111, 3, 3)]                                         # the last two: register-staged kernel
+    rng = np.random.default_rng(15)
+    plan = binding.Plan(shapes, grad_dtype=binding.RSDGC_BF16 if bf16 else binding.RSDGC_F32, alpha=0.5,
+                        flags=binding.KEEP_AT_LEAST_ONE | binding.MOMENTUM)
+    res = [np.zeros(r * c, np.float32) for r, c, _, _ in shapes]
+    vel = [np.zeros(r * c, np.float32) for r, c, _, _ in shapes]
+    ratios = [0.02, 0.05, 0.5, 0.01, 0.03, 0.004]
+    gc = parity.GpuCompress(plan, max_ratio=0.5)
+    for it in range(5):
+        g = [(rng.standard_normal(r * c) * 1e-2).astype(np.float32) for r, c, _, _ in shapes]
+        if bf16:
+            g = [synth.f32_to_bf16_bits(x) for x in g]
+        gc.idx.fill_(-1)
+        gc.val.fill_(float(parity.CANARY))
+        res, refs, _ = parity.compress_and_check(oracle, plan, shapes, g, res, ratios, 0.5, gc=gc,
+                                                 what="momentum it%d" % it, velocities=vel, momentum=0.9)
+        vel = [r.velocity for r in refs]
+    # a momentum plan refuses the plain entry point, and the other way round
+    with pytest.raises(binding.RsdgcError):
+        gc.run(parity.dev(parity.to_arena(plan, res)), parity.dev(parity.to_arena(plan, res)),
+               torch.tensor(ratios, device="cuda:0"))
+    plain = binding.Plan(shapes, alpha=0.5)
+    with pytest.raises(binding.RsdgcError):
+        parity.GpuCompress(plain).run(parity.dev(parity.to_arena(plain, res)), parity.dev(parity.to_arena(plain, res)),
+                                      torch.tensor(ratios, device="cuda:0"),
+                                      velocity=parity.dev(parity.to_arena(plain, res)), momentum=0.9)

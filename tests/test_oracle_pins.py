@@ -212,6 +212,32 @@ def test_accumulate_bf16_widens_exactly(oracle):
     np.testing.assert_array_equal(v, (t.to(torch.float32) + torch.from_numpy(r)).numpy())
 
 
+def test_momentum_correction_closed_forms(oracle):
+    """Eq. 12, first two lines: with a constant gradient and nothing sent, u_T = g (1 - m^T) / (1 - m)
+    and v_T = sum_t u_t; with m = 0 the step is the plain accumulation."""
+    rng = np.random.default_rng(14)
+    g = rng.standard_normal(257).astype(np.float32)
+    r0 = rng.standard_normal(257).astype(np.float32)
+    u1, v1 = oracle.accumulate_momentum(g, np.zeros_like(g), r0, 0.0)
+    np.testing.assert_array_equal(u1, g)
+    np.testing.assert_array_equal(v1, oracle.accumulate(g, r0))
+    m, T = 0.9, 25
+    u, v = np.zeros_like(g), np.zeros_like(g)
+    for _ in range(T):
+        u, v = oracle.accumulate_momentum(g, u, v, m)
+    m32 = float(np.float32(m))
+    g64 = g.astype(np.float64)
+    u_exact = g64 * (1 - m32 ** T) / (1 - m32)
+    v_exact = g64 * (T - m32 * (1 - m32 ** T) / (1 - m32)) / (1 - m32)
+    np.testing.assert_allclose(u, u_exact, rtol=2e-6)
+    np.testing.assert_allclose(v, v_exact, rtol=4e-6)
+    # one step by hand: the product is rounded before the sum (no fused multiply-add)
+    u0 = rng.standard_normal(257).astype(np.float32)
+    u2, v2 = oracle.accumulate_momentum(g, u0, r0, m)
+    np.testing.assert_array_equal(u2, np.float32(m) * u0 + g)
+    np.testing.assert_array_equal(v2, r0 + u2)
+
+
 # ---------------------------------------------------------------------------------------------
 # keep count (Eq. 11) and selection
 # ---------------------------------------------------------------------------------------------
