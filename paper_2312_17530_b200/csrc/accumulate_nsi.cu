@@ -704,6 +704,9 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
         fence_async_smem();
     }
     __syncthreads();
+    // launched with programmatic stream serialization: everything above overlapped the tail of the
+    // previous kernel in the stream; nothing below may run before that kernel has completed
+    grid_dependency_wait();
     // prologue: the first kLookahead items start loading
     if (tid == 0) {
         for (int j = 0; j < kLookahead && begin + j < end; ++j) {
@@ -837,9 +840,21 @@ static void launch_k1_typed(rsdgc_plan *p, const void *grads, float *resid, floa
 {
     const G *g = reinterpret_cast<const G *>(grads);
     if (p->n_items_bulk > 0) {
-        k1_bulk<G, MOM><<<p->grid_bulk, kBulkThreads, sizeof(K1BulkShared<MOM>), s>>>(
-            g, resid, vel, mom, keys, p->d_layers, p->d_items, p->d_cta_begin_bulk, p->d_hist, p->d_state, ratios,
-            counts, p->d_status, p->alpha, p->flags);
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3((unsigned)p->grid_bulk);
+        cfg.blockDim = dim3(kBulkThreads);
+        cfg.dynamicSmemBytes = sizeof(K1BulkShared<MOM>);
+        cfg.stream = s;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        const LayerDev *layers = p->d_layers;
+        const ItemDev *items = p->d_items;
+        const int32_t *cta_begin = p->d_cta_begin_bulk;
+        (void)cudaLaunchKernelEx(&cfg, k1_bulk<G, MOM>, g, resid, vel, mom, keys, layers, items, cta_begin, p->d_hist,
+                                 p->d_state, ratios, counts, p->d_status, p->alpha, (unsigned int)p->flags);
         ++*launches;
     }
     if (p->n_items_reg > 0) {
