@@ -2,9 +2,10 @@
 """Benchmark of the RS-DGC compression path on B200.
 
 Workload: the VGG-19-shaped gradient set (38 tensors, 139,754,605 fp32 elements per worker),
-4 simulated workers per GPU, uniform keep ratio 1/64, alpha 0.5.  One step = every worker's
-rsdgc_compress() (accumulate, NSI, threshold select, pack, residual update) followed by one
-rsdgc_decompress_accumulate() of the 4 payloads into a dense buffer on the same GPU.  The
+4 simulated workers per GPU, uniform keep ratio 1/64, alpha 0.5.  One step = the 4 workers'
+compression (accumulate, NSI, threshold select, pack, residual update) through one
+rsdgc_compress_workers() call, followed by one rsdgc_decompress_accumulate() of the 4 payloads
+into a dense buffer on the same GPU.  The
 per-epoch ratio rule (rsdgc_update_ratios) is timed separately and reported in "extra".
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl b200|reference]
@@ -35,8 +36,8 @@ N_WORKERS = 4
 KEEP_RATIO = 1.0 / 64.0
 ALPHA = 0.5
 WORKLOAD = ("VGG-19-shaped gradient set (38 tensors, 139754605 fp32 elements per worker), %d workers per GPU, "
-            "keep 1/64 of the neighborhoods per layer, alpha 0.5; step = %d x compress + 1 x "
-            "decompress_accumulate" % (N_WORKERS, N_WORKERS))
+            "keep 1/64 of the neighborhoods per layer, alpha 0.5; step = compress of the %d workers (one "
+            "compress_workers call) + 1 x decompress_accumulate" % (N_WORKERS, N_WORKERS))
 
 
 def measured_peaks():
@@ -204,15 +205,15 @@ def run_b200(args):
     d_idx = [torch.zeros(ni, dtype=torch.int32, device=device) for _ in range(N_WORKERS)]
     d_val = [torch.zeros(nv, dtype=torch.float32, device=device) for _ in range(N_WORKERS)]
     d_cnt = [torch.zeros(plan.n_layers, dtype=torch.int32, device=device) for _ in range(N_WORKERS)]
-    d_ws = torch.empty(plan.info.workspace_bytes, dtype=torch.uint8, device=device)
+    d_ws = torch.empty(N_WORKERS * plan.info.workspace_bytes, dtype=torch.uint8, device=device)
+    plan.reserve_workers(N_WORKERS)
     d_ratios = torch.full((plan.n_layers,), KEEP_RATIO, dtype=torch.float32, device=device)
     d_dense = torch.zeros(arena, dtype=torch.float32, device=device)
     d_r0 = d_r[0]
     torch.cuda.synchronize()
 
     def step():
-        for w in range(N_WORKERS):
-            plan.compress(d_g[w], d_r[w], d_ratios, d_idx[w], d_val[w], d_cnt[w], workspace=d_ws)
+        plan.compress_workers(d_g, d_r, d_ratios, d_idx, d_val, d_cnt, d_ws)
         plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
 
     # ---- device-resident timing: W warm-up steps, then exactly K steps between two events
@@ -230,8 +231,7 @@ def run_b200(args):
     launches0 = binding.launch_count()
     ev0.record()
     for s in range(args.steps):
-        for w in range(N_WORKERS):
-            plan.compress(d_g[w], d_r[w], d_ratios, d_idx[w], d_val[w], d_cnt[w], workspace=d_ws)
+        plan.compress_workers(d_g, d_r, d_ratios, d_idx, d_val, d_cnt, d_ws)
         ev_dec[s][0].record()
         plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
         ev_dec[s][1].record()
@@ -257,6 +257,11 @@ def run_b200(args):
         step()
     torch.cuda.synchronize()
     breakdown_ms, breakdown_calls = plan.profile_read()
+    for _ in range(2):  # the same stages of single-worker rsdgc_compress() calls, for comparison
+        for w in range(N_WORKERS):
+            plan.compress(d_g[w], d_r[w], d_ratios, d_idx[w], d_val[w], d_cnt[w], workspace=d_ws)
+    torch.cuda.synchronize()
+    single_ms, single_calls = plan.profile_read()
     plan.profile_enable(0)
 
     # ---- end to end: host buffers in, payload out, through rsdgc_compress_host()
@@ -384,17 +389,20 @@ def run_b200(args):
 
     if rank == 0:
         peak, peak_src = measured_peaks()
-        k1_s = kernel_ms[0] / 1e3 / max(n_calls, 1)
+        # level-1 events bracket the N_WORKERS back-to-back first passes of a call
+        k1_s = kernel_ms[0] / 1e3 / max(n_calls * N_WORKERS, 1)
         # one worker's compress inside the timed steps: step time minus the aggregation, per worker
         compress_s = (elapsed_s / args.steps - dec_ms / 1e3) / N_WORKERS
         alg_bytes = 12.0 * n  # read g, read r, write v: 12 B per element for fp32 gradients
         achieved = alg_bytes / k1_s / 1e9
         per_kernel_us = {name: 1e3 * ms / max(breakdown_calls, 1)
                          for name, ms in zip(binding.COMPRESS_KERNELS, breakdown_ms)}
+        single_us = {name: 1e3 * ms / max(single_calls, 1) for name, ms in zip(binding.COMPRESS_KERNELS, single_ms)}
         extra.update({
             "us_per_model_iteration": compress_s * 1e6,
             "layers_per_s": plan.n_layers / compress_s,
-            "compress_kernels_us_with_events_between": per_kernel_us,
+            "compress_workers_stage_us_with_events_between": per_kernel_us,  # one call = all the workers
+            "single_worker_compress_stage_us_with_events_between": single_us,
             "compress_roofline_frac": alg_bytes / compress_s / 1e9 / peak,
             "compress_roofline_frac_of_nominal_8TBs": alg_bytes / compress_s / 1e9 / 8000.0,
             "decompress_accumulate_us": dec_ms * 1e3,

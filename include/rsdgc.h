@@ -220,6 +220,31 @@ int rsdgc_compress_momentum(rsdgc_plan *plan, const void *grads_dev, float *velo
                             float *nsi_dev, void *workspace_dev, void *stream);
 
 /*
+ * The same step for the n_workers data-parallel workers that share this GPU (Sec. III-A: every
+ * node k compresses its own gradient with the same per-layer ratios; Eq. 12 per worker k), in
+ * one call: one accumulate+NSI pass per worker, then the selection, index and gather kernels
+ * run once each over all workers.  Results per worker are exactly those of n_workers calls of
+ * rsdgc_compress().
+ * rsdgc_plan_reserve_workers() gives the plan the selection tables of n_workers workers (a few
+ * MB of device memory each; allocates, so call it once outside any stream capture);
+ * rsdgc_compress_workers() returns CAPACITY if fewer workers were reserved.
+ * grads_dev_host / residual_dev_host / idx_dev_host / val_dev_host / counts_dev_host: HOST
+ * arrays of n_workers DEVICE pointers, one arena / payload per worker (no two workers may share
+ * an accumulator or a payload buffer); idx_capacity / val_capacity hold for every worker.
+ * workspace_dev: n_workers * workspace_bytes bytes, 16-byte aligned.  Not for plans created
+ * with RSDGC_MOMENTUM.  With rsdgc_profile_enable() a call records one set of events per group
+ * of up to 16 workers: stage 0 spans the accumulate+NSI passes of all the workers of the group,
+ * the later stages the single launches that serve them all.
+ * Errors: INVALID, ALIGNMENT, CAPACITY, CUDA / NOMEM.
+ */
+int rsdgc_plan_reserve_workers(rsdgc_plan *plan, int32_t n_workers);
+int rsdgc_compress_workers(rsdgc_plan *plan, int32_t n_workers, const void *const *grads_dev_host,
+                           float *const *residual_dev_host, const float *ratios_dev,
+                           int32_t *const *idx_dev_host, int64_t idx_capacity,
+                           float *const *val_dev_host, int64_t val_capacity,
+                           int32_t *const *counts_dev_host, void *workspace_dev, void *stream);
+
+/*
  * Same step with the gradient and the payload in HOST memory: copies grads_host into
  * grads_dev (a caller-owned staging arena), runs rsdgc_compress(), waits, and copies
  * counts and exactly the used part of idx/val back to the host buffers (which must hold

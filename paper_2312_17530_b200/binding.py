@@ -25,7 +25,8 @@ EXPORTS = [
     "rsdgc_plan_payload_bound", "rsdgc_plan_worklist", "rsdgc_update_ratios", "rsdgc_compress",
     "rsdgc_compress_host", "rsdgc_decompress_accumulate", "rsdgc_get_status", "rsdgc_launch_count",
     "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
-    "rsdgc_update_ratios_noalloc", "rsdgc_compress_momentum",
+    "rsdgc_update_ratios_noalloc", "rsdgc_compress_momentum", "rsdgc_plan_reserve_workers",
+    "rsdgc_compress_workers",
 ]
 NOALLOC_MAX_LAYERS = 64
 N_COMPRESS_KERNELS = 6
@@ -83,6 +84,9 @@ def lib():
         L.rsdgc_update_ratios.argtypes = [vp, vp, f32, vp, vp]
         L.rsdgc_compress.argtypes = [vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
         L.rsdgc_compress_momentum.argtypes = [vp, vp, vp, f32, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp]
+        L.rsdgc_plan_reserve_workers.argtypes = [vp, i32]
+        L.rsdgc_compress_workers.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), vp, C.POINTER(vp), i64,
+                                             C.POINTER(vp), i64, C.POINTER(vp), vp, vp]
         L.rsdgc_compress_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, vp,
                                           C.POINTER(i64), C.POINTER(i64), vp]
         L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
@@ -189,6 +193,22 @@ class Plan:
                                              _ptr(ratios), _ptr(idx), idx.numel(), _ptr(val), val.numel(),
                                              _ptr(counts), _ptr(nsi), _ptr(workspace), _stream()),
                "rsdgc_compress_momentum")
+
+    def reserve_workers(self, n_workers: int) -> None:
+        _check(lib().rsdgc_plan_reserve_workers(self._h, int(n_workers)), "rsdgc_plan_reserve_workers")
+
+    def compress_workers(self, grads, residuals, ratios, idx, val, counts, workspace) -> None:
+        """One call for several workers: ``grads``, ``residuals``, ``idx``, ``val``, ``counts`` are
+        sequences with one device tensor per worker; ``workspace`` holds n_workers * workspace_bytes."""
+        n = len(grads)
+        A = C.c_void_p * max(1, n)
+        ga, ra, ia, va, ca = A(), A(), A(), A(), A()
+        for w in range(n):
+            ga[w], ra[w], ca[w] = grads[w].data_ptr(), residuals[w].data_ptr(), counts[w].data_ptr()
+            ia[w], va[w] = idx[w].data_ptr(), val[w].data_ptr()
+        _check(lib().rsdgc_compress_workers(self._h, n, ga, ra, _ptr(ratios), ia, min(t.numel() for t in idx), va,
+                                            min(t.numel() for t in val), ca, _ptr(workspace), _stream()),
+               "rsdgc_compress_workers")
 
     def compress_host(self, grads_host, grads_dev, residual, ratios, idx, val, counts, workspace,
                       idx_host, val_host, counts_host) -> Tuple[int, int]:

@@ -835,8 +835,9 @@ int k1_reg_ctas_per_sm(int dtype, bool momentum)
 }
 
 template <typename G, bool MOM>
-static void launch_k1_typed(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
-                            const float *ratios, int32_t *counts, uint32_t *keys, cudaStream_t s, int *launches)
+static void launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
+                            float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
+                            cudaStream_t s, int *launches)
 {
     const G *g = reinterpret_cast<const G *>(grads);
     if (p->n_items_bulk > 0) {
@@ -853,30 +854,31 @@ static void launch_k1_typed(rsdgc_plan *p, const void *grads, float *resid, floa
         const LayerDev *layers = p->d_layers;
         const ItemDev *items = p->d_items;
         const int32_t *cta_begin = p->d_cta_begin_bulk;
-        (void)cudaLaunchKernelEx(&cfg, k1_bulk<G, MOM>, g, resid, vel, mom, keys, layers, items, cta_begin, p->d_hist,
-                                 p->d_state, ratios, counts, p->d_status, p->alpha, (unsigned int)p->flags);
+        (void)cudaLaunchKernelEx(&cfg, k1_bulk<G, MOM>, g, resid, vel, mom, keys, layers, items, cta_begin, hist,
+                                 state, ratios, counts, p->d_status, p->alpha, (unsigned int)p->flags);
         ++*launches;
     }
     if (p->n_items_reg > 0) {
         k1_reg<G, MOM><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
-            g, resid, vel, mom, keys, p->d_layers, p->d_items + p->n_items_bulk, p->d_cta_begin_reg, p->d_hist,
-            p->d_state, ratios, counts, p->d_status, p->alpha, p->flags);
+            g, resid, vel, mom, keys, p->d_layers, p->d_items + p->n_items_bulk, p->d_cta_begin_reg, hist,
+            state, ratios, counts, p->d_status, p->alpha, p->flags);
         ++*launches;
     }
 }
 
 // vel == nullptr: plain accumulation v = g + r; otherwise u = mom * u + g, v = r + u.
-int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
-                          const float *ratios, int32_t *counts, uint32_t *keys, cudaStream_t s)
+int launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
+                          float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
+                          cudaStream_t s)
 {
     int launches = 0;
     if (configure_once() != cudaSuccess) return 0;
     if (p->dtype == RSDGC_BF16) {
-        if (vel) launch_k1_typed<__nv_bfloat16, true>(p, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
-        else launch_k1_typed<__nv_bfloat16, false>(p, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+        if (vel) launch_k1_typed<__nv_bfloat16, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+        else launch_k1_typed<__nv_bfloat16, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
     } else {
-        if (vel) launch_k1_typed<float, true>(p, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
-        else launch_k1_typed<float, false>(p, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+        if (vel) launch_k1_typed<float, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+        else launch_k1_typed<float, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
     }
     count_launch(launches);
     return launches;

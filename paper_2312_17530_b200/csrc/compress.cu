@@ -28,10 +28,14 @@ struct RefineShared {
 // of the layer then knows the threshold key T and how many keys equal to T are taken.
 template <int LEVEL>
 __global__ void __launch_bounds__(kThreads)
-k_refine(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
-         const Chunk *__restrict__ chunks, unsigned int *hist, LayerState *state)
+k_refine(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
+         const Chunk *__restrict__ chunks)
 {
     __shared__ RefineShared sh;
+    const Lane &ln = lanes.l[blockIdx.y];
+    const uint32_t *__restrict__ keys = ln.keys;
+    unsigned int *hist = ln.hist;
+    LayerState *state = ln.state;
     constexpr int SHIFT_HI = (LEVEL == 2) ? kL1Shift : kL2Shift;
     constexpr int SHIFT_LO = (LEVEL == 2) ? kL2Shift : 0;
     constexpr int NBITS = (LEVEL == 2) ? kL2Bits : kL3Bits;
@@ -128,11 +132,15 @@ struct CountShared {
 };
 
 __global__ void __launch_bounds__(kThreads)
-k_count(const uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers,
-        const Chunk *__restrict__ chunks, LayerState *state, uint2 *chunk_cnt, unsigned char *__restrict__ codes,
-        int n_layers, long long idx_cap, long long val_cap, StatusDev *status)
+k_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
+        const Chunk *__restrict__ chunks, int n_layers, long long idx_cap, long long val_cap, StatusDev *status)
 {
     __shared__ CountShared sh;
+    const Lane &ln = lanes.l[blockIdx.y];
+    const uint32_t *__restrict__ keys = ln.keys;
+    LayerState *state = ln.state;
+    uint2 *chunk_cnt = ln.chunk_cnt;
+    unsigned char *__restrict__ codes = ln.codes;
     const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     LayerState &st = state[c.layer];
@@ -254,11 +262,15 @@ struct MarkShared {
 };
 
 __global__ void __launch_bounds__(kThreads)
-k_mark(const unsigned char *__restrict__ codes, const LayerDev *__restrict__ layers,
-       const Chunk *__restrict__ chunks, const LayerState *__restrict__ state,
-       const uint2 *__restrict__ chunk_cnt, int32_t *__restrict__ idx, long long idx_cap)
+k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
+       const Chunk *__restrict__ chunks, long long idx_cap)
 {
     __shared__ MarkShared sh;
+    const Lane &ln = lanes.l[blockIdx.y];
+    const unsigned char *__restrict__ codes = ln.codes;
+    const LayerState *__restrict__ state = ln.state;
+    const uint2 *__restrict__ chunk_cnt = ln.chunk_cnt;
+    int32_t *__restrict__ idx = ln.idx;
     const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x;
     grid_dependency_wait();
@@ -337,87 +349,97 @@ k_mark(const unsigned char *__restrict__ codes, const LayerDev *__restrict__ lay
 constexpr int kCopyBatch = RSDGC_COPY_BATCH;
 
 __global__ void __launch_bounds__(kThreads)
-k_gather(float *__restrict__ resid, const LayerDev *__restrict__ layers, const LayerState *__restrict__ state,
-         int n_layers, const int32_t *__restrict__ idx, long long idx_cap, float *__restrict__ val, long long val_cap)
+k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *__restrict__ layers, int n_layers,
+         long long idx_cap, long long val_cap)
 {
     __shared__ long long val_off[kMaxLayers + 1];
     __shared__ long long idx_off[kMaxLayers];
     const int tid = threadIdx.x;
     grid_dependency_wait();
-    for (int l = tid; l < n_layers; l += kThreads) {
-        val_off[l] = state[l].val_off;
-        idx_off[l] = state[l].idx_off;
-    }
-    if (tid == 0) {
-        const LayerState &last = state[n_layers - 1];
-        val_off[n_layers] = last.val_off + (long long)last.k * layers[n_layers - 1].slot;
-    }
-    __syncthreads();
-    const long long total = val_off[n_layers];
-    // a CTA takes blocks of kThreads * kCopyBatch consecutive payload values: almost always one
-    // layer per block, so the layer search is done once per block, not once per value
-    constexpr long long kBlock = (long long)kThreads * kCopyBatch;
-    auto find_layer = [&](long long j) {
-        int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (val_off[mid] <= j) lo = mid; else hi = mid;
+    // the workers one after the other: the scattered accesses of the CTAs that run at the same
+    // time then fall into one worker's arena
+    for (int lane = 0; lane < n_lanes; ++lane) {
+        const Lane &ln = lanes.l[lane];
+        float *__restrict__ resid = ln.resid;
+        const LayerState *__restrict__ state = ln.state;
+        const int32_t *__restrict__ idx = ln.idx;
+        float *__restrict__ val = ln.val;
+        if (lane) __syncthreads();  // everyone is done with the previous worker's tables
+        for (int l = tid; l < n_layers; l += kThreads) {
+            val_off[l] = state[l].val_off;
+            idx_off[l] = state[l].idx_off;
         }
-        return lo;
-    };
-    for (long long jb = (long long)blockIdx.x * kBlock; jb < total; jb += (long long)gridDim.x * kBlock) {
-        const long long jend = min(total, jb + kBlock) - 1;
-        const int l_first = find_layer(jb);
-        const bool one_layer = val_off[l_first + 1] > jend;
-        long long ga[kCopyBatch], vo[kCopyBatch];
-        int tile[kCopyBatch], lay[kCopyBatch], el[kCopyBatch];
-        float xv[kCopyBatch];
-#pragma unroll
-        for (int u = 0; u < kCopyBatch; ++u) {
-            const long long j = jb + u * kThreads + tid;
-            ga[u] = -1;
-            vo[u] = -1;
-            tile[u] = -1;
-            if (j < total) {
-                const int lo = one_layer ? l_first : find_layer(j);
-                const int slot = layers[lo].slot;
-                const long long jl = j - val_off[lo];
-                // 32-bit division whenever the layer's payload is below 2^31 values (the usual case)
-                long long s;
-                if (jl < 0x7FFFFFFFll) {
-                    int q, r;
-                    divmod_small((int)jl, slot, &q, &r);
-                    s = q;
-                    el[u] = r;
-                } else {
-                    s = jl / slot;
-                    el[u] = (int)(jl - s * slot);
-                }
-                lay[u] = lo;
-                // tiles that do not fit the payload buffers are not sent and stay in the residual
-                if (idx_off[lo] + s < idx_cap && val_off[lo] + (s + 1) * slot <= val_cap) {
-                    tile[u] = __ldg(idx + idx_off[lo] + s);
-                    vo[u] = j;
+        if (tid == 0) {
+            const LayerState &last = state[n_layers - 1];
+            val_off[n_layers] = last.val_off + (long long)last.k * layers[n_layers - 1].slot;
+        }
+        __syncthreads();
+        const long long total = val_off[n_layers];
+        // a CTA takes blocks of kThreads * kCopyBatch consecutive payload values: almost always one
+        // layer per block, so the layer search is done once per block, not once per value
+        constexpr long long kBlock = (long long)kThreads * kCopyBatch;
+        auto find_layer = [&](long long j) {
+            int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (val_off[mid] <= j) lo = mid; else hi = mid;
+            }
+            return lo;
+        };
+        for (long long jb = (long long)blockIdx.x * kBlock; jb < total; jb += (long long)gridDim.x * kBlock) {
+            const long long jend = min(total, jb + kBlock) - 1;
+            const int l_first = find_layer(jb);
+            const bool one_layer = val_off[l_first + 1] > jend;
+            long long ga[kCopyBatch], vo[kCopyBatch];
+            int tile[kCopyBatch], lay[kCopyBatch], el[kCopyBatch];
+            float xv[kCopyBatch];
+    #pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) {
+                const long long j = jb + u * kThreads + tid;
+                ga[u] = -1;
+                vo[u] = -1;
+                tile[u] = -1;
+                if (j < total) {
+                    const int lo = one_layer ? l_first : find_layer(j);
+                    const int slot = layers[lo].slot;
+                    const long long jl = j - val_off[lo];
+                    // 32-bit division whenever the layer's payload is below 2^31 values (the usual case)
+                    long long s;
+                    if (jl < 0x7FFFFFFFll) {
+                        int q, r;
+                        divmod_small((int)jl, slot, &q, &r);
+                        s = q;
+                        el[u] = r;
+                    } else {
+                        s = jl / slot;
+                        el[u] = (int)(jl - s * slot);
+                    }
+                    lay[u] = lo;
+                    // tiles that do not fit the payload buffers are not sent and stay in the residual
+                    if (idx_off[lo] + s < idx_cap && val_off[lo] + (s + 1) * slot <= val_cap) {
+                        tile[u] = __ldg(idx + idx_off[lo] + s);
+                        vo[u] = j;
+                    }
                 }
             }
-        }
-#pragma unroll
-        for (int u = 0; u < kCopyBatch; ++u) {
-            if (tile[u] >= 0) {
-                const LayerDev &L = layers[lay[u]];
-                const int tr = tile[u] / L.TC, tc = tile[u] - tr * L.TC;
-                int a, b;
-                divmod_small(el[u], L.nw, &a, &b);
-                const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
-                if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+    #pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) {
+                if (tile[u] >= 0) {
+                    const LayerDev &L = layers[lay[u]];
+                    const int tr = tile[u] / L.TC, tc = tile[u] - tr * L.TC;
+                    int a, b;
+                    divmod_small(el[u], L.nw, &a, &b);
+                    const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
+                    if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+                }
             }
-        }
-#pragma unroll
-        for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
-#pragma unroll
-        for (int u = 0; u < kCopyBatch; ++u) {
-            if (ga[u] >= 0) resid[ga[u]] = 0.0f;
-            if (vo[u] >= 0) val[vo[u]] = xv[u];
+    #pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
+    #pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) {
+                if (ga[u] >= 0) resid[ga[u]] = 0.0f;
+                if (vo[u] >= 0) val[vo[u]] = xv[u];
+            }
         }
     }
 }
@@ -440,10 +462,10 @@ static cudaError_t record_event(rsdgc_plan *p, cudaStream_t s)
 // while its predecessor drains; it calls grid_dependency_wait() before touching that kernel's
 // results.
 template <typename... KArgs, typename... Args>
-static cudaError_t launch_chained(void (*kernel)(KArgs...), int grid, cudaStream_t s, Args... args)
+static cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, cudaStream_t s, Args... args)
 {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)grid);
+    cfg.gridDim = grid;
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = s;
@@ -455,39 +477,84 @@ static cudaError_t launch_chained(void (*kernel)(KArgs...), int grid, cudaStream
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
+// The five kernels after the accumulate+NSI pass, one launch each for all the lanes of the call.
+static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n_lanes, int64_t idx_cap,
+                                    int64_t val_cap, int prof, cudaStream_t s)
+{
+    const dim3 grid((unsigned)p->chunks.size(), (unsigned)n_lanes);
+    const dim3 grid_gather((unsigned)(p->n_sm * 8));  // grid-stride loops over each lane's payload
+    cudaError_t e = cudaSuccess;
+#define RSDGC_MARK(level)                              \
+    if (prof >= (level) && e == cudaSuccess) e = record_event(p, s)
+    if (e == cudaSuccess) e = launch_chained(k_refine<2>, grid, s, lanes, p->d_layers, p->d_chunks);
+    RSDGC_MARK(2);
+    if (e == cudaSuccess) e = launch_chained(k_refine<3>, grid, s, lanes, p->d_layers, p->d_chunks);
+    RSDGC_MARK(2);
+    if (e == cudaSuccess)
+        e = launch_chained(k_count, grid, s, lanes, p->d_layers, p->d_chunks, p->n_layers, (long long)idx_cap,
+                           (long long)val_cap, p->d_status);
+    RSDGC_MARK(2);
+    if (e == cudaSuccess) e = launch_chained(k_mark, grid, s, lanes, p->d_layers, p->d_chunks, (long long)idx_cap);
+    RSDGC_MARK(2);
+    if (e == cudaSuccess)
+        e = launch_chained(k_gather, grid_gather, s, lanes, n_lanes, p->d_layers, p->n_layers, (long long)idx_cap,
+                           (long long)val_cap);
+    RSDGC_MARK(2);
+#undef RSDGC_MARK
+    count_launch(5);
+    return e;
+}
+
 cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
                             const float *ratios, int32_t *idx, int64_t idx_cap, float *val, int64_t val_cap,
                             int32_t *counts, uint32_t *keys, cudaStream_t s)
 {
-    const int n_chunks = (int)p->chunks.size();
     const int prof = p->profile;
     cudaError_t e = cudaSuccess;
-#define RSDGC_MARK(level)                              \
-    if (prof >= (level) && e == cudaSuccess) e = record_event(p, s)
     if (prof) p->profile_recorded = prof;
-    RSDGC_MARK(1);
-    launch_accumulate_nsi(p, grads, resid, vel, mom, ratios, counts, keys, s);
-    RSDGC_MARK(1);
-    if (e == cudaSuccess)
-        e = launch_chained(k_refine<2>, n_chunks, s, keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
-    RSDGC_MARK(2);
-    if (e == cudaSuccess)
-        e = launch_chained(k_refine<3>, n_chunks, s, keys, p->d_layers, p->d_chunks, p->d_hist, p->d_state);
-    RSDGC_MARK(2);
-    if (e == cudaSuccess)
-        e = launch_chained(k_count, n_chunks, s, keys, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt,
-                           p->d_codes, p->n_layers, (long long)idx_cap, (long long)val_cap, p->d_status);
-    RSDGC_MARK(2);
-    if (e == cudaSuccess)
-        e = launch_chained(k_mark, n_chunks, s, p->d_codes, p->d_layers, p->d_chunks, p->d_state, p->d_chunk_cnt, idx,
-                           (long long)idx_cap);
-    RSDGC_MARK(2);
-    if (e == cudaSuccess)
-        e = launch_chained(k_gather, p->n_sm * 8, s, resid, p->d_layers, p->d_state, p->n_layers, idx,
-                           (long long)idx_cap, val, (long long)val_cap);
-    RSDGC_MARK(2);
-#undef RSDGC_MARK
-    count_launch(5);
+    if (prof >= 1) e = record_event(p, s);
+    launch_accumulate_nsi(p, p->d_hist, p->d_state, grads, resid, vel, mom, ratios, counts, keys, s);
+    if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
+    LaneTable lanes{};
+    lanes.l[0] = Lane{keys, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid, idx, val};
+    if (e == cudaSuccess) e = launch_selection(p, lanes, 1, idx_cap, val_cap, prof, s);
+    if (e != cudaSuccess) return e;
+    return cudaGetLastError();
+}
+
+// Several workers' gradients in one call (the data-parallel replicas that share a GPU): one
+// accumulate+NSI launch per worker, back to back, then ONE launch of each selection kernel and of
+// the gather for all the workers (blockIdx.y = worker).  The short, latency-bound kernels so
+// serve several workers at a time.  With profiling on, stage 0 of a record covers the first
+// passes of all the workers of a group (up to kMaxLanes workers form a group).
+cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *const *grads, float *const *resid,
+                                    const float *ratios, int32_t *const *idx, int64_t idx_cap, float *const *val,
+                                    int64_t val_cap, int32_t *const *counts, uint32_t *keys_all, cudaStream_t s)
+{
+    const size_t key_stride = (size_t)p->info.workspace_bytes / sizeof(uint32_t);
+    const int prof = p->profile;
+    if (prof) p->profile_recorded = prof;
+    cudaError_t e = cudaSuccess;
+    for (int w0 = 0; w0 < n_workers && e == cudaSuccess; w0 += kMaxLanes) {
+        const int n = n_workers - w0 < kMaxLanes ? n_workers - w0 : kMaxLanes;
+        LaneTable lanes{};
+        if (prof >= 1) e = record_event(p, s);
+        for (int j = 0; j < n; ++j) {
+            const int w = w0 + j;
+            Lane &ln = lanes.l[j];
+            if (w == 0) {
+                ln = Lane{keys_all, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid[0], idx[0], val[0]};
+            } else {
+                const rsdgc_plan::LaneScratch &x = p->extra_lanes[(size_t)w - 1];
+                ln = Lane{keys_all + (size_t)w * key_stride, x.hist, x.state, x.chunk_cnt, x.codes, resid[w], idx[w],
+                          val[w]};
+            }
+            launch_accumulate_nsi(p, ln.hist, ln.state, grads[w], ln.resid, nullptr, 0.0f, ratios, counts[w], ln.keys,
+                                  s);
+        }
+        if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
+        if (e == cudaSuccess) e = launch_selection(p, lanes, n, idx_cap, val_cap, prof, s);
+    }
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

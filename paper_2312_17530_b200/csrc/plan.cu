@@ -76,6 +76,13 @@ void free_device_tables(rsdgc_plan *p)
     cudaFree(p->d_survivors);
     cudaFree(p->d_rstate);
     cudaFree(p->d_status);
+    for (rsdgc_plan::LaneScratch &x : p->extra_lanes) {
+        cudaFree(x.state);
+        cudaFree(x.hist);
+        cudaFree(x.codes);
+        cudaFree(x.chunk_cnt);
+    }
+    p->extra_lanes.clear();
     for (cudaEvent_t ev : p->events) cudaEventDestroy(ev);
     p->events.clear();
 }
@@ -470,6 +477,71 @@ extern "C" int rsdgc_compress_momentum(rsdgc_plan *plan, const void *grads_dev, 
     if (!(momentum >= 0.0f && momentum <= 1.0f)) return RSDGC_ERR_INVALID;
     return compress_common(plan, grads_dev, velocity_dev, momentum, residual_dev, ratios_dev, idx_dev, idx_capacity,
                            val_dev, val_capacity, counts_dev, nsi_dev, workspace_dev, stream);
+}
+
+extern "C" int rsdgc_plan_reserve_workers(rsdgc_plan *plan, int32_t n_workers)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (n_workers < 1) return RSDGC_ERR_INVALID;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    while ((int)plan->extra_lanes.size() + 1 < n_workers) {
+        rsdgc_plan::LaneScratch x;
+        cudaError_t e = alloc_zero(&x.state, (size_t)plan->n_layers);
+        if (e == cudaSuccess) e = alloc_zero(&x.hist, (size_t)plan->n_layers * kHistStride);
+        if (e == cudaSuccess) e = alloc_zero(&x.chunk_cnt, plan->chunks.size());
+        if (e == cudaSuccess)
+            e = alloc_zero(&x.codes, (size_t)plan->info.total_tiles_padded / 4 + kChunkKeys / 4 + 16);
+        if (e == cudaSuccess) e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) {
+            cudaFree(x.state);
+            cudaFree(x.hist);
+            cudaFree(x.chunk_cnt);
+            cudaFree(x.codes);
+            return e == cudaErrorMemoryAllocation ? RSDGC_ERR_NOMEM : cuda_fail(e);
+        }
+        plan->extra_lanes.push_back(x);
+    }
+    return RSDGC_OK;
+}
+
+extern "C" int rsdgc_compress_workers(rsdgc_plan *plan, int32_t n_workers, const void *const *grads_dev_host,
+                                      float *const *residual_dev_host, const float *ratios_dev,
+                                      int32_t *const *idx_dev_host, int64_t idx_capacity,
+                                      float *const *val_dev_host, int64_t val_capacity,
+                                      int32_t *const *counts_dev_host, void *workspace_dev, void *stream)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (plan->flags & RSDGC_MOMENTUM) return RSDGC_ERR_INVALID;
+    if (n_workers < 1 || !grads_dev_host || !residual_dev_host || !ratios_dev || !counts_dev_host || !workspace_dev)
+        return RSDGC_ERR_INVALID;
+    if (idx_capacity < 0 || val_capacity < 0) return RSDGC_ERR_INVALID;
+    if ((idx_capacity > 0 && !idx_dev_host) || (val_capacity > 0 && !val_dev_host)) return RSDGC_ERR_INVALID;
+    if ((int)plan->extra_lanes.size() + 1 < n_workers) return RSDGC_ERR_CAPACITY;  // rsdgc_plan_reserve_workers()
+    if (!aligned16(workspace_dev)) return RSDGC_ERR_ALIGNMENT;
+    std::vector<int32_t *> idx((size_t)n_workers, nullptr);
+    std::vector<float *> val((size_t)n_workers, nullptr);
+    for (int w = 0; w < n_workers; ++w) {
+        if (!grads_dev_host[w] || !residual_dev_host[w] || !counts_dev_host[w]) return RSDGC_ERR_INVALID;
+        if (idx_capacity > 0) idx[w] = idx_dev_host[w];
+        if (val_capacity > 0) val[w] = val_dev_host[w];
+        if ((idx_capacity > 0 && !idx[w]) || (val_capacity > 0 && !val[w])) return RSDGC_ERR_INVALID;
+        if (!aligned16(grads_dev_host[w]) || !aligned16(residual_dev_host[w]) || !aligned16(idx[w]) ||
+            !aligned16(val[w]))
+            return RSDGC_ERR_ALIGNMENT;
+        for (int v = 0; v < w; ++v)  // every worker has its own accumulator and payload
+            if (residual_dev_host[v] == residual_dev_host[w] || counts_dev_host[v] == counts_dev_host[w] ||
+                (idx[w] && idx[v] == idx[w]) || (val[w] && val[v] == val[w]))
+                return RSDGC_ERR_INVALID;
+    }
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaError_t e = launch_compress_workers(plan, n_workers, grads_dev_host, residual_dev_host, ratios_dev, idx.data(),
+                                            idx_capacity, val.data(), val_capacity, counts_dev_host,
+                                            reinterpret_cast<uint32_t *>(workspace_dev), (cudaStream_t)stream);
+    return e == cudaSuccess ? RSDGC_OK : cuda_fail(e);
 }
 
 extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_dev, float *residual_dev,

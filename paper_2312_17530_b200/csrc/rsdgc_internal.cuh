@@ -95,6 +95,24 @@ struct LayerState {
     int64_t idx_off, val_off;  // payload offsets of the layer
 };
 
+// One worker of a compress call: its buffers and its own copy of the selection tables.  The
+// selection and gather kernels of a call that serves several workers take one launch each;
+// blockIdx.y picks the lane.
+constexpr int kMaxLanes = 16;
+struct Lane {
+    uint32_t *keys;
+    unsigned int *hist;        // n_layers * kHistStride
+    LayerState *state;         // n_layers
+    uint2 *chunk_cnt;          // one entry per key chunk
+    unsigned char *codes;      // one byte per 4 tiles
+    float *resid;
+    int32_t *idx;
+    float *val;
+};
+struct LaneTable {
+    Lane l[kMaxLanes];
+};
+
 struct RatioState {
     unsigned int ticket;
     uint32_t prefix;
@@ -141,6 +159,14 @@ struct rsdgc_plan {
     uint32_t *d_hist = nullptr;        // n_layers * kHistStride
     unsigned char *d_codes = nullptr;  // one byte per 4 tiles: above / equal flags left by k_count for k_mark
     uint2 *d_chunk_cnt = nullptr;      // per key chunk: (#key > T, #key == T), then exclusive bases
+    // the same four tables for workers 1.. of rsdgc_compress_workers() (worker 0 uses the ones above)
+    struct LaneScratch {
+        rsdgc::LayerState *state = nullptr;
+        uint32_t *hist = nullptr;
+        unsigned char *codes = nullptr;
+        uint2 *chunk_cnt = nullptr;
+    };
+    std::vector<LaneScratch> extra_lanes;
     long long *d_survivors = nullptr;  // ratio rule: per-layer survivor counts
     rsdgc::RatioState *d_rstate = nullptr;
     rsdgc::StatusDev *d_status = nullptr;
@@ -161,6 +187,9 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *layers, int n_layer
 cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
                             const float *ratios, int32_t *idx, int64_t idx_cap, float *val, int64_t val_cap,
                             int32_t *counts, uint32_t *keys, cudaStream_t s);
+cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *const *grads, float *const *resid,
+                                    const float *ratios, int32_t *const *idx, int64_t idx_cap, float *const *val,
+                                    int64_t val_cap, int32_t *const *counts, uint32_t *keys_all, cudaStream_t s);
 cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long n_keep,
                                  float *ratios, cudaStream_t s);
 cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const float *const *val,
@@ -169,7 +198,8 @@ void count_launch(int n);
 void set_last_cuda_error(int e);
 int k1_reg_ctas_per_sm(int dtype, bool momentum);
 int k1_bulk_ctas_per_sm(bool momentum);
-int launch_accumulate_nsi(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
-                          const float *ratios, int32_t *counts, uint32_t *keys, cudaStream_t s);
+int launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
+                          float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
+                          cudaStream_t s);
 
 }  // namespace rsdgc

@@ -169,6 +169,54 @@ def compress_and_check(oracle, plan: binding.Plan, shapes, grads: Sequence[np.nd
     return new_res, refs, gc
 
 
+def compress_workers_and_check(oracle, plan: binding.Plan, shapes, grads_w, residuals_w, ratios, alpha: float,
+                               clamp: bool = True, what: str = "", max_ratio: float = 1.0, device="cuda:0"):
+    """One rsdgc_compress_workers() call for len(grads_w) workers; every worker's outputs are
+    checked against the oracle like a single rsdgc_compress() call (the indicators are read from
+    the worker's part of the workspace, where the call leaves them as keys).  Returns
+    (new residuals per worker and layer, oracle results per worker, payload tensors per worker)."""
+    W = len(grads_w)
+    plan.reserve_workers(W)
+    ni, nv = plan.payload_bound(max_ratio)
+    d_g = [dev(to_arena(plan, g, np.uint16 if g[0].dtype == np.uint16 else np.float32)) for g in grads_w]
+    r_arenas = [to_arena(plan, r) for r in residuals_w]
+    d_r = [dev(a) for a in r_arenas]
+    idx = [torch.full((max(ni, 4),), -1, dtype=torch.int32, device=device) for _ in range(W)]
+    val = [torch.full((max(nv, 4),), float(CANARY), dtype=torch.float32, device=device) for _ in range(W)]
+    cnt = [torch.full((plan.n_layers,), -1, dtype=torch.int32, device=device) for _ in range(W)]
+    stride = plan.info.workspace_bytes // 4
+    ws = torch.full((W * stride,), float(CANARY), dtype=torch.float32, device=device)
+    d_ratios = torch.tensor(np.asarray(ratios, dtype=np.float32), device=device)
+    plan.compress_workers(d_g, d_r, d_ratios, idx, val, cnt, ws)
+    torch.cuda.synchronize()
+    st = plan.status()
+    assert st.flags == 0, "%s: status flags %d" % (what, st.flags)
+    pad = padding_mask(plan)
+    keys = ws.cpu().numpy()
+    new_res_w, refs_w = [], []
+    for w in range(W):
+        res_arena = d_r[w].cpu().numpy()
+        assert (res_arena[pad] == CANARY).all(), what + ": padding of a residual arena was written"
+        counts, ix, vl = cnt[w].cpu().numpy(), idx[w].cpu().numpy(), val[w].cpu().numpy()
+        nsi = keys[w * stride:(w + 1) * stride]
+        io = vo = 0
+        refs, new_res = [], []
+        for l, (li, shape) in enumerate(zip(plan.layers, shapes)):
+            k, slot = int(counts[l]), shape[2] * shape[3]
+            ref = check_layer(oracle, li, shape, grads_w[w][l], residuals_w[w][l], float(np.float32(ratios[l])),
+                              alpha, clamp, nsi[li.tile_offset:li.tile_offset + li.n_tiles], k, ix[io:io + k],
+                              vl[vo:vo + k * slot], res_arena[li.elem_offset:li.elem_offset + li.rows * li.cols],
+                              what="%s worker %d layer %d %r" % (what, w, l, tuple(shape)))
+            io, vo = io + k, vo + k * slot
+            refs.append(ref)
+            new_res.append(ref.residual)
+        assert st.idx_needed == io and st.val_needed == vo
+        assert (ix[io:] == -1).all() and (vl[vo:] == CANARY).all(), what + ": payload written past its end"
+        new_res_w.append(new_res)
+        refs_w.append(refs)
+    return new_res_w, refs_w, list(zip(idx, val, cnt))
+
+
 def check_decompress(dense_gpu: np.ndarray, dense_ref: np.ndarray, abs_sent_sum: np.ndarray, exact: bool = True):
     """R3 (and bit-exactness, which holds because workers are added in order on both sides)."""
     assert (np.abs(dense_gpu.astype(np.float64) - dense_ref) <= 1e-6 * abs_sent_sum + 1e-45).all()

@@ -52,6 +52,26 @@ def test_vgg19_four_workers_full_size(oracle):
     fc6_tiles = np.concatenate([refs_all[w].layers[32].idx for w in range(4)])
     assert int((np.bincount(fc6_tiles) > 1).sum()) > 1000
 
+    # the same four workers through one rsdgc_compress_workers() call (what the benchmark times):
+    # bit-identical payloads and residuals to the per-worker calls checked above
+    plan.reserve_workers(4)
+    d_g = [parity.dev(parity.to_arena(plan, grads[w])) for w in range(4)]
+    d_r = [torch.zeros(plan.info.arena_elems, device="cuda:0") for _ in range(4)]
+    ni, nv = plan.payload_bound(1 / 64)
+    idx = [torch.full((ni,), -1, dtype=torch.int32, device="cuda:0") for _ in range(4)]
+    val = [torch.full((nv,), float(parity.CANARY), device="cuda:0") for _ in range(4)]
+    cnt = [torch.zeros(plan.n_layers, dtype=torch.int32, device="cuda:0") for _ in range(4)]
+    ws = torch.empty(4 * plan.info.workspace_bytes, dtype=torch.uint8, device="cuda:0")
+    plan.compress_workers(d_g, d_r, torch.tensor(ratios, device="cuda:0"), idx, val, cnt, ws)
+    torch.cuda.synchronize()
+    assert plan.status().flags == 0
+    for w in range(4):
+        assert torch.equal(idx[w], payloads[w][0]) and torch.equal(cnt[w], payloads[w][2])
+        assert torch.equal(val[w].view(torch.int32), payloads[w][1].view(torch.int32))
+        res = parity.from_arena(plan, d_r[w].cpu().numpy())
+        for l in (0, 17, 32, 34, 36, 37):
+            np.testing.assert_array_equal(res[l].view(np.uint32), refs_all[w].layers[l].residual.view(np.uint32))
+
 
 # ---------------------------------------------------------------------------------------------
 # config 4: ResNet-50-shaped set, 100 iterations, scales drift, ratios refreshed every 10

@@ -211,6 +211,50 @@ def test_decompress_accumulate_four_workers(oracle, scale):
     assert torch.equal(before, d_dense)
 
 
+# ---------------------------------------------------------------------------------------------
+# several workers in one call: the selection kernels run once over all workers
+# ---------------------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("n_workers", [1, 3])
+def test_compress_workers_two_iterations(oracle, n_workers):
+    shapes = [(300, 515, 3, 3), (256, 64 * 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3), (1200, 1536, 3, 3),
+              (64, 7 * 7 * 3, 1, 49), (5, 5, 3, 3)]
+    tensors = [("t%d" % i, (s[0], s[1])) for i, s in enumerate(shapes)]
+    plan = binding.Plan(shapes, alpha=0.5)
+    sig = synth.log_uniform_scales(len(shapes), (21,))
+    ratios = np.array([1 / 16, 1 / 50, 0.3, 1.0, 1 / 64, 0.0, 0.5], np.float32)
+    res = [[np.zeros(s[0] * s[1], np.float32) for s in shapes] for _ in range(n_workers)]
+    for it in range(2):                     # the second call starts from the tables the first one left
+        grads = synth.multi_worker_gradients(tensors, n_workers, (21, it), sig)
+        res, refs, payloads = parity.compress_workers_and_check(oracle, plan, shapes, grads, res, ratios, 0.5,
+                                                                what="iteration %d" % it)
+    for w in range(n_workers):
+        assert int(payloads[w][2].sum()) == sum(r.k for r in refs[w])
+
+
+def test_compress_workers_argument_errors():
+    plan = binding.Plan([(64, 64, 3, 3)], alpha=0.5)
+    dev = "cuda:0"
+    g = [torch.zeros(plan.info.arena_elems, device=dev) for _ in range(2)]
+    r = [torch.zeros(plan.info.arena_elems, device=dev) for _ in range(2)]
+    ni, nv = plan.payload_bound(1.0)
+    idx = [torch.zeros(ni, dtype=torch.int32, device=dev) for _ in range(2)]
+    val = [torch.zeros(nv, device=dev) for _ in range(2)]
+    cnt = [torch.zeros(1, dtype=torch.int32, device=dev) for _ in range(2)]
+    ws = torch.zeros(2 * plan.info.workspace_bytes, dtype=torch.uint8, device=dev)
+    rat = torch.ones(1, device=dev)
+    with pytest.raises(binding.RsdgcError) as e:      # lanes not reserved
+        plan.compress_workers(g, r, rat, idx, val, cnt, ws)
+    assert e.value.code == binding.ERR_CAPACITY
+    plan.reserve_workers(2)
+    with pytest.raises(binding.RsdgcError) as e:      # two workers share an accumulator
+        plan.compress_workers(g, [r[0], r[0]], rat, idx, val, cnt, ws)
+    assert e.value.code == binding.ERR_INVALID
+    plan.compress_workers(g, r, rat, idx, val, cnt, ws)
+    torch.cuda.synchronize()
+    assert plan.status().flags == 0 and int(cnt[1][0]) == plan.layers[0].n_tiles
+
+
 def test_bf16_gradients(oracle):
     shapes = [(300, 515, 3, 3), (128, 64 * 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3)]
     rng = np.random.default_rng(9)
