@@ -315,6 +315,14 @@ def run_b200(args):
         ev1.record()
         torch.cuda.synchronize()
         extra["dense_zero_fill_us"] = ev0.elapsed_time(ev1) / 3 * 1e3
+        payloads = [(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)]
+        plan.decompress_assign(payloads, d_dense, 1.0)
+        ev0.record()
+        for _ in range(3):
+            plan.decompress_assign(payloads, d_dense, 1.0)  # zero fill + aggregation in one launch
+        ev1.record()
+        torch.cuda.synchronize()
+        extra["decompress_assign_us"] = ev0.elapsed_time(ev1) / 3 * 1e3
 
     # ---- separately timed: the momentum-corrected variant (20 algorithmic bytes per element)
     if rank == 0 and args.workload == "vgg19":

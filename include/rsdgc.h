@@ -277,6 +277,18 @@ int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,
                                 float *dense_dev, void *stream);
 
 /*
+ * The same aggregation into a dense arena that holds nothing yet (Eq. 12, third line, as an
+ * assignment: g_t = scale * sum over workers of sparse(v)):
+ *   dense[i] = +0, then dense[i] = dense[i] + scale * sent_w[i] for w = 0 .. n_workers-1,
+ * i.e. exactly a zero fill of every layer's elements followed by rsdgc_decompress_accumulate(),
+ * in the same launch (no separate pass over the arena).  Padding elements between layers are
+ * not written.  n_workers = 0 gives all +0.  Arguments and errors as above.
+ */
+int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
+                            const float *const *val_dev_host, const int32_t *const *counts_dev_host,
+                            float scale, float *dense_dev, void *stream);
+
+/*
  * Optional per-kernel timing of rsdgc_compress().  While enabled, every rsdgc_compress() on
  * this plan records CUDA events on its stream: with level 1 only before and after the first
  * pass (accumulate+NSI, the kernel that moves all the bytes), with level 2 after each of the

@@ -251,3 +251,11 @@ def decompress_accumulate(shapes: Sequence[LayerShape], dense: Sequence[np.ndarr
     for w in payloads:
         for shape, d, lr in zip(shapes, dense, w.layers):
             decompress_into(d, shape, lr.idx, lr.val, scale)
+
+
+def decompress_assign(shapes: Sequence[LayerShape], dense: Sequence[np.ndarray],
+                      payloads: Sequence[CompressResult], scale: float = 1.0) -> None:
+    """Eq. 12 third line as an assignment: dense_l = +0, then the workers are added in order."""
+    for d in dense:
+        d[...] = np.float32(0.0)
+    decompress_accumulate(shapes, dense, payloads, scale)

@@ -26,7 +26,7 @@ EXPORTS = [
     "rsdgc_compress_host", "rsdgc_decompress_accumulate", "rsdgc_get_status", "rsdgc_launch_count",
     "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
     "rsdgc_update_ratios_noalloc", "rsdgc_compress_momentum", "rsdgc_plan_reserve_workers",
-    "rsdgc_compress_workers",
+    "rsdgc_compress_workers", "rsdgc_decompress_assign",
 ]
 NOALLOC_MAX_LAYERS = 64
 N_COMPRESS_KERNELS = 6
@@ -90,6 +90,7 @@ def lib():
         L.rsdgc_compress_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, vp,
                                           C.POINTER(i64), C.POINTER(i64), vp]
         L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
+        L.rsdgc_decompress_assign.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
         L.rsdgc_get_status.argtypes = [vp, vp, C.POINTER(Status)]
         L.rsdgc_profile_enable.argtypes = [vp, i32]
         L.rsdgc_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
@@ -219,15 +220,20 @@ class Plan:
                                          C.byref(ni), C.byref(nv), _stream()), "rsdgc_compress_host")
         return ni.value, nv.value
 
-    def decompress_accumulate(self, payloads, dense, scale: float = 1.0) -> None:
-        """``payloads``: sequence of (idx, val, counts) device tensors, one per worker."""
+    def decompress_accumulate(self, payloads, dense, scale: float = 1.0, assign: bool = False) -> None:
+        """``payloads``: sequence of (idx, val, counts) device tensors, one per worker.  ``assign``:
+        rsdgc_decompress_assign() (the arena is zero-filled by the same launch)."""
         n = len(payloads)
         A = C.c_void_p * max(1, n)
         ia, va, ca = A(), A(), A()
         for w, (i, v, c) in enumerate(payloads):
             ia[w], va[w], ca[w] = i.data_ptr(), v.data_ptr(), c.data_ptr()
-        _check(lib().rsdgc_decompress_accumulate(self._h, n, ia, va, ca, scale, _ptr(dense), _stream()),
-               "rsdgc_decompress_accumulate")
+        fn = lib().rsdgc_decompress_assign if assign else lib().rsdgc_decompress_accumulate
+        _check(fn(self._h, n, ia, va, ca, scale, _ptr(dense), _stream()),
+               "rsdgc_decompress_assign" if assign else "rsdgc_decompress_accumulate")
+
+    def decompress_assign(self, payloads, dense, scale: float = 1.0) -> None:
+        self.decompress_accumulate(payloads, dense, scale, assign=True)
 
     def profile_enable(self, level: int) -> None:
         """0 off; 1 events around the first pass only; 2 events around every kernel."""

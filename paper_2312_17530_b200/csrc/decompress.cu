@@ -9,6 +9,10 @@
 // dense arena is only ever touched by the CTA that owns its tile, in worker order, with plain
 // read-modify-write, so the binary32 sums are reproducible (no atomics) although all workers
 // are processed by one launch.
+//
+// The ASSIGN variant first stores +0 to every element of the chunk's tiles (the dense arena then
+// needs no separate zero fill, and the read-modify-writes that follow find their lines in L2),
+// so that dense = scale * sum of the workers' payloads.
 #include "device_utils.cuh"
 
 namespace rsdgc {
@@ -50,6 +54,46 @@ __device__ __forceinline__ int warp_lower_bound(const int32_t *a, int n, int key
     return lo;
 }
 
+// Stores +0 to dense[begin, end): scalar stores up to the first 16-byte boundary and after the
+// last one, 128-bit stores in between; all threads of the CTA take part.
+__device__ __forceinline__ void zero_span(float *__restrict__ dense, long long begin, long long end)
+{
+    if (end <= begin) return;
+    const int tid = threadIdx.x;
+    const long long body0 = min(end, (begin + 3) & ~3ll), body1 = max(body0, end & ~3ll);
+    if (begin + tid < body0) dense[begin + tid] = 0.0f;
+    if (body1 + tid < end) dense[body1 + tid] = 0.0f;
+    float4 *d4 = reinterpret_cast<float4 *>(dense + body0);
+    const long long n4 = (body1 - body0) >> 2;
+    for (long long i = tid; i < n4; i += kThreads) d4[i] = make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+}
+
+// +0 to every element of the tiles [c.start, c.start + c.n) of layer L: a partial first tile
+// row, a contiguous run of whole tile rows, a partial last tile row.
+__device__ __forceinline__ void zero_chunk(float *__restrict__ dense, const LayerDev &L, const Chunk &c)
+{
+    const int t_last = c.start + c.n - 1;
+    const int tr0 = c.start / L.TC, tc0 = c.start - tr0 * L.TC;
+    const int tr1 = t_last / L.TC, tc1 = t_last - tr1 * L.TC;
+    const bool head_partial = tc0 != 0, tail_partial = tc1 != L.TC - 1;
+    auto rows_of = [&](int tr, long long cb, long long ce) {  // columns [cb, ce) of the rows of tile row tr
+        const long long r_end = min((long long)L.rows, ((long long)tr + 1) * L.nh);
+        for (long long r = (long long)tr * L.nh; r < r_end; ++r)
+            zero_span(dense, L.elem_off + r * L.cols + cb, L.elem_off + r * L.cols + ce);
+    };
+    if (tr0 == tr1 && (head_partial || tail_partial)) {
+        rows_of(tr0, (long long)tc0 * L.nw, min((long long)L.cols, ((long long)tc1 + 1) * L.nw));
+        return;
+    }
+    if (head_partial) rows_of(tr0, (long long)tc0 * L.nw, L.cols);
+    if (tail_partial) rows_of(tr1, 0, min((long long)L.cols, ((long long)tc1 + 1) * L.nw));
+    const long long full0 = tr0 + (head_partial ? 1 : 0), full1 = tr1 - (tail_partial ? 1 : 0);  // inclusive
+    if (full1 >= full0)
+        zero_span(dense, L.elem_off + full0 * L.nh * L.cols,
+                  L.elem_off + min((long long)L.rows, (full1 + 1) * L.nh) * L.cols);
+}
+
+template <bool ASSIGN>
 __global__ void __launch_bounds__(kThreads)
 k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restrict__ layers,
              const Chunk *__restrict__ chunks, float scale, float *__restrict__ dense)
@@ -59,6 +103,7 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
     const LayerDev L = layers[c.layer];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int W = wp.n_workers;
+    if (ASSIGN) zero_chunk(dense, L, c);  // made visible to the whole CTA by the barrier below
 
     // ---- per worker (one warp each, round-robin): payload offsets of this layer = sums of the
     // counts of the preceding layers, and the run of entries that falls into the chunk
@@ -126,12 +171,16 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
     }
 }
 
-// Applies workers [0, n_workers) in order; groups of kMaxWorkersPerLaunch go into one launch
+// Applies workers [0, n_workers) in order (after the zero fill of the ASSIGN variant); groups of kMaxWorkersPerLaunch go into one launch
 // each, and the stream orders the groups.
 cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const float *const *val,
-                              const int32_t *const *counts, float scale, float *dense, cudaStream_t s)
+                              const int32_t *const *counts, float scale, float *dense, bool assign, cudaStream_t s)
 {
     const int n_chunks = (int)p->chunks.size();
+    if (assign && n_workers == 0) {  // nothing was sent: the result is all +0
+        k_decompress<true><<<n_chunks, kThreads, 0, s>>>(WorkerPayloads{}, p->d_layers, p->d_chunks, scale, dense);
+        count_launch(1);
+    }
     for (int w0 = 0; w0 < n_workers; w0 += kMaxWorkersPerLaunch) {
         WorkerPayloads wp{};
         wp.n_workers = n_workers - w0 < kMaxWorkersPerLaunch ? n_workers - w0 : kMaxWorkersPerLaunch;
@@ -140,7 +189,8 @@ cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const
             wp.val[w] = val[w0 + w];
             wp.counts[w] = counts[w0 + w];
         }
-        k_decompress<<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense);
+        if (assign && w0 == 0) k_decompress<true><<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense);
+        else k_decompress<false><<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense);
         count_launch(1);
     }
     return cudaGetLastError();

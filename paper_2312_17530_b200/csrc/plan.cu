@@ -584,10 +584,11 @@ extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, voi
     return RSDGC_OK;
 }
 
-extern "C" int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
-                                           const float *const *val_dev_host,
-                                           const int32_t *const *counts_dev_host, float scale, float *dense_dev,
-                                           void *stream)
+namespace {
+
+int decompress_common(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
+                      const float *const *val_dev_host, const int32_t *const *counts_dev_host, float scale,
+                      float *dense_dev, bool assign, void *stream)
 {
     int rc = check_plan_device(plan);
     if (rc) return rc;
@@ -601,12 +602,31 @@ extern "C" int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers, 
     DeviceGuard guard(plan->device);
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
     // every dense element is updated by one CTA, worker after worker: reproducible binary32 sums
-    if (n_workers > 0) {
+    if (n_workers > 0 || assign) {
         cudaError_t e = launch_decompress(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, scale,
-                                          dense_dev, (cudaStream_t)stream);
+                                          dense_dev, assign, (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return RSDGC_OK;
+}
+
+}  // namespace
+
+extern "C" int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
+                                           const float *const *val_dev_host,
+                                           const int32_t *const *counts_dev_host, float scale, float *dense_dev,
+                                           void *stream)
+{
+    return decompress_common(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, scale, dense_dev, false,
+                             stream);
+}
+
+extern "C" int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
+                                       const float *const *val_dev_host, const int32_t *const *counts_dev_host,
+                                       float scale, float *dense_dev, void *stream)
+{
+    return decompress_common(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, scale, dense_dev, true,
+                             stream);
 }
 
 extern "C" int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *out_host)

@@ -193,7 +193,8 @@ cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *co
 cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long n_keep,
                                  float *ratios, cudaStream_t s);
 cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const float *const *val,
-                              const int32_t *const *counts, float scale, float *dense, cudaStream_t s);
+                              const int32_t *const *counts, float scale, float *dense, bool assign,
+                              cudaStream_t s);
 void count_launch(int n);
 void set_last_cuda_error(int e);
 int k1_reg_ctas_per_sm(int dtype, bool momentum);

@@ -48,6 +48,12 @@ def test_vgg19_four_workers_full_size(oracle):
     oracle.decompress_accumulate(shapes, dense_ref, refs_all, 1.0)
     for got, ref in zip(parity.from_arena(plan, d_dense.cpu().numpy()), dense_ref):
         np.testing.assert_array_equal(got.view(np.uint32), ref.view(np.uint32))
+    d_dense2 = torch.full((plan.info.arena_elems,), float("nan"), device="cuda:0")
+    plan.decompress_assign(payloads, d_dense2, 1.0)          # zero fill fused into the same launch
+    torch.cuda.synchronize()
+    assert torch.equal(d_dense.view(torch.int32)[~torch.from_numpy(parity.padding_mask(plan)).cuda()],
+                       d_dense2.view(torch.int32)[~torch.from_numpy(parity.padding_mask(plan)).cuda()])
+    del d_dense2
     # the workers' selections overlap (shared gradient component): the scatter-add does collide
     fc6_tiles = np.concatenate([refs_all[w].layers[32].idx for w in range(4)])
     assert int((np.bincount(fc6_tiles) > 1).sum()) > 1000

@@ -202,6 +202,21 @@ def test_decompress_accumulate_four_workers(oracle, scale):
         collisions += int((hit > 1).sum())
         parity.check_decompress(got, ref, abs_sum)
     assert collisions > 1000                                   # the workers' selections do overlap
+    # the assigning variant: whatever the arena held is replaced, the padding is left alone
+    d_dense2 = parity.dev(parity.to_arena(plan, [np.full(synth.numel(s), np.nan, np.float32) for _, s in tensors]))
+    plan.decompress_assign(payloads, d_dense2, scale)
+    torch.cuda.synchronize()
+    assign_ref = [np.full(synth.numel(s), 3.0, np.float32) for _, s in tensors]
+    oracle.decompress_assign(shapes, assign_ref, refs_all, scale)
+    out2 = d_dense2.cpu().numpy()
+    assert (out2[parity.padding_mask(plan)] == parity.CANARY).all()
+    for got, ref in zip(parity.from_arena(plan, out2), assign_ref):
+        np.testing.assert_array_equal(got.view(np.uint32), ref.view(np.uint32))
+    plan.decompress_assign([], d_dense2, scale)               # no worker: all +0
+    torch.cuda.synchronize()
+    out2 = d_dense2.cpu().numpy()
+    assert (out2[parity.padding_mask(plan)] == parity.CANARY).all()
+    assert all((x.view(np.uint32) == 0).all() for x in parity.from_arena(plan, out2))
     # empty payload: nothing changes
     before = d_dense.clone()
     zc = torch.zeros(plan.n_layers, dtype=torch.int32, device="cuda:0")
@@ -253,6 +268,31 @@ def test_compress_workers_argument_errors():
     plan.compress_workers(g, r, rat, idx, val, cnt, ws)
     torch.cuda.synchronize()
     assert plan.status().flags == 0 and int(cnt[1][0]) == plan.layers[0].n_tiles
+
+
+def test_decompress_assign_ragged_layers(oracle):
+    shapes = [(300, 515, 3, 3), (5, 5, 3, 3), (1, 1000, 1, 9), (77, 45, 3, 3), (64, 147, 1, 49), (1, 1, 3, 3),
+              (40000, 3, 3, 3), (2, 70001, 3, 3), (131, 131, 7, 5)]
+    tensors = [("t%d" % i, (s[0], s[1])) for i, s in enumerate(shapes)]
+    plan = binding.Plan(shapes, alpha=0.5)
+    sig = synth.log_uniform_scales(len(shapes), (31,))
+    grads = synth.multi_worker_gradients(tensors, 2, (31,), sig)
+    ratios = np.array([0.1, 1.0, 0.3, 0.02, 0.5, 1.0, 0.01, 0.2, 0.05], np.float32)
+    zeros = [np.zeros(s[0] * s[1], np.float32) for s in shapes]
+    payloads, refs_all = [], []
+    for w in range(2):
+        _, refs, gc = parity.compress_and_check(oracle, plan, shapes, grads[w], zeros, ratios, 0.5, what="w%d" % w)
+        payloads.append(gc.payload())
+        refs_all.append(oracle.CompressResult(layers=refs))
+    d_dense = parity.dev(parity.to_arena(plan, [np.full(s[0] * s[1], -5.0, np.float32) for s in shapes]))
+    plan.decompress_assign(payloads, d_dense, 0.5)
+    torch.cuda.synchronize()
+    ref = [np.full(s[0] * s[1], 9.0, np.float32) for s in shapes]
+    oracle.decompress_assign(shapes, ref, refs_all, 0.5)
+    out = d_dense.cpu().numpy()
+    assert (out[parity.padding_mask(plan)] == parity.CANARY).all()
+    for l, (got, want) in enumerate(zip(parity.from_arena(plan, out), ref)):
+        np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32), err_msg="layer %d" % l)
 
 
 def test_bf16_gradients(oracle):

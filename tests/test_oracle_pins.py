@@ -374,6 +374,12 @@ def test_decompress_special_cases(oracle):
     d2 = np.ones(100, np.float32)
     oracle.decompress_into(d2, shape, res.idx, res.val, 0.25)
     np.testing.assert_array_equal(d2, np.float32(1) + np.float32(0.25) * sent)
+    # the assigning form forgets what the buffer held and is otherwise the same sum
+    d3 = [np.full(100, np.nan, np.float32)]
+    cr = oracle.CompressResult(layers=[res])
+    oracle.decompress_assign([shape], d3, [cr, cr], 0.5)
+    np.testing.assert_array_equal(d3[0], sent)                      # 0 + sent/2 + sent/2, exact in binary
+    assert not np.signbit(d3[0][sent == 0]).any()                   # untouched entries are +0
 
 
 # ---------------------------------------------------------------------------------------------
