@@ -72,6 +72,10 @@ def lib():
         L.rsdgc_oracle_select.argtypes = [p, i64, i64, p]
         L.rsdgc_oracle_pack.restype = None
         L.rsdgc_oracle_pack.argtypes = [p, i64, i64, i32, i32, p, i64, p, p]
+        L.rsdgc_oracle_pack_bf16.restype = None
+        L.rsdgc_oracle_pack_bf16.argtypes = [p, i64, i64, i32, i32, p, i64, p, p]
+        L.rsdgc_oracle_f32_to_bf16.restype = C.c_uint16
+        L.rsdgc_oracle_f32_to_bf16.argtypes = [f32]
         L.rsdgc_oracle_decompress.restype = None
         L.rsdgc_oracle_decompress.argtypes = [p, i64, i64, i32, i32, p, p, i64, f32]
         L.rsdgc_oracle_update_ratios.restype = i64
@@ -164,6 +168,24 @@ def pack(v: np.ndarray, shape: LayerShape, sel: np.ndarray):
     return idx, val, res
 
 
+def f32_to_bf16(x: float) -> int:
+    """Bit pattern of the bfloat16 nearest to the binary32 ``x`` (ties to even)."""
+    return int(lib().rsdgc_oracle_f32_to_bf16(float(np.float32(x))))
+
+
+def pack_bf16(v: np.ndarray, shape: LayerShape, sel: np.ndarray):
+    """(idx, val_bits uint16, new_residual): the payload with bfloat16 values; the rounding
+    error of every sent value stays in the accumulator."""
+    rows, cols, nh, nw = shape
+    res = _f32(v).copy()
+    sel = np.ascontiguousarray(sel, dtype=np.int32)
+    k = sel.size
+    idx = np.empty(k, dtype=np.int32)
+    bits = np.empty(k * nh * nw, dtype=np.uint16)
+    lib().rsdgc_oracle_pack_bf16(_ptr(res), rows, cols, nh, nw, _ptr(sel), k, _ptr(idx), _ptr(bits))
+    return idx, bits, res
+
+
 def decompress_into(dense: np.ndarray, shape: LayerShape, idx: np.ndarray, val: np.ndarray, scale: float) -> None:
     """dense += scale * payload for one layer and one worker, in place (Eq. 12, Eq. 2)."""
     rows, cols, nh, nw = shape
@@ -202,6 +224,7 @@ class LayerResult:
     residual: np.ndarray     # float32 [rows * cols], new accumulator
     nonfinite: int = 0
     velocity: Optional[np.ndarray] = None  # new u when momentum correction is on
+    val_bf16: Optional[np.ndarray] = None  # uint16 [k * nh * nw] when the payload values are bfloat16
 
 
 @dataclass
@@ -215,7 +238,8 @@ class CompressResult:
 
 def compress_layer(g: np.ndarray, r: np.ndarray, shape: LayerShape, ratio: float, alpha: float,
                    clamp_min1: bool = True, forced_sel: Optional[np.ndarray] = None,
-                   velocity: Optional[np.ndarray] = None, momentum: float = 0.0) -> LayerResult:
+                   velocity: Optional[np.ndarray] = None, momentum: float = 0.0,
+                   payload_bf16: bool = False) -> LayerResult:
     """One layer of the per-iteration half of Algorithm 1.
 
     ``forced_sel`` replaces the ranking step by a given ascending tile set (used by the
@@ -232,9 +256,14 @@ def compress_layer(g: np.ndarray, r: np.ndarray, shape: LayerShape, ratio: float
     else:
         sel = np.ascontiguousarray(forced_sel, dtype=np.int32)
         thr = float(f32[sel].min()) if sel.size else 0.0
-    idx, val, res = pack(v, shape, sel)
+    bits = None
+    if payload_bf16:
+        idx, bits, res = pack_bf16(v, shape, sel)
+        val = (bits.astype(np.uint32) << 16).view(np.float32)  # the values the receiver sees
+    else:
+        idx, val, res = pack(v, shape, sel)
     return LayerResult(v=v, nsi_ref=ref, nsi_f32=f32, k=k, sel=sel, threshold=thr, idx=idx, val=val,
-                       residual=res, nonfinite=nonfinite, velocity=u_new)
+                       residual=res, nonfinite=nonfinite, velocity=u_new, val_bf16=bits)
 
 
 def compress(shapes: Sequence[LayerShape], grads: Sequence[np.ndarray], residuals: Sequence[np.ndarray],

@@ -232,6 +232,54 @@ void rsdgc_oracle_pack(float *v, int64_t rows, int64_t cols, int32_t nh, int32_t
     }
 }
 
+/* binary32 -> bfloat16 (1 sign, 8 exponent, 7 fraction bits: the upper half of a binary32
+ * word), round to nearest, ties to even; overflow goes to infinity as IEEE rounding does.
+ * NaN stays a quiet NaN with its sign. */
+uint16_t rsdgc_oracle_f32_to_bf16(float x)
+{
+    uint32_t b;
+    memcpy(&b, &x, sizeof b);
+    if ((b & 0x7FFFFFFFu) > 0x7F800000u) return (uint16_t)((b >> 16) | 0x0040u);
+    const uint32_t lower = b & 0xFFFFu, upper = b >> 16;
+    uint32_t q = upper;
+    if (lower > 0x8000u || (lower == 0x8000u && (upper & 1u))) q = upper + 1u; /* carries into the exponent as it must */
+    return (uint16_t)q;
+}
+
+float rsdgc_oracle_bf16_to_f32(uint16_t h)
+{
+    const uint32_t b = (uint32_t)h << 16;
+    float x;
+    memcpy(&x, &b, sizeof x);
+    return x;
+}
+
+/* The same payload with 16-bit values (an option of this implementation, not of the paper):
+ * q = bfloat16(v) is what is sent, and the accumulator keeps v - q, the part of v that was
+ * not sent (Eq. 12: what is not transmitted stays in v); the subtraction is exact in
+ * binary32.  Clipped tiles are padded with +0. */
+void rsdgc_oracle_pack_bf16(float *v, int64_t rows, int64_t cols, int32_t nh, int32_t nw,
+                            const int32_t *sel, int64_t k, int32_t *idx, uint16_t *val)
+{
+    const int64_t TC = ceil_div(cols, nw);
+    const int64_t slot = (int64_t)nh * nw;
+    for (int64_t s = 0; s < k; ++s) {
+        const int64_t t = sel[s], tr = t / TC, tc = t % TC;
+        idx[s] = (int32_t)t;
+        for (int32_t a = 0; a < nh; ++a)
+            for (int32_t b = 0; b < nw; ++b) {
+                const int64_t i = tr * nh + a, j = tc * nw + b;
+                uint16_t q = 0;
+                if (i < rows && j < cols) {
+                    const float x = v[i * cols + j];
+                    q = rsdgc_oracle_f32_to_bf16(x);
+                    v[i * cols + j] = x - rsdgc_oracle_bf16_to_f32(q);
+                }
+                val[s * slot + a * nw + b] = q;
+            }
+    }
+}
+
 /* Aggregation of one worker's payload into the dense gradient of one layer
  * (Eq. 12, third line: sum over workers of sparse(v); Eq. 2, Sync):
  * dense[i] = dense[i] + scale * sent[i], product then sum, each rounded to binary32.

@@ -383,6 +383,66 @@ def test_decompress_special_cases(oracle):
 
 
 # ---------------------------------------------------------------------------------------------
+# payload with bfloat16 values (an option of the implementation; Eq. 12: the unsent part stays)
+# ---------------------------------------------------------------------------------------------
+
+def test_bf16_rounding_known_values_and_library_routine(oracle):
+    two = lambda e: float(2.0 ** e)
+    cases = [
+        (1.0, 0x3F80), (-1.0, 0xBF80), (0.0, 0x0000), (-0.0, 0x8000),
+        (1.0 + two(-8), 0x3F80),                    # tie between 0x3F80 and 0x3F81: even wins
+        (1.0 + two(-8) + two(-23), 0x3F81),         # just above the tie
+        (1.0 + 3 * two(-8), 0x3F82),                # tie between 0x3F81 and 0x3F82: even wins
+        (1.0 + two(-7), 0x3F81),                    # exactly representable
+        (float(np.float32(3.4028234663852886e38)), 0x7F80),   # largest binary32 rounds up to +inf
+        (two(-133), 0x0001),                        # a bfloat16 subnormal, exact
+        (two(-134), 0x0000),                        # tie between 0 and the smallest subnormal: even (0)
+        (3 * two(-134), 0x0002),                    # tie between 1 and 2 subnormal steps: even (2)
+        (float("inf"), 0x7F80), (float("-inf"), 0xFF80),
+    ]
+    for x, bits in cases:
+        assert oracle.f32_to_bf16(x) == bits, (x, hex(oracle.f32_to_bf16(x)), hex(bits))
+    assert (oracle.f32_to_bf16(float("nan")) & 0x7FFF) > 0x7F80
+    # the same conversion as the tensor library's cast on random finite values of every magnitude
+    import torch
+    rng = np.random.default_rng(5)
+    x = (rng.standard_normal(20000) * np.exp(rng.uniform(-80, 80, 20000))).astype(np.float32)
+    want = torch.from_numpy(x).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    got = np.array([oracle.f32_to_bf16(float(v)) for v in x], dtype=np.uint16)
+    np.testing.assert_array_equal(got, want)
+
+
+def test_bf16_payload_keeps_the_rounding_error(oracle):
+    shape = (10, 11, 3, 3)
+    rng = np.random.default_rng(12)
+    g = rng.standard_normal(110).astype(np.float32)
+    r = (rng.standard_normal(110) * 0.1).astype(np.float32)
+    full = oracle.compress_layer(g, r, shape, 0.3, 0.5)
+    half = oracle.compress_layer(g, r, shape, 0.3, 0.5, payload_bf16=True)
+    np.testing.assert_array_equal(half.idx, full.idx)               # the selection does not depend on it
+    assert half.val_bf16.dtype == np.uint16 and half.val_bf16.size == full.val.size
+    # sent + kept = v, exactly, on every element; unsent tiles keep v untouched
+    sent = np.zeros(110, np.float32)
+    oracle.decompress_into(sent, shape, half.idx, half.val, 1.0)
+    np.testing.assert_array_equal(sent.astype(np.float64) + half.residual.astype(np.float64),
+                                  half.v.astype(np.float64))
+    untouched = full.residual != 0
+    np.testing.assert_array_equal(half.residual[untouched], half.v[untouched])
+    # every sent value is the nearest bfloat16: error at most half a unit in the 8th significant bit
+    kept = ~untouched
+    assert (np.abs(half.residual[kept]) <= np.abs(half.v[kept]) * 2.0 ** -8).all()
+    assert np.abs(half.residual[kept]).max() > 0                    # and the error is really there
+    # padded slots of clipped tiles are +0; the 16 low bits of what the receiver sees are zero
+    assert (half.val.view(np.uint32) & 0xFFFF == 0).all()
+    # values that bfloat16 holds exactly: identical to the 32-bit payload, nothing stays behind
+    g2 = (rng.integers(-100, 100, 110) / 4.0).astype(np.float32)
+    a = oracle.compress_layer(g2, np.zeros(110, np.float32), shape, 0.3, 0.5)
+    b = oracle.compress_layer(g2, np.zeros(110, np.float32), shape, 0.3, 0.5, payload_bf16=True)
+    np.testing.assert_array_equal(a.val, b.val)
+    np.testing.assert_array_equal(a.residual, b.residual)
+
+
+# ---------------------------------------------------------------------------------------------
 # layer-wise ratio rule (Eq. 3-5)
 # ---------------------------------------------------------------------------------------------
 
