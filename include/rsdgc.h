@@ -33,7 +33,12 @@
  *  - Payload: idx_dev[idx_offset_l + s] is the s-th kept tile of layer l (ascending),
  *    val_dev[val_offset_l + s*nh*nw + a*nw + b] its element (a, b) (+0 where the tile is
  *    clipped), with idx_offset_l = sum_{l'<l} k_l' and val_offset_l = sum_{l'<l}
- *    k_l' * nh_l' * nw_l'; counts_dev[l] = k_l.
+ *    k_l' * nh_l' * nw_l'; counts_dev[l] = k_l.  The values are binary32.  A plan created
+ *    with RSDGC_PAYLOAD_BF16 uses bfloat16 values instead (an option of this library; the
+ *    paper sends binary32): val_dev is then an array of 16-bit words, the value sent is
+ *    q = v rounded to the nearest bfloat16 (ties to even), and the accumulator keeps v - q
+ *    (exact in binary32) instead of +0, so the rounding error is sent later like everything
+ *    else that was not sent (Eq. 12).  Capacities and offsets count values, not bytes.
  */
 #ifndef RSDGC_H_
 #define RSDGC_H_
@@ -61,6 +66,7 @@ typedef enum {
 #define RSDGC_KEEP_AT_LEAST_ONE 1u /* k_l = max(1, ceil(K_l * ratio_l)): every layer sends >= 1 tile */
 #define RSDGC_NO_BULK_COPY 2u      /* first pass: register-staged kernel for every item           */
 #define RSDGC_MOMENTUM 4u          /* the plan is used with rsdgc_compress_momentum() (Eq. 12 l.1) */
+#define RSDGC_PAYLOAD_BF16 8u      /* payload values are bfloat16 instead of binary32 (see below)  */
 
 /* bits of rsdgc_status.flags */
 #define RSDGC_STATUS_NONFINITE 1u         /* some indicator was NaN/Inf (ranked first as +Inf)  */
@@ -104,7 +110,8 @@ typedef struct {
  * Builds the plan for a set of layers (Algorithm 1's loop over l = 1..L with the
  * neighborhoods of Eq. 7): arena offsets, tile counts, the work lists the kernels walk and
  * the per-layer device tables.  `alpha` is the hyper-parameter of Eq. 8 (0 <= alpha <= 1).
- * `flags`: an OR of RSDGC_KEEP_AT_LEAST_ONE, RSDGC_NO_BULK_COPY and RSDGC_MOMENTUM, or 0.  `device` is the CUDA device ordinal.  On success
+ * `flags`: an OR of RSDGC_KEEP_AT_LEAST_ONE, RSDGC_NO_BULK_COPY, RSDGC_MOMENTUM and
+ * RSDGC_PAYLOAD_BF16, or 0.  `device` is the CUDA device ordinal.  On success
  * *out owns host memory and a few MB of device memory until rsdgc_plan_destroy().
  * Errors: INVALID (null, n_layers < 1, rows/cols/nh/nw < 1, alpha outside [0,1] or NaN,
  * unknown dtype), CAPACITY (a layer with more than 2^31-1 tiles or nh*nw > 4096),
@@ -201,7 +208,7 @@ int rsdgc_update_ratios_noalloc(const float *weights_dev, const int64_t *layer_o
  */
 int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *residual_dev,
                    const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity,
-                   float *val_dev, int64_t val_capacity, int32_t *counts_dev, float *nsi_dev,
+                   void *val_dev, int64_t val_capacity, int32_t *counts_dev, float *nsi_dev,
                    void *workspace_dev, void *stream);
 
 /*
@@ -216,7 +223,7 @@ int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *residual_dev,
  */
 int rsdgc_compress_momentum(rsdgc_plan *plan, const void *grads_dev, float *velocity_dev, float momentum,
                             float *residual_dev, const float *ratios_dev, int32_t *idx_dev,
-                            int64_t idx_capacity, float *val_dev, int64_t val_capacity, int32_t *counts_dev,
+                            int64_t idx_capacity, void *val_dev, int64_t val_capacity, int32_t *counts_dev,
                             float *nsi_dev, void *workspace_dev, void *stream);
 
 /*
@@ -241,7 +248,7 @@ int rsdgc_plan_reserve_workers(rsdgc_plan *plan, int32_t n_workers);
 int rsdgc_compress_workers(rsdgc_plan *plan, int32_t n_workers, const void *const *grads_dev_host,
                            float *const *residual_dev_host, const float *ratios_dev,
                            int32_t *const *idx_dev_host, int64_t idx_capacity,
-                           float *const *val_dev_host, int64_t val_capacity,
+                           void *const *val_dev_host, int64_t val_capacity,
                            int32_t *const *counts_dev_host, void *workspace_dev, void *stream);
 
 /*
@@ -254,9 +261,9 @@ int rsdgc_compress_workers(rsdgc_plan *plan, int32_t n_workers, const void *cons
  */
 int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_dev,
                         float *residual_dev, const float *ratios_dev, int32_t *idx_dev,
-                        int64_t idx_capacity, float *val_dev, int64_t val_capacity,
+                        int64_t idx_capacity, void *val_dev, int64_t val_capacity,
                         int32_t *counts_dev, void *workspace_dev, int32_t *idx_host,
-                        float *val_host, int32_t *counts_host, int64_t *idx_used_host,
+                        void *val_host, int32_t *counts_host, int64_t *idx_used_host,
                         int64_t *val_used_host, void *stream);
 
 /*
@@ -272,7 +279,7 @@ int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_de
  */
 int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,
                                 const int32_t *const *idx_dev_host,
-                                const float *const *val_dev_host,
+                                const void *const *val_dev_host,
                                 const int32_t *const *counts_dev_host, float scale,
                                 float *dense_dev, void *stream);
 
@@ -285,7 +292,7 @@ int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,
  * not written.  n_workers = 0 gives all +0.  Arguments and errors as above.
  */
 int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
-                            const float *const *val_dev_host, const int32_t *const *counts_dev_host,
+                            const void *const *val_dev_host, const int32_t *const *counts_dev_host,
                             float scale, float *dense_dev, void *stream);
 
 /*

@@ -17,6 +17,7 @@ RSDGC_F32, RSDGC_BF16 = 0, 1
 KEEP_AT_LEAST_ONE = 1
 NO_BULK_COPY = 2
 MOMENTUM = 4
+PAYLOAD_BF16 = 8
 STATUS_NONFINITE, STATUS_PAYLOAD_OVERFLOW, STATUS_TIMEOUT = 1, 2, 4
 OK, ERR_INVALID, ERR_ALIGNMENT, ERR_CAPACITY, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
 
@@ -140,6 +141,7 @@ class Plan:
         self.device = device
         self.n_layers = len(layers)
         self.grad_dtype = grad_dtype
+        self.flags = int(flags)
         info = Info()
         _check(lib().rsdgc_plan_info(self._h, C.byref(info)), "rsdgc_plan_info")
         self.info = info

@@ -6,6 +6,8 @@
 // CTA.  The per-layer histograms and tickets are reset by the CTA that consumes them, so the
 // plan's tables are all-zero again when a compress call has run to completion.
 
+#include <cuda_bf16.h>
+
 #include "device_utils.cuh"
 
 namespace rsdgc {
@@ -359,6 +361,7 @@ struct GatherShared {
     int extent[kThreads];        // rows << 16 | columns of the tile that lie inside the layer
 };
 
+template <bool BF16VAL>
 __global__ void __launch_bounds__(kThreads)
 k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *__restrict__ layers, int n_layers,
          long long idx_cap, long long val_cap)
@@ -376,7 +379,8 @@ k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *_
         float *__restrict__ resid = ln.resid;
         const LayerState *__restrict__ state = ln.state;
         const int32_t *__restrict__ idx = ln.idx;
-        float *__restrict__ val = ln.val;
+        float *__restrict__ val = reinterpret_cast<float *>(ln.val);
+        __nv_bfloat16 *__restrict__ val16 = reinterpret_cast<__nv_bfloat16 *>(ln.val);
         if (lane) __syncthreads();  // everyone is done with the previous worker's tables
         for (int l = tid; l < n_layers; l += kThreads) {
             val_off[l] = state[l].val_off;
@@ -453,8 +457,14 @@ k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *_
                         for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
 #pragma unroll
                         for (int u = 0; u < kCopyBatch; ++u) {
-                            if (ga[u] >= 0) resid[ga[u]] = 0.0f;
-                            if (rel[u] >= 0) val[base + rel[u]] = xv[u];
+                            if (BF16VAL) {  // q = bfloat16(v) is sent, v - q stays (exact in binary32)
+                                const __nv_bfloat16 q = __float2bfloat16_rn(xv[u]);
+                                if (ga[u] >= 0) resid[ga[u]] = __fsub_rn(xv[u], __bfloat162float(q));
+                                if (rel[u] >= 0) val16[base + rel[u]] = q;
+                            } else {
+                                if (ga[u] >= 0) resid[ga[u]] = 0.0f;
+                                if (rel[u] >= 0) val[base + rel[u]] = xv[u];
+                            }
                         }
                     }
                 }
@@ -516,9 +526,13 @@ static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n
     RSDGC_MARK(2);
     if (e == cudaSuccess) e = launch_chained(k_mark, grid, 0, s, lanes, p->d_layers, p->d_chunks, (long long)idx_cap);
     RSDGC_MARK(2);
+    const size_t gather_smem = (size_t)(2 * p->n_layers + 1) * sizeof(long long);
     if (e == cudaSuccess)
-        e = launch_chained(k_gather, grid_gather, (size_t)(2 * p->n_layers + 1) * sizeof(long long), s, lanes, n_lanes,
-                           p->d_layers, p->n_layers, (long long)idx_cap, (long long)val_cap);
+        e = (p->flags & RSDGC_PAYLOAD_BF16)
+                ? launch_chained(k_gather<true>, grid_gather, gather_smem, s, lanes, n_lanes, p->d_layers, p->n_layers,
+                                 (long long)idx_cap, (long long)val_cap)
+                : launch_chained(k_gather<false>, grid_gather, gather_smem, s, lanes, n_lanes, p->d_layers,
+                                 p->n_layers, (long long)idx_cap, (long long)val_cap);
     RSDGC_MARK(2);
 #undef RSDGC_MARK
     count_launch(5);
@@ -526,7 +540,7 @@ static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n
 }
 
 cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
-                            const float *ratios, int32_t *idx, int64_t idx_cap, float *val, int64_t val_cap,
+                            const float *ratios, int32_t *idx, int64_t idx_cap, void *val, int64_t val_cap,
                             int32_t *counts, uint32_t *keys, cudaStream_t s)
 {
     const int prof = p->profile;
@@ -548,7 +562,7 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, floa
 // serve several workers at a time.  With profiling on, stage 0 of a record covers the first
 // passes of all the workers of a group (up to kMaxLanes workers form a group).
 cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *const *grads, float *const *resid,
-                                    const float *ratios, int32_t *const *idx, int64_t idx_cap, float *const *val,
+                                    const float *ratios, int32_t *const *idx, int64_t idx_cap, void *const *val,
                                     int64_t val_cap, int32_t *const *counts, uint32_t *keys_all, cudaStream_t s)
 {
     const size_t key_stride = (size_t)p->info.workspace_bytes / sizeof(uint32_t);

@@ -13,6 +13,8 @@
 // The ASSIGN variant first stores +0 to every element of the chunk's tiles (the dense arena then
 // needs no separate zero fill, and the read-modify-writes that follow find their lines in L2),
 // so that dense = scale * sum of the workers' payloads.
+#include <cuda_bf16.h>
+
 #include "device_utils.cuh"
 
 namespace rsdgc {
@@ -22,7 +24,7 @@ constexpr int kScatterBatch = 8;  // independent entries in flight per thread
 
 struct WorkerPayloads {
     const int32_t *idx[kMaxWorkersPerLaunch];
-    const float *val[kMaxWorkersPerLaunch];
+    const void *val[kMaxWorkersPerLaunch];  // binary32 or bfloat16 values
     const int32_t *counts[kMaxWorkersPerLaunch];
     int n_workers;
 };
@@ -93,7 +95,7 @@ __device__ __forceinline__ void zero_chunk(float *__restrict__ dense, const Laye
                   L.elem_off + min((long long)L.rows, (full1 + 1) * L.nh) * L.cols);
 }
 
-template <bool ASSIGN>
+template <bool ASSIGN, bool BF16VAL>
 __global__ void __launch_bounds__(kThreads)
 k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restrict__ layers,
              const Chunk *__restrict__ chunks, float scale, float *__restrict__ dense)
@@ -139,7 +141,9 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
         const int lo = sh.lo[w];
         const int n_copy = (sh.hi[w] - lo) * slot;
         const int32_t *idx = wp.idx[w] + sh.idx_off[w] + lo;
-        const float *val = wp.val[w] + sh.val_off[w] + (long long)lo * slot;
+        const long long v_first = sh.val_off[w] + (long long)lo * slot;
+        const float *val = reinterpret_cast<const float *>(wp.val[w]) + v_first;
+        const __nv_bfloat16 *val16 = reinterpret_cast<const __nv_bfloat16 *>(wp.val[w]) + v_first;
         for (int j0 = 0; j0 < n_copy; j0 += kThreads * kScatterBatch) {
             long long ga[kScatterBatch];
             float pv[kScatterBatch], dv[kScatterBatch];
@@ -151,7 +155,7 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
                     int r, el;
                     divmod_small(j, slot, &r, &el);
                     const int tile = __ldg(idx + r);
-                    pv[u] = __ldg(val + j);
+                    pv[u] = BF16VAL ? __bfloat162float(val16[j]) : __ldg(val + j);
                     if (tile >= c.start && tile < c.start + c.n) {  // always true for ascending lists
                         const int tr = tile / L.TC, tc = tile - tr * L.TC;
                         int a, b;
@@ -173,12 +177,13 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
 
 // Applies workers [0, n_workers) in order (after the zero fill of the ASSIGN variant); groups of kMaxWorkersPerLaunch go into one launch
 // each, and the stream orders the groups.
-cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const float *const *val,
+cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const void *const *val,
                               const int32_t *const *counts, float scale, float *dense, bool assign, cudaStream_t s)
 {
     const int n_chunks = (int)p->chunks.size();
+    const bool half = (p->flags & RSDGC_PAYLOAD_BF16) != 0;
     if (assign && n_workers == 0) {  // nothing was sent: the result is all +0
-        k_decompress<true><<<n_chunks, kThreads, 0, s>>>(WorkerPayloads{}, p->d_layers, p->d_chunks, scale, dense);
+        k_decompress<true, false><<<n_chunks, kThreads, 0, s>>>(WorkerPayloads{}, p->d_layers, p->d_chunks, scale, dense);
         count_launch(1);
     }
     for (int w0 = 0; w0 < n_workers; w0 += kMaxWorkersPerLaunch) {
@@ -189,8 +194,10 @@ cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const
             wp.val[w] = val[w0 + w];
             wp.counts[w] = counts[w0 + w];
         }
-        if (assign && w0 == 0) k_decompress<true><<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense);
-        else k_decompress<false><<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense);
+        const bool zero_first = assign && w0 == 0;
+        auto kernel = zero_first ? (half ? k_decompress<true, true> : k_decompress<true, false>)
+                                 : (half ? k_decompress<false, true> : k_decompress<false, false>);
+        kernel<<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense);
         count_launch(1);
     }
     return cudaGetLastError();

@@ -276,7 +276,8 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
     if (n_layers > kMaxLayers) return RSDGC_ERR_CAPACITY;
     if (grad_dtype != RSDGC_F32 && grad_dtype != RSDGC_BF16) return RSDGC_ERR_INVALID;
     if (!(alpha >= 0.0f && alpha <= 1.0f)) return RSDGC_ERR_INVALID;
-    if (flags & ~(RSDGC_KEEP_AT_LEAST_ONE | RSDGC_NO_BULK_COPY | RSDGC_MOMENTUM)) return RSDGC_ERR_INVALID;
+    if (flags & ~(RSDGC_KEEP_AT_LEAST_ONE | RSDGC_NO_BULK_COPY | RSDGC_MOMENTUM | RSDGC_PAYLOAD_BF16))
+        return RSDGC_ERR_INVALID;
 
     rsdgc_plan *p = new (std::nothrow) rsdgc_plan();
     if (!p) return RSDGC_ERR_NOMEM;
@@ -436,7 +437,7 @@ extern "C" int rsdgc_update_ratios(rsdgc_plan *plan, const float *weights_dev, f
 namespace {
 
 int compress_common(rsdgc_plan *plan, const void *grads_dev, float *velocity_dev, float momentum, float *residual_dev,
-                    const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, float *val_dev,
+                    const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, void *val_dev,
                     int64_t val_capacity, int32_t *counts_dev, float *nsi_dev, void *workspace_dev, void *stream)
 {
     int rc = check_plan_device(plan);
@@ -459,7 +460,7 @@ int compress_common(rsdgc_plan *plan, const void *grads_dev, float *velocity_dev
 }  // namespace
 
 extern "C" int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *residual_dev,
-                              const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, float *val_dev,
+                              const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, void *val_dev,
                               int64_t val_capacity, int32_t *counts_dev, float *nsi_dev, void *workspace_dev,
                               void *stream)
 {
@@ -470,7 +471,7 @@ extern "C" int rsdgc_compress(rsdgc_plan *plan, const void *grads_dev, float *re
 
 extern "C" int rsdgc_compress_momentum(rsdgc_plan *plan, const void *grads_dev, float *velocity_dev, float momentum,
                                        float *residual_dev, const float *ratios_dev, int32_t *idx_dev,
-                                       int64_t idx_capacity, float *val_dev, int64_t val_capacity,
+                                       int64_t idx_capacity, void *val_dev, int64_t val_capacity,
                                        int32_t *counts_dev, float *nsi_dev, void *workspace_dev, void *stream)
 {
     if (!plan || !(plan->flags & RSDGC_MOMENTUM) || !velocity_dev) return RSDGC_ERR_INVALID;
@@ -509,7 +510,7 @@ extern "C" int rsdgc_plan_reserve_workers(rsdgc_plan *plan, int32_t n_workers)
 extern "C" int rsdgc_compress_workers(rsdgc_plan *plan, int32_t n_workers, const void *const *grads_dev_host,
                                       float *const *residual_dev_host, const float *ratios_dev,
                                       int32_t *const *idx_dev_host, int64_t idx_capacity,
-                                      float *const *val_dev_host, int64_t val_capacity,
+                                      void *const *val_dev_host, int64_t val_capacity,
                                       int32_t *const *counts_dev_host, void *workspace_dev, void *stream)
 {
     int rc = check_plan_device(plan);
@@ -522,7 +523,7 @@ extern "C" int rsdgc_compress_workers(rsdgc_plan *plan, int32_t n_workers, const
     if ((int)plan->extra_lanes.size() + 1 < n_workers) return RSDGC_ERR_CAPACITY;  // rsdgc_plan_reserve_workers()
     if (!aligned16(workspace_dev)) return RSDGC_ERR_ALIGNMENT;
     std::vector<int32_t *> idx((size_t)n_workers, nullptr);
-    std::vector<float *> val((size_t)n_workers, nullptr);
+    std::vector<void *> val((size_t)n_workers, nullptr);
     for (int w = 0; w < n_workers; ++w) {
         if (!grads_dev_host[w] || !residual_dev_host[w] || !counts_dev_host[w]) return RSDGC_ERR_INVALID;
         if (idx_capacity > 0) idx[w] = idx_dev_host[w];
@@ -545,9 +546,9 @@ extern "C" int rsdgc_compress_workers(rsdgc_plan *plan, int32_t n_workers, const
 }
 
 extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_dev, float *residual_dev,
-                                   const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, float *val_dev,
+                                   const float *ratios_dev, int32_t *idx_dev, int64_t idx_capacity, void *val_dev,
                                    int64_t val_capacity, int32_t *counts_dev, void *workspace_dev,
-                                   int32_t *idx_host, float *val_host, int32_t *counts_host,
+                                   int32_t *idx_host, void *val_host, int32_t *counts_host,
                                    int64_t *idx_used_host, int64_t *val_used_host, void *stream)
 {
     int rc = check_plan_device(plan);
@@ -576,7 +577,8 @@ extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, voi
     if (nv > val_capacity) nv = val_capacity;
     if (ni > 0) e = cudaMemcpyAsync(idx_host, idx_dev, (size_t)ni * sizeof(int32_t), cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess && nv > 0)
-        e = cudaMemcpyAsync(val_host, val_dev, (size_t)nv * sizeof(float), cudaMemcpyDeviceToHost, s);
+        e = cudaMemcpyAsync(val_host, val_dev, (size_t)nv * ((plan->flags & RSDGC_PAYLOAD_BF16) ? 2 : 4),
+                            cudaMemcpyDeviceToHost, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(e);
     *idx_used_host = ni;
@@ -587,7 +589,7 @@ extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, voi
 namespace {
 
 int decompress_common(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
-                      const float *const *val_dev_host, const int32_t *const *counts_dev_host, float scale,
+                      const void *const *val_dev_host, const int32_t *const *counts_dev_host, float scale,
                       float *dense_dev, bool assign, void *stream)
 {
     int rc = check_plan_device(plan);
@@ -613,7 +615,7 @@ int decompress_common(rsdgc_plan *plan, int32_t n_workers, const int32_t *const 
 }  // namespace
 
 extern "C" int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
-                                           const float *const *val_dev_host,
+                                           const void *const *val_dev_host,
                                            const int32_t *const *counts_dev_host, float scale, float *dense_dev,
                                            void *stream)
 {
@@ -622,7 +624,7 @@ extern "C" int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers, 
 }
 
 extern "C" int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
-                                       const float *const *val_dev_host, const int32_t *const *counts_dev_host,
+                                       const void *const *val_dev_host, const int32_t *const *counts_dev_host,
                                        float scale, float *dense_dev, void *stream)
 {
     return decompress_common(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, scale, dense_dev, true,

@@ -107,7 +107,7 @@ struct Lane {
     unsigned char *codes;      // one byte per 4 tiles
     float *resid;
     int32_t *idx;
-    float *val;
+    void *val;                 // binary32 or bfloat16 payload values
 };
 struct LaneTable {
     Lane l[kMaxLanes];
@@ -185,14 +185,14 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *layers, int n_layer
 
 // launches (defined in the .cu files); each returns a cudaError_t
 cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
-                            const float *ratios, int32_t *idx, int64_t idx_cap, float *val, int64_t val_cap,
+                            const float *ratios, int32_t *idx, int64_t idx_cap, void *val, int64_t val_cap,
                             int32_t *counts, uint32_t *keys, cudaStream_t s);
 cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *const *grads, float *const *resid,
-                                    const float *ratios, int32_t *const *idx, int64_t idx_cap, float *const *val,
+                                    const float *ratios, int32_t *const *idx, int64_t idx_cap, void *const *val,
                                     int64_t val_cap, int32_t *const *counts, uint32_t *keys_all, cudaStream_t s);
 cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long n_keep,
                                  float *ratios, cudaStream_t s);
-cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const float *const *val,
+cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const void *const *val,
                               const int32_t *const *counts, float scale, float *dense, bool assign,
                               cudaStream_t s);
 void count_launch(int n);

@@ -21,6 +21,7 @@ from paper_2312_17530_b200 import binding
 
 TAU = 1e-5
 FLT_MIN = float(np.finfo(np.float32).tiny)
+CANARY16 = 0x7A5A   # 16-bit filler of bfloat16 payload buffers
 CANARY = np.float32(-7.25)
 
 
@@ -62,7 +63,9 @@ class GpuCompress:
         self.plan, self.device = plan, device
         ni, nv = plan.payload_bound(max_ratio)
         self.idx = torch.full((max(ni, 4),), -1, dtype=torch.int32, device=device)
-        self.val = torch.full((max(nv, 4),), float(CANARY), dtype=torch.float32, device=device)
+        self.half = bool(plan.flags & binding.PAYLOAD_BF16)   # payload values are bfloat16 words
+        self.val = (torch.full((max(nv, 8),), CANARY16, dtype=torch.int16, device=device) if self.half else
+                    torch.full((max(nv, 4),), float(CANARY), dtype=torch.float32, device=device))
         self.counts = torch.full((plan.n_layers,), -1, dtype=torch.int32, device=device)
         self.nsi = torch.full((plan.info.total_tiles_padded,), float(CANARY), dtype=torch.float32,
                               device=device) if with_nsi else None
@@ -85,9 +88,12 @@ class GpuCompress:
 
 
 def check_layer(oracle, li, shape, g, r, ratio, alpha, clamp, gpu_nsi, gpu_count, gpu_idx, gpu_val, gpu_res,
-                strict_keys: bool = True, what: str = "", velocity=None, momentum: float = 0.0):
-    """Applies R1 and R2 to one layer; returns the oracle's LayerResult."""
-    ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp, velocity=velocity, momentum=momentum)
+                strict_keys: bool = True, what: str = "", velocity=None, momentum: float = 0.0,
+                payload_bf16: bool = False):
+    """Applies R1 and R2 to one layer; returns the oracle's LayerResult.  With ``payload_bf16``
+    gpu_val holds the 16-bit words of the payload."""
+    ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp, velocity=velocity, momentum=momentum,
+                                payload_bf16=payload_bf16)
     K = ref.nsi_f32.size
     # R1
     err = np.abs(gpu_nsi.astype(np.float64) - ref.nsi_ref)
@@ -111,9 +117,12 @@ def check_layer(oracle, li, shape, g, r, ratio, alpha, clamp, gpu_nsi, gpu_count
             assert not kept[must_not].any(), what + ": a tile clearly below the threshold was kept"
     if not np.array_equal(gpu_idx, ref.idx):
         ref = oracle.compress_layer(g, r, shape, ratio, alpha, clamp_min1=clamp, forced_sel=gpu_idx,
-                                    velocity=velocity, momentum=momentum)
+                                    velocity=velocity, momentum=momentum, payload_bf16=payload_bf16)
     np.testing.assert_array_equal(gpu_idx, ref.idx, err_msg=what)
-    np.testing.assert_array_equal(gpu_val.view(np.uint32), ref.val.view(np.uint32), err_msg=what + " val")
+    if payload_bf16:
+        np.testing.assert_array_equal(gpu_val.view(np.uint16), ref.val_bf16, err_msg=what + " val (bfloat16)")
+    else:
+        np.testing.assert_array_equal(gpu_val.view(np.uint32), ref.val.view(np.uint32), err_msg=what + " val")
     np.testing.assert_array_equal(gpu_res.view(np.uint32), ref.residual.view(np.uint32), err_msg=what + " residual")
     return ref
 
@@ -147,6 +156,7 @@ def compress_and_check(oracle, plan: binding.Plan, shapes, grads: Sequence[np.nd
         assert (vel_arena[pad] == CANARY).all(), what + ": padding of the velocity arena was written"
     counts = gc.counts.cpu().numpy()
     idx, val, nsi = gc.idx.cpu().numpy(), gc.val.cpu().numpy(), gc.nsi.cpu().numpy()
+    half = gc.half
     assert st.idx_needed == counts.sum()
     io = vo = 0
     refs, new_res = [], []
@@ -156,7 +166,8 @@ def compress_and_check(oracle, plan: binding.Plan, shapes, grads: Sequence[np.nd
                           nsi[li.tile_offset:li.tile_offset + li.n_tiles], k, idx[io:io + k],
                           val[vo:vo + k * slot], res_arena[li.elem_offset:li.elem_offset + li.rows * li.cols],
                           strict_keys=strict_keys, what="%s layer %d %r" % (what, l, tuple(shape)),
-                          velocity=None if velocities is None else velocities[l], momentum=momentum)
+                          velocity=None if velocities is None else velocities[l], momentum=momentum,
+                          payload_bf16=half)
         if vel_arena is not None:
             np.testing.assert_array_equal(
                 vel_arena[li.elem_offset:li.elem_offset + li.rows * li.cols].view(np.uint32),
@@ -165,7 +176,8 @@ def compress_and_check(oracle, plan: binding.Plan, shapes, grads: Sequence[np.nd
         refs.append(ref)
         new_res.append(ref.residual)
     assert st.val_needed == vo
-    assert (idx[io:] == -1).all() and (val[vo:] == CANARY).all(), what + ": payload written past its end"
+    assert (idx[io:] == -1).all() and (val[vo:] == (CANARY16 if half else CANARY)).all(), \
+        what + ": payload written past its end"
     return new_res, refs, gc
 
 

@@ -446,3 +446,48 @@ def test_momentum_correction_five_iterations(oracle, bf16):
         parity.GpuCompress(plain).run(parity.dev(parity.to_arena(plain, res)), parity.dev(parity.to_arena(plain, res)),
                                       torch.tensor(ratios, device="cuda:0"),
                                       velocity=parity.dev(parity.to_arena(plain, res)), momentum=0.9)
+
+
+# ---------------------------------------------------------------------------------------------
+# payload with bfloat16 values: q = bfloat16(v) is sent, v - q stays in the accumulator
+# ---------------------------------------------------------------------------------------------
+
+def test_bf16_payload_three_iterations_and_aggregation(oracle):
+    shapes = [(300, 515, 3, 3), (256 * 16, 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3), (64, 147, 1, 49),
+              (1200, 1536, 3, 3), (5, 5, 3, 3)]
+    tensors = [("t%d" % i, (s[0], s[1])) for i, s in enumerate(shapes)]
+    plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE | binding.PAYLOAD_BF16)
+    sig = synth.log_uniform_scales(len(shapes), (41,))
+    ratios = np.array([1 / 16, 1 / 50, 0.3, 1.0, 0.1, 1 / 64, 0.5], np.float32)
+    n_workers = 2
+    res = [[np.zeros(s[0] * s[1], np.float32) for s in shapes] for _ in range(n_workers)]
+    gcs = [parity.GpuCompress(plan) for _ in range(n_workers)]
+    for it in range(3):
+        grads = synth.multi_worker_gradients(tensors, n_workers, (41, it), sig)
+        refs_all = []
+        for w in range(n_workers):
+            gcs[w].idx.fill_(-1)
+            gcs[w].val.fill_(parity.CANARY16)
+            res[w], refs, _ = parity.compress_and_check(oracle, plan, shapes, grads[w], res[w], ratios, 0.5,
+                                                        gc=gcs[w], what="bf16 payload it%d w%d" % (it, w))
+            refs_all.append(oracle.CompressResult(layers=refs))
+    # what the receivers rebuild from the 16-bit payloads
+    payloads = [gc.payload() for gc in gcs]
+    rng = np.random.default_rng(9)
+    dense0 = [(rng.standard_normal(s[0] * s[1]) * 1e-3).astype(np.float32) for s in shapes]
+    d_dense = parity.dev(parity.to_arena(plan, dense0))
+    plan.decompress_accumulate(payloads, d_dense, 0.5)
+    d_assign = parity.dev(parity.to_arena(plan, dense0))
+    plan.decompress_assign(payloads, d_assign, 0.5)
+    torch.cuda.synchronize()
+    ref_acc = [d.copy() for d in dense0]
+    oracle.decompress_accumulate(shapes, ref_acc, refs_all, 0.5)
+    ref_asg = [d.copy() for d in dense0]
+    oracle.decompress_assign(shapes, ref_asg, refs_all, 0.5)
+    for got, want in zip(parity.from_arena(plan, d_dense.cpu().numpy()), ref_acc):
+        np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+    for got, want in zip(parity.from_arena(plan, d_assign.cpu().numpy()), ref_asg):
+        np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+    # bytes: 4 per index + 2 per value
+    k = int(payloads[0][2].sum())
+    assert gcs[0].val.element_size() == 2 and k > 0

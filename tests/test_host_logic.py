@@ -33,7 +33,7 @@ def test_library_exports_every_declared_symbol(lib):
 def test_plan_create_rejects_bad_arguments(lib):
     ok = [(8, 8, 3, 3)]
     for layers, kw in [([], {}), ([(0, 8, 3, 3)], {}), ([(8, 8, 0, 3)], {}), (ok, {"alpha": 1.5}),
-                       (ok, {"alpha": float("nan")}), (ok, {"grad_dtype": 7}), (ok, {"flags": 8})]:
+                       (ok, {"alpha": float("nan")}), (ok, {"grad_dtype": 7}), (ok, {"flags": 16})]:
         with pytest.raises(binding.RsdgcError) as e:
             binding.Plan(layers, device=-1, **kw)
         assert e.value.code == binding.ERR_INVALID
