@@ -296,6 +296,21 @@ int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, const int32_t *
                             float scale, float *dense_dev, void *stream);
 
 /*
+ * Per-element (coordinate) view of a payload.  The payload of Sec. III-C names neighborhoods;
+ * this expands the indices to one arena position per payload value, for receivers that scatter
+ * element by element:
+ *   coo_index_dev[j] = elem_offset_l + i * cols_l + jj   for payload value j = val_offset_l +
+ *   s * nh * nw + a * nw + b of tile idx[idx_offset_l + s] = (tr, tc), i = tr * nh + a,
+ *   jj = tc * nw + b, and -1 where (i, jj) lies outside the layer (the +0 padding of clipped
+ *   tiles) or the tile index is not one of the layer's.
+ * The values are not touched: (coo_index_dev[j], val_dev[j]) are the pairs.  At most
+ * coo_capacity entries are written (payload order).  idx_dev / counts_dev as produced by
+ * rsdgc_compress().  Errors: INVALID, ALIGNMENT, CUDA.
+ */
+int rsdgc_payload_to_coo(rsdgc_plan *plan, const int32_t *idx_dev, const int32_t *counts_dev,
+                         int64_t *coo_index_dev, int64_t coo_capacity, void *stream);
+
+/*
  * Optional per-kernel timing of rsdgc_compress().  While enabled, every rsdgc_compress() on
  * this plan records CUDA events on its stream: with level 1 only before and after the first
  * pass (accumulate+NSI, the kernel that moves all the bytes), with level 2 after each of the

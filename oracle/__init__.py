@@ -288,3 +288,22 @@ def decompress_assign(shapes: Sequence[LayerShape], dense: Sequence[np.ndarray],
     for d in dense:
         d[...] = np.float32(0.0)
     decompress_accumulate(shapes, dense, payloads, scale)
+
+
+def payload_to_coo(shape: LayerShape, idx: np.ndarray, elem_offset: int = 0) -> np.ndarray:
+    """Position (int64) of every payload value of one layer in a flat buffer in which the layer
+    starts at ``elem_offset``: value s*nh*nw + a*nw + b of tile idx[s] = (tr, tc) is element
+    (tr*nh + a, tc*nw + b) of the row-major layer (Sec. III-C: the neighborhood index stands
+    for all the positions of the neighborhood); -1 where that element lies outside the layer."""
+    rows, cols, nh, nw = shape
+    TC = -(-cols // nw)
+    out = np.empty(idx.size * nh * nw, dtype=np.int64)
+    n = 0
+    for t in np.asarray(idx, dtype=np.int64):
+        tr, tc = divmod(int(t), TC)
+        for a in range(nh):
+            for b in range(nw):
+                i, j = tr * nh + a, tc * nw + b
+                out[n] = elem_offset + i * cols + j if (i < rows and j < cols) else -1
+                n += 1
+    return out

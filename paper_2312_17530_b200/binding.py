@@ -27,7 +27,7 @@ EXPORTS = [
     "rsdgc_compress_host", "rsdgc_decompress_accumulate", "rsdgc_get_status", "rsdgc_launch_count",
     "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
     "rsdgc_update_ratios_noalloc", "rsdgc_compress_momentum", "rsdgc_plan_reserve_workers",
-    "rsdgc_compress_workers", "rsdgc_decompress_assign",
+    "rsdgc_compress_workers", "rsdgc_decompress_assign", "rsdgc_payload_to_coo",
 ]
 NOALLOC_MAX_LAYERS = 64
 N_COMPRESS_KERNELS = 6
@@ -92,6 +92,7 @@ def lib():
                                           C.POINTER(i64), C.POINTER(i64), vp]
         L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
         L.rsdgc_decompress_assign.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
+        L.rsdgc_payload_to_coo.argtypes = [vp, vp, vp, vp, i64, vp]
         L.rsdgc_get_status.argtypes = [vp, vp, C.POINTER(Status)]
         L.rsdgc_profile_enable.argtypes = [vp, i32]
         L.rsdgc_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
@@ -236,6 +237,11 @@ class Plan:
 
     def decompress_assign(self, payloads, dense, scale: float = 1.0) -> None:
         self.decompress_accumulate(payloads, dense, scale, assign=True)
+
+    def payload_to_coo(self, idx, counts, coo_index) -> None:
+        """Arena position (int64) of every payload value, -1 for padding slots."""
+        _check(lib().rsdgc_payload_to_coo(self._h, _ptr(idx), _ptr(counts), _ptr(coo_index), coo_index.numel(),
+                                          _stream()), "rsdgc_payload_to_coo")
 
     def profile_enable(self, level: int) -> None:
         """0 off; 1 events around the first pass only; 2 events around every kernel."""

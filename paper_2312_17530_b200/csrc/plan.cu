@@ -631,6 +631,22 @@ extern "C" int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, cons
                              stream);
 }
 
+extern "C" int rsdgc_payload_to_coo(rsdgc_plan *plan, const int32_t *idx_dev, const int32_t *counts_dev,
+                                    int64_t *coo_index_dev, int64_t coo_capacity, void *stream)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (!idx_dev || !counts_dev || coo_capacity < 0 || (coo_capacity > 0 && !coo_index_dev)) return RSDGC_ERR_INVALID;
+    if (!aligned16(idx_dev) || !aligned16(coo_index_dev)) return RSDGC_ERR_ALIGNMENT;
+    if (coo_capacity == 0) return RSDGC_OK;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    static_assert(sizeof(long long) == sizeof(int64_t), "coordinate entries are 64-bit");
+    cudaError_t e = launch_payload_to_coo(plan, idx_dev, counts_dev, reinterpret_cast<long long *>(coo_index_dev),
+                                          (long long)coo_capacity, (cudaStream_t)stream);
+    return e == cudaSuccess ? RSDGC_OK : cuda_fail(e);
+}
+
 extern "C" int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *out_host)
 {
     int rc = check_plan_device(plan);

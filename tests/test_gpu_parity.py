@@ -491,3 +491,40 @@ def test_bf16_payload_three_iterations_and_aggregation(oracle):
     # bytes: 4 per index + 2 per value
     k = int(payloads[0][2].sum())
     assert gcs[0].val.element_size() == 2 and k > 0
+
+
+# ---------------------------------------------------------------------------------------------
+# coordinate view of a payload: one arena position per value
+# ---------------------------------------------------------------------------------------------
+
+def test_payload_to_coo(oracle):
+    shapes = [(300, 515, 3, 3), (256, 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3), (64, 147, 1, 49), (5, 5, 3, 3),
+              (131, 131, 7, 5), (4, 4, 3, 3)]
+    plan = binding.Plan(shapes, alpha=0.5)
+    rng = np.random.default_rng(17)
+    g = [(rng.standard_normal(s[0] * s[1]) * 1e-2).astype(np.float32) for s in shapes]
+    zeros = [np.zeros(s[0] * s[1], np.float32) for s in shapes]
+    ratios = np.array([0.1, 0.5, 0.2, 1.0, 0.3, 1.0, 0.25, 0.0], np.float32)
+    _, refs, gc = parity.compress_and_check(oracle, plan, shapes, g, zeros, ratios, 0.5, what="coo")
+    n_val = sum(r.val.size for r in refs)
+    coo = torch.full((n_val + 8,), -7, dtype=torch.int64, device="cuda:0")
+    plan.payload_to_coo(gc.idx, gc.counts, coo[:n_val])
+    torch.cuda.synchronize()
+    got = coo.cpu().numpy()
+    assert (got[n_val:] == -7).all()                                  # nothing past the capacity given
+    want = np.concatenate([oracle.payload_to_coo(s, r.idx, li.elem_offset)
+                           for s, r, li in zip(shapes, refs, plan.layers)])
+    np.testing.assert_array_equal(got[:n_val], want)
+    # scattering the pairs into an arena gives the aggregation's result
+    d_dense = torch.zeros(plan.info.arena_elems, device="cuda:0")
+    ok = coo[:n_val] >= 0
+    d_dense.index_put_((coo[:n_val][ok],), gc.val[:n_val][ok], accumulate=True)
+    d_ref = torch.zeros(plan.info.arena_elems, device="cuda:0")
+    plan.decompress_accumulate([gc.payload()], d_ref, 1.0)
+    torch.cuda.synchronize()
+    assert torch.equal(d_dense, d_ref)
+    # a smaller capacity writes a prefix
+    coo2 = torch.full((n_val,), -7, dtype=torch.int64, device="cuda:0")
+    plan.payload_to_coo(gc.idx, gc.counts, coo2[:1000])
+    torch.cuda.synchronize()
+    assert torch.equal(coo2[:1000], coo[:1000]) and bool((coo2[1000:] == -7).all())

@@ -382,6 +382,33 @@ def test_decompress_special_cases(oracle):
     assert not np.signbit(d3[0][sent == 0]).any()                   # untouched entries are +0
 
 
+def test_coordinate_view_scatters_like_the_aggregation(oracle):
+    # scattering (position, value) pairs one by one rebuilds exactly what the tile-wise
+    # aggregation builds; clipped tiles mark their padding with -1
+    rng = np.random.default_rng(13)
+    for shape in [(10, 11, 3, 3), (7, 9, 1, 9), (1, 20, 1, 9), (9, 9, 3, 3), (5, 4, 7, 5)]:
+        n = shape[0] * shape[1]
+        g = rng.standard_normal(n).astype(np.float32)
+        res = oracle.compress_layer(g, np.zeros(n, np.float32), shape, 0.5, 0.5)
+        coo = oracle.payload_to_coo(shape, res.idx, elem_offset=64)
+        assert coo.size == res.val.size
+        dense = np.zeros(64 + n, np.float32)
+        for p, x in zip(coo, res.val):
+            if p >= 0:
+                dense[p] += x
+            else:
+                assert x == 0 and not np.signbit(x)
+        want = np.zeros(n, np.float32)
+        oracle.decompress_into(want, shape, res.idx, res.val, 1.0)
+        np.testing.assert_array_equal(dense[64:], want)
+        assert (dense[:64] == 0).all()
+        valid = coo[coo >= 0]
+        assert np.unique(valid).size == valid.size                   # tiles do not overlap
+        n_pad = int((coo < 0).sum())
+        if shape[0] % shape[2] == 0 and shape[1] % shape[3] == 0:
+            assert n_pad == 0
+
+
 # ---------------------------------------------------------------------------------------------
 # payload with bfloat16 values (an option of the implementation; Eq. 12: the unsent part stays)
 # ---------------------------------------------------------------------------------------------
