@@ -202,9 +202,19 @@ def run_b200(args):
     host_g = [to_arena(grads[w], pin=True) for w in range(N_WORKERS)]
     d_g = [h.to(device, non_blocking=True) for h in host_g]
     d_r = [torch.zeros(arena, dtype=torch.float32, device=device) for _ in range(N_WORKERS)]
-    d_idx = [torch.zeros(ni, dtype=torch.int32, device=device) for _ in range(N_WORKERS)]
-    d_val = [torch.zeros(nv, dtype=torch.float32, device=device) for _ in range(N_WORKERS)]
-    d_cnt = [torch.zeros(plan.n_layers, dtype=torch.int32, device=device) for _ in range(N_WORKERS)]
+    exchange = None
+    if args.sync:
+        # optional: the ranks all-gather their workers' payloads and every rank aggregates all of them
+        # (the exchange step after the timed path; off by default: the default job has no collective)
+        from paper_2312_17530_b200 import sync
+
+        exchange = sync.PayloadExchange(plan.n_layers, ni, nv, N_WORKERS, world, rank, device)
+        views = [exchange.local_views(w) for w in range(N_WORKERS)]
+        d_idx, d_val, d_cnt = [v[0] for v in views], [v[1] for v in views], [v[2] for v in views]
+    else:
+        d_idx = [torch.zeros(ni, dtype=torch.int32, device=device) for _ in range(N_WORKERS)]
+        d_val = [torch.zeros(nv, dtype=torch.float32, device=device) for _ in range(N_WORKERS)]
+        d_cnt = [torch.zeros(plan.n_layers, dtype=torch.int32, device=device) for _ in range(N_WORKERS)]
     d_ws = torch.empty(N_WORKERS * plan.info.workspace_bytes, dtype=torch.uint8, device=device)
     plan.reserve_workers(N_WORKERS)
     d_ratios = torch.full((plan.n_layers,), KEEP_RATIO, dtype=torch.float32, device=device)
@@ -212,9 +222,16 @@ def run_b200(args):
     d_r0 = d_r[0]
     torch.cuda.synchronize()
 
+    def aggregate():
+        if exchange is not None:
+            exchange.exchange()
+            exchange.aggregate(plan, d_dense, 1.0)
+        else:
+            plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
+
     def step():
         plan.compress_workers(d_g, d_r, d_ratios, d_idx, d_val, d_cnt, d_ws)
-        plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
+        aggregate()
 
     # ---- device-resident timing: W warm-up steps, then exactly K steps between two events
     for _ in range(args.warmup):
@@ -233,7 +250,7 @@ def run_b200(args):
     for s in range(args.steps):
         plan.compress_workers(d_g, d_r, d_ratios, d_idx, d_val, d_cnt, d_ws)
         ev_dec[s][0].record()
-        plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
+        aggregate()
         ev_dec[s][1].record()
     ev1.record()
     torch.cuda.synchronize()
@@ -425,7 +442,8 @@ def run_b200(args):
             "config": {"workload": WORKLOAD if args.workload == "vgg19" else
                        "fc6 25088x4096 alone, 1 worker (small case for profiler captures, not the benchmark)",
                        "l2": "inputs larger than L2 (4 x 1.1 GB streamed per step)",
-                       "parallelism": "dp%d (independent replicas, no collective)" % args.gpus},
+                       "parallelism": ("dp%d (payload all-gather + aggregation of every rank's workers)" if args.sync
+                                       else "dp%d (independent replicas, no collective)") % args.gpus},
             "clocks": clocks,
             "e2e": {"value": e2e_bps / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(4 * arena * N_WORKERS),
                     "d2h_bytes_per_step": int(d2h)},
@@ -458,6 +476,8 @@ def main():
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sync", action="store_true",
+                    help="all-gather the payloads between the ranks and aggregate all of them on every rank")
     ap.add_argument("--workload", choices=["vgg19", "fc6"], default="vgg19",
                     help="vgg19: the benchmark; fc6: its largest layer alone, for profiler captures")
     args = ap.parse_args()

@@ -528,3 +528,65 @@ def test_payload_to_coo(oracle):
     plan.payload_to_coo(gc.idx, gc.counts, coo2[:1000])
     torch.cuda.synchronize()
     assert torch.equal(coo2[:1000], coo[:1000]) and bool((coo2[1000:] == -7).all())
+
+
+# ---------------------------------------------------------------------------------------------
+# the exchange step (Eq. 2 Sync) through NCCL: one rank on one GPU, the collective really runs
+# ---------------------------------------------------------------------------------------------
+
+NCCL_CHILD = r"""
+import os, sys
+sys.path.insert(0, %r); sys.path.insert(0, os.path.join(%r, "tests"))
+import numpy as np, torch
+import torch.distributed as td
+import oracle, parity
+from paper_2312_17530_b200 import binding, sync, synth
+td.init_process_group("nccl", rank=0, world_size=1)
+torch.cuda.set_device(0)
+shapes = [(300, 515, 3, 3), (256, 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3)]
+tensors = [("t%%d" %% i, (s[0], s[1])) for i, s in enumerate(shapes)]
+plan = binding.Plan(shapes, alpha=0.5)
+n_local = 3
+plan.reserve_workers(n_local)
+ratios = np.array([0.1, 0.3, 0.2, 0.05], np.float32)
+ni, nv = plan.payload_bound(0.3)
+ex = sync.PayloadExchange(plan.n_layers, ni, nv, n_local, 1, 0, "cuda:0", always_gather=True)
+sig = synth.log_uniform_scales(len(shapes), (61,))
+grads = synth.multi_worker_gradients(tensors, n_local, (61,), sig)
+zeros = [np.zeros(s[0] * s[1], np.float32) for s in shapes]
+d_g = [parity.dev(parity.to_arena(plan, g)) for g in grads]
+d_r = [parity.dev(parity.to_arena(plan, zeros)) for _ in range(n_local)]
+views = [ex.local_views(w) for w in range(n_local)]
+ws = torch.empty(n_local * plan.info.workspace_bytes, dtype=torch.uint8, device="cuda:0")
+plan.compress_workers(d_g, d_r, torch.tensor(ratios, device="cuda:0"), [v[0] for v in views], [v[1] for v in views],
+                      [v[2] for v in views], ws)
+ex.exchange()
+d_dense = torch.zeros(plan.info.arena_elems, device="cuda:0")
+ex.aggregate(plan, d_dense, 0.5, assign=True)
+torch.cuda.synchronize()
+assert plan.status().flags == 0
+refs = [oracle.compress(shapes, g, zeros, ratios, 0.5) for g in grads]
+want = [np.zeros(s[0] * s[1], np.float32) for s in shapes]
+oracle.decompress_assign(shapes, want, refs, 0.5)
+for got, w in zip(parity.from_arena(plan, d_dense.cpu().numpy()), want):
+    assert np.array_equal(got.view(np.uint32), w.view(np.uint32))
+assert ex.recv.data_ptr() != ex.send.data_ptr() and torch.equal(ex.recv, ex.send)
+td.destroy_process_group()
+print("nccl exchange ok")
+"""
+
+
+def test_payload_exchange_through_nccl_one_rank():
+    import os
+    import socket
+    import subprocess
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    out = subprocess.run([sys.executable, "-c", NCCL_CHILD % (root, root)], env=env, capture_output=True, text=True,
+                         timeout=300)
+    assert out.returncode == 0 and "nccl exchange ok" in out.stdout, out.stdout + out.stderr
