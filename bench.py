@@ -49,18 +49,65 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """nvidia-smi sampling of SM clocks and throttle reasons while the timed region runs."""
+    """SM clock and throttle reasons (read-only NVML queries) sampled by a thread while the timed
+    region runs; the region may last only milliseconds, so the samples are taken in-process every
+    millisecond rather than by a separate nvidia-smi process.  Falls back to nvidia-smi when the NVML
+    binding is missing."""
 
     FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.gpu_index = gpu_index
+    def __init__(self, gpu_index: int, uuid: str = ""):
+        self.gpu_index, self.uuid = gpu_index, uuid
         self.proc = None
+        self.thread = None
+        self.samples, self.reason_bits, self.smax = [], 0, None
         self.path = os.path.join("/tmp", "rsdgc_clocks_%d_%d.csv" % (os.getpid(), gpu_index))
 
+    def _nvml_handle(self):
+        import pynvml
+
+        pynvml.nvmlInit()
+        if self.uuid:
+            try:
+                return pynvml, pynvml.nvmlDeviceGetHandleByUUID(self.uuid.encode() if hasattr(self.uuid, "encode")
+                                                                 else self.uuid)
+            except pynvml.NVMLError:
+                pass
+        visible = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+        index = self.gpu_index
+        if visible:
+            tok = visible.split(",")[self.gpu_index].strip()
+            if tok.isdigit():
+                index = int(tok)
+            else:
+                return pynvml, pynvml.nvmlDeviceGetHandleByUUID(tok.encode())
+        return pynvml, pynvml.nvmlDeviceGetHandleByIndex(index)
+
     def start(self):
+        try:
+            nv, h = self._nvml_handle()
+            self.smax = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+        except Exception:
+            return self._start_smi()
+        import threading
+
+        self._stop = threading.Event()
+
+        def run():
+            while not self._stop.is_set():
+                try:
+                    self.samples.append(float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)))
+                    self.reason_bits |= int(nv.nvmlDeviceGetCurrentClocksEventReasons(h))
+                except Exception:
+                    pass
+                self._stop.wait(0.001)
+
+        self.thread = threading.Thread(target=run, daemon=True)
+        self.thread.start()
+
+    def _start_smi(self):
         try:
             self.out = open(self.path, "w")
             self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu_index), "--query-gpu=" + self.FIELDS,
@@ -70,8 +117,21 @@ class ClockSampler:
             self.proc = None
 
     def stop(self):
+        if self.thread is not None:
+            import pynvml as nv
+
+            self._stop.set()
+            self.thread.join(timeout=5)
+            names = [("hw_slowdown", nv.nvmlClocksEventReasonHwSlowdown),
+                     ("hw_thermal_slowdown", nv.nvmlClocksEventReasonHwThermalSlowdown),
+                     ("sw_thermal_slowdown", nv.nvmlClocksEventReasonSwThermalSlowdown),
+                     ("sw_power_cap", nv.nvmlClocksEventReasonSwPowerCap),
+                     ("hw_power_brake_slowdown", nv.nvmlClocksEventReasonHwPowerBrakeSlowdown)]
+            reasons = [n for n, bit in names if self.reason_bits & bit]
+            return {"sm_mhz": statistics.median(self.samples) if self.samples else None, "sm_max_mhz": self.smax,
+                    "samples": len(self.samples), "reasons": reasons, "source": "nvml"}
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return {"sm_mhz": None, "sm_max_mhz": None, "samples": 0, "reasons": ["clock query unavailable"]}
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
@@ -97,7 +157,7 @@ class ClockSampler:
         except OSError:
             pass
         return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "source": "nvidia-smi"}
 
 
 def vgg_inputs(rank: int, n_workers: int = N_WORKERS, only_fc6: bool = False):
@@ -239,7 +299,11 @@ def run_b200(args):
     torch.cuda.synchronize()
     assert plan.status().flags == 0
     plan.profile_enable(1)  # events around the first pass only: the roofline kernel's duration
-    sampler = ClockSampler(local_rank)
+    try:
+        gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        gpu_uuid = ""
+    sampler = ClockSampler(local_rank, gpu_uuid)
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev_dec = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
@@ -471,7 +535,7 @@ K1_TRAFFIC_BYTES = int(1236.01e6 * 139754605 / 102760448)
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")

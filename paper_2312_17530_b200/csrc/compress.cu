@@ -301,65 +301,57 @@ k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
             }
         }
     }
-    unsigned int gt = 0, eq = 0;
+    // 64-bit masks in key order: bit 4 * byte + c of `above` (`equal`) is set when key c of that
+    // code byte lies above (equals) the threshold
+    unsigned long long above = 0, equal = 0;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-        gt += __popc(w[j] & 0x0F0F0F0Fu);
-        eq += __popc(w[j] & 0xF0F0F0F0u);
+        const unsigned int lo = w[j] & 0x0F0F0F0Fu, hi = (w[j] >> 4) & 0x0F0F0F0Fu;
+        const unsigned int a16 = (lo & 0xFu) | ((lo >> 4) & 0xF0u) | ((lo >> 8) & 0xF00u) | ((lo >> 12) & 0xF000u);
+        const unsigned int e16 = (hi & 0xFu) | ((hi >> 4) & 0xF0u) | ((hi >> 8) & 0xF00u) | ((hi >> 12) & 0xF000u);
+        above |= (unsigned long long)a16 << (16 * j);
+        equal |= (unsigned long long)e16 << (16 * j);
     }
+    const unsigned int gt = __popcll(above), eq = __popcll(equal);
     unsigned long long total;
     const unsigned long long ex =
         block_exclusive_scan<unsigned long long>(((unsigned long long)eq << 32) | gt, sh.scan_tmp, &total);
-    unsigned int gt_before = (unsigned int)(ex & 0xFFFFFFFFull), eq_before = (unsigned int)(ex >> 32);
-    if ((gt | eq) == 0) return;
+    const unsigned int gt_before = (unsigned int)(ex & 0xFFFFFFFFull), eq_before = (unsigned int)(ex >> 32);
+    // equal keys from this thread on are no longer taken once eq_room is used up
+    unsigned long long todo = above | (((long long)eq_before < eq_room) ? equal : 0ull);
+    if (todo == 0) return;
     // payload position of this chunk's first kept tile
     const long long slot0 = st.idx_off + (long long)base.x + min((long long)base.y, (long long)st.e);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-#pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            const unsigned int byte = (w[j] >> (8 * b)) & 0xFFu;
-            if (byte == 0) continue;
-            const int p0 = c.start + tid * kKeysPerThread + (j * 4 + b) * 4;
-#pragma unroll
-            for (int k = 0; k < 4; ++k) {
-                long long s = -1;
-                if (byte & (1u << k)) {
-                    s = slot0 + gt_before + min((long long)eq_before, eq_room);
-                    ++gt_before;
-                } else if (byte & (16u << k)) {
-                    if ((long long)eq_before < eq_room) s = slot0 + gt_before + eq_before;
-                    ++eq_before;
-                }
-                if (s >= 0 && s < idx_cap) idx[s] = p0 + k;
-            }
-        }
+    const int p0 = c.start + tid * kKeysPerThread;
+    // only the set bits are visited: a warp takes as many rounds as its busiest lane has kept tiles
+    while (todo) {
+        const int p = __ffsll((long long)todo) - 1;
+        todo &= todo - 1;
+        const unsigned long long below = (1ull << p) - 1ull;
+        const long long g_rank = (long long)gt_before + __popcll(above & below);
+        const long long e_rank = (long long)eq_before + __popcll(equal & below);
+        long long s;
+        if ((above >> p) & 1ull) s = slot0 + g_rank + min(e_rank, eq_room);
+        else if (e_rank < eq_room) s = slot0 + g_rank + e_rank;
+        else continue;
+        if (s < idx_cap) idx[s] = p0 + p;
     }
 }
 
 // ------------------------------------------------------------------------------------------
-// K6: gather.  Payload value j of a worker belongs to layer l (val_off_l <= j < val_off_l +
-// k_l * slot_l), payload slot s = (j - val_off_l) / slot_l, element el of the tile
+// K6: gather.  Payload value j of the whole call belongs to layer l (val_off_l <= j <
+// val_off_l + k_l * slot_l), payload slot s = (j - val_off_l) / slot_l, element el of the tile
 // idx[idx_off_l + s].  The value is moved from the residual to val and the residual entry
-// becomes +0 (Eq. 12: what is sent leaves the accumulator).
-//
-// A CTA takes blocks of kGatherBlock consecutive payload values, so the work is spread evenly
-// whatever the spatial pattern of the kept tiles and the writes to val are contiguous.  Inside
-// a block the tiles are resolved first, one thread per tile (index -> arena address of the
-// tile's corner and its clipped extent, kept in shared memory); the values then need only a
-// division by small constants each.  kCopyBatch independent values are in flight per thread.
+// becomes +0 (Eq. 12: what is sent leaves the accumulator); with 16-bit payload values
+// q = bfloat16(v) is sent and v - q stays.  Grid-stride over blocks of consecutive payload values
+// (so the work is even whatever the spatial pattern of the kept tiles, and the payload stores are
+// contiguous) with kCopyBatch independent entries in flight per thread.
 // ------------------------------------------------------------------------------------------
 
 #ifndef RSDGC_COPY_BATCH
 #define RSDGC_COPY_BATCH 8
 #endif
 constexpr int kCopyBatch = RSDGC_COPY_BATCH;
-constexpr int kGatherBlock = kThreads * kCopyBatch;
-
-struct GatherShared {
-    long long corner[kThreads];  // arena index of the tile's first element, or -1: tile not sent
-    int extent[kThreads];        // rows << 16 | columns of the tile that lie inside the layer
-};
 
 template <bool BF16VAL>
 __global__ void __launch_bounds__(kThreads)
@@ -369,7 +361,6 @@ k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *_
     extern __shared__ __align__(16) unsigned char gather_smem_raw[];
     long long *val_off = reinterpret_cast<long long *>(gather_smem_raw);  // n_layers + 1
     long long *idx_off = val_off + n_layers + 1;                          // n_layers
-    __shared__ GatherShared sh;
     const int tid = threadIdx.x;
     grid_dependency_wait();
     // the workers one after the other: the scattered accesses of the CTAs that run at the same
@@ -392,83 +383,76 @@ k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *_
         }
         __syncthreads();
         const long long total = val_off[n_layers];
-        const long long stride = (long long)gridDim.x * kGatherBlock;
-        for (long long jb = (long long)blockIdx.x * kGatherBlock; jb < total; jb += stride) {
-            const long long jend = min(total, jb + kGatherBlock);
-            long long ja = jb;
-            while (ja < jend) {  // one round per layer that has values in [jb, jend): almost always one
-                int lo = 0, hi = n_layers;  // layer with val_off[lo] <= ja < val_off[lo + 1]
-                while (hi - lo > 1) {
-                    const int mid = (lo + hi) >> 1;
-                    if (val_off[mid] <= ja) lo = mid; else hi = mid;
-                }
-                while (val_off[lo + 1] <= ja) ++lo;  // layers without payload share their offset
-                const LayerDev &L = layers[lo];
-                const long long v0 = val_off[lo], i0 = idx_off[lo];
-                const long long jz = min(jend, val_off[lo + 1]);
-                const int slot = L.slot, nh = L.nh, nw = L.nw, TC = L.TC;
-                const long long cols = L.cols;
-                const long long s_first = (ja - v0) / slot, s_last = (jz - 1 - v0) / slot;
-                for (long long s0 = s_first; s0 <= s_last; s0 += kThreads) {
-                    const int nt = (int)min((long long)kThreads, s_last - s0 + 1);
-                    __syncthreads();  // the previous round's tiles are no longer in use
-                    if (tid < nt) {
-                        const long long sl = s0 + tid;
-                        long long corner = -1;
-                        int extent = 0;
-                        // tiles that do not fit the payload buffers are not sent and stay in the residual
-                        if (i0 + sl < idx_cap && v0 + (sl + 1) * slot <= val_cap) {
-                            const int tile = __ldg(idx + i0 + sl);
-                            const int tr = tile / TC, tc = tile - tr * TC;
-                            const long long r0 = (long long)tr * nh, c0 = (long long)tc * nw;
-                            corner = L.elem_off + r0 * cols + c0;
-                            extent = ((int)min((long long)nh, L.rows - r0) << 16) | (int)min((long long)nw, cols - c0);
-                        }
-                        sh.corner[tid] = corner;
-                        sh.extent[tid] = extent;
+        // a CTA takes blocks of kThreads * kCopyBatch consecutive payload values: almost always one
+        // layer per block, so the layer search is done once per block, not once per value
+        constexpr long long kBlock = (long long)kThreads * kCopyBatch;
+        auto find_layer = [&](long long j) {
+            int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (val_off[mid] <= j) lo = mid; else hi = mid;
+            }
+            return lo;
+        };
+        for (long long jb = (long long)blockIdx.x * kBlock; jb < total; jb += (long long)gridDim.x * kBlock) {
+            const long long jend = min(total, jb + kBlock) - 1;
+            const int l_first = find_layer(jb);
+            const bool one_layer = val_off[l_first + 1] > jend;
+            long long ga[kCopyBatch], vo[kCopyBatch];
+            int tile[kCopyBatch], lay[kCopyBatch], el[kCopyBatch];
+            float xv[kCopyBatch];
+#pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) {
+                const long long j = jb + u * kThreads + tid;
+                ga[u] = -1;
+                vo[u] = -1;
+                tile[u] = -1;
+                if (j < total) {
+                    const int lo = one_layer ? l_first : find_layer(j);
+                    const int slot = layers[lo].slot;
+                    const long long jl = j - val_off[lo];
+                    // 32-bit division whenever the layer's payload is below 2^31 values (the usual case)
+                    long long s;
+                    if (jl < 0x7FFFFFFFll) {
+                        int q, r;
+                        divmod_small((int)jl, slot, &q, &r);
+                        s = q;
+                        el[u] = r;
+                    } else {
+                        s = jl / slot;
+                        el[u] = (int)(jl - s * slot);
                     }
-                    __syncthreads();
-                    // values of this round: slots [s0, s0 + nt) cut to [ja, jz)
-                    const long long base = v0 + s0 * slot;
-                    const int r_begin = (int)max(0ll, ja - base);
-                    const int r_end = (int)min((long long)nt * slot, jz - base);
-                    for (int rb = r_begin; rb < r_end; rb += kGatherBlock) {
-                        long long ga[kCopyBatch];
-                        int rel[kCopyBatch];
-                        float xv[kCopyBatch];
-#pragma unroll
-                        for (int u = 0; u < kCopyBatch; ++u) {
-                            const int r = rb + u * kThreads + tid;
-                            ga[u] = -1;
-                            rel[u] = -1;
-                            if (r < r_end) {
-                                int t, el, a, b;
-                                divmod_small(r, slot, &t, &el);
-                                divmod_small(el, nw, &a, &b);
-                                const long long corner = sh.corner[t];
-                                const int extent = sh.extent[t];
-                                if (corner >= 0) {
-                                    rel[u] = r;
-                                    if (a < (extent >> 16) && b < (extent & 0xFFFF)) ga[u] = corner + a * cols + b;
-                                }
-                            }
-                        }
-#pragma unroll
-                        for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
-#pragma unroll
-                        for (int u = 0; u < kCopyBatch; ++u) {
-                            if (BF16VAL) {  // q = bfloat16(v) is sent, v - q stays (exact in binary32)
-                                const __nv_bfloat16 q = __float2bfloat16_rn(xv[u]);
-                                if (ga[u] >= 0) resid[ga[u]] = __fsub_rn(xv[u], __bfloat162float(q));
-                                if (rel[u] >= 0) val16[base + rel[u]] = q;
-                            } else {
-                                if (ga[u] >= 0) resid[ga[u]] = 0.0f;
-                                if (rel[u] >= 0) val[base + rel[u]] = xv[u];
-                            }
-                        }
+                    lay[u] = lo;
+                    // tiles that do not fit the payload buffers are not sent and stay in the residual
+                    if (idx_off[lo] + s < idx_cap && val_off[lo] + (s + 1) * slot <= val_cap) {
+                        tile[u] = __ldg(idx + idx_off[lo] + s);
+                        vo[u] = j;
                     }
                 }
-                ja = jz;
+            }
+#pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) {
+                if (tile[u] >= 0) {
+                    const LayerDev &L = layers[lay[u]];
+                    const int tr = tile[u] / L.TC, tc = tile[u] - tr * L.TC;
+                    int a, b;
+                    divmod_small(el[u], L.nw, &a, &b);
+                    const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
+                    if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
+#pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) {
+                if (BF16VAL) {  // q = bfloat16(v) is sent, v - q stays (exact in binary32)
+                    const __nv_bfloat16 q = __float2bfloat16_rn(xv[u]);
+                    if (ga[u] >= 0) resid[ga[u]] = __fsub_rn(xv[u], __bfloat162float(q));
+                    if (vo[u] >= 0) val16[vo[u]] = q;
+                } else {
+                    if (ga[u] >= 0) resid[ga[u]] = 0.0f;
+                    if (vo[u] >= 0) val[vo[u]] = xv[u];
+                }
             }
         }
     }
