@@ -8,6 +8,8 @@
 
 #include <cuda_bf16.h>
 
+#include <algorithm>
+
 #include "device_utils.cuh"
 
 namespace rsdgc {
@@ -17,6 +19,7 @@ namespace rsdgc {
 // ------------------------------------------------------------------------------------------
 
 constexpr int kKeyVecBatch = 8;  // 128-bit key loads in flight per thread in the key passes
+constexpr int kRefineCtasPerSm = 6;  // resident CTAs per SM of k_refine (40 registers, 8 KB of shared memory)
 
 struct RefineShared {
     unsigned int hist[kL2Bins];
@@ -25,32 +28,108 @@ struct RefineShared {
     int is_last;
 };
 
+// Adds the CTA's histogram of `layer` (it covers n_done chunks of the layer) to the layer's
+// global one and clears it; the CTA that accounts for the layer's last chunk finds the bin the
+// threshold falls into and extends the layer's prefix (level 2) or fixes T and e (level 3).
+template <int LEVEL>
+__device__ __forceinline__ void refine_flush(RefineShared &sh, const Lane &ln, const LayerDev *__restrict__ layers,
+                                             int layer, int n_done)
+{
+    constexpr int NBITS = (LEVEL == 2) ? kL2Bits : kL3Bits;
+    constexpr int NBINS = 1 << NBITS;
+    const int tid = threadIdx.x;
+    LayerState &st = ln.state[layer];
+    unsigned int *gh = ln.hist + (size_t)layer * kHistStride;
+    __syncthreads();
+    for (int b = tid; b < NBINS; b += kThreads) {
+        const unsigned int n = sh.hist[b];
+        if (n) {
+            atomicAdd(gh + b, n);
+            sh.hist[b] = 0;
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned int t = atomicAdd(&st.ticket[LEVEL - 1], (unsigned int)n_done);
+        sh.is_last = (t + (unsigned int)n_done == (unsigned int)layers[layer].n_chunks);
+    }
+    __syncthreads();
+    if (!sh.is_last) return;
+    __threadfence();
+    {
+        unsigned int h[NBINS / kThreads];
+#pragma unroll
+        for (int j = 0; j < NBINS / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + tid);
+#pragma unroll
+        for (int j = 0; j < NBINS / kThreads; ++j) {
+            sh.hist[j * kThreads + tid] = h[j];
+            gh[j * kThreads + tid] = 0;
+        }
+    }
+    __syncthreads();
+    const uint32_t prefix = st.prefix;
+    const int remaining = st.remaining;
+    if (prefix != kTakeNone)
+        find_bin_from_top<NBINS>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
+    if (tid == 0) {
+        st.ticket[LEVEL - 1] = 0;
+        if (prefix != kTakeNone) {
+            const uint32_t next = (prefix << NBITS) | (uint32_t)sh.found[0];
+            if (LEVEL == 2) {
+                st.prefix = next;
+                st.remaining = (int32_t)sh.found[1];
+            } else {
+                st.T = next;
+                st.e = (int32_t)sh.found[1];
+            }
+        } else if (LEVEL == 3) {
+            st.T = kTakeNone;
+            st.e = 0;
+        }
+    }
+    __syncthreads();
+    for (int b = tid; b < NBINS; b += kThreads) sh.hist[b] = 0;  // it held the layer's totals
+    __syncthreads();
+}
+
 // LEVEL 2: among keys whose bits 30..21 equal the layer's prefix, histogram bits 20..10.
 // LEVEL 3: among keys whose bits 30..10 equal the prefix, histogram bits 9..0; the last CTA
 // of the layer then knows the threshold key T and how many keys equal to T are taken.
+// Every CTA takes a contiguous range of the key chunks (one chunk when the grid is as large as
+// the chunk list) and keeps one shared-memory histogram per layer it passes through.
 template <int LEVEL>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, kRefineCtasPerSm)
 k_refine(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
-         const Chunk *__restrict__ chunks)
+         const Chunk *__restrict__ chunks, int n_chunks_all)
 {
     __shared__ RefineShared sh;
     const Lane &ln = lanes.l[blockIdx.y];
     const uint32_t *__restrict__ keys = ln.keys;
-    unsigned int *hist = ln.hist;
-    LayerState *state = ln.state;
     constexpr int SHIFT_HI = (LEVEL == 2) ? kL1Shift : kL2Shift;
     constexpr int SHIFT_LO = (LEVEL == 2) ? kL2Shift : 0;
     constexpr int NBITS = (LEVEL == 2) ? kL2Bits : kL3Bits;
     constexpr int NBINS = 1 << NBITS;
-    const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x;
-    LayerState &st = state[c.layer];
+    const int chunk_begin = (int)((long long)blockIdx.x * n_chunks_all / gridDim.x);
+    const int chunk_end = (int)((long long)(blockIdx.x + 1) * n_chunks_all / gridDim.x);
     for (int b = tid; b < NBINS; b += kThreads) sh.hist[b] = 0;
     grid_dependency_wait();
     grid_dependency_launch_next();
-    const uint32_t prefix = st.prefix;
     __syncthreads();
-    if (prefix != kTakeNone) {
+    int cur_layer = -1, n_done = 0;
+    uint32_t prefix = kTakeNone;
+    for (int chunk_id = chunk_begin; chunk_id < chunk_end; ++chunk_id) {
+        const Chunk c = chunks[chunk_id];
+        if (c.layer != cur_layer) {
+            if (n_done) refine_flush<LEVEL>(sh, ln, layers, cur_layer, n_done);
+            cur_layer = c.layer;
+            n_done = 0;
+            // not yet extended by this pass: this CTA still owes the layer a chunk
+            prefix = ln.state[c.layer].prefix;
+        }
+        ++n_done;
+        if (prefix == kTakeNone) continue;
         const uint32_t *kp = keys + layers[c.layer].tile_off + c.start;
         const int nvec = c.n >> 2;
         for (int base = 0; base < nvec; base += kThreads * kKeyVecBatch) {
@@ -74,51 +153,7 @@ k_refine(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ l
             if ((q >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q >> SHIFT_LO) & (NBINS - 1)], 1u);
         }
     }
-    __syncthreads();
-    unsigned int *gh = hist + (size_t)c.layer * kHistStride;
-    for (int b = tid; b < NBINS; b += kThreads) {
-        const unsigned int n = sh.hist[b];
-        if (n) atomicAdd(gh + b, n);
-    }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const unsigned int t = atomicAdd(&st.ticket[LEVEL - 1], 1u);
-        sh.is_last = (t + 1u == (unsigned int)layers[c.layer].n_chunks);
-    }
-    __syncthreads();
-    if (!sh.is_last) return;
-    __threadfence();
-    {
-        unsigned int h[NBINS / kThreads];
-#pragma unroll
-        for (int j = 0; j < NBINS / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + tid);
-#pragma unroll
-        for (int j = 0; j < NBINS / kThreads; ++j) {
-            sh.hist[j * kThreads + tid] = h[j];
-            gh[j * kThreads + tid] = 0;
-        }
-    }
-    __syncthreads();
-    const int remaining = st.remaining;
-    if (prefix != kTakeNone)
-        find_bin_from_top<NBINS>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
-    if (tid == 0) {
-        st.ticket[LEVEL - 1] = 0;
-        if (prefix != kTakeNone) {
-            const uint32_t next = (prefix << NBITS) | (uint32_t)sh.found[0];
-            if (LEVEL == 2) {
-                st.prefix = next;
-                st.remaining = (int32_t)sh.found[1];
-            } else {
-                st.T = next;
-                st.e = (int32_t)sh.found[1];
-            }
-        } else if (LEVEL == 3) {
-            st.T = kTakeNone;
-            st.e = 0;
-        }
-    }
+    if (n_done) refine_flush<LEVEL>(sh, ln, layers, cur_layer, n_done);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -500,9 +535,19 @@ static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n
     cudaError_t e = cudaSuccess;
 #define RSDGC_MARK(level)                              \
     if (prof >= (level) && e == cudaSuccess) e = record_event(p, s)
-    if (e == cudaSuccess) e = launch_chained(k_refine<2>, grid, 0, s, lanes, p->d_layers, p->d_chunks);
+    // the two full key passes: one wave of resident CTAs with a contiguous chunk range each when
+    // the chunk list is much longer than that, else one CTA per chunk
+    const int n_chunks = (int)p->chunks.size();
+    const int resident = p->n_sm * kRefineCtasPerSm;
+    const dim3 grid_refine((unsigned)((long long)n_chunks * n_lanes <= 2ll * resident
+                                          ? n_chunks
+                                          : std::max(1, std::min(n_chunks, resident / n_lanes))),
+                           (unsigned)n_lanes);
+    if (e == cudaSuccess)
+        e = launch_chained(k_refine<2>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks);
     RSDGC_MARK(2);
-    if (e == cudaSuccess) e = launch_chained(k_refine<3>, grid, 0, s, lanes, p->d_layers, p->d_chunks);
+    if (e == cudaSuccess)
+        e = launch_chained(k_refine<3>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks);
     RSDGC_MARK(2);
     if (e == cudaSuccess)
         e = launch_chained(k_count, grid, 0, s, lanes, p->d_layers, p->d_chunks, p->n_layers, (long long)idx_cap,
