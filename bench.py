@@ -307,15 +307,18 @@ def run_b200(args):
     sampler.start()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev_dec = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    ev_step = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     dist.barrier()
     torch.cuda.synchronize()
     launches0 = binding.launch_count()
     ev0.record()
     for s in range(args.steps):
+        ev_step[s].record()
         plan.compress_workers(d_g, d_r, d_ratios, d_idx, d_val, d_cnt, d_ws)
         ev_dec[s][0].record()
         aggregate()
         ev_dec[s][1].record()
+    ev_step[args.steps].record()
     ev1.record()
     torch.cuda.synchronize()
     dist.barrier()
@@ -325,6 +328,7 @@ def run_b200(args):
     kernel_ms, n_calls = plan.profile_read()
     plan.profile_enable(0)
     dec_ms = sum(a.elapsed_time(b) for a, b in ev_dec) / args.steps
+    step_ms = [ev_step[i].elapsed_time(ev_step[i + 1]) for i in range(args.steps)]
     st = plan.status()
     assert st.flags == 0, "status flags %d after the timed region" % st.flags
 
@@ -435,45 +439,64 @@ def run_b200(args):
         from paper_2312_17530_b200 import synth
 
         flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)  # larger than L2
-        for name, tens in (("resnet18", synth.resnet18_tensors()), ("resnet50", synth.resnet50_tensors())):
-            sp = binding.Plan(synth.layer_shapes(tens), alpha=ALPHA, device=local_rank)
+
+        def time_set(shapes_s, ratio, dtype=binding.RSDGC_F32, reps=20):
+            """One worker, residual carried, uniform ratio; 20 repeats each of: L2 flushed between repeats
+            (stream launches and CUDA-graph replay) and hot (no flush).  Median and best in microseconds."""
+            sp = binding.Plan(shapes_s, alpha=ALPHA, device=local_rank, grad_dtype=dtype)
             a = sp.info.arena_elems
             g_s = torch.randn(a, device=device) * 1e-3
+            if dtype == binding.RSDGC_BF16:
+                g_s = g_s.to(torch.bfloat16)
             r_s = torch.zeros(a, device=device)
-            bi, bv = sp.payload_bound(1 / 50)
+            bi, bv = sp.payload_bound(ratio)
             i_s = torch.zeros(bi, dtype=torch.int32, device=device)
             v_s = torch.zeros(bv, device=device)
             c_s = torch.zeros(sp.n_layers, dtype=torch.int32, device=device)
             w_s = torch.empty(sp.info.workspace_bytes, dtype=torch.uint8, device=device)
-            q_s = torch.full((sp.n_layers,), 1 / 50, device=device)
-            for _ in range(3):
+            q_s = torch.full((sp.n_layers,), ratio, device=device)
+
+            def call():
                 sp.compress(g_s, r_s, q_s, i_s, v_s, c_s, workspace=w_s)
+
+            for _ in range(3):
+                call()
             torch.cuda.synchronize()
             graph = torch.cuda.CUDAGraph()
             with torch.cuda.graph(graph):
-                sp.compress(g_s, r_s, q_s, i_s, v_s, c_s, workspace=w_s)
-            tot = tot_graph = 0.0
-            for _ in range(5):
-                flush.zero_()
-                ev0.record()
-                sp.compress(g_s, r_s, q_s, i_s, v_s, c_s, workspace=w_s)
-                ev1.record()
-                torch.cuda.synchronize()
-                tot += ev0.elapsed_time(ev1)
-                flush.zero_()
-                ev0.record()
-                graph.replay()
-                ev1.record()
-                torch.cuda.synchronize()
-                tot_graph += ev0.elapsed_time(ev1)
-            us, us_g = tot / 5 * 1e3, tot_graph / 5 * 1e3
-            extra[name] = {"elements": int(sp.info.total_elems), "layers": sp.n_layers,
-                           "us_per_model_iteration_l2_flushed": us, "us_per_model_iteration_cuda_graph": us_g,
-                           "layers_per_s": sp.n_layers / (us_g * 1e-6),
-                           "gradient_GBps": 4.0 * sp.info.total_elems / (us_g * 1e-6) / 1e9,
-                           "roofline_frac_12B_per_elem": 12.0 * sp.info.total_elems / (us_g * 1e-6) / 1e9 / measured_peaks()[0]}
+                call()
+            out = {}
+            for key, fn, do_flush in (("l2_flushed", call, True), ("cuda_graph_l2_flushed", graph.replay, True),
+                                      ("hot", call, False)):
+                ts = []
+                for _ in range(reps):
+                    if do_flush:
+                        flush.zero_()
+                    ev0.record()
+                    fn()
+                    ev1.record()
+                    torch.cuda.synchronize()
+                    ts.append(ev0.elapsed_time(ev1) * 1e3)
+                out["us_" + key + "_median"] = statistics.median(ts)
+                out["us_" + key + "_best"] = min(ts)
+            n_el = int(sp.info.total_elems)
+            bpe = 10.0 if dtype == binding.RSDGC_BF16 else 12.0
+            us_ref = out["us_cuda_graph_l2_flushed_median"]
+            out.update({"elements": n_el, "layers": sp.n_layers, "layers_per_s": sp.n_layers / (us_ref * 1e-6),
+                        "gradient_GBps": (bpe - 8.0) * n_el / (us_ref * 1e-6) / 1e9,
+                        "roofline_frac": bpe * n_el / (us_ref * 1e-6) / 1e9 / measured_peaks()[0]})
             del graph
             sp.close()
+            return out
+
+        extra["resnet18"] = time_set(synth.layer_shapes(synth.resnet18_tensors()), 1 / 50)
+        extra["resnet50"] = time_set(synth.layer_shapes(synth.resnet50_tensors()), 1 / 50)
+        extra["single_512x512"] = time_set([(512, 512, 3, 3)], 1 / 64)
+        extra["sweep"] = {}
+        for rows_s, cols_s in ((1024, 1024), (4096, 4096), (7840, 1280), (16384, 16384)):
+            for dt, tag in ((binding.RSDGC_F32, "f32"), (binding.RSDGC_BF16, "bf16")):
+                extra["sweep"]["%dx%d_%s_keep_1_100" % (rows_s, cols_s, tag)] = time_set(
+                    [(rows_s, cols_s, 3, 3)], 1 / 100, dtype=dt, reps=10)
         del flush
 
     if rank == 0:
@@ -488,6 +511,7 @@ def run_b200(args):
                          for name, ms in zip(binding.COMPRESS_KERNELS, breakdown_ms)}
         single_us = {name: 1e3 * ms / max(single_calls, 1) for name, ms in zip(binding.COMPRESS_KERNELS, single_ms)}
         extra.update({
+            "step_ms_median": statistics.median(step_ms), "step_ms_best": min(step_ms),
             "us_per_model_iteration": compress_s * 1e6,
             "layers_per_s": plan.n_layers / compress_s,
             "compress_workers_stage_us_with_events_between": per_kernel_us,  # one call = all the workers

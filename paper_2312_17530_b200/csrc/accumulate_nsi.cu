@@ -2,11 +2,12 @@
 // (Eq. 8-10), and the level-1 histogram of the keys per layer.
 //
 // Two kernels share the work list:
-//  * k1_bulk: one persistent 512-thread CTA per SM.  The g and r blocks of an item are brought
-//    into shared memory by the bulk-copy engine (cp.async.bulk + mbarrier) two items ahead
-//    of their use, v is formed in shared memory and written back with a bulk store, and the
-//    tiles are reduced from shared memory.  Bytes in flight do not occupy registers.
-//    It takes every item whose rows are 16-byte aligned in memory (all the usual shapes).
+//  * k1_bulk: three persistent 256-thread CTAs per SM (two with momentum correction).  The g and
+//    r blocks of an item are brought into shared memory by the bulk-copy engine (cp.async.bulk +
+//    mbarrier) one item ahead of their use, v is formed in shared memory and written back with a
+//    bulk store, and the tiles are reduced from shared memory.  Bytes in flight do not occupy
+//    registers.  It takes every item whose rows are 16-byte aligned in memory (all the usual
+//    shapes).
 //  * k1_reg: 256-thread CTAs that stage an item in registers (128-bit loads where possible,
 //    scalar otherwise).  It takes the remaining items (odd pitches, unaligned starts).
 //
@@ -76,89 +77,6 @@ __device__ __forceinline__ float tile_nsi_fixed(const float *p, int pitch, float
     return __fadd_rn(__fmul_rn(alpha, mean_abs), __fmul_rn(__fsub_rn(1.0f, alpha), s));
 }
 
-#ifndef RSDGC_PAIR_MODE
-#define RSDGC_PAIR_MODE 0
-#endif
-
-// Packed binary32x2 arithmetic of sm_100 with explicit round-to-nearest (never fused).
-__device__ __forceinline__ float2 add2_rn(float2 a, float2 b)
-{
-    unsigned long long ra, rb, rd;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
-    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
-    float2 d;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
-    return d;
-}
-__device__ __forceinline__ float2 mul2_rn(float2 a, float2 b)
-{
-    unsigned long long ra, rb, rd;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(ra) : "f"(a.x), "f"(a.y));
-    asm("mov.b64 %0, {%1, %2};" : "=l"(rb) : "f"(b.x), "f"(b.y));
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(rd) : "l"(ra), "l"(rb));
-    float2 d;
-    asm("mov.b64 {%0, %1}, %2;" : "=f"(d.x), "=f"(d.y) : "l"(rd));
-    return d;
-}
-
-// Two full HH x WW tiles at once (component x = tile A, y = tile B): each component goes
-// through exactly the operations of tile_nsi_generic, in the same order, with the same
-// per-operation rounding; the two independent chains hide each other's latency.
-template <int HH, int WW>
-__device__ __forceinline__ float2 tile_pair_nsi(const float *pa, const float *pb, int pitch, float alpha)
-{
-    float2 x[HH * WW];
-#pragma unroll
-    for (int a = 0; a < HH; ++a)
-#pragma unroll
-        for (int b = 0; b < WW; ++b) x[a * WW + b] = make_float2(pa[a * pitch + b], pb[a * pitch + b]);
-    const float inv_n = __fdiv_rn(1.0f, (float)(HH * WW));  // folded at compile time
-    const float one_minus = __fsub_rn(1.0f, alpha);
-#if RSDGC_PAIR_MODE == 2
-    float2 sa = make_float2(0.0f, 0.0f), sv = make_float2(0.0f, 0.0f);
-#pragma unroll
-    for (int i = 0; i < HH * WW; ++i) {
-        sa = add2_rn(sa, make_float2(fabsf(x[i].x), fabsf(x[i].y)));
-        sv = add2_rn(sv, x[i]);
-    }
-    const float2 inv2 = make_float2(inv_n, inv_n);
-    const float2 mean_abs = mul2_rn(sa, inv2);
-    const float2 m = mul2_rn(sv, inv2);
-    const float2 neg_m = make_float2(-m.x, -m.y);  // x - m == x + (-m) in IEEE arithmetic
-    float2 sq = make_float2(0.0f, 0.0f);
-#pragma unroll
-    for (int i = 0; i < HH * WW; ++i) {
-        const float2 d = add2_rn(x[i], neg_m);
-        sq = add2_rn(sq, mul2_rn(d, d));
-    }
-    const float2 var = mul2_rn(sq, inv2);
-    const float2 s = make_float2(__fsqrt_rn(var.x), __fsqrt_rn(var.y));
-    return add2_rn(mul2_rn(make_float2(alpha, alpha), mean_abs), mul2_rn(make_float2(one_minus, one_minus), s));
-#else
-    float sa0 = 0.0f, sv0 = 0.0f, sa1 = 0.0f, sv1 = 0.0f;
-#pragma unroll
-    for (int i = 0; i < HH * WW; ++i) {
-        sa0 = __fadd_rn(sa0, fabsf(x[i].x));
-        sa1 = __fadd_rn(sa1, fabsf(x[i].y));
-        sv0 = __fadd_rn(sv0, x[i].x);
-        sv1 = __fadd_rn(sv1, x[i].y);
-    }
-    const float a0 = __fmul_rn(sa0, inv_n), a1 = __fmul_rn(sa1, inv_n);
-    const float m0 = __fmul_rn(sv0, inv_n), m1 = __fmul_rn(sv1, inv_n);
-    float sq0 = 0.0f, sq1 = 0.0f;
-#pragma unroll
-    for (int i = 0; i < HH * WW; ++i) {
-        const float d0 = __fsub_rn(x[i].x, m0), d1 = __fsub_rn(x[i].y, m1);
-        sq0 = __fadd_rn(sq0, __fmul_rn(d0, d0));
-        sq1 = __fadd_rn(sq1, __fmul_rn(d1, d1));
-    }
-    const float s0 = __fsqrt_rn(__fmul_rn(sq0, inv_n)), s1 = __fsqrt_rn(__fmul_rn(sq1, inv_n));
-    return make_float2(__fadd_rn(__fmul_rn(alpha, a0), __fmul_rn(one_minus, s0)),
-                       __fadd_rn(__fmul_rn(alpha, a1), __fmul_rn(one_minus, s1)));
-#endif
-}
-
 // Key of one indicator value; counts it in the CTA's level-1 histogram.
 __device__ __forceinline__ void emit_key(float nsi, uint32_t *dst, unsigned int *hist_smem, unsigned int &nonfinite)
 {
@@ -183,33 +101,16 @@ __device__ __forceinline__ unsigned int item_tile_keys(const ItemDev &d, const f
     const int ntile = ntr * ntc;
     uint32_t *kout = keys + d.kbase;
     unsigned int nonfinite = 0;
-    const bool noclip = (d.flags & kItemNoClip) != 0;
-    if (RSDGC_PAIR_MODE != 0 && noclip && ((nh == 3 && nw == 3) || (nh == 1 && nw == 9))) {
-        // two tiles per thread and step: t and t + NTHREADS
-        for (int t = threadIdx.x; t < ntile; t += 2 * NTHREADS) {
-            const int t2 = t + NTHREADS;
-            const bool two = t2 < ntile;
-            const int ti = (ntr == 1) ? 0 : fast_div(t, d.inv_ntc), tj = t - ti * ntc;
-            const int tb = two ? t2 : t;
-            const int ti2 = (ntr == 1) ? 0 : fast_div(tb, d.inv_ntc), tj2 = tb - ti2 * ntc;
-            const float *pa = sv + (ti * nh) * P + tj * nw;
-            const float *pb = sv + (ti2 * nh) * P + tj2 * nw;
-            const float2 nsi = (nh == 3) ? tile_pair_nsi<3, 3>(pa, pb, P, alpha) : tile_pair_nsi<1, 9>(pa, pb, P, alpha);
-            emit_key(nsi.x, kout + ti * d.TC + tj, hist_smem, nonfinite);
-            if (two) emit_key(nsi.y, kout + ti2 * d.TC + tj2, hist_smem, nonfinite);
-        }
-    } else {
-        for (int t = threadIdx.x; t < ntile; t += NTHREADS) {
-            const int ti = (ntr == 1) ? 0 : fast_div(t, d.inv_ntc);
-            const int tj = t - ti * ntc;
-            const int hh = min(nh, R - ti * nh);
-            const int ww = min(nw, W - tj * nw);
-            const float *pt = sv + (ti * nh) * P + tj * nw;
-            const float nsi = (hh == 3 && ww == 3) ? tile_nsi_fixed<3, 3>(pt, P, alpha)
-                              : (hh == 1 && ww == 9) ? tile_nsi_fixed<1, 9>(pt, P, alpha)
-                                                     : tile_nsi_generic(pt, P, hh, ww, alpha);
-            emit_key(nsi, kout + ti * d.TC + tj, hist_smem, nonfinite);
-        }
+    for (int t = threadIdx.x; t < ntile; t += NTHREADS) {
+        const int ti = (ntr == 1) ? 0 : fast_div(t, d.inv_ntc);
+        const int tj = t - ti * ntc;
+        const int hh = min(nh, R - ti * nh);
+        const int ww = min(nw, W - tj * nw);
+        const float *pt = sv + (ti * nh) * P + tj * nw;
+        const float nsi = (hh == 3 && ww == 3) ? tile_nsi_fixed<3, 3>(pt, P, alpha)
+                          : (hh == 1 && ww == 9) ? tile_nsi_fixed<1, 9>(pt, P, alpha)
+                                                 : tile_nsi_generic(pt, P, hh, ww, alpha);
+        emit_key(nsi, kout + ti * d.TC + tj, hist_smem, nonfinite);
     }
     return nonfinite;
 }
