@@ -590,3 +590,36 @@ def test_payload_exchange_through_nccl_one_rank():
     out = subprocess.run([sys.executable, "-c", NCCL_CHILD % (root, root)], env=env, capture_output=True, text=True,
                          timeout=300)
     assert out.returncode == 0 and "nccl exchange ok" in out.stdout, out.stdout + out.stderr
+
+
+# ---------------------------------------------------------------------------------------------
+# more workers than one launch serves (groups of 16): compress_workers and the aggregation
+# ---------------------------------------------------------------------------------------------
+
+def test_eighteen_workers_in_one_call(oracle):
+    shapes = [(120, 99, 3, 3), (64, 9, 1, 9), (1, 100, 1, 9)]
+    tensors = [("t%d" % i, (s[0], s[1])) for i, s in enumerate(shapes)]
+    plan = binding.Plan(shapes, alpha=0.5)
+    n_workers = 18
+    sig = synth.log_uniform_scales(len(shapes), (71,))
+    grads = synth.multi_worker_gradients(tensors, n_workers, (71,), sig)
+    ratios = np.array([0.1, 0.25, 0.5], np.float32)
+    zeros = [[np.zeros(s[0] * s[1], np.float32) for s in shapes] for _ in range(n_workers)]
+    _, refs, payloads = parity.compress_workers_and_check(oracle, plan, shapes, grads, zeros, ratios, 0.5,
+                                                          what="18 workers")
+    rng = np.random.default_rng(72)
+    dense0 = [(rng.standard_normal(s[0] * s[1]) * 1e-3).astype(np.float32) for s in shapes]
+    d_dense = parity.dev(parity.to_arena(plan, dense0))
+    plan.decompress_accumulate(payloads, d_dense, 0.125)          # two launches: 16 + 2 workers, in order
+    d_assign = parity.dev(parity.to_arena(plan, dense0))
+    plan.decompress_assign(payloads, d_assign, 0.125)
+    torch.cuda.synchronize()
+    results = [oracle.CompressResult(layers=r) for r in refs]
+    want = [d.copy() for d in dense0]
+    oracle.decompress_accumulate(shapes, want, results, 0.125)
+    for got, w in zip(parity.from_arena(plan, d_dense.cpu().numpy()), want):
+        np.testing.assert_array_equal(got.view(np.uint32), w.view(np.uint32))
+    want = [d.copy() for d in dense0]
+    oracle.decompress_assign(shapes, want, results, 0.125)
+    for got, w in zip(parity.from_arena(plan, d_assign.cpu().numpy()), want):
+        np.testing.assert_array_equal(got.view(np.uint32), w.view(np.uint32))
