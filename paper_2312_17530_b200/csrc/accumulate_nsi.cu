@@ -482,6 +482,8 @@ constexpr int kBulkCtasPerSmMomentum = 2;  // a third block per stage: 110 KB of
 constexpr int kStages = RSDGC_BULK_STAGES;  // shared-memory stages; loads run kStages - 1 items ahead
 constexpr int kLookahead = kStages - 1;
 constexpr unsigned int kSpinLimit = 1u << 22;  // bounded mbarrier waits
+constexpr int kOverlapPrev = 1;  // k1_bulk: the previous kernel in the stream is another worker's first pass
+constexpr int kOverlapNext = 2;  // k1_bulk: the next one is
 
 template <bool MOM>
 struct K1BulkShared {
@@ -591,12 +593,17 @@ __global__ void __launch_bounds__(kBulkThreads, MOM ? kBulkCtasPerSmMomentum : k
 k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict__ vel, float mom,
         uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
         const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
-        const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags)
+        const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags,
+        int overlap)
 {
     extern __shared__ __align__(128) unsigned char k1_bulk_smem_raw[];
     K1BulkShared<MOM> &sh = *reinterpret_cast<K1BulkShared<MOM> *>(k1_bulk_smem_raw);
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
-    if (begin >= end) return;
+    const bool wait_late = (overlap & kOverlapPrev) != 0;
+    if (begin >= end) {
+        if (wait_late) grid_dependency_wait();
+        return;
+    }
     const int tid = threadIdx.x;
     for (int b = tid; b < kL1Bins; b += kBulkThreads) sh.hist[b] = 0;
     if (tid == 0) {
@@ -605,9 +612,17 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
         fence_async_smem();
     }
     __syncthreads();
-    // launched with programmatic stream serialization: everything above overlapped the tail of the
-    // previous kernel in the stream; nothing below may run before that kernel has completed
-    grid_dependency_wait();
+    // Launched with programmatic stream serialization: everything above overlapped the tail of the
+    // previous kernel in the stream.  Normally nothing below may run before that kernel has
+    // completed.  kOverlapPrev: the previous kernel is the first pass of another worker of the same
+    // call, which touches none of this worker's buffers or tables and has itself passed its own wait
+    // (so everything older is complete): this launch runs alongside that kernel's last CTAs, and
+    // waits for it only before it exits, which keeps completion transitive along the stream.
+    // kOverlapNext: the next kernel is such a first pass; it may be scheduled as soon as CTAs of
+    // this one leave.  (Other successors are not released early: their few CTAs would crowd onto
+    // the first SMs that become free.)
+    if (!wait_late) grid_dependency_wait();
+    if (overlap & kOverlapNext) grid_dependency_launch_next();
     // prologue: the first kLookahead items start loading
     if (tid == 0) {
         for (int j = 0; j < kLookahead && begin + j < end; ++j) {
@@ -686,6 +701,7 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
         atomicOr(&status->flags, RSDGC_STATUS_NONFINITE);
     }
     if (timed_out) atomicOr(&status->flags, RSDGC_STATUS_TIMEOUT);
+    if (wait_late) grid_dependency_wait();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -738,7 +754,7 @@ int k1_reg_ctas_per_sm(int dtype, bool momentum)
 template <typename G, bool MOM>
 static void launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                             float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                            cudaStream_t s, int *launches)
+                            cudaStream_t s, int *launches, int overlap)
 {
     const G *g = reinterpret_cast<const G *>(grads);
     if (p->n_items_bulk > 0) {
@@ -756,7 +772,8 @@ static void launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *state, co
         const ItemDev *items = p->d_items;
         const int32_t *cta_begin = p->d_cta_begin_bulk;
         (void)cudaLaunchKernelEx(&cfg, k1_bulk<G, MOM>, g, resid, vel, mom, keys, layers, items, cta_begin, hist,
-                                 state, ratios, counts, p->d_status, p->alpha, (unsigned int)p->flags);
+                                 state, ratios, counts, p->d_status, p->alpha, (unsigned int)p->flags,
+                                 overlap);
         ++*launches;
     }
     if (p->n_items_reg > 0) {
@@ -768,18 +785,24 @@ static void launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *state, co
 }
 
 // vel == nullptr: plain accumulation v = g + r; otherwise u = mom * u + g, v = r + u.
+// after_sibling / before_sibling: the kernel launched just before / next on this stream is the first
+// pass of another worker of the same call (see k1_bulk); only honoured when a first pass is a
+// single bulk-copy kernel.
 int launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                           float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                          cudaStream_t s)
+                          cudaStream_t s, bool after_sibling, bool before_sibling)
 {
+    int overlap = 0;
+    if (p->n_items_reg == 0)  // the register-staged kernel is launched without overlap
+        overlap = (after_sibling ? kOverlapPrev : 0) | (before_sibling ? kOverlapNext : 0);
     int launches = 0;
     if (configure_once() != cudaSuccess) return 0;
     if (p->dtype == RSDGC_BF16) {
-        if (vel) launch_k1_typed<__nv_bfloat16, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
-        else launch_k1_typed<__nv_bfloat16, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+        if (vel) launch_k1_typed<__nv_bfloat16, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
+        else launch_k1_typed<__nv_bfloat16, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
     } else {
-        if (vel) launch_k1_typed<float, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
-        else launch_k1_typed<float, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches);
+        if (vel) launch_k1_typed<float, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
+        else launch_k1_typed<float, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
     }
     count_launch(launches);
     return launches;

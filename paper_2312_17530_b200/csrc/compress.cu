@@ -612,8 +612,9 @@ cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *co
                 ln = Lane{keys_all + (size_t)w * key_stride, x.hist, x.state, x.chunk_cnt, x.codes, resid[w], idx[w],
                           val[w]};
             }
+            // the first passes of a group's workers share nothing: all but the first start without waiting
             launch_accumulate_nsi(p, ln.hist, ln.state, grads[w], ln.resid, nullptr, 0.0f, ratios, counts[w], ln.keys,
-                                  s);
+                                  s, j > 0, j + 1 < n);
         }
         if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
         if (e == cudaSuccess) e = launch_selection(p, lanes, n, idx_cap, val_cap, prof, s);

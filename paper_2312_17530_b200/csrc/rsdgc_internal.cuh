@@ -203,6 +203,6 @@ int k1_reg_ctas_per_sm(int dtype, bool momentum);
 int k1_bulk_ctas_per_sm(bool momentum);
 int launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                           float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                          cudaStream_t s);
+                          cudaStream_t s, bool after_sibling = false, bool before_sibling = false);
 
 }  // namespace rsdgc
