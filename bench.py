@@ -556,10 +556,10 @@ def run_b200(args):
 
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k1_bulk launch on the benchmark workload:
-# 12.02 B/element measured by ncu on the fc6 layer alone (1235.53 MB for 102,760,448 elements,
+# 12.03 B/element measured by ncu on the fc6 layer alone (1235.73 MB for 102,760,448 elements,
 # profiles/k1_bulk_fc6_25088x4096.md), scaled to the 139,754,605 elements of one launch here
 # (traffic is proportional to the elements streamed).  Set to None when k1_bulk changes.
-K1_TRAFFIC_BYTES = int(1235.53e6 * 139754605 / 102760448)
+K1_TRAFFIC_BYTES = int(1235.73e6 * 139754605 / 102760448)
 
 
 def main():
