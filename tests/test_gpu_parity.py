@@ -375,6 +375,65 @@ def test_compress_and_aggregate_replay_from_a_cuda_graph(oracle):
     assert plan.status().flags == 0
 
 
+def test_compress_workers_replay_from_a_cuda_graph():
+    """The call that serves several workers lets their first passes run into one another (only the
+    first waits for what precedes it in the stream).  Captured in a CUDA graph and replayed, it must
+    give what the same calls give on a stream: three iterations, residuals carried, compared bit for bit."""
+    tensors = synth.resnet18_tensors()
+    shapes = synth.layer_shapes(tensors)
+    dev, W, ratio = "cuda:0", 3, 1 / 32
+    gen = torch.Generator(device=dev).manual_seed(77)
+    outs = {}
+    grads = None
+    for mode in ("stream", "graph"):
+        plan = binding.Plan(shapes, alpha=0.5)
+        plan.reserve_workers(W)
+        n = plan.info.arena_elems
+        ni, nv = plan.payload_bound(ratio)
+        if grads is None:
+            grads = [[torch.randn(n, device=dev, generator=gen) * 1e-2 for _ in range(W)] for _ in range(3)]
+        d_g = [torch.zeros(n, device=dev) for _ in range(W)]
+        d_r = [torch.zeros(n, device=dev) for _ in range(W)]
+        idx = [torch.zeros(ni, dtype=torch.int32, device=dev) for _ in range(W)]
+        val = [torch.zeros(nv, device=dev) for _ in range(W)]
+        cnt = [torch.zeros(len(shapes), dtype=torch.int32, device=dev) for _ in range(W)]
+        ws = torch.empty(W * plan.info.workspace_bytes, dtype=torch.uint8, device=dev)
+        ratios = torch.full((len(shapes),), ratio, device=dev)
+        d_dense = torch.zeros(n, device=dev)
+
+        def step():
+            plan.compress_workers(d_g, d_r, ratios, idx, val, cnt, ws)
+            plan.decompress_accumulate(list(zip(idx, val, cnt)), d_dense, 0.5)
+
+        graph = None
+        if mode == "graph":
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                step()                                   # warm-up outside the capture
+            side.synchronize()
+            for t in d_r + [d_dense]:
+                t.zero_()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            for t in d_r + [d_dense]:
+                t.zero_()
+        got = []
+        for it in range(3):
+            for w in range(W):
+                d_g[w].copy_(grads[it][w])
+            graph.replay() if graph is not None else step()
+            torch.cuda.synchronize()
+            got.append([t.cpu().numpy().copy() for t in idx + val + cnt + d_r + [d_dense]])
+        assert plan.status().flags == 0
+        outs[mode] = got
+        plan.close()
+    for a_it, b_it in zip(outs["stream"], outs["graph"]):
+        for a, b in zip(a_it, b_it):
+            np.testing.assert_array_equal(a.view(np.uint32), b.view(np.uint32))
+    assert int(outs["graph"][2][2 * W].sum()) > 0
+
+
 # ---------------------------------------------------------------------------------------------
 # the ablation rows of Table I as settings of the same path: "Neighbor" only (alpha = 1), no
 # "Dynamic" (one fixed ratio), and plain Top-k as the 1x1-neighborhood special case
