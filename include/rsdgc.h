@@ -132,10 +132,12 @@ int rsdgc_plan_layer_info(const rsdgc_plan *plan, int32_t layer, rsdgc_layer_inf
 int rsdgc_plan_payload_bound(const rsdgc_plan *plan, float max_ratio, int64_t *idx_capacity_host,
                              int64_t *val_capacity_host);
 
-/* Diagnostic: copies the work list of the accumulate+NSI pass, 7 int32 per item: layer,
+/* Diagnostic: copies the work list of the accumulate+NSI pass, 9 int32 per item: layer,
  * first tile row, tile rows, first tile col, tile cols (the items of a layer partition its
  * tile grid), the kernel that takes the item (0 = bulk-copy kernel, 1 = register-staged
- * kernel) and the CTA of that kernel that owns it; grids_host[0..1] receive the two kernels'
+ * kernel), the CTA of that kernel that owns it, the row pitch (elements) of the item's block in
+ * shared memory, and the item's flags (1 = one contiguous run, 2 = 128-bit accesses, 4 = bulk
+ * copies, 8 = no clipped tile); grids_host[0..1] receive the two kernels'
  * grid sizes and n_flush_host[l] how many (kernel, CTA) pairs touch layer l.  Any pointer
  * may be NULL.  Returns the number of items (or a negative rsdgc_error).  Host only. */
 int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,

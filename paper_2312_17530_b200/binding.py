@@ -171,11 +171,13 @@ class Plan:
         return a.value, b.value
 
     def worklist(self):
-        """(items [n,7] int32: layer, tr0, ntr, tc0, ntc, kernel, cta; grids [2]; n_flush [L])."""
+        """(items [n,9] int32: layer, tr0, ntr, tc0, ntc, kernel, cta, shared-memory pitch, item
+        flags (1 contiguous, 2 128-bit accesses, 4 bulk copies, 8 no clipped tile); grids [2];
+        n_flush [L])."""
         import numpy as np
 
         n = lib().rsdgc_plan_worklist(self._h, None, 0, None, None)
-        items = np.zeros((n, 7), dtype=np.int32)
+        items = np.zeros((n, 9), dtype=np.int32)
         grids = np.zeros(2, dtype=np.int32)
         nf = np.zeros(self.n_layers, dtype=np.int32)
         lib().rsdgc_plan_worklist(self._h, items.ctypes.data, n, grids.ctypes.data, nf.ctypes.data)

@@ -146,6 +146,11 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
             if (round_up64(ntc, 8) <= ntc_max) ntc = round_up64(ntc, 8);
             else if (ntc_max >= 8) ntc = ntc_max & ~(int64_t)7;
             chunk_w[l] = std::min<int64_t>(ntc * d.nw, d.cols);
+            // the chunk width is also the row pitch of the block in shared memory: a multiple of 8
+            // elements keeps every row of the block 16-byte aligned there for both element sizes
+            // (neighborhoods of more than 550 elements leave fewer than 8 tile columns per item, so
+            // the width itself need not be one)
+            if (round_up64(chunk_w[l], 8) * d.nh <= kItemElems) chunk_w[l] = round_up64(chunk_w[l], 8);
             for (int64_t tr = 0; tr < L.TR; ++tr)
                 for (int64_t tc0 = 0; tc0 < L.TC; tc0 += ntc) {
                     Item it{l, (int32_t)tr, 1, (int32_t)tc0, (int32_t)std::min<int64_t>(ntc, L.TC - tc0)};
@@ -180,6 +185,8 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
     std::vector<ItemDev> all(n_items);
     p->item_path.assign(n_items, 0);
     p->item_cta.assign(n_items, 0);
+    p->item_pitch.assign(n_items, 0);
+    p->item_flags.assign(n_items, 0);
     std::vector<double> cost(n_items);
     for (size_t i = 0; i < n_items; ++i) {
         const Item &it = p->items[i];
@@ -197,19 +204,23 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
         d.nw = (int16_t)L.nw;
         d.layer = it.layer;
         const bool full = (d.W == L.cols) || d.R == 1;  // one contiguous run
-        const bool vec = (d.gbase % 4 == 0) && (full || (L.cols % 4 == 0 && d.W % 4 == 0));
-        const bool bulk = !(p->flags & RSDGC_NO_BULK_COPY) && (d.gbase % gran == 0) &&
-                          (full || (L.cols % gran == 0 && d.W % gran == 0));
-        const bool noclip = (d.R % L.nh == 0) && (d.W % L.nw == 0);
-        d.flags = (full ? kItemFull : 0) | (vec ? kItemVec : 0) | (bulk ? kItemBulk : 0) | (noclip ? kItemNoClip : 0);
         // shared-memory pitch: the width of the layer's regular column chunk, so that every item
         // of a layer maps threads to elements the same way (the last chunk of a row is narrower)
         d.P = full ? d.W : (int32_t)chunk_w[it.layer];
+        // 128-bit accesses / bulk copies need every row of the item 16-byte aligned in global
+        // memory (start, row stride, width) AND in the shared-memory block (pitch)
+        const bool vec = (d.gbase % 4 == 0) && (full || (L.cols % 4 == 0 && d.W % 4 == 0 && d.P % 4 == 0));
+        const bool bulk = !(p->flags & RSDGC_NO_BULK_COPY) && (d.gbase % gran == 0) &&
+                          (full || (L.cols % gran == 0 && d.W % gran == 0 && d.P % gran == 0));
+        const bool noclip = (d.R % L.nh == 0) && (d.W % L.nw == 0);
+        d.flags = (full ? kItemFull : 0) | (vec ? kItemVec : 0) | (bulk ? kItemBulk : 0) | (noclip ? kItemNoClip : 0);
         d.inv_ntc = magic(d.ntc);
         d.inv_p = magic(d.P);
         d.inv_pv = magic(d.P / 4);
         all[i] = d;
         p->item_path[i] = bulk ? 0 : 1;
+        p->item_pitch[i] = d.P;
+        p->item_flags[i] = d.flags;
         cost[i] = (double)d.R * d.W + 512.0;  // elements + a fixed cost per item
         // the first item of a layer pays for the previous layer's histogram flush in its CTA
         if (i > 0 && p->items[i - 1].layer != it.layer) cost[i] += 6000.0;
@@ -386,8 +397,9 @@ extern "C" int rsdgc_plan_payload_bound(const rsdgc_plan *plan, float max_ratio,
     return RSDGC_OK;
 }
 
-// Diagnostic: the accumulate+NSI work list (7 int32 per item: layer, tr0, ntr, tc0, ntc, kernel,
-// CTA), the two grid sizes and the per-layer flush counts; used by the host-logic tests.
+// Diagnostic: the accumulate+NSI work list (9 int32 per item: layer, tr0, ntr, tc0, ntc, kernel,
+// CTA, shared-memory pitch, item flags), the two grid sizes and the per-layer flush counts; used by
+// the host-logic tests.
 extern "C" int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,
                                        int32_t *grids_host, int32_t *n_flush_host)
 {
@@ -396,9 +408,10 @@ extern "C" int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_ho
     if (items_host)
         for (int64_t i = 0; i < n && i < items_capacity; ++i) {
             const Item &it = plan->items[i];
-            int32_t *o = items_host + 7 * i;
+            int32_t *o = items_host + 9 * i;
             o[0] = it.layer, o[1] = it.tr0, o[2] = it.ntr, o[3] = it.tc0, o[4] = it.ntc;
             o[5] = plan->item_path[i], o[6] = plan->item_cta[i];
+            o[7] = plan->item_pitch[i], o[8] = plan->item_flags[i];
         }
     if (grids_host) grids_host[0] = plan->grid_bulk, grids_host[1] = plan->grid_reg;
     if (n_flush_host)

@@ -143,6 +143,7 @@ struct rsdgc_plan {
     std::vector<rsdgc::Item> items;
     std::vector<rsdgc::ItemDev> items_dev;
     std::vector<int32_t> item_path, item_cta;          // per host item: kernel (0 bulk, 1 reg) and CTA
+    std::vector<int32_t> item_pitch, item_flags;       // per host item: shared-memory row pitch, kItem* bits
     std::vector<int32_t> cta_begin_bulk, cta_begin_reg;  // grid + 1 indices into each kernel's item list
     std::vector<rsdgc::Chunk> chunks;
     std::vector<rsdgc::EChunk> echunks;

@@ -46,14 +46,20 @@ def test_plan_create_rejects_bad_arguments(lib):
     assert lib.rsdgc_compress(p._h, 16, 16, 16, 16, 1, 16, 1, 16, None, 16, None) == binding.ERR_INVALID
 
 
-@pytest.mark.parametrize("net", ["resnet18", "resnet50", "vgg19", "odd"])
-def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net):
-    if net == "odd":
+@pytest.mark.parametrize("net,dtype", [("resnet18", 0), ("resnet50", 0), ("vgg19", 0), ("odd", 0), ("odd", 1),
+                                       ("wide_tiles", 0), ("wide_tiles", 1)])
+def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net, dtype):
+    gran = 8 if dtype == binding.RSDGC_BF16 else 4      # elements per 16 bytes of the gradient arena
+    if net == "wide_tiles":
+        # neighborhoods of more than 550 elements: fewer than 8 tile columns fit an item, so the
+        # column chunks are not multiples of 8 tiles wide
+        shapes = [(50, 400, 25, 25), (40, 480, 20, 30), (75, 1000, 25, 25), (64, 4096, 32, 32), (30, 777, 30, 21)]
+    elif net == "odd":
         shapes = [(7, 11, 3, 3), (1, 5, 1, 9), (4096, 45, 3, 3), (3, 20000, 3, 3), (100, 4401, 2, 5),
                   (5000, 7, 1, 7), (1, 100000, 1, 9), (64, 64, 64, 64), (9, 9, 1, 1)]
     else:
         shapes = synth.layer_shapes(getattr(synth, net + "_tensors")())
-    p = binding.Plan(shapes, device=-1)
+    p = binding.Plan(shapes, device=-1, grad_dtype=dtype)
     assert p.info.n_layers == len(shapes)
     assert p.info.total_elems == sum(r * c for r, c, _, _ in shapes)
     tiles = [(-(-r // nh)) * (-(-c // nw)) for r, c, nh, nw in shapes]
@@ -74,21 +80,28 @@ def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net):
         TR, TC = -(-r // nh), -(-c // nw)
         cover = np.zeros((TR, TC), dtype=np.int32)
         sel = items[items[:, 0] == l]
-        for _, tr0, ntr, tc0, ntc, path, cta in sel.tolist():
+        for _, tr0, ntr, tc0, ntc, path, cta, pitch, flags in sel.tolist():
             assert ntr >= 1 and ntc >= 1 and tr0 + ntr <= TR and tc0 + ntc <= TC
             rows = min(r, (tr0 + ntr) * nh) - tr0 * nh
             cols = min(c, (tc0 + ntc) * nw) - tc0 * nw
             assert rows * cols <= 4400
             assert ntr == 1 or (tc0 == 0 and ntc == TC)   # several tile rows only at full width
             assert path in (0, 1) and 0 <= cta < grids[path]
-            # the bulk-copy kernel only takes items whose rows start on 16-byte boundaries
             start = p.layers[l].elem_offset + tr0 * nh * c + tc0 * nw
             contiguous = cols == c or rows == 1
-            aligned = start % 4 == 0 and (contiguous or (c % 4 == 0 and cols % 4 == 0))
-            assert (path == 0) == aligned
+            assert bool(flags & 1) == contiguous
+            # the block in shared memory: rows of `pitch` elements, all of it inside one stage
+            assert pitch >= cols and (pitch == cols if contiguous else rows * pitch <= 4400)
+            # 128-bit accesses (flag 2) and bulk copies (flag 4, the bulk-copy kernel) need every row of
+            # the item 16-byte aligned in global memory (start, row stride, width) and, through the
+            # pitch, in shared memory; bulk copies need that for the gradient's element size too
+            def aligned(g):
+                return start % g == 0 and (contiguous or (c % g == 0 and cols % g == 0 and pitch % g == 0))
+            assert bool(flags & 2) == aligned(4)
+            assert bool(flags & 4) == aligned(gran) and (path == 0) == bool(flags & 4)
             cover[tr0:tr0 + ntr, tc0:tc0 + ntc] += 1
         assert (cover == 1).all()
-        assert nflush[l] == len(set((pa, ct) for *_, pa, ct in sel.tolist()))
+        assert nflush[l] == len(set((it[5], it[6]) for it in sel.tolist()))
     # within a kernel the CTA of consecutive items never decreases, and the static partition is
     # balanced: no CTA holds much more than the mean cost
     for path in (0, 1):
@@ -97,11 +110,11 @@ def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net):
             continue
         assert (np.diff(sel[:, 6]) >= 0).all()
         cost = np.zeros(grids[path])
-        for l, tr0, ntr, tc0, ntc, _, cta in sel.tolist():
+        for l, tr0, ntr, tc0, ntc, _, cta, _, _ in sel.tolist():
             r, c, nh, nw = shapes[l]
             cost[cta] += (min(r, (tr0 + ntr) * nh) - tr0 * nh) * (min(c, (tc0 + ntc) * nw) - tc0 * nw) + 512
         assert cost.max() <= cost.sum() / len(cost) + 4400 + 512 + 1
-    if net != "odd":
+    if net not in ("odd", "wide_tiles"):
         assert (items[:, 5] == 0).mean() > 0.99       # the usual shapes go to the bulk-copy kernel
 
 
