@@ -1,8 +1,9 @@
 """GPU parity on the full-size workloads: the VGG-19-shaped set with 4 workers and their
 aggregation (the configuration the benchmark times), the ResNet-50-shaped set over 100 iterations
 with drifting scales and refreshed ratios, and the single-matrix sweep from 1M to 1B elements in
-binary32 and bfloat16.  Sizes the oracle can sort are compared element by element; above that,
-sampled tiles go through the oracle and the rest is checked by exact properties."""
+binary32 and bfloat16.  Sizes the oracle can sort are compared through its own selection; above that,
+every key still goes through the oracle's indicator and the kept set is the oracle's rule evaluated with
+a partition instead of its full sort."""
 import numpy as np
 import pytest
 import torch
@@ -124,15 +125,6 @@ def _sweep_inputs(rows, cols, bf16):
     return synth.f32_to_bf16_bits(x) if bf16 else x
 
 
-def _run_single(plan, g, ratio):
-    gc = parity.GpuCompress(plan, max_ratio=ratio)
-    d_g = parity.dev(parity.to_arena(plan, [g], np.uint16 if g.dtype == np.uint16 else np.float32))
-    d_r = torch.zeros(plan.info.arena_elems, device="cuda:0")            # a real buffer, still read
-    st = gc.run(d_g, d_r, torch.tensor([ratio], dtype=torch.float32, device="cuda:0"))
-    assert st.flags == 0
-    return gc, d_r
-
-
 @pytest.mark.parametrize("rows,cols", [(1024, 1024), (4096, 4096), (2450, 400), (7840, 1280)])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_sweep_small_full_oracle(oracle, rows, cols, bf16):
@@ -154,21 +146,42 @@ def test_sweep_medium_full_oracle(oracle, rows, cols, bf16, ratio):
                               max_ratio=ratio, what="sweep %dx%d" % (rows, cols))
 
 
-@pytest.mark.parametrize("rows,cols,bf16,ratio", [(8192, 8192, True, 1 / 10), (16384, 16384, False, 1 / 10),
-                                                  (32768, 32768, True, 1 / 100), (78400, 12800, False, 1 / 1000)])
-def test_sweep_large_sampled(oracle, rows, cols, bf16, ratio):
+# (rows, cols, dtypes, ratios): every key of the layer goes through the oracle; one input per shape, the
+# bfloat16 variant is the rounded binary32 draw; all three ratios at 268 M elements in both dtypes, the
+# 1 B-element matrices in both dtypes
+LARGE = [(8192, 8192, (True,), (1 / 10,)),
+         (25088, 4096, (True,), (1 / 100,)),
+         (16384, 16384, (False, True), synth.SWEEP_RATIOS),
+         (32768, 32768, (False, True), (1 / 100,)),
+         (78400, 12800, (False, True), (1 / 1000,))]
+
+
+@pytest.mark.parametrize("rows,cols,dtypes,ratios", LARGE, ids=["%dx%d" % (c[0], c[1]) for c in LARGE])
+def test_sweep_large_every_key(oracle, rows, cols, dtypes, ratios):
     shape = (rows, cols, 3, 3)
-    g = _sweep_inputs(rows, cols, bf16)
-    plan = binding.Plan([shape], grad_dtype=binding.RSDGC_BF16 if bf16 else binding.RSDGC_F32, alpha=0.5)
-    gc, d_r = _run_single(plan, g, ratio)
-    k = int(gc.counts.cpu().numpy()[0])
-    li = plan.layers[0]
-    nsi = gc.nsi.cpu().numpy()[:li.n_tiles]
-    idx = gc.idx.cpu().numpy()[:k]
-    val = gc.val.cpu().numpy()[:k * 9]
-    res = d_r.cpu().numpy()[:rows * cols]
-    del gc, d_r
-    torch.cuda.empty_cache()
-    parity.check_single_layer_sampled(oracle, shape, g, np.zeros(rows * cols, np.float32), float(np.float32(ratio)),
-                                      0.5, nsi, k, idx, val, res,
-                                      what="sweep %dx%d bf16=%s 1/%d" % (rows, cols, bf16, round(1 / ratio)))
+    x = synth.clustered_matrix(rows, cols, seed=5)
+    zeros = np.zeros(rows * cols, np.float32)
+    for bf16 in dtypes:
+        g = synth.f32_to_bf16_bits(x) if bf16 else x
+        ref = parity.LargeLayerReference(oracle, shape, g, zeros, 0.5)
+        plan = binding.Plan([shape], grad_dtype=binding.RSDGC_BF16 if bf16 else binding.RSDGC_F32, alpha=0.5)
+        li = plan.layers[0]
+        d_g = parity.dev(parity.to_arena(plan, [g], np.uint16 if bf16 else np.float32))
+        for ratio in ratios:
+            gc = parity.GpuCompress(plan, max_ratio=ratio)
+            d_r = torch.zeros(plan.info.arena_elems, device="cuda:0")        # a real buffer, still read
+            st = gc.run(d_g, d_r, torch.tensor([ratio], dtype=torch.float32, device="cuda:0"))
+            assert st.flags == 0
+            k = int(gc.counts.cpu().numpy()[0])
+            nsi = gc.nsi.cpu().numpy()[:li.n_tiles]
+            idx = gc.idx.cpu().numpy()[:k]
+            val = gc.val.cpu().numpy()[:k * 9]
+            assert (gc.idx.cpu().numpy()[k:] == -1).all() and (gc.val.cpu().numpy()[k * 9:] == parity.CANARY).all()
+            res = d_r.cpu().numpy()[:rows * cols]
+            del gc, d_r
+            torch.cuda.empty_cache()
+            ref.check(float(np.float32(ratio)), nsi, k, idx, val, res,
+                      what="sweep %dx%d bf16=%s 1/%d" % (rows, cols, bf16, round(1 / ratio)))
+            del nsi, idx, val, res
+        del d_g, plan, ref, g
+        torch.cuda.empty_cache()

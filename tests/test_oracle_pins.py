@@ -238,6 +238,50 @@ def test_momentum_correction_closed_forms(oracle):
     np.testing.assert_array_equal(v2, r0 + u2)
 
 
+def test_momentum_correction_with_bfloat16_gradients(oracle):
+    """Eq. 12, first two lines, with the gradient stored as bfloat16: the stored 16 bits are widened
+    exactly (they are the upper half of the binary32), then u = fl(m u0) + g and v = r + u with the
+    product rounded before the sum.  Expected values are built with NumPy / torch binary32 ops from the
+    bit patterns; m = 0 reduces to the plain accumulation; a plausible mistake (rounding g again, using
+    the unwidened binary32 draw, a fused multiply-add, u and r swapped) changes some element."""
+    from paper_2312_17530_b200 import synth
+
+    rng = np.random.default_rng(21)
+    n = 4099
+    x = (rng.standard_normal(n) * 10.0 ** rng.uniform(-6, 1, n)).astype(np.float32)
+    x[:6] = [0.0, -0.0, 1.0 + 2.0 ** -8, 3.0e38, 1.0e-40, -2.5]       # tie, near-overflow, subnormal
+    bits = synth.f32_to_bf16_bits(x)
+    widened = (bits.astype(np.uint32) << 16).view(np.float32)         # exact by construction of the format
+    assert not np.array_equal(widened, x)                             # the 16-bit storage does lose bits
+    np.testing.assert_array_equal(widened, torch.from_numpy(bits.view(np.int16)).view(torch.bfloat16)
+                                  .to(torch.float32).numpy())
+    u0 = rng.standard_normal(n).astype(np.float32)
+    r0 = (rng.standard_normal(n) * 1e-2).astype(np.float32)
+    m = 0.9
+    u1, v1 = oracle.accumulate_momentum(bits, u0, r0, m)
+    prod = np.float32(m) * u0                                         # one rounding
+    want_u = prod + widened                                           # one rounding
+    np.testing.assert_array_equal(u1.view(np.uint32), want_u.view(np.uint32))
+    np.testing.assert_array_equal(v1.view(np.uint32), (r0 + want_u).view(np.uint32))
+    # the same through torch's binary32 arithmetic
+    tu = torch.from_numpy(u0) * torch.tensor(np.float32(m)) + torch.from_numpy(widened)
+    np.testing.assert_array_equal(u1, tu.numpy())
+    # not fused: the exactly rounded m*u0 + g differs somewhere from the two-step result
+    fused = (np.float64(np.float32(m)) * u0.astype(np.float64) + widened.astype(np.float64)).astype(np.float32)
+    assert (fused != u1).any()
+    # m = 0: u = g exactly, v = the plain accumulation of Eq. 12's second line
+    u2, v2 = oracle.accumulate_momentum(bits, u0, r0, 0.0)
+    np.testing.assert_array_equal(u2.view(np.uint32) & 0x7FFFFFFF, widened.view(np.uint32) & 0x7FFFFFFF)
+    np.testing.assert_array_equal(v2, oracle.accumulate(bits, r0))
+    # the binary32 entry point on the widened values gives the same bits: the two variants differ only
+    # in how the gradient is stored
+    u3, v3 = oracle.accumulate_momentum(widened, u0, r0, m)
+    np.testing.assert_array_equal(u1.view(np.uint32), u3.view(np.uint32))
+    np.testing.assert_array_equal(v1.view(np.uint32), v3.view(np.uint32))
+    # inputs are not modified
+    np.testing.assert_array_equal(bits, synth.f32_to_bf16_bits(x))
+
+
 # ---------------------------------------------------------------------------------------------
 # keep count (Eq. 11) and selection
 # ---------------------------------------------------------------------------------------------
@@ -254,6 +298,47 @@ def test_keep_count_examples(oracle):
     # the ratio is a binary32 number; the product is taken in binary64
     assert oracle.keep_count(10, 0.1) == math.ceil(10 * float(np.float32(0.1)))
     assert oracle.keep_count(1 << 20, 0.001) == math.ceil((1 << 20) * float(np.float32(0.001)))
+
+
+def test_partition_form_of_the_selection_equals_the_oracles_sort(oracle):
+    """The GPU tests on layers of 10^8 tiles evaluate the oracle's selection rule with a partition
+    (parity.select_by_partition) because the oracle's full sort takes minutes there; here the two
+    are held together on inputs with few distinct values (many ties at the threshold), all-equal
+    keys, zeros, an infinity, and k at both ends."""
+    import parity
+
+    rng = np.random.default_rng(31)
+    cases = [rng.standard_normal(5000).astype(np.float32) ** 2,
+             rng.integers(0, 4, 3000).astype(np.float32) * np.float32(0.25),      # four distinct values
+             np.full(777, 0.5, np.float32), np.zeros(100, np.float32),
+             np.concatenate([rng.random(500).astype(np.float32), [np.inf, 0.0, np.inf]]).astype(np.float32)]
+    for keys in cases:
+        for k in (0, 1, 2, keys.size // 64 + 1, keys.size // 3, keys.size - 1, keys.size):
+            want, _ = oracle.select(keys, k)
+            np.testing.assert_array_equal(parity.select_by_partition(keys, k), want)
+
+
+def test_large_layer_reference_agrees_with_the_layer_oracle(oracle):
+    """parity.LargeLayerReference (bands of tile rows through oracle.nsi, partition selection, oracle.pack)
+    must reproduce oracle.compress_layer, ragged edges and a band boundary inside the layer included."""
+    import parity
+    from paper_2312_17530_b200 import synth
+
+    rng = np.random.default_rng(32)
+    for shape, bf16 in (((100, 131, 3, 3), False), ((64, 50, 3, 3), True), ((10, 90, 1, 9), False)):
+        rows, cols = shape[:2]
+        x = (rng.standard_normal(rows * cols) * 1e-2).astype(np.float32)
+        g = synth.f32_to_bf16_bits(x) if bf16 else x
+        r = (rng.standard_normal(rows * cols) * 1e-3).astype(np.float32)
+        big = parity.LargeLayerReference(oracle, shape, g, r, 0.5, band_tile_rows=7)
+        for ratio in (0.1, 0.01):
+            ratio = float(np.float32(ratio))
+            ref = oracle.compress_layer(g, r, shape, ratio, 0.5)
+            big.check(ratio, ref.nsi_f32, ref.k, ref.idx, ref.val, ref.residual)
+            wrong = ref.residual.copy()
+            wrong[int(ref.idx[0]) // big.TC * shape[2] * cols] = 1.0      # a sent entry not cleared
+            with pytest.raises(AssertionError):
+                big.check(ratio, ref.nsi_f32, ref.k, ref.idx, ref.val, wrong)
 
 
 def test_select_1x1_alpha1_is_library_topk(oracle):

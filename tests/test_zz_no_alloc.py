@@ -4,8 +4,10 @@ through their own pool, loops that cannot take an allocation's implicit synchron
 
 The entry point keeps its scratch in a fixed array inside the library instead of in a plan, so
 this test calls it through the C ABI and requires the same ratios, bit for bit, as the plan-based
-rsdgc_update_ratios() on the same weights -- twice in a row with different inputs, because the
-array is shared by all calls and still holds the previous call's contents when the next one starts.
+rsdgc_update_ratios() on the same weights AND as the CPU oracle's ratio rule (the two GPU kernels are
+close relatives, so agreement between them alone would not see a mistake they share) -- twice in a
+row with different inputs, because the array is shared by all calls and still holds the previous
+call's contents when the next one starts.
 This file is collected last on purpose: a failure here cannot hide a failure elsewhere.
 """
 import numpy as np
@@ -24,7 +26,7 @@ def _weights_arena(plan, weights):
     return torch.from_numpy(a).to("cuda:0")
 
 
-def test_noalloc_matches_plan_based_entry_point_twice_in_a_row():
+def test_noalloc_matches_plan_based_entry_point_twice_in_a_row(oracle):
     assert torch.cuda.is_available()
     tensors = synth.resnet18_tensors()[:binding.NOALLOC_MAX_LAYERS - 2] + [("tail.weight", (1000, 37)),
                                                                            ("tail.bias", (5,))]
@@ -43,9 +45,15 @@ def test_noalloc_matches_plan_based_entry_point_twice_in_a_row():
         want = torch.full((len(shapes),), -1.0, device="cuda:0")
         got = torch.full((len(shapes),), -2.0, device="cuda:0")
         plan.update_ratios(d_w, rho, want)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]      # the driver's view: sees any cudaMalloc in the library
         binding.update_ratios_noalloc(d_w, offsets, sizes, rho, got)
         torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
         np.testing.assert_array_equal(got.cpu().numpy(), want.cpu().numpy())
+        ref_ratios, survivors, n_keep = oracle.update_ratios(weights, rho)
+        np.testing.assert_array_equal(got.cpu().numpy(), ref_ratios)
+        assert int(survivors.sum()) == n_keep
         assert 0.0 < float(got.max()) <= 1.0
         del d_w, want, got
     assert torch.cuda.memory_allocated() == mem_before
