@@ -275,15 +275,18 @@ int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_de
  * product then sum, each rounded to binary32 (scale = 1 gives the paper's plain sum).
  * idx_dev_host / val_dev_host / counts_dev_host: HOST arrays of n_workers DEVICE pointers
  * to payloads produced by rsdgc_compress() with this plan (or an identical one): the tile
- * indices of a layer must be ascending.  dense_dev: binary32 arena, in/out.  Entries whose tile
- * index breaks that order or lies outside the layer are skipped.
+ * indices of a layer must be ascending.  idx_capacity / val_capacity: the number of entries
+ * every worker's idx / val buffer holds (the capacities given to rsdgc_compress()); a payload
+ * that did not fit them (RSDGC_STATUS_PAYLOAD_OVERFLOW: counts say more than was written) is
+ * aggregated as far as it was written, nothing is read past the buffers.  dense_dev: binary32
+ * arena, in/out.  Entries whose tile index breaks the order or lies outside the layer are skipped.
  * Errors: INVALID, ALIGNMENT, CUDA.
  */
 int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,
                                 const int32_t *const *idx_dev_host,
                                 const void *const *val_dev_host,
-                                const int32_t *const *counts_dev_host, float scale,
-                                float *dense_dev, void *stream);
+                                const int32_t *const *counts_dev_host, int64_t idx_capacity,
+                                int64_t val_capacity, float scale, float *dense_dev, void *stream);
 
 /*
  * The same aggregation into a dense arena that holds nothing yet (Eq. 12, third line, as an
@@ -295,7 +298,8 @@ int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers,
  */
 int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
                             const void *const *val_dev_host, const int32_t *const *counts_dev_host,
-                            float scale, float *dense_dev, void *stream);
+                            int64_t idx_capacity, int64_t val_capacity, float scale, float *dense_dev,
+                            void *stream);
 
 /*
  * Per-element (coordinate) view of a payload.  The payload of Sec. III-C names neighborhoods;

@@ -90,8 +90,10 @@ def lib():
                                              C.POINTER(vp), i64, C.POINTER(vp), vp, vp]
         L.rsdgc_compress_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, vp,
                                           C.POINTER(i64), C.POINTER(i64), vp]
-        L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
-        L.rsdgc_decompress_assign.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), f32, vp, vp]
+        L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), i64, i64, f32,
+                                                  vp, vp]
+        L.rsdgc_decompress_assign.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), i64, i64, f32, vp,
+                                              vp]
         L.rsdgc_payload_to_coo.argtypes = [vp, vp, vp, vp, i64, vp]
         L.rsdgc_get_status.argtypes = [vp, vp, C.POINTER(Status)]
         L.rsdgc_profile_enable.argtypes = [vp, i32]
@@ -234,7 +236,9 @@ class Plan:
         for w, (i, v, c) in enumerate(payloads):
             ia[w], va[w], ca[w] = i.data_ptr(), v.data_ptr(), c.data_ptr()
         fn = lib().rsdgc_decompress_assign if assign else lib().rsdgc_decompress_accumulate
-        _check(fn(self._h, n, ia, va, ca, scale, _ptr(dense), _stream()),
+        idx_cap = min((i.numel() for i, _, _ in payloads), default=0)
+        val_cap = min((v.numel() for _, v, _ in payloads), default=0)
+        _check(fn(self._h, n, ia, va, ca, idx_cap, val_cap, scale, _ptr(dense), _stream()),
                "rsdgc_decompress_assign" if assign else "rsdgc_decompress_accumulate")
 
     def decompress_assign(self, payloads, dense, scale: float = 1.0) -> None:

@@ -712,9 +712,19 @@ static cudaError_t allow_smem(K kernel, size_t bytes)
     return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
 }
 
+// Raises the kernels' dynamic shared-memory limits, once per device (the attribute belongs to the
+// device's context); a failure is not cached, so a later call tries again instead of silently
+// launching nothing.  The caller has made the plan's device current.
 static cudaError_t configure_once()
 {
-    static cudaError_t result = [] {
+    constexpr int kMaxDevices = 64;
+    static bool done[kMaxDevices] = {};
+    int dev = 0;
+    cudaError_t ed = cudaGetDevice(&dev);
+    if (ed != cudaSuccess) return ed;
+    const bool tracked = dev >= 0 && dev < kMaxDevices;
+    if (tracked && done[dev]) return cudaSuccess;
+    const cudaError_t result = [] {
         cudaError_t e = allow_smem(k1_reg<float, false>, sizeof(K1RegShared));
         if (e == cudaSuccess) e = allow_smem(k1_reg<float, true>, sizeof(K1RegShared));
         if (e == cudaSuccess) e = allow_smem(k1_reg<__nv_bfloat16, false>, sizeof(K1RegShared));
@@ -725,6 +735,7 @@ static cudaError_t configure_once()
         if (e == cudaSuccess) e = allow_smem(k1_bulk<__nv_bfloat16, true>, sizeof(K1BulkShared<true>));
         return e;
     }();
+    if (tracked) done[dev] = (result == cudaSuccess);
     return result;
 }
 
@@ -752,11 +763,12 @@ int k1_reg_ctas_per_sm(int dtype, bool momentum)
 }
 
 template <typename G, bool MOM>
-static void launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
-                            float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                            cudaStream_t s, int *launches, int overlap)
+static cudaError_t launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
+                                   float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
+                                   cudaStream_t s, int *launches, int overlap)
 {
     const G *g = reinterpret_cast<const G *>(grads);
+    cudaError_t e = cudaSuccess;
     if (p->n_items_bulk > 0) {
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)p->grid_bulk);
@@ -771,41 +783,47 @@ static void launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *state, co
         const LayerDev *layers = p->d_layers;
         const ItemDev *items = p->d_items;
         const int32_t *cta_begin = p->d_cta_begin_bulk;
-        (void)cudaLaunchKernelEx(&cfg, k1_bulk<G, MOM>, g, resid, vel, mom, keys, layers, items, cta_begin, hist,
-                                 state, ratios, counts, p->d_status, p->alpha, (unsigned int)p->flags,
-                                 overlap);
+        e = cudaLaunchKernelEx(&cfg, k1_bulk<G, MOM>, g, resid, vel, mom, keys, layers, items, cta_begin, hist,
+                               state, ratios, counts, p->d_status, p->alpha, (unsigned int)p->flags, overlap);
+        if (e != cudaSuccess) return e;
         ++*launches;
     }
     if (p->n_items_reg > 0) {
         k1_reg<G, MOM><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
             g, resid, vel, mom, keys, p->d_layers, p->d_items + p->n_items_bulk, p->d_cta_begin_reg, hist,
             state, ratios, counts, p->d_status, p->alpha, p->flags);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
         ++*launches;
     }
+    return e;
 }
 
 // vel == nullptr: plain accumulation v = g + r; otherwise u = mom * u + g, v = r + u.
 // after_sibling / before_sibling: the kernel launched just before / next on this stream is the first
 // pass of another worker of the same call (see k1_bulk); only honoured when a first pass is a
 // single bulk-copy kernel.
-int launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
-                          float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                          cudaStream_t s, bool after_sibling, bool before_sibling)
+// Returns the first error of the kernel configuration or of a launch: the selection kernels must
+// not run on keys no first pass has written.
+cudaError_t launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
+                                  float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
+                                  cudaStream_t s, bool after_sibling, bool before_sibling)
 {
     int overlap = 0;
     if (p->n_items_reg == 0)  // the register-staged kernel is launched without overlap
         overlap = (after_sibling ? kOverlapPrev : 0) | (before_sibling ? kOverlapNext : 0);
     int launches = 0;
-    if (configure_once() != cudaSuccess) return 0;
+    cudaError_t e = configure_once();
+    if (e != cudaSuccess) return e;
     if (p->dtype == RSDGC_BF16) {
-        if (vel) launch_k1_typed<__nv_bfloat16, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
-        else launch_k1_typed<__nv_bfloat16, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
+        if (vel) e = launch_k1_typed<__nv_bfloat16, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
+        else e = launch_k1_typed<__nv_bfloat16, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
     } else {
-        if (vel) launch_k1_typed<float, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
-        else launch_k1_typed<float, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
+        if (vel) e = launch_k1_typed<float, true>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
+        else e = launch_k1_typed<float, false>(p, hist, state, grads, resid, vel, mom, ratios, counts, keys, s, &launches, overlap);
     }
     count_launch(launches);
-    return launches;
+    return e;
 }
 
 }  // namespace rsdgc

@@ -20,12 +20,13 @@
 namespace rsdgc {
 
 constexpr int kMaxWorkersPerLaunch = 16;
-constexpr int kScatterBatch = 8;  // independent entries in flight per thread
+constexpr int kScatterBatch = 9;  // independent entries in flight per thread (one 3x3 tile's worth)
 
 struct WorkerPayloads {
     const int32_t *idx[kMaxWorkersPerLaunch];
     const void *val[kMaxWorkersPerLaunch];  // binary32 or bfloat16 values
     const int32_t *counts[kMaxWorkersPerLaunch];
+    long long idx_cap, val_cap;  // entries every worker's idx / val buffer holds
     int n_workers;
 };
 
@@ -33,6 +34,8 @@ struct DecompressShared {
     long long idx_off[kMaxWorkersPerLaunch];  // payload offsets of the chunk's layer, per worker
     long long val_off[kMaxWorkersPerLaunch];
     int lo[kMaxWorkersPerLaunch], hi[kMaxWorkersPerLaunch];  // the worker's entries inside the chunk
+    long long gbase[kThreads];  // per tile of the current block: arena position of its element (0, 0), or -1
+    int hw[kThreads];           // rows << 16 | columns of the tile inside the layer (clipped)
 };
 
 // First position in a[0, n) whose value is >= key (a ascending); all 32 lanes of the warp take
@@ -122,8 +125,13 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
             si += __shfl_xor_sync(0xFFFFFFFFu, si, d);
             sv += __shfl_xor_sync(0xFFFFFFFFu, sv, d);
         }
-        int k = wp.counts[w][c.layer];
-        if (k < 0) k = 0;
+        long long kk = wp.counts[w][c.layer];
+        if (kk < 0) kk = 0;
+        // a payload cut short by its buffers (RSDGC_STATUS_PAYLOAD_OVERFLOW) holds, of this layer,
+        // only the tiles that fit both of them: the rest was neither written nor sent
+        kk = min(kk, max(0ll, wp.idx_cap - si));
+        kk = min(kk, max(0ll, (wp.val_cap - sv) / layers[c.layer].slot));
+        const int k = (int)kk;
         const int32_t *a = wp.idx[w] + si;
         const int lo = warp_lower_bound(a, k, c.start);
         const int hi = lo + warp_lower_bound(a + lo, k - lo, c.start + c.n);
@@ -136,49 +144,71 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
     }
     __syncthreads();
 
-    const int slot = L.slot;
+    const int slot = L.slot, nw = L.nw;
+    const long long cols = L.cols;
     for (int w = 0; w < W; ++w) {
         const int lo = sh.lo[w];
-        const int n_copy = (sh.hi[w] - lo) * slot;
+        const int n_run = sh.hi[w] - lo;  // the worker's tiles inside this chunk
         const int32_t *idx = wp.idx[w] + sh.idx_off[w] + lo;
         const long long v_first = sh.val_off[w] + (long long)lo * slot;
         const float *val = reinterpret_cast<const float *>(wp.val[w]) + v_first;
         const __nv_bfloat16 *val16 = reinterpret_cast<const __nv_bfloat16 *>(wp.val[w]) + v_first;
-        for (int j0 = 0; j0 < n_copy; j0 += kThreads * kScatterBatch) {
-            long long ga[kScatterBatch];
-            float pv[kScatterBatch], dv[kScatterBatch];
-#pragma unroll
-            for (int u = 0; u < kScatterBatch; ++u) {
-                const int j = j0 + u * kThreads + tid;
-                ga[u] = -1;
-                if (j < n_copy) {
-                    int r, el;
-                    divmod_small(j, slot, &r, &el);
-                    const int tile = __ldg(idx + r);
-                    pv[u] = BF16VAL ? __bfloat162float(val16[j]) : __ldg(val + j);
-                    if (tile >= c.start && tile < c.start + c.n) {  // always true for ascending lists
-                        const int tr = tile / L.TC, tc = tile - tr * L.TC;
-                        int a, b;
-                        divmod_small(el, L.nw, &a, &b);
-                        const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
-                        if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
-                    }
+        // blocks of kThreads tiles: every thread first resolves one tile (index load, tile row / column,
+        // clipping) into shared memory; the value loop then needs one division by the slot size per
+        // value and its loads do not depend on the index list
+        for (int t0 = 0; t0 < n_run; t0 += kThreads) {
+            long long gb = -1;
+            int hw = 0;
+            if (t0 + tid < n_run) {
+                const int tile = __ldg(idx + t0 + tid);
+                if (tile >= c.start && tile < c.start + c.n) {  // always true for ascending lists
+                    const int tr = tile / L.TC, tc = tile - tr * L.TC;
+                    const long long i0 = (long long)tr * L.nh, j0 = (long long)tc * L.nw;
+                    gb = L.elem_off + i0 * cols + j0;
+                    hw = ((int)min((long long)L.nh, L.rows - i0) << 16) | (int)min((long long)L.nw, cols - j0);
                 }
             }
+            sh.gbase[tid] = gb;
+            sh.hw[tid] = hw;
+            __syncthreads();
+            const int n_vals = min(kThreads, n_run - t0) * slot;
+            const long long v0 = (long long)t0 * slot;
+            for (int j0 = 0; j0 < n_vals; j0 += kThreads * kScatterBatch) {
+                long long ga[kScatterBatch];
+                float pv[kScatterBatch], dv[kScatterBatch];
 #pragma unroll
-            for (int u = 0; u < kScatterBatch; ++u) dv[u] = (ga[u] >= 0) ? dense[ga[u]] : 0.0f;
+                for (int u = 0; u < kScatterBatch; ++u) {
+                    const int j = j0 + u * kThreads + tid;
+                    ga[u] = -1;
+                    pv[u] = 0.0f;
+                    if (j < n_vals) {
+                        int q, el, a, b;
+                        divmod_small(j, slot, &q, &el);
+                        divmod_small(el, nw, &a, &b);
+                        const long long g0 = sh.gbase[q];
+                        const int thw = sh.hw[q];
+                        if (g0 >= 0 && a < (thw >> 16) && b < (thw & 0xFFFF)) {
+                            ga[u] = g0 + a * cols + b;
+                            pv[u] = BF16VAL ? __bfloat162float(val16[v0 + j]) : __ldg(val + v0 + j);
+                        }
+                    }
+                }
 #pragma unroll
-            for (int u = 0; u < kScatterBatch; ++u)
-                if (ga[u] >= 0) dense[ga[u]] = __fadd_rn(dv[u], __fmul_rn(scale, pv[u]));
+                for (int u = 0; u < kScatterBatch; ++u) dv[u] = (ga[u] >= 0) ? dense[ga[u]] : 0.0f;
+#pragma unroll
+                for (int u = 0; u < kScatterBatch; ++u)
+                    if (ga[u] >= 0) dense[ga[u]] = __fadd_rn(dv[u], __fmul_rn(scale, pv[u]));
+            }
+            __syncthreads();  // the tables are reused; the next worker may touch the same elements
         }
-        __syncthreads();  // the next worker may touch the same elements
     }
 }
 
 // Applies workers [0, n_workers) in order (after the zero fill of the ASSIGN variant); groups of kMaxWorkersPerLaunch go into one launch
 // each, and the stream orders the groups.
 cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const void *const *val,
-                              const int32_t *const *counts, float scale, float *dense, bool assign, cudaStream_t s)
+                              const int32_t *const *counts, long long idx_cap, long long val_cap, float scale,
+                              float *dense, bool assign, cudaStream_t s)
 {
     const int n_chunks = (int)p->chunks.size();
     const bool half = (p->flags & RSDGC_PAYLOAD_BF16) != 0;
@@ -189,6 +219,8 @@ cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const
     for (int w0 = 0; w0 < n_workers; w0 += kMaxWorkersPerLaunch) {
         WorkerPayloads wp{};
         wp.n_workers = n_workers - w0 < kMaxWorkersPerLaunch ? n_workers - w0 : kMaxWorkersPerLaunch;
+        wp.idx_cap = idx_cap;
+        wp.val_cap = val_cap;
         for (int w = 0; w < wp.n_workers; ++w) {
             wp.idx[w] = idx[w0 + w];
             wp.val[w] = val[w0 + w];

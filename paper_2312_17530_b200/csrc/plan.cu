@@ -602,12 +602,12 @@ extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, voi
 namespace {
 
 int decompress_common(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
-                      const void *const *val_dev_host, const int32_t *const *counts_dev_host, float scale,
-                      float *dense_dev, bool assign, void *stream)
+                      const void *const *val_dev_host, const int32_t *const *counts_dev_host, int64_t idx_capacity,
+                      int64_t val_capacity, float scale, float *dense_dev, bool assign, void *stream)
 {
     int rc = check_plan_device(plan);
     if (rc) return rc;
-    if (n_workers < 0 || !dense_dev) return RSDGC_ERR_INVALID;
+    if (n_workers < 0 || !dense_dev || idx_capacity < 0 || val_capacity < 0) return RSDGC_ERR_INVALID;
     if (n_workers > 0 && (!idx_dev_host || !val_dev_host || !counts_dev_host)) return RSDGC_ERR_INVALID;
     if (!aligned16(dense_dev)) return RSDGC_ERR_ALIGNMENT;
     for (int w = 0; w < n_workers; ++w) {
@@ -618,8 +618,9 @@ int decompress_common(rsdgc_plan *plan, int32_t n_workers, const int32_t *const 
     if (guard.err != cudaSuccess) return cuda_fail(guard.err);
     // every dense element is updated by one CTA, worker after worker: reproducible binary32 sums
     if (n_workers > 0 || assign) {
-        cudaError_t e = launch_decompress(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, scale,
-                                          dense_dev, assign, (cudaStream_t)stream);
+        cudaError_t e = launch_decompress(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host,
+                                          (long long)idx_capacity, (long long)val_capacity, scale, dense_dev, assign,
+                                          (cudaStream_t)stream);
         if (e != cudaSuccess) return cuda_fail(e);
     }
     return RSDGC_OK;
@@ -629,19 +630,20 @@ int decompress_common(rsdgc_plan *plan, int32_t n_workers, const int32_t *const 
 
 extern "C" int rsdgc_decompress_accumulate(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
                                            const void *const *val_dev_host,
-                                           const int32_t *const *counts_dev_host, float scale, float *dense_dev,
-                                           void *stream)
+                                           const int32_t *const *counts_dev_host, int64_t idx_capacity,
+                                           int64_t val_capacity, float scale, float *dense_dev, void *stream)
 {
-    return decompress_common(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, scale, dense_dev, false,
-                             stream);
+    return decompress_common(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, idx_capacity,
+                             val_capacity, scale, dense_dev, false, stream);
 }
 
 extern "C" int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, const int32_t *const *idx_dev_host,
                                        const void *const *val_dev_host, const int32_t *const *counts_dev_host,
-                                       float scale, float *dense_dev, void *stream)
+                                       int64_t idx_capacity, int64_t val_capacity, float scale, float *dense_dev,
+                                       void *stream)
 {
-    return decompress_common(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, scale, dense_dev, true,
-                             stream);
+    return decompress_common(plan, n_workers, idx_dev_host, val_dev_host, counts_dev_host, idx_capacity,
+                             val_capacity, scale, dense_dev, true, stream);
 }
 
 extern "C" int rsdgc_payload_to_coo(rsdgc_plan *plan, const int32_t *idx_dev, const int32_t *counts_dev,

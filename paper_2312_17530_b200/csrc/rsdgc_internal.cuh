@@ -194,15 +194,15 @@ cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *co
 cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long n_keep,
                                  float *ratios, cudaStream_t s);
 cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const *idx, const void *const *val,
-                              const int32_t *const *counts, float scale, float *dense, bool assign,
-                              cudaStream_t s);
+                              const int32_t *const *counts, long long idx_cap, long long val_cap, float scale,
+                              float *dense, bool assign, cudaStream_t s);
 cudaError_t launch_payload_to_coo(rsdgc_plan *p, const int32_t *idx, const int32_t *counts, long long *coo,
                                   long long coo_cap, cudaStream_t s);
 void count_launch(int n);
 void set_last_cuda_error(int e);
 int k1_reg_ctas_per_sm(int dtype, bool momentum);
 int k1_bulk_ctas_per_sm(bool momentum);
-int launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
+cudaError_t launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                           float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
                           cudaStream_t s, bool after_sibling = false, bool before_sibling = false);
 

@@ -131,6 +131,14 @@ def test_payload_overflow_is_reported_and_nothing_is_lost(oracle):
     sent = np.zeros(8100, np.float32)
     oracle.decompress_into(sent, shapes[0], idx[:cap], val[:cap * 9], 1.0)
     assert (sent + res[0] == g[0]).all() and (res[1] == g[1]).all()
+    # the GPU aggregation of the cut-short payload: counts say k0 + k1 tiles, the buffers hold `cap` of
+    # them; the capacities keep it inside the buffers and it adds exactly what was sent
+    d_dense = torch.full((plan.info.arena_elems,), float(parity.CANARY), device="cuda:0")
+    plan.decompress_assign([gc.payload()], d_dense, 1.0)
+    torch.cuda.synchronize()
+    dense = parity.from_arena(plan, d_dense.cpu().numpy())
+    np.testing.assert_array_equal(dense[0], sent)
+    assert (dense[0] + res[0] == g[0]).all() and (dense[1] == 0).all()
 
 
 # ---------------------------------------------------------------------------------------------
