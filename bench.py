@@ -176,11 +176,10 @@ def vgg_inputs(rank: int, n_workers: int = N_WORKERS, only_fc6: bool = False):
 
 
 def run_reference(args):
-    """The CPU oracle as it stands, timed on the host cores.  One step = the oracle's compress of a
-    bounded sample of the workload: one worker's gradient without its largest layer (37 of the 38
-    tensors, 36,994,157 elements, about a second per step on one core), so that the default
-    --steps/--warmup run ends within a few minutes.  The metric (gradient bytes per second) does
-    not depend on the sample's size."""
+    """The CPU oracle as it stands, timed on the host cores, on the benchmark's own configuration.
+    One step = the oracle's compress of ONE of the step's workers: the full VGG-19-shaped gradient,
+    all 38 tensors, 139,754,605 elements, 3 to 4 seconds on one core (the other workers of a step
+    repeat the same work on other values, so the sample is bounded by taking one of them)."""
     from paper_2312_17530_b200 import dist
 
     rank, _, world = dist.env_world()
@@ -190,9 +189,7 @@ def run_reference(args):
 
     oracle.build()
     tensors, shapes, grads, _ = vgg_inputs(0, 1)
-    keep = [i for i, t in enumerate(tensors) if t[0] != "fc6.weight"]
-    shapes = [shapes[i] for i in keep]
-    g = [grads[0][i] for i in keep]
+    g = grads[0]
     n = sum(x.size for x in g)
     res = [np.zeros(x.size, np.float32) for x in g]
     ratios = [KEEP_RATIO] * len(shapes)
@@ -206,8 +203,8 @@ def run_reference(args):
             times.append(dt)
     total = sum(times)
     value = 4.0 * n * len(times) / total / 1e9
-    sample = ("oracle compress of 1 worker's VGG-19-shaped gradient without fc6 (%d tensors, %d elements) per step"
-              % (len(shapes), n))
+    sample = ("oracle compress of 1 of the %d workers of a step: the full VGG-19-shaped gradient (%d tensors, %d "
+              "elements) per step" % (N_WORKERS, len(shapes), n))
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
@@ -355,21 +352,17 @@ def run_b200(args):
     single_ms, single_calls = plan.profile_read()
     plan.profile_enable(0)
 
-    # ---- end to end: host buffers in, payload out, through rsdgc_compress_host()
-    h_idx = torch.zeros(ni, dtype=torch.int32, pin_memory=True)
-    h_val = torch.zeros(nv, dtype=torch.float32, pin_memory=True)
-    h_cnt = torch.zeros(plan.n_layers, dtype=torch.int32, pin_memory=True)
-    d_stage = torch.empty(arena, dtype=torch.float32, device=device)
+    # ---- end to end: host buffers in, payloads out, through rsdgc_compress_workers_host() (two staging
+    # arenas: the next worker's gradient is copied in while the current one is compressed)
+    h_idx = [torch.zeros(ni, dtype=torch.int32, pin_memory=True) for _ in range(N_WORKERS)]
+    h_val = [torch.zeros(nv, dtype=torch.float32, pin_memory=True) for _ in range(N_WORKERS)]
+    h_cnt = [torch.zeros(plan.n_layers, dtype=torch.int32, pin_memory=True) for _ in range(N_WORKERS)]
+    d_stage = [torch.empty(arena, dtype=torch.float32, device=device) for _ in range(2)]
     e2e_steps = 0 if args.no_e2e else max(1, min(args.steps, 5))
-    d2h = 0
+    d2h = N_WORKERS * 4 * (plan.n_layers + ni + nv)   # counts and the whole payload buffers come back
 
     def e2e_step():
-        nonlocal d2h
-        d2h = 0
-        for w in range(N_WORKERS):
-            a, b = plan.compress_host(host_g[w], d_stage, d_r[w], d_ratios, d_idx[w], d_val[w], d_cnt[w], d_ws,
-                                      h_idx, h_val, h_cnt)
-            d2h += 4 * a + 4 * b + 4 * plan.n_layers
+        plan.compress_workers_host(host_g, d_stage, d_r, d_ratios, d_idx, d_val, d_cnt, d_ws, h_idx, h_val, h_cnt)
         plan.decompress_accumulate([(d_idx[w], d_val[w], d_cnt[w]) for w in range(N_WORKERS)], d_dense, 1.0)
 
     e2e_bps = 0.0
@@ -542,9 +535,15 @@ def run_b200(args):
             "e2e": {"value": e2e_bps / 1e9, "unit": UNIT, "h2d_bytes_per_step": int(4 * arena * N_WORKERS),
                     "d2h_bytes_per_step": int(d2h)},
             "gpu_launches": int(launches),
+            # frac: the dominant kernel (the first pass) alone.  compress_step_frac: one worker's whole
+            # compress (first pass, selection, pack, residual update) = 12 B/element / its share of the
+            # step.  step_frac: the same algorithmic bytes over the whole step, aggregation included.
             "roofline": {"bound": "hbm", "kernel": "k1_bulk", "achieved": achieved, "peak": peak,
-                         "unit": "GB/s", "frac": achieved / peak, "traffic": K1_TRAFFIC_BYTES if args.workload == "vgg19" else None,
-                         "peak_source": peak_src, "algorithmic_bytes": alg_bytes, "launch_us": k1_s * 1e6},
+                         "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": k1_traffic_bytes(n) if args.workload == "vgg19" else None,
+                         "peak_source": peak_src, "algorithmic_bytes": alg_bytes, "launch_us": k1_s * 1e6,
+                         "compress_step_frac": alg_bytes / compress_s / 1e9 / peak,
+                         "step_frac": alg_bytes * N_WORKERS / (elapsed_s / args.steps) / 1e9 / peak},
             "extra": extra,
         }
         if args.gpus == 1 and not args.no_cpu_baseline:
@@ -555,17 +554,40 @@ def run_b200(args):
     return 0
 
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one k1_bulk launch on the benchmark workload:
-# 12.03 B/element measured by ncu on the fc6 layer alone (1235.73 MB for 102,760,448 elements,
-# profiles/k1_bulk_fc6_25088x4096.md), scaled to the 139,754,605 elements of one launch here
-# (traffic is proportional to the elements streamed).  Set to None when k1_bulk changes.
-K1_TRAFFIC_BYTES = int(1235.73e6 * 139754605 / 102760448)
+def k1_traffic_bytes(n_elems: int):
+    """dram__bytes_read.sum + dram__bytes_write.sum of one first-pass launch over n_elems elements,
+    from the ncu capture summarised in profiles/k1_bulk_fc6_25088x4096.md (taken on the largest
+    layer alone and scaled by elements: the traffic is proportional to the elements streamed).  The
+    summary records the SHA-256 of the kernel's source files at capture time; when they have
+    changed since, the figure is stale and None is returned."""
+    import re
+
+    path = os.path.join(ROOT, "profiles", "k1_bulk_fc6_25088x4096.md")
+    try:
+        text = open(path).read()
+        per_elem = float(re.search(r"^traffic_bytes_per_element:\s*([0-9.]+)", text, re.M).group(1))
+        want = re.search(r"^kernel_source_sha256:\s*([0-9a-f]{64})", text, re.M).group(1)
+    except (OSError, AttributeError, ValueError):
+        return None
+    return int(per_elem * n_elems) if kernel_source_sha256() == want else None
+
+
+def kernel_source_sha256() -> str:
+    """Hash of the sources the first-pass kernel is compiled from."""
+    import hashlib
+
+    h = hashlib.sha256()
+    for name in ("accumulate_nsi.cu", "device_utils.cuh", "rsdgc_internal.cuh"):
+        with open(os.path.join(ROOT, "paper_2312_17530_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default 100; 10 for --impl reference, whose step takes seconds)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["b200", "reference"], default="b200")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -575,6 +597,8 @@ def main():
     ap.add_argument("--workload", choices=["vgg19", "fc6"], default="vgg19",
                     help="vgg19: the benchmark; fc6: its largest layer alone, for profiler captures")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 100 if args.impl == "b200" else 10
     if args.warmup < 3 and args.impl == "b200":
         args.warmup = 3
     if args.impl == "reference":

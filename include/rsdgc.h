@@ -269,6 +269,29 @@ int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, void *grads_de
                         int64_t *val_used_host, void *stream);
 
 /*
+ * rsdgc_compress_host() for the n_workers workers of a GPU (Sec. III-A: every node compresses its
+ * own gradient), pipelined: staging_dev_host holds TWO caller-owned device arenas of the
+ * gradient's type; worker w + 1's gradient is copied into one (on a stream the plan owns) while
+ * worker w is compressed out of the other on `stream`, and worker w's counts and payload buffers
+ * are copied back right behind its compress.  The payload sizes are not known on the host before
+ * the end, so idx_host[w] / val_host[w] must hold idx_capacity / val_capacity entries and receive
+ * the whole buffers; idx_used_host[w] / val_used_host[w] say how much of them is payload.
+ * grads_host / residual_dev_host / idx_dev_host / val_dev_host / counts_dev_host / idx_host /
+ * val_host / counts_host: HOST arrays of n_workers pointers; workspace_dev: workspace_bytes bytes
+ * (the workers take turns).  Pinned host memory lets the copies overlap the compression.  Waits
+ * for both streams once, at the end; not for use during stream capture.  The first call on a plan
+ * creates the copy stream and events.  Not for plans created with RSDGC_MOMENTUM.
+ * Errors: INVALID, ALIGNMENT, CUDA.
+ */
+int rsdgc_compress_workers_host(rsdgc_plan *plan, int32_t n_workers, const void *const *grads_host,
+                                void *const *staging_dev_host, float *const *residual_dev_host,
+                                const float *ratios_dev, int32_t *const *idx_dev_host, int64_t idx_capacity,
+                                void *const *val_dev_host, int64_t val_capacity,
+                                int32_t *const *counts_dev_host, void *workspace_dev,
+                                int32_t *const *idx_host, void *const *val_host, int32_t *const *counts_host,
+                                int64_t *idx_used_host, int64_t *val_used_host, void *stream);
+
+/*
  * Aggregation of n_workers payloads into a dense gradient on the same device (Eq. 12,
  * third line: sum over workers of sparse(v); Eq. 2 "Sync"):
  *   dense[i] = dense[i] + scale * sent_w[i]   for w = 0 .. n_workers-1 in that order,

@@ -27,7 +27,7 @@ EXPORTS = [
     "rsdgc_compress_host", "rsdgc_decompress_accumulate", "rsdgc_get_status", "rsdgc_launch_count",
     "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
     "rsdgc_update_ratios_noalloc", "rsdgc_compress_momentum", "rsdgc_plan_reserve_workers",
-    "rsdgc_compress_workers", "rsdgc_decompress_assign", "rsdgc_payload_to_coo",
+    "rsdgc_compress_workers", "rsdgc_decompress_assign", "rsdgc_payload_to_coo", "rsdgc_compress_workers_host",
 ]
 NOALLOC_MAX_LAYERS = 64
 N_COMPRESS_KERNELS = 6
@@ -90,6 +90,9 @@ def lib():
                                              C.POINTER(vp), i64, C.POINTER(vp), vp, vp]
         L.rsdgc_compress_host.argtypes = [vp, vp, vp, vp, vp, vp, i64, vp, i64, vp, vp, vp, vp, vp,
                                           C.POINTER(i64), C.POINTER(i64), vp]
+        pp = C.POINTER(vp)
+        L.rsdgc_compress_workers_host.argtypes = [vp, i32, pp, pp, pp, vp, pp, i64, pp, i64, pp, vp, pp, pp, pp,
+                                                  C.POINTER(i64), C.POINTER(i64), vp]
         L.rsdgc_decompress_accumulate.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), i64, i64, f32,
                                                   vp, vp]
         L.rsdgc_decompress_assign.argtypes = [vp, i32, C.POINTER(vp), C.POINTER(vp), C.POINTER(vp), i64, i64, f32, vp,
@@ -226,6 +229,25 @@ class Plan:
                                          _ptr(workspace), _ptr(idx_host), _ptr(val_host), _ptr(counts_host),
                                          C.byref(ni), C.byref(nv), _stream()), "rsdgc_compress_host")
         return ni.value, nv.value
+
+    def compress_workers_host(self, grads_host, staging, residuals, ratios, idx, val, counts, workspace,
+                              idx_host, val_host, counts_host):
+        """rsdgc_compress_workers_host(): per-worker sequences of host gradients / host payload buffers and
+        device residuals / payload buffers, ``staging`` = two device arenas.  Returns the per-worker
+        (idx_used, val_used) lists."""
+        n = len(grads_host)
+        A = C.c_void_p * max(1, n)
+        gh, rd, ia, va, ca, ih, vh, ch = A(), A(), A(), A(), A(), A(), A(), A()
+        for w in range(n):
+            gh[w], rd[w], ca[w] = grads_host[w].data_ptr(), residuals[w].data_ptr(), counts[w].data_ptr()
+            ia[w], va[w] = idx[w].data_ptr(), val[w].data_ptr()
+            ih[w], vh[w], ch[w] = idx_host[w].data_ptr(), val_host[w].data_ptr(), counts_host[w].data_ptr()
+        st = (C.c_void_p * 2)(staging[0].data_ptr(), staging[1].data_ptr())
+        ni, nv = (C.c_int64 * max(1, n))(), (C.c_int64 * max(1, n))()
+        _check(lib().rsdgc_compress_workers_host(
+            self._h, n, gh, st, rd, _ptr(ratios), ia, min(t.numel() for t in idx), va, min(t.numel() for t in val),
+            ca, _ptr(workspace), ih, vh, ch, ni, nv, _stream()), "rsdgc_compress_workers_host")
+        return list(ni)[:n], list(nv)[:n]
 
     def decompress_accumulate(self, payloads, dense, scale: float = 1.0, assign: bool = False) -> None:
         """``payloads``: sequence of (idx, val, counts) device tensors, one per worker.  ``assign``:

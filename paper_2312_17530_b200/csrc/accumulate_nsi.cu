@@ -493,6 +493,7 @@ struct K1BulkShared {
     unsigned int hist[kL1Bins];
     __align__(8) unsigned long long full[kStages];  // mbarriers: stage loaded
     FlushShared fs;
+    int dead_at;  // first item whose loads did not arrive within the bound (see k1_bulk)
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -632,7 +633,12 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
         }
     }
     unsigned int nonfinite = 0;
-    bool timed_out = false;
+    // `dead` (the same value in every thread): a bounded wait gave up.  From then on the CTA moves no
+    // more data: the items it has not finished keep their old accumulator (v is not stored), no further
+    // loads are issued, no keys are written; it still takes part in the layers' histogram tickets so
+    // that the plan's tables are left consistent, and raises RSDGC_STATUS_TIMEOUT (the payload of this
+    // call is then invalid).
+    bool dead = false;
     ItemDev cur = load_item(items, begin);
     // the producer thread keeps the descriptor of the next item to load one iteration ahead
     ItemDev ahead = cur;
@@ -648,59 +654,77 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
         // ---- wait for this item's blocks (bounded), form v in place
         float *sr = sh.r[stage];
         const G *sg = reinterpret_cast<const G *>(sh.g[stage]);
-        if (!mbar_wait_bounded(&sh.full[stage], (uint32_t)((rel / kStages) & 1))) timed_out = true;
-        const int nb = bulk_elems<G>(cur);
-        const int nvec = nb >> 2;
         float *su = sh.u[MOM ? stage : 0];
-        for (int i = tid; i < nvec; i += kBulkThreads) {
-            float4 g = smem_grad4(sg, i);
-            if (MOM) {  // u = m * u + g takes the gradient's place (Eq. 12, first line)
-                g = momentum_step4(mom, reinterpret_cast<const float4 *>(su)[i], g);
-                reinterpret_cast<float4 *>(su)[i] = g;
-            }
-            reinterpret_cast<float4 *>(sr)[i] = add4_rn(g, reinterpret_cast<const float4 *>(sr)[i]);
-        }
-        fence_async_smem();  // the bulk stores below read what the threads just wrote
-        if (cur.flags & kItemFull) k1_tail<G, MOM>(cur, (sizeof(G) == 2) ? 8 : 4, grads, resid, sr, vel, mom);
-        __syncthreads();
-        if (tid == 0) {
-            if (cur.flags & kItemFull) {
-                if (nb > 0) {
-                    bulk_store(resid + cur.gbase, sr, (uint32_t)(nb * sizeof(float)));
-                    if (MOM) bulk_store(vel + cur.gbase, su, (uint32_t)(nb * sizeof(float)));
+        const int nb = bulk_elems<G>(cur);
+        bool arrived = true;
+        if (!dead) {
+            arrived = mbar_wait_bounded(&sh.full[stage], (uint32_t)((rel / kStages) & 1));
+            const int nvec = nb >> 2;
+            for (int i = tid; i < nvec; i += kBulkThreads) {
+                float4 g = smem_grad4(sg, i);
+                if (MOM) {  // u = m * u + g takes the gradient's place (Eq. 12, first line)
+                    g = momentum_step4(mom, reinterpret_cast<const float4 *>(su)[i], g);
+                    reinterpret_cast<float4 *>(su)[i] = g;
                 }
-            } else {
-                for (int row = 0; row < cur.R; ++row) {
-                    const long long gi = cur.gbase + (long long)row * cur.cols;
-                    bulk_store(resid + gi, sr + row * cur.P, (uint32_t)(cur.W * sizeof(float)));
-                    if (MOM) bulk_store(vel + gi, su + row * cur.P, (uint32_t)(cur.W * sizeof(float)));
+                reinterpret_cast<float4 *>(sr)[i] = add4_rn(g, reinterpret_cast<const float4 *>(sr)[i]);
+            }
+            fence_async_smem();  // the bulk stores below read what the threads just wrote
+            // the elements beyond the last 16-byte group of a contiguous item: plain loads and stores of
+            // g and r themselves, so they are right whether or not the bulk copies arrived
+            if (cur.flags & kItemFull) k1_tail<G, MOM>(cur, (sizeof(G) == 2) ? 8 : 4, grads, resid, sr, vel, mom);
+        }
+        // the barrier that orders the threads' writes before the bulk store also tells every thread
+        // whether some thread's wait ran out (nothing of the item has left shared memory yet)
+        if (__syncthreads_or(!arrived)) {
+            if (!dead && tid == 0) sh.dead_at = it;
+            dead = true;
+        }
+        if (!dead) {
+            if (tid == 0) {
+                if (cur.flags & kItemFull) {
+                    if (nb > 0) {
+                        bulk_store(resid + cur.gbase, sr, (uint32_t)(nb * sizeof(float)));
+                        if (MOM) bulk_store(vel + cur.gbase, su, (uint32_t)(nb * sizeof(float)));
+                    }
+                } else {
+                    for (int row = 0; row < cur.R; ++row) {
+                        const long long gi = cur.gbase + (long long)row * cur.cols;
+                        bulk_store(resid + gi, sr + row * cur.P, (uint32_t)(cur.W * sizeof(float)));
+                        if (MOM) bulk_store(vel + gi, su + row * cur.P, (uint32_t)(cur.W * sizeof(float)));
+                    }
+                }
+                bulk_commit();
+                // ---- producer: item it + kLookahead goes into the stage item it - 1 used.  Every
+                // thread finished that item's tiles before the barrier above, and its bulk store
+                // has finished reading shared memory once only the store just committed is pending.
+                if (it + kLookahead < end) {
+                    bulk_wait_read<1>();
+                    const int ps = (rel + kLookahead) % kStages;
+                    bulk_issue_item<G, MOM>(ahead, grads, resid, vel, sh.r[ps], reinterpret_cast<G *>(sh.g[ps]),
+                                            sh.u[MOM ? ps : 0], &sh.full[ps]);
+                    if (it + 1 + kLookahead < end) ahead = load_item(items, it + 1 + kLookahead);
                 }
             }
-            bulk_commit();
-            // ---- producer: item it + kLookahead goes into the stage item it - 1 used.  Every
-            // thread finished that item's tiles before the barrier above, and its bulk store
-            // has finished reading shared memory once only the store just committed is pending.
-            if (it + kLookahead < end) {
-                bulk_wait_read<1>();
-                const int ps = (rel + kLookahead) % kStages;
-                bulk_issue_item<G, MOM>(ahead, grads, resid, vel, sh.r[ps], reinterpret_cast<G *>(sh.g[ps]),
-                                        sh.u[MOM ? ps : 0], &sh.full[ps]);
-                if (it + 1 + kLookahead < end) ahead = load_item(items, it + 1 + kLookahead);
-            }
+            // ---- NSI of every tile of the item
+            nonfinite += item_tile_keys<kBulkThreads>(cur, sr, keys, sh.hist, alpha);
         }
-
-        // ---- NSI of every tile of the item
-        nonfinite += item_tile_keys<kBulkThreads>(cur, sr, keys, sh.hist, alpha);
         if (!has_next || nxt.layer != cur.layer)
             k1_flush_layer<kBulkThreads>(sh.hist, sh.fs, cur.layer, layers, hist, state, ratios, counts, flags);
         cur = nxt;
+    }
+    if (dead && tid == 0) {
+        // the loads already started still target this CTA's shared memory: give them the same bounded
+        // chance to land before the CTA leaves
+        // (when the CTA gave up at item d, items d .. d + kLookahead - 1 had been started)
+        for (int j = sh.dead_at; j < sh.dead_at + kLookahead && j < end; ++j)
+            (void)mbar_wait_bounded(&sh.full[(j - begin) % kStages], (uint32_t)(((j - begin) / kStages) & 1));
     }
     if (tid == 0) bulk_wait_all<0>();  // all stores of this CTA have landed before it exits
     if (nonfinite) {
         atomicAdd(&status->nonfinite, (unsigned long long)nonfinite);
         atomicOr(&status->flags, RSDGC_STATUS_NONFINITE);
     }
-    if (timed_out) atomicOr(&status->flags, RSDGC_STATUS_TIMEOUT);
+    if (dead && tid == 0) atomicOr(&status->flags, RSDGC_STATUS_TIMEOUT);
     if (wait_late) grid_dependency_wait();
 }
 

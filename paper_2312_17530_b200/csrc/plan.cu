@@ -85,6 +85,10 @@ void free_device_tables(rsdgc_plan *p)
     p->extra_lanes.clear();
     for (cudaEvent_t ev : p->events) cudaEventDestroy(ev);
     p->events.clear();
+    for (cudaEvent_t ev : p->order_events) cudaEventDestroy(ev);
+    p->order_events.clear();
+    if (p->copy_stream) cudaStreamDestroy(p->copy_stream);
+    p->copy_stream = nullptr;
 }
 
 }  // namespace
@@ -596,6 +600,90 @@ extern "C" int rsdgc_compress_host(rsdgc_plan *plan, const void *grads_host, voi
     if (e != cudaSuccess) return cuda_fail(e);
     *idx_used_host = ni;
     *val_used_host = nv;
+    return RSDGC_OK;
+}
+
+// The host-buffer path for all the workers of a GPU, pipelined over two staging arenas: while
+// worker w is compressed on the caller's stream, worker w + 1's gradient is already on its way into
+// the other arena on the plan's copy stream, and worker w's payload leaves right behind its
+// compress.  One synchronisation, at the end.
+extern "C" int rsdgc_compress_workers_host(rsdgc_plan *plan, int32_t n_workers, const void *const *grads_host,
+                                           void *const *staging_dev_host, float *const *residual_dev_host,
+                                           const float *ratios_dev, int32_t *const *idx_dev_host,
+                                           int64_t idx_capacity, void *const *val_dev_host, int64_t val_capacity,
+                                           int32_t *const *counts_dev_host, void *workspace_dev,
+                                           int32_t *const *idx_host, void *const *val_host,
+                                           int32_t *const *counts_host, int64_t *idx_used_host,
+                                           int64_t *val_used_host, void *stream)
+{
+    int rc = check_plan_device(plan);
+    if (rc) return rc;
+    if (n_workers < 1 || !grads_host || !staging_dev_host || !residual_dev_host || !idx_dev_host || !val_dev_host ||
+        !counts_dev_host || !idx_host || !val_host || !counts_host || !idx_used_host || !val_used_host)
+        return RSDGC_ERR_INVALID;
+    if (!staging_dev_host[0] || !staging_dev_host[1] || staging_dev_host[0] == staging_dev_host[1])
+        return RSDGC_ERR_INVALID;
+    if (idx_capacity < 0 || val_capacity < 0) return RSDGC_ERR_INVALID;
+    for (int w = 0; w < n_workers; ++w)
+        if (!grads_host[w] || !counts_host[w] || (idx_capacity > 0 && !idx_host[w]) || (val_capacity > 0 && !val_host[w]))
+            return RSDGC_ERR_INVALID;
+    cudaStream_t s = (cudaStream_t)stream;
+    DeviceGuard guard(plan->device);
+    if (guard.err != cudaSuccess) return cuda_fail(guard.err);
+    cudaError_t e = cudaSuccess;
+    if (!plan->copy_stream) e = cudaStreamCreateWithFlags(&plan->copy_stream, cudaStreamNonBlocking);
+    while (e == cudaSuccess && plan->order_events.size() < (size_t)(2 * n_workers + 1)) {
+        cudaEvent_t ev;
+        e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e == cudaSuccess) plan->order_events.push_back(ev);
+    }
+    if (e != cudaSuccess) return cuda_fail(e);
+    cudaEvent_t *copied = plan->order_events.data();                 // [w]: worker w's gradient has arrived
+    cudaEvent_t *consumed = plan->order_events.data() + n_workers;   // [w]: worker w's compress has run
+    cudaEvent_t begin = plan->order_events[2 * (size_t)n_workers];
+    const size_t esz = plan->dtype == RSDGC_BF16 ? 2 : 4, vsz = (plan->flags & RSDGC_PAYLOAD_BF16) ? 2 : 4;
+    const size_t arena_bytes = (size_t)plan->info.arena_elems * esz;
+    // the staging arenas may still be read by work the caller queued before this call
+    e = cudaEventRecord(begin, s);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(plan->copy_stream, begin, 0);
+    for (int w = 0; w < n_workers && e == cudaSuccess; ++w) {
+        void *stage = staging_dev_host[w & 1];
+        if (w >= 2) e = cudaStreamWaitEvent(plan->copy_stream, consumed[w - 2], 0);  // the arena is free again
+        if (e == cudaSuccess) e = cudaMemcpyAsync(stage, grads_host[w], arena_bytes, cudaMemcpyHostToDevice, plan->copy_stream);
+        if (e == cudaSuccess) e = cudaEventRecord(copied[w], plan->copy_stream);
+        if (e == cudaSuccess) e = cudaStreamWaitEvent(s, copied[w], 0);
+        if (e != cudaSuccess) break;
+        rc = rsdgc_compress(plan, stage, residual_dev_host[w], ratios_dev, idx_dev_host[w], idx_capacity,
+                            val_dev_host[w], val_capacity, counts_dev_host[w], nullptr, workspace_dev, stream);
+        if (rc) break;
+        e = cudaEventRecord(consumed[w], s);
+        // the payload sizes are only known on the device: the buffers travel whole (their capacity is
+        // the payload bound, a few tiles per layer above the payload itself)
+        if (e == cudaSuccess)
+            e = cudaMemcpyAsync(counts_host[w], counts_dev_host[w], (size_t)plan->n_layers * sizeof(int32_t),
+                                cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess && idx_capacity > 0)
+            e = cudaMemcpyAsync(idx_host[w], idx_dev_host[w], (size_t)idx_capacity * sizeof(int32_t),
+                                cudaMemcpyDeviceToHost, s);
+        if (e == cudaSuccess && val_capacity > 0)
+            e = cudaMemcpyAsync(val_host[w], val_dev_host[w], (size_t)val_capacity * vsz, cudaMemcpyDeviceToHost, s);
+    }
+    // whatever happened, nothing of this call is left in flight when it returns
+    cudaError_t e2 = cudaStreamSynchronize(plan->copy_stream);
+    cudaError_t e3 = cudaStreamSynchronize(s);
+    if (rc) return rc;
+    if (e == cudaSuccess) e = e2;
+    if (e == cudaSuccess) e = e3;
+    if (e != cudaSuccess) return cuda_fail(e);
+    for (int w = 0; w < n_workers; ++w) {
+        int64_t ni = 0, nv = 0;
+        for (int l = 0; l < plan->n_layers; ++l) {
+            ni += counts_host[w][l];
+            nv += (int64_t)counts_host[w][l] * plan->layers[l].slot;
+        }
+        idx_used_host[w] = ni < idx_capacity ? ni : idx_capacity;
+        val_used_host[w] = nv < val_capacity ? nv : val_capacity;
+    }
     return RSDGC_OK;
 }
 

@@ -172,6 +172,11 @@ struct rsdgc_plan {
     rsdgc::RatioState *d_rstate = nullptr;
     rsdgc::StatusDev *d_status = nullptr;
 
+    // rsdgc_compress_workers_host(): a second stream for the host-to-device copies and the events that
+    // order it against the caller's stream (created on first use)
+    cudaStream_t copy_stream = nullptr;
+    std::vector<cudaEvent_t> order_events;
+
     // optional per-kernel timing of compress calls
     int profile = 0;                  // 0 off, 1 first pass only, 2 every stage
     int profile_recorded = 0;         // level of the calls recorded since the last read

@@ -257,6 +257,45 @@ def test_compress_workers_two_iterations(oracle, n_workers):
         assert int(payloads[w][2].sum()) == sum(r.k for r in refs[w])
 
 
+def test_compress_workers_host_pipelined(oracle):
+    """Host buffers in, host payloads out, three workers over two staging arenas (the third reuses the
+    first worker's arena): every worker's payload and accumulator match the oracle, twice in a row."""
+    shapes = [(300, 515, 3, 3), (256, 64 * 9, 1, 9), (1, 1000, 1, 9), (1200, 1536, 3, 3)]
+    tensors = [("t%d" % i, (s[0], s[1])) for i, s in enumerate(shapes)]
+    plan = binding.Plan(shapes, alpha=0.5)
+    W, dev = 3, "cuda:0"
+    sig = synth.log_uniform_scales(len(shapes), (22,))
+    ratios = np.array([1 / 16, 1 / 50, 0.3, 1 / 64], np.float32)
+    ni, nv = plan.payload_bound(0.3)
+    d_r = [torch.zeros(plan.info.arena_elems, device=dev) for _ in range(W)]
+    d_idx = [torch.full((ni,), -1, dtype=torch.int32, device=dev) for _ in range(W)]
+    d_val = [torch.full((nv,), float(parity.CANARY), device=dev) for _ in range(W)]
+    d_cnt = [torch.zeros(len(shapes), dtype=torch.int32, device=dev) for _ in range(W)]
+    h_idx = [torch.zeros(ni, dtype=torch.int32, pin_memory=True) for _ in range(W)]
+    h_val = [torch.zeros(nv, dtype=torch.float32, pin_memory=True) for _ in range(W)]
+    h_cnt = [torch.zeros(len(shapes), dtype=torch.int32, pin_memory=True) for _ in range(W)]
+    stage = [torch.full((plan.info.arena_elems,), float("nan"), device=dev) for _ in range(2)]
+    ws = torch.empty(plan.info.workspace_bytes, dtype=torch.uint8, device=dev)
+    res = [[np.zeros(s[0] * s[1], np.float32) for s in shapes] for _ in range(W)]
+    for it in range(2):
+        grads = synth.multi_worker_gradients(tensors, W, (22, it), sig)
+        h_g = [torch.from_numpy(parity.to_arena(plan, grads[w])).pin_memory() for w in range(W)]
+        used_i, used_v = plan.compress_workers_host(h_g, stage, d_r, torch.tensor(ratios, device=dev), d_idx, d_val,
+                                                    d_cnt, ws, h_idx, h_val, h_cnt)
+        assert plan.status().flags == 0
+        for w in range(W):
+            ref = oracle.compress(shapes, grads[w], res[w], ratios, 0.5)
+            assert h_cnt[w].numpy().tolist() == ref.counts.tolist()
+            k = int(ref.counts.sum())
+            assert (used_i[w], used_v[w]) == (k, sum(l.val.size for l in ref.layers))
+            np.testing.assert_array_equal(h_idx[w].numpy()[:k], np.concatenate([l.idx for l in ref.layers]))
+            np.testing.assert_array_equal(h_val[w].numpy()[:used_v[w]].view(np.uint32),
+                                          np.concatenate([l.val for l in ref.layers]).view(np.uint32))
+            res[w] = [l.residual for l in ref.layers]
+            for got, want in zip(parity.from_arena(plan, d_r[w].cpu().numpy()), res[w]):
+                np.testing.assert_array_equal(got.view(np.uint32), want.view(np.uint32))
+
+
 def test_compress_workers_argument_errors():
     plan = binding.Plan([(64, 64, 3, 3)], alpha=0.5)
     dev = "cuda:0"
