@@ -114,8 +114,8 @@ typedef struct {
  * RSDGC_PAYLOAD_BF16, or 0.  `device` is the CUDA device ordinal.  On success
  * *out owns host memory and a few MB of device memory until rsdgc_plan_destroy().
  * Errors: INVALID (null, n_layers < 1, rows/cols/nh/nw < 1, alpha outside [0,1] or NaN,
- * unknown dtype), CAPACITY (a layer with more than 2^31-1 tiles or nh*nw > 4096),
- * CUDA / NOMEM.
+ * unknown dtype), CAPACITY (a layer with more than 2^31-1 elements, nh*nw > 4096, or more
+ * than 2048 layers), CUDA / NOMEM.
  */
 int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_layers, int32_t grad_dtype,
                       float alpha, uint32_t flags, int32_t device, rsdgc_plan **out);
@@ -132,17 +132,6 @@ int rsdgc_plan_layer_info(const rsdgc_plan *plan, int32_t layer, rsdgc_layer_inf
 int rsdgc_plan_payload_bound(const rsdgc_plan *plan, float max_ratio, int64_t *idx_capacity_host,
                              int64_t *val_capacity_host);
 
-/* Diagnostic: copies the work list of the accumulate+NSI pass, 9 int32 per item: layer,
- * first tile row, tile rows, first tile col, tile cols (the items of a layer partition its
- * tile grid), the kernel that takes the item (0 = bulk-copy kernel, 1 = register-staged
- * kernel), the CTA of that kernel that owns it, the row pitch (elements) of the item's block in
- * shared memory, and the item's flags (1 = one contiguous run, 2 = 128-bit accesses, 4 = bulk
- * copies, 8 = no clipped tile); grids_host[0..1] receive the two kernels'
- * grid sizes and n_flush_host[l] how many (kernel, CTA) pairs touch layer l.  Any pointer
- * may be NULL.  Returns the number of items (or a negative rsdgc_error).  Host only. */
-int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,
-                            int32_t *grids_host, int32_t *n_flush_host);
-
 /*
  * Layer-wise dynamic compression ratio (Eq. 3-5; Algorithm 1, per-epoch part): importance
  * |w| (Eq. 3), one ranking over all layers of the plan, the ceil(global_keep * G) largest
@@ -151,6 +140,8 @@ int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t
  * the magnitude bits: no sort, three reads of the weights.
  * weights_dev: binary32 arena with the plan's layer offsets (read only).
  * ratios_dev: out, n_layers floats.  global_keep in [0, 1].
+ * The call takes no workspace: its per-layer histograms and counters are among the small device
+ * tables the plan owns.
  * Errors: INVALID, ALIGNMENT, CUDA.
  */
 int rsdgc_update_ratios(rsdgc_plan *plan, const float *weights_dev, float global_keep,
@@ -339,6 +330,29 @@ int rsdgc_decompress_assign(rsdgc_plan *plan, int32_t n_workers, const int32_t *
 int rsdgc_payload_to_coo(rsdgc_plan *plan, const int32_t *idx_dev, const int32_t *counts_dev,
                          int64_t *coo_index_dev, int64_t coo_capacity, void *stream);
 
+/* Waits for the stream, copies the device status word to *out_host and clears it. */
+int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *out_host);
+
+/* Text for an rsdgc_error; the cudaError_t of the last RSDGC_ERR_CUDA of this thread. */
+const char *rsdgc_strerror(int code);
+int rsdgc_last_cuda_error(void);
+
+/* =========================================================================================
+ * Diagnostics.  Nothing below is needed to run the method; these calls exist for tests, timing
+ * breakdowns and the host-logic checks.
+ * ========================================================================================= */
+
+/* Diagnostic: copies the work list of the accumulate+NSI pass, 9 int32 per item: layer,
+ * first tile row, tile rows, first tile col, tile cols (the items of a layer partition its
+ * tile grid), the kernel that takes the item (0 = bulk-copy kernel, 1 = register-staged
+ * kernel), the CTA of that kernel that owns it, the row pitch (elements) of the item's block in
+ * shared memory, and the item's flags (1 = one contiguous run, 2 = 128-bit accesses, 4 = bulk
+ * copies, 8 = no clipped tile); grids_host[0..1] receive the two kernels'
+ * grid sizes and n_flush_host[l] how many (kernel, CTA) pairs touch layer l.  Any pointer
+ * may be NULL.  Returns the number of items (or a negative rsdgc_error).  Host only. */
+int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,
+                            int32_t *grids_host, int32_t *n_flush_host);
+
 /*
  * Optional per-kernel timing of rsdgc_compress().  While enabled, every rsdgc_compress() on
  * this plan records CUDA events on its stream: with level 1 only before and after the first
@@ -355,15 +369,17 @@ int rsdgc_payload_to_coo(rsdgc_plan *plan, const int32_t *idx_dev, const int32_t
 int rsdgc_profile_enable(rsdgc_plan *plan, int32_t level);
 int rsdgc_profile_read(rsdgc_plan *plan, double *ms_per_kernel_host, int64_t *n_calls_host);
 
-/* Waits for the stream, copies the device status word to *out_host and clears it. */
-int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *out_host);
-
 /* Number of kernels this library has launched in this process (all plans). */
 int64_t rsdgc_launch_count(void);
 
-/* Text for an rsdgc_error; the cudaError_t of the last RSDGC_ERR_CUDA of this thread. */
-const char *rsdgc_strerror(int code);
-int rsdgc_last_cuda_error(void);
+/*
+ * Self-test of the bounded on-chip wait the first pass relies on (the paper has no counterpart):
+ * launches one warp that arms a shared-memory barrier for bytes no copy will ever deliver (nothing
+ * is in flight before or after), polls it `polls` times (1 .. 2^20) with the library's bounded
+ * wait, gives up and raises RSDGC_STATUS_TIMEOUT in the plan's status word, which the next
+ * rsdgc_get_status() returns and clears.  The context stays usable.  Errors: INVALID, CUDA.
+ */
+int rsdgc_selftest_bounded_wait(rsdgc_plan *plan, int32_t polls, void *stream);
 
 #ifdef __cplusplus
 }

@@ -28,6 +28,7 @@ EXPORTS = [
     "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
     "rsdgc_update_ratios_noalloc", "rsdgc_compress_momentum", "rsdgc_plan_reserve_workers",
     "rsdgc_compress_workers", "rsdgc_decompress_assign", "rsdgc_payload_to_coo", "rsdgc_compress_workers_host",
+    "rsdgc_selftest_bounded_wait",
 ]
 NOALLOC_MAX_LAYERS = 64
 N_COMPRESS_KERNELS = 6
@@ -102,6 +103,7 @@ def lib():
         L.rsdgc_profile_enable.argtypes = [vp, i32]
         L.rsdgc_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
         L.rsdgc_update_ratios_noalloc.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), i32, f32, vp, vp]
+        L.rsdgc_selftest_bounded_wait.argtypes = [vp, i32, vp]
         L.rsdgc_launch_count.argtypes = []
         L.rsdgc_launch_count.restype = i64
         L.rsdgc_strerror.argtypes = [C.c_int]
@@ -281,6 +283,10 @@ class Plan:
         n = C.c_int64()
         _check(lib().rsdgc_profile_read(self._h, ms, C.byref(n)), "rsdgc_profile_read")
         return list(ms), n.value
+
+    def selftest_bounded_wait(self, polls: int = 256) -> None:
+        """Diagnostic: a bounded on-chip wait that is certain to give up; sets STATUS_TIMEOUT."""
+        _check(lib().rsdgc_selftest_bounded_wait(self._h, int(polls), _stream()), "rsdgc_selftest_bounded_wait")
 
     def status(self) -> Status:
         st = Status()

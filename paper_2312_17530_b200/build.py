@@ -30,6 +30,10 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC,-Wall", "-shared", "-I", os.path.join(_ROOT, "include"), "-I", CSRC,
            "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
+    # NVTX ranges around the entry points (header-only NVTX 3; RSDGC_NVTX=0 compiles them out)
+    if os.environ.get("RSDGC_NVTX", "1") != "0":
+        cmd[1:1] = ["-DRSDGC_NVTX"]
+        cmd += ["-ldl"]
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

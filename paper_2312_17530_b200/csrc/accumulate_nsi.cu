@@ -517,10 +517,11 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long *bar, uint32_t 
         : "memory");
     return ok != 0;
 }
-// Bounded wait; returns false if the barrier did not complete within the limit.
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, uint32_t parity)
+// Bounded wait; returns false if the barrier did not complete within `limit` polls.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long *bar, uint32_t parity,
+                                                  unsigned int limit = kSpinLimit)
 {
-    for (unsigned int i = 0; i < kSpinLimit; ++i)
+    for (unsigned int i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
@@ -726,6 +727,35 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
     }
     if (dead && tid == 0) atomicOr(&status->flags, RSDGC_STATUS_TIMEOUT);
     if (wait_late) grid_dependency_wait();
+}
+
+// ------------------------------------------------------------------------------------------
+// Self-test of the bounded wait: one warp arms a barrier for 16 bytes that no copy will ever
+// deliver (nothing is in flight, before or after), polls it `polls` times with the same helper the
+// first pass uses, and reports the give-up through the status word like the first pass does.
+// ------------------------------------------------------------------------------------------
+
+__global__ void k_selftest_bounded_wait(StatusDev *status, unsigned int polls)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) mbar_arrive_expect_tx(&bar, 16);
+    __syncwarp();
+    const bool arrived = mbar_wait_bounded(&bar, 0, polls);
+    if (__syncthreads_or(!arrived) && threadIdx.x == 0) atomicOr(&status->flags, RSDGC_STATUS_TIMEOUT);
+    __syncthreads();
+    if (threadIdx.x == 0) asm volatile("mbarrier.inval.shared::cta.b64 [%0];" ::"r"(smem_u32(&bar)) : "memory");
+}
+
+cudaError_t launch_selftest_bounded_wait(rsdgc_plan *p, unsigned int polls, cudaStream_t s)
+{
+    k_selftest_bounded_wait<<<1, 32, 0, s>>>(p->d_status, polls);
+    count_launch(1);
+    return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------------------------------

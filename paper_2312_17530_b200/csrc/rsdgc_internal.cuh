@@ -203,6 +203,7 @@ cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const
                               float *dense, bool assign, cudaStream_t s);
 cudaError_t launch_payload_to_coo(rsdgc_plan *p, const int32_t *idx, const int32_t *counts, long long *coo,
                                   long long coo_cap, cudaStream_t s);
+cudaError_t launch_selftest_bounded_wait(rsdgc_plan *p, unsigned int polls, cudaStream_t s);
 void count_launch(int n);
 void set_last_cuda_error(int e);
 int k1_reg_ctas_per_sm(int dtype, bool momentum);

@@ -108,6 +108,26 @@ def test_nonfinite_inputs_are_flagged_and_deterministic(oracle):
     np.testing.assert_array_equal(outs[0][0][:ref0.k], ref0.idx)      # non-finite tiles rank first
 
 
+def test_bounded_wait_gives_up_and_reports_timeout():
+    """The first pass waits for its bulk copies with a bounded poll loop; this runs that loop on a
+    barrier that nothing will ever complete (no copy is issued, so nothing is left in flight), and the
+    give-up must surface as STATUS_TIMEOUT, once, with the context and the plan still usable."""
+    plan = binding.Plan([(64, 64, 3, 3)], alpha=0.5)
+    assert plan.status().flags == 0
+    plan.selftest_bounded_wait(300)
+    st = plan.status()                       # synchronises, returns and clears the status word
+    assert st.flags == binding.STATUS_TIMEOUT
+    assert plan.status().flags == 0
+    with pytest.raises(binding.RsdgcError):
+        plan.selftest_bounded_wait(0)
+    # the same plan still compresses correctly afterwards
+    gc = parity.GpuCompress(plan)
+    g = torch.randn(plan.info.arena_elems, device="cuda:0")
+    r = torch.zeros(plan.info.arena_elems, device="cuda:0")
+    st = gc.run(g, r, torch.tensor([0.1], device="cuda:0"))
+    assert st.flags == 0 and int(gc.counts[0]) == 49
+
+
 def test_payload_overflow_is_reported_and_nothing_is_lost(oracle):
     shapes = [(90, 90, 3, 3), (60, 60, 3, 3)]
     rng = np.random.default_rng(7)
