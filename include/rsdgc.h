@@ -67,6 +67,8 @@ typedef enum {
 #define RSDGC_NO_BULK_COPY 2u      /* first pass: register-staged kernel for every item           */
 #define RSDGC_MOMENTUM 4u          /* the plan is used with rsdgc_compress_momentum() (Eq. 12 l.1) */
 #define RSDGC_PAYLOAD_BF16 8u      /* payload values are bfloat16 instead of binary32 (see below)  */
+#define RSDGC_NO_FUSED_TAIL 16u    /* always the chained selection kernels, also on plans of small  */
+                                   /* layers (which otherwise select and pack in one kernel)        */
 
 /* bits of rsdgc_status.flags */
 #define RSDGC_STATUS_NONFINITE 1u         /* some indicator was NaN/Inf (ranked first as +Inf)  */
@@ -110,8 +112,8 @@ typedef struct {
  * Builds the plan for a set of layers (Algorithm 1's loop over l = 1..L with the
  * neighborhoods of Eq. 7): arena offsets, tile counts, the work lists the kernels walk and
  * the per-layer device tables.  `alpha` is the hyper-parameter of Eq. 8 (0 <= alpha <= 1).
- * `flags`: an OR of RSDGC_KEEP_AT_LEAST_ONE, RSDGC_NO_BULK_COPY, RSDGC_MOMENTUM and
- * RSDGC_PAYLOAD_BF16, or 0.  `device` is the CUDA device ordinal.  On success
+ * `flags`: an OR of RSDGC_KEEP_AT_LEAST_ONE, RSDGC_NO_BULK_COPY, RSDGC_MOMENTUM,
+ * RSDGC_PAYLOAD_BF16 and RSDGC_NO_FUSED_TAIL, or 0.  `device` is the CUDA device ordinal.  On success
  * *out owns host memory and a few MB of device memory until rsdgc_plan_destroy().
  * Errors: INVALID (null, n_layers < 1, rows/cols/nh/nw < 1, alpha outside [0,1] or NaN,
  * unknown dtype), CAPACITY (a layer with more than 2^31-1 elements, nh*nw > 4096, or more
@@ -353,12 +355,24 @@ int rsdgc_last_cuda_error(void);
 int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_host, int64_t items_capacity,
                             int32_t *grids_host, int32_t *n_flush_host);
 
+/* Diagnostic: plans whose layers all have at most 262144 tiles select and pack in one kernel per
+ * layer-size class instead of the chained selection kernels (unless RSDGC_NO_FUSED_TAIL is set or the
+ * layers need more thread-block clusters than the device holds at a time).  Copies that kernel's
+ * work list, 6 int32 per CTA: layer, first tile, tiles (0: a cluster rank without work), CTAs that
+ * share the layer, this CTA's rank among them, cluster rank of the first of them; the cluster
+ * variant's CTAs first (8 per cluster), then the one-CTA layers.  info_host[0..2] receive the two
+ * counts and the number of clusters.  Returns the number of CTAs (0: the plan takes the chained
+ * kernels) or a negative rsdgc_error.  Host only. */
+int64_t rsdgc_plan_tail_slices(const rsdgc_plan *plan, int32_t *slices_host, int64_t capacity,
+                               int32_t *info_host);
+
 /*
  * Optional per-kernel timing of rsdgc_compress().  While enabled, every rsdgc_compress() on
  * this plan records CUDA events on its stream: with level 1 only before and after the first
  * pass (accumulate+NSI, the kernel that moves all the bytes), with level 2 after each of the
  * RSDGC_N_COMPRESS_KERNELS stages as well (accumulate+NSI, refine level 2, refine level 3,
- * count, mark, gather).  Events between kernels cost about 3 us each, so level 2 is for
+ * count, mark, gather; on plans that select and pack in one kernel per layer-size class: accumulate+NSI,
+ * the cluster kernel, the one-CTA kernel, and three empty stages).  Events between kernels cost about 3 us each, so level 2 is for
  * breakdowns, not for throughput numbers.  rsdgc_profile_read() waits for the recorded events,
  * adds the elapsed milliseconds of every timed stage over all recorded calls into
  * ms_per_kernel_host[RSDGC_N_COMPRESS_KERNELS] (untimed stages stay 0), stores the number of

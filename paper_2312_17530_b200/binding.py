@@ -18,6 +18,7 @@ KEEP_AT_LEAST_ONE = 1
 NO_BULK_COPY = 2
 MOMENTUM = 4
 PAYLOAD_BF16 = 8
+NO_FUSED_TAIL = 16
 STATUS_NONFINITE, STATUS_PAYLOAD_OVERFLOW, STATUS_TIMEOUT = 1, 2, 4
 OK, ERR_INVALID, ERR_ALIGNMENT, ERR_CAPACITY, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
 
@@ -28,7 +29,7 @@ EXPORTS = [
     "rsdgc_strerror", "rsdgc_last_cuda_error", "rsdgc_profile_enable", "rsdgc_profile_read",
     "rsdgc_update_ratios_noalloc", "rsdgc_compress_momentum", "rsdgc_plan_reserve_workers",
     "rsdgc_compress_workers", "rsdgc_decompress_assign", "rsdgc_payload_to_coo", "rsdgc_compress_workers_host",
-    "rsdgc_selftest_bounded_wait",
+    "rsdgc_selftest_bounded_wait", "rsdgc_plan_tail_slices",
 ]
 NOALLOC_MAX_LAYERS = 64
 N_COMPRESS_KERNELS = 6
@@ -104,6 +105,8 @@ def lib():
         L.rsdgc_profile_read.argtypes = [vp, C.POINTER(C.c_double), C.POINTER(i64)]
         L.rsdgc_update_ratios_noalloc.argtypes = [vp, C.POINTER(i64), C.POINTER(i64), i32, f32, vp, vp]
         L.rsdgc_selftest_bounded_wait.argtypes = [vp, i32, vp]
+        L.rsdgc_plan_tail_slices.argtypes = [vp, vp, i64, vp]
+        L.rsdgc_plan_tail_slices.restype = i64
         L.rsdgc_launch_count.argtypes = []
         L.rsdgc_launch_count.restype = i64
         L.rsdgc_strerror.argtypes = [C.c_int]
@@ -189,6 +192,18 @@ class Plan:
         nf = np.zeros(self.n_layers, dtype=np.int32)
         lib().rsdgc_plan_worklist(self._h, items.ctypes.data, n, grids.ctypes.data, nf.ctypes.data)
         return items, grids, nf
+
+    def tail_slices(self):
+        """(slices [n,6] int32: layer, first tile, tiles, CTAs of the layer, rank, leader rank; info [3]:
+        cluster-variant CTAs, one-CTA layers, clusters) of the single-kernel selection + pack; n = 0 when
+        the plan takes the chained kernels."""
+        import numpy as np
+
+        n = lib().rsdgc_plan_tail_slices(self._h, None, 0, None)
+        sl = np.zeros((max(n, 0), 6), dtype=np.int32)
+        info = np.zeros(3, dtype=np.int32)
+        lib().rsdgc_plan_tail_slices(self._h, sl.ctypes.data, n, info.ctypes.data)
+        return sl, info
 
     # ---- device calls (torch tensors on the plan's device) -------------------------------
     def update_ratios(self, weights, global_keep: float, ratios) -> None:

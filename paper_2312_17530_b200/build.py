@@ -9,7 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "librsdgc_b200.so")
-SOURCES = ["plan.cu", "accumulate_nsi.cu", "compress.cu", "ratio.cu", "decompress.cu", "ratio_noalloc.cu", "coo.cu"]
+SOURCES = ["plan.cu", "accumulate_nsi.cu", "compress.cu", "ratio.cu", "decompress.cu", "ratio_noalloc.cu", "coo.cu", "tail.cu"]
 HEADERS = ["rsdgc_internal.cuh", "device_utils.cuh"]
 
 

@@ -20,6 +20,9 @@
 
 namespace rsdgc {
 
+constexpr int kNoHistogram = 4;  // launch mode bit of both kernels: keys only, no level-1 histogram (the kernel
+                                 // that follows selects from the keys alone)
+
 // ------------------------------------------------------------------------------------------
 // NSI of one tile
 // ------------------------------------------------------------------------------------------
@@ -86,7 +89,7 @@ __device__ __forceinline__ void emit_key(float nsi, uint32_t *dst, unsigned int 
         ++nonfinite;
     }
     *dst = key;
-    atomicAdd(&hist_smem[key >> kL1Shift], 1u);
+    if (hist_smem) atomicAdd(&hist_smem[key >> kL1Shift], 1u);
 }
 
 // Keys of all tiles of one item from its v block in shared memory (row pitch d.P).
@@ -423,9 +426,11 @@ __global__ void __launch_bounds__(kThreads)
 k1_reg(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict__ vel, float mom,
        uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
        const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
-       const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags)
+       const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags,
+       int mode)
 {
     extern __shared__ __align__(16) unsigned char k1_smem_raw[];
+    const bool with_hist = (mode & kNoHistogram) == 0;
     K1RegShared &sh = *reinterpret_cast<K1RegShared *>(k1_smem_raw);
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     if (begin >= end) return;
@@ -451,8 +456,8 @@ k1_reg(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict
         // the next item's g and r stream in while this item's tiles are reduced
         if (has_next) k1_issue_loads<G, MOM>(nxt, grads, resid, vel, x, map);
         __syncthreads();
-        nonfinite += item_tile_keys<kThreads>(cur, sv, keys, sh.hist, alpha);
-        if (!has_next || nxt.layer != cur.layer)
+        nonfinite += item_tile_keys<kThreads>(cur, sv, keys, with_hist ? sh.hist : nullptr, alpha);
+        if (with_hist && (!has_next || nxt.layer != cur.layer))
             k1_flush_layer<kThreads>(sh.hist, sh.fs, cur.layer, layers, hist, state, ratios, counts, flags);
         cur = nxt;
         buf ^= 1;
@@ -602,6 +607,7 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
     K1BulkShared<MOM> &sh = *reinterpret_cast<K1BulkShared<MOM> *>(k1_bulk_smem_raw);
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     const bool wait_late = (overlap & kOverlapPrev) != 0;
+    const bool with_hist = (overlap & kNoHistogram) == 0;
     if (begin >= end) {
         if (wait_late) grid_dependency_wait();
         return;
@@ -707,9 +713,9 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
                 }
             }
             // ---- NSI of every tile of the item
-            nonfinite += item_tile_keys<kBulkThreads>(cur, sr, keys, sh.hist, alpha);
+            nonfinite += item_tile_keys<kBulkThreads>(cur, sr, keys, with_hist ? sh.hist : nullptr, alpha);
         }
-        if (!has_next || nxt.layer != cur.layer)
+        if (with_hist && (!has_next || nxt.layer != cur.layer))
             k1_flush_layer<kBulkThreads>(sh.hist, sh.fs, cur.layer, layers, hist, state, ratios, counts, flags);
         cur = nxt;
     }
@@ -845,7 +851,7 @@ static cudaError_t launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *st
     if (p->n_items_reg > 0) {
         k1_reg<G, MOM><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
             g, resid, vel, mom, keys, p->d_layers, p->d_items + p->n_items_bulk, p->d_cta_begin_reg, hist,
-            state, ratios, counts, p->d_status, p->alpha, p->flags);
+            state, ratios, counts, p->d_status, p->alpha, p->flags, overlap & kNoHistogram);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         ++*launches;
@@ -861,11 +867,12 @@ static cudaError_t launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *st
 // not run on keys no first pass has written.
 cudaError_t launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                                   float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                                  cudaStream_t s, bool after_sibling, bool before_sibling)
+                                  cudaStream_t s, bool after_sibling, bool before_sibling, bool no_histogram)
 {
     int overlap = 0;
     if (p->n_items_reg == 0)  // the register-staged kernel is launched without overlap
         overlap = (after_sibling ? kOverlapPrev : 0) | (before_sibling ? kOverlapNext : 0);
+    if (no_histogram) overlap |= kNoHistogram;
     int launches = 0;
     cudaError_t e = configure_once();
     if (e != cudaSuccess) return e;

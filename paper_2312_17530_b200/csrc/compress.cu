@@ -374,28 +374,25 @@ k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
 }
 
 // ------------------------------------------------------------------------------------------
-// K6: gather.  Payload tile s of the whole call (0 <= s < sum of k_l) belongs to the layer l with
-// idx_off_l <= s < idx_off_l + k_l; its values are the nh x nw elements of tile idx[s] of that
-// layer and go to val[val_off_l + (s - idx_off_l) * slot_l ...].  The values are moved from the
-// residual to val and the residual entries become +0 (Eq. 12: what is sent leaves the accumulator);
-// with 16-bit payload values q = bfloat16(v) is sent and v - q stays.
+// K6: gather.  Payload value j of the whole call belongs to layer l (val_off_l <= j <
+// val_off_l + k_l * slot_l), payload slot s = (j - val_off_l) / slot_l, element el of the tile
+// idx[idx_off_l + s].  The value is moved from the residual to val and the residual entry
+// becomes +0 (Eq. 12: what is sent leaves the accumulator); with 16-bit payload values
+// q = bfloat16(v) is sent and v - q stays.  Grid-stride over blocks of consecutive payload values
+// (so the work is even whatever the spatial pattern of the kept tiles, and the payload stores are
+// contiguous) with kCopyBatch independent entries in flight per thread.
 //
-// A CTA takes blocks of kGatherTiles consecutive payload tiles (grid-stride, so the work is even
-// whatever the spatial pattern of the kept tiles, and the payload stores are contiguous).  Per
-// block, every thread first resolves ONE tile (layer search, index load, tile row / column, clipping)
-// and leaves its first element's position in shared memory; the value loop that follows then needs
-// per value only a division by the slot size and one shared-memory read, and all its loads are
-// independent of each other and of the index list.
+// "Read v, leave +0" is ONE atomic exchange per element, executed where the line lives (L2): a
+// plain load followed by a store of 0 to the same sector is 3x slower on this memory system (the
+// store meets the sector while its fill is still in flight) and fetches twice the bytes from DRAM
+// (127 against 84 bytes per 12-byte row segment of a 3x3 tile).  No two threads touch the same
+// element, so the exchange is only a fused read-and-clear, not a synchronisation.
 // ------------------------------------------------------------------------------------------
 
-constexpr int kGatherTiles = kThreads;  // payload tiles per block: one per thread in the resolve phase
-constexpr int kGatherBatch = 9;         // independent values in flight per thread (one 3x3 tile's worth)
-
-struct GatherShared {
-    long long gbase[kGatherTiles];  // arena position of element (0, 0) of the tile, or -1: not sent
-    int hw[kGatherTiles];           // rows << 16 | columns of the tile inside the layer (clipped)
-    int block_layers[2];            // layers of the block's first and last tile
-};
+#ifndef RSDGC_COPY_BATCH
+#define RSDGC_COPY_BATCH 4
+#endif
+constexpr int kCopyBatch = RSDGC_COPY_BATCH;
 
 template <bool BF16VAL>
 __global__ void __launch_bounds__(kThreads)
@@ -403,9 +400,8 @@ k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *_
          long long idx_cap, long long val_cap)
 {
     extern __shared__ __align__(16) unsigned char gather_smem_raw[];
-    long long *val_off = reinterpret_cast<long long *>(gather_smem_raw);  // n_layers
-    long long *idx_off = val_off + n_layers;                              // n_layers + 1
-    __shared__ GatherShared sh;
+    long long *val_off = reinterpret_cast<long long *>(gather_smem_raw);  // n_layers + 1
+    long long *idx_off = val_off + n_layers + 1;                          // n_layers
     const int tid = threadIdx.x;
     grid_dependency_wait();
     // the workers one after the other: the scattered accesses of the CTAs that run at the same
@@ -424,107 +420,86 @@ k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *_
         }
         if (tid == 0) {
             const LayerState &last = state[n_layers - 1];
-            idx_off[n_layers] = last.idx_off + (long long)last.k;
+            val_off[n_layers] = last.val_off + (long long)last.k * layers[n_layers - 1].slot;
         }
         __syncthreads();
-        const long long total = idx_off[n_layers];  // payload tiles of this worker
-        auto find_layer = [&](long long s) {
-            int lo = 0, hi = n_layers;  // last layer with idx_off[lo] <= s (layers that keep nothing are skipped)
+        const long long total = val_off[n_layers];
+        // a CTA takes blocks of kThreads * kCopyBatch consecutive payload values: almost always one
+        // layer per block, so the layer search is done once per block, not once per value
+        constexpr long long kBlock = (long long)kThreads * kCopyBatch;
+        auto find_layer = [&](long long j) {
+            int lo = 0, hi = n_layers;  // layer with val_off[lo] <= j < val_off[lo + 1]
             while (hi - lo > 1) {
                 const int mid = (lo + hi) >> 1;
-                if (idx_off[mid] <= s) lo = mid; else hi = mid;
+                if (val_off[mid] <= j) lo = mid; else hi = mid;
             }
             return lo;
         };
-        for (long long tb = (long long)blockIdx.x * kGatherTiles; tb < total; tb += (long long)gridDim.x * kGatherTiles) {
-            // ---- resolve: one payload tile per thread
-            const long long s = tb + tid;
-            long long gb = -1;
-            int hw = 0, my_layer = -1;
-            if (s < total) {
-                my_layer = find_layer(s);
-                const LayerDev &L = layers[my_layer];
-                const long long sl = s - idx_off[my_layer];
-                // tiles that do not fit the payload buffers are not sent and stay in the residual
-                if (s < idx_cap && val_off[my_layer] + (sl + 1) * L.slot <= val_cap) {
-                    const int tile = __ldg(idx + s);
-                    const int tr = tile / L.TC, tc = tile - tr * L.TC;
-                    const long long i0 = (long long)tr * L.nh, j0 = (long long)tc * L.nw;
-                    gb = L.elem_off + i0 * L.cols + j0;
-                    hw = ((int)min((long long)L.nh, L.rows - i0) << 16) | (int)min((long long)L.nw, L.cols - j0);
-                }
-            }
-            sh.gbase[tid] = gb;
-            sh.hw[tid] = hw;
-            if (tid == 0) sh.block_layers[0] = my_layer;
-            if (s == min(total, tb + kGatherTiles) - 1) sh.block_layers[1] = my_layer;
-            __syncthreads();
-            const int n_tiles = (int)min((long long)kGatherTiles, total - tb);
-            if (sh.block_layers[0] == sh.block_layers[1]) {
-                // ---- the usual case, one layer per block: value j of the block is element el = j % slot
-                // of its tile q = j / slot, at payload position vbase + j
-                const LayerDev &L = layers[sh.block_layers[0]];
-                const int slot = L.slot, nw = L.nw;
-                const long long cols = L.cols;
-                const long long vbase = val_off[sh.block_layers[0]] + (tb - idx_off[sh.block_layers[0]]) * slot;
-                const int n_vals = n_tiles * slot;
-                for (int j0 = 0; j0 < n_vals; j0 += kThreads * kGatherBatch) {
-                    long long ga[kGatherBatch];
-                    float xv[kGatherBatch];
-                    bool sent[kGatherBatch];
+        for (long long jb = (long long)blockIdx.x * kBlock; jb < total; jb += (long long)gridDim.x * kBlock) {
+            const long long jend = min(total, jb + kBlock) - 1;
+            const int l_first = find_layer(jb);
+            const bool one_layer = val_off[l_first + 1] > jend;
+            long long ga[kCopyBatch], vo[kCopyBatch];
+            int tile[kCopyBatch], lay[kCopyBatch], el[kCopyBatch];
+            float xv[kCopyBatch];
 #pragma unroll
-                    for (int u = 0; u < kGatherBatch; ++u) {
-                        const int j = j0 + u * kThreads + tid;
-                        ga[u] = -1;
-                        sent[u] = false;
-                        if (j < n_vals) {
-                            int q, el, a, b;
-                            divmod_small(j, slot, &q, &el);
-                            divmod_small(el, nw, &a, &b);
-                            const long long g0 = sh.gbase[q];
-                            const int thw = sh.hw[q];
-                            sent[u] = g0 >= 0;
-                            if (g0 >= 0 && a < (thw >> 16) && b < (thw & 0xFFFF)) ga[u] = g0 + a * cols + b;
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < kGatherBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
-#pragma unroll
-                    for (int u = 0; u < kGatherBatch; ++u) {
-                        const long long vo = vbase + j0 + u * kThreads + tid;
-                        if (BF16VAL) {  // q = bfloat16(v) is sent, v - q stays (exact in binary32)
-                            const __nv_bfloat16 q = __float2bfloat16_rn(xv[u]);
-                            if (ga[u] >= 0) resid[ga[u]] = __fsub_rn(xv[u], __bfloat162float(q));
-                            if (sent[u]) val16[vo] = q;
-                        } else {
-                            if (ga[u] >= 0) resid[ga[u]] = 0.0f;
-                            if (sent[u]) val[vo] = xv[u];
-                        }
-                    }
-                }
-            } else if (gb >= 0) {
-                // ---- a block that spans a layer boundary (at most one per layer): every thread moves its
-                // own tile
-                const LayerDev &L = layers[my_layer];
-                const long long vo0 = val_off[my_layer] + (s - idx_off[my_layer]) * L.slot;
-                for (int el = 0; el < L.slot; ++el) {
-                    int a, b;
-                    divmod_small(el, L.nw, &a, &b);
-                    float x = 0.0f;
-                    const bool inside = a < (hw >> 16) && b < (hw & 0xFFFF);
-                    const long long g1 = gb + a * L.cols + b;
-                    if (inside) x = resid[g1];
-                    if (BF16VAL) {
-                        const __nv_bfloat16 q = __float2bfloat16_rn(x);
-                        if (inside) resid[g1] = __fsub_rn(x, __bfloat162float(q));
-                        val16[vo0 + el] = q;
+            for (int u = 0; u < kCopyBatch; ++u) {
+                const long long j = jb + u * kThreads + tid;
+                ga[u] = -1;
+                vo[u] = -1;
+                tile[u] = -1;
+                if (j < total) {
+                    const int lo = one_layer ? l_first : find_layer(j);
+                    const int slot = layers[lo].slot;
+                    const long long jl = j - val_off[lo];
+                    // 32-bit division whenever the layer's payload is below 2^31 values (the usual case)
+                    long long s;
+                    if (jl < 0x7FFFFFFFll) {
+                        int q, r;
+                        divmod_small((int)jl, slot, &q, &r);
+                        s = q;
+                        el[u] = r;
                     } else {
-                        if (inside) resid[g1] = 0.0f;
-                        val[vo0 + el] = x;
+                        s = jl / slot;
+                        el[u] = (int)(jl - s * slot);
+                    }
+                    lay[u] = lo;
+                    // tiles that do not fit the payload buffers are not sent and stay in the residual
+                    if (idx_off[lo] + s < idx_cap && val_off[lo] + (s + 1) * slot <= val_cap) {
+                        tile[u] = __ldg(idx + idx_off[lo] + s);
+                        vo[u] = j;
                     }
                 }
             }
-            __syncthreads();  // the block's tables are reused
+#pragma unroll
+            for (int u = 0; u < kCopyBatch; ++u) {
+                if (tile[u] >= 0) {
+                    const LayerDev &L = layers[lay[u]];
+                    const int tr = tile[u] / L.TC, tc = tile[u] - tr * L.TC;
+                    int a, b;
+                    divmod_small(el[u], L.nw, &a, &b);
+                    const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
+                    if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+                }
+            }
+            if (BF16VAL) {  // q = bfloat16(v) is sent, v - q stays (exact in binary32)
+#pragma unroll
+                for (int u = 0; u < kCopyBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
+#pragma unroll
+                for (int u = 0; u < kCopyBatch; ++u) {
+                    const __nv_bfloat16 q = __float2bfloat16_rn(xv[u]);
+                    if (ga[u] >= 0) resid[ga[u]] = __fsub_rn(xv[u], __bfloat162float(q));
+                    if (vo[u] >= 0) val16[vo[u]] = q;
+                }
+            } else {
+#pragma unroll
+                for (int u = 0; u < kCopyBatch; ++u)
+                    xv[u] = (ga[u] >= 0) ? __uint_as_float(atomicExch(reinterpret_cast<unsigned int *>(resid) + ga[u], 0u))
+                                         : 0.0f;
+#pragma unroll
+                for (int u = 0; u < kCopyBatch; ++u)
+                    if (vo[u] >= 0) val[vo[u]] = xv[u];
+            }
         }
     }
 }
@@ -604,6 +579,24 @@ static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n
     return e;
 }
 
+// Plans whose layers all fit the single-kernel tail take it when the call's clusters (one set per
+// worker) can all be resident at once; otherwise the chained kernels.
+static bool use_fused_tail(const rsdgc_plan *p, int n_lanes)
+{
+    if (p->n_tail_big + p->n_tail_small == 0) return false;
+    return (long long)p->n_tail_clusters * n_lanes <= p->tail_max_clusters;
+}
+
+// The single-kernel tail in the event layout of the chained path: stage 1 = the cluster kernel,
+// stage 2 = the one-CTA kernel, stages 3..5 empty.
+static cudaError_t launch_fused_tail(rsdgc_plan *p, const LaneTable &lanes, int n_lanes, const float *ratios,
+                                     int64_t idx_cap, int64_t val_cap, int prof, cudaStream_t s)
+{
+    cudaError_t e = launch_tail(p, lanes, n_lanes, ratios, (long long)idx_cap, (long long)val_cap, prof, s, record_event);
+    for (int k = 0; k < 3 && prof >= 2 && e == cudaSuccess; ++k) e = record_event(p, s);
+    return e;
+}
+
 cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, float *vel, float mom,
                             const float *ratios, int32_t *idx, int64_t idx_cap, void *val, int64_t val_cap,
                             int32_t *counts, uint32_t *keys, cudaStream_t s)
@@ -612,12 +605,16 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, floa
     cudaError_t e = cudaSuccess;
     if (prof) p->profile_recorded = prof;
     if (prof >= 1) e = record_event(p, s);
+    const bool fused = use_fused_tail(p, 1);
     if (e == cudaSuccess)
-        e = launch_accumulate_nsi(p, p->d_hist, p->d_state, grads, resid, vel, mom, ratios, counts, keys, s);
+        e = launch_accumulate_nsi(p, p->d_hist, p->d_state, grads, resid, vel, mom, ratios, counts, keys, s, false,
+                                  false, fused);
     if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
     LaneTable lanes{};
-    lanes.l[0] = Lane{keys, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid, idx, val};
-    if (e == cudaSuccess) e = launch_selection(p, lanes, 1, idx_cap, val_cap, prof, s);
+    lanes.l[0] = Lane{keys, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid, idx, val, counts};
+    if (e == cudaSuccess)
+        e = fused ? launch_fused_tail(p, lanes, 1, ratios, idx_cap, val_cap, prof, s)
+                  : launch_selection(p, lanes, 1, idx_cap, val_cap, prof, s);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
@@ -637,24 +634,27 @@ cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *co
     cudaError_t e = cudaSuccess;
     for (int w0 = 0; w0 < n_workers && e == cudaSuccess; w0 += kMaxLanes) {
         const int n = n_workers - w0 < kMaxLanes ? n_workers - w0 : kMaxLanes;
+        const bool fused = use_fused_tail(p, n);
         LaneTable lanes{};
         if (prof >= 1) e = record_event(p, s);
         for (int j = 0; j < n && e == cudaSuccess; ++j) {
             const int w = w0 + j;
             Lane &ln = lanes.l[j];
             if (w == 0) {
-                ln = Lane{keys_all, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid[0], idx[0], val[0]};
+                ln = Lane{keys_all, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid[0], idx[0], val[0], counts[0]};
             } else {
                 const rsdgc_plan::LaneScratch &x = p->extra_lanes[(size_t)w - 1];
                 ln = Lane{keys_all + (size_t)w * key_stride, x.hist, x.state, x.chunk_cnt, x.codes, resid[w], idx[w],
-                          val[w]};
+                          val[w], counts[w]};
             }
             // the first passes of a group's workers share nothing: all but the first start without waiting
             e = launch_accumulate_nsi(p, ln.hist, ln.state, grads[w], ln.resid, nullptr, 0.0f, ratios, counts[w],
-                                      ln.keys, s, j > 0, j + 1 < n);
+                                      ln.keys, s, j > 0, j + 1 < n, fused);
         }
         if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
-        if (e == cudaSuccess) e = launch_selection(p, lanes, n, idx_cap, val_cap, prof, s);
+        if (e == cudaSuccess)
+            e = fused ? launch_fused_tail(p, lanes, n, ratios, idx_cap, val_cap, prof, s)
+                      : launch_selection(p, lanes, n, idx_cap, val_cap, prof, s);
     }
     if (e != cudaSuccess) return e;
     return cudaGetLastError();

@@ -1,4 +1,5 @@
 // Host side of the RS-DGC library: plan tables, argument checks, the C entry points.
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdlib>
@@ -83,6 +84,7 @@ void free_device_tables(rsdgc_plan *p)
     cudaFree(p->d_cta_begin_bulk);
     cudaFree(p->d_cta_begin_reg);
     cudaFree(p->d_chunks);
+    cudaFree(p->d_tail_slices);
     cudaFree(p->d_echunks);
     cudaFree(p->d_state);
     cudaFree(p->d_hist);
@@ -279,6 +281,62 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
         while (next_cta <= (size_t)G) cta_begin[next_cta++] = (int32_t)mine.size();
     }
 
+    // --- single-kernel tail (tail.cu): possible when every layer's keys fit one cluster's shared memory
+    p->tail_slices.clear();
+    p->n_tail_big = p->n_tail_small = p->n_tail_clusters = 0;
+    bool tail_ok = !(p->flags & RSDGC_NO_FUSED_TAIL);
+    for (const LayerDev &L : p->layers)
+        if ((int64_t)L.K > (int64_t)kTailCluster * kTailKeysBig) tail_ok = false;
+    if (tail_ok) {
+        // layers above the one-CTA size: m slices each, all in one cluster; first fit, largest first
+        struct Big {
+            int layer, m;
+        };
+        std::vector<Big> big;
+        for (int l = 0; l < n_layers; ++l)
+            if (p->layers[l].K > kTailKeysSmall)
+                big.push_back(Big{l, (int)ceil_div64(p->layers[l].K, kTailKeysBig)});
+        std::stable_sort(big.begin(), big.end(), [](const Big &a, const Big &b) { return a.m > b.m; });
+        std::vector<std::vector<Big>> clusters;
+        std::vector<int> used;
+        for (const Big &b : big) {
+            size_t c = 0;
+            while (c < clusters.size() && used[c] + b.m > kTailCluster) ++c;
+            if (c == clusters.size()) {
+                clusters.emplace_back();
+                used.push_back(0);
+            }
+            clusters[c].push_back(b);
+            used[c] += b.m;
+        }
+        for (const std::vector<Big> &cl : clusters) {
+            int rank = 0;
+            for (const Big &b : cl) {
+                const int32_t K = p->layers[b.layer].K;
+                // equal slices, starts on multiples of 64 keys (16-byte aligned loads)
+                const int32_t per = (int32_t)round_up64(ceil_div64(K, b.m), 64);
+                for (int j = 0; j < b.m; ++j) {
+                    const int32_t start = j * per;
+                    const int32_t n = std::max<int32_t>(0, std::min<int32_t>(per, K - start));
+                    p->tail_slices.push_back(TailSlice{b.layer, start, n, b.m, j, rank, {0, 0}});
+                }
+                rank += b.m;
+            }
+            for (; rank < kTailCluster; ++rank) p->tail_slices.push_back(TailSlice{0, 0, 0, 0, 0, 0, {0, 0}});
+        }
+        p->n_tail_clusters = (int)clusters.size();
+        p->n_tail_big = p->n_tail_clusters * kTailCluster;
+        for (int l = 0; l < n_layers; ++l)
+            if (p->layers[l].K <= kTailKeysSmall) {
+                p->tail_slices.push_back(TailSlice{l, 0, p->layers[l].K, 1, 0, 0, {0, 0}});
+                ++p->n_tail_small;
+            }
+        if (p->n_tail_clusters > p->tail_max_clusters) {  // more than one wave of clusters: the chained kernels do better
+            p->tail_slices.clear();
+            p->n_tail_big = p->n_tail_small = p->n_tail_clusters = 0;
+        }
+    }
+
     rsdgc_info &I = p->info;
     I.n_layers = n_layers;
     I.grad_dtype = p->dtype;
@@ -306,7 +364,8 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
     if (n_layers > kMaxLayers) return RSDGC_ERR_CAPACITY;
     if (grad_dtype != RSDGC_F32 && grad_dtype != RSDGC_BF16) return RSDGC_ERR_INVALID;
     if (!(alpha >= 0.0f && alpha <= 1.0f)) return RSDGC_ERR_INVALID;
-    if (flags & ~(RSDGC_KEEP_AT_LEAST_ONE | RSDGC_NO_BULK_COPY | RSDGC_MOMENTUM | RSDGC_PAYLOAD_BF16))
+    if (flags & ~(RSDGC_KEEP_AT_LEAST_ONE | RSDGC_NO_BULK_COPY | RSDGC_MOMENTUM | RSDGC_PAYLOAD_BF16 |
+                  RSDGC_NO_FUSED_TAIL))
         return RSDGC_ERR_INVALID;
 
     rsdgc_plan *p = new (std::nothrow) rsdgc_plan();
@@ -328,6 +387,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         DeviceGuard guard(device);
         // one CTA per resident slot: the static partitions assume all CTAs run concurrently
         p->reg_ctas_per_sm = k1_reg_ctas_per_sm(grad_dtype, (flags & RSDGC_MOMENTUM) != 0);
+        p->tail_max_clusters = tail_max_active_clusters();
     }
 
     int rc;
@@ -349,6 +409,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         if (e == cudaSuccess) e = upload(&p->d_cta_begin_bulk, p->cta_begin_bulk);
         if (e == cudaSuccess) e = upload(&p->d_cta_begin_reg, p->cta_begin_reg);
         if (e == cudaSuccess) e = upload(&p->d_chunks, p->chunks);
+        if (e == cudaSuccess) e = upload(&p->d_tail_slices, p->tail_slices);
         if (e == cudaSuccess) e = upload(&p->d_echunks, p->echunks);
         if (e == cudaSuccess) e = alloc_zero(&p->d_state, (size_t)n_layers);
         if (e == cudaSuccess) e = alloc_zero(&p->d_hist, (size_t)n_layers * kHistStride);
@@ -435,6 +496,24 @@ extern "C" int64_t rsdgc_plan_worklist(const rsdgc_plan *plan, int32_t *items_ho
     if (grids_host) grids_host[0] = plan->grid_bulk, grids_host[1] = plan->grid_reg;
     if (n_flush_host)
         for (int l = 0; l < plan->n_layers; ++l) n_flush_host[l] = plan->layers[l].n_flush1;
+    return n;
+}
+
+// Diagnostic: the slices of the single-kernel tail (6 int32 per slice: layer, first tile, tiles,
+// CTAs of the layer, rank among them, cluster rank of the first), cluster slices first; info_host
+// receives their number, the number of one-CTA slices and the number of clusters.
+extern "C" int64_t rsdgc_plan_tail_slices(const rsdgc_plan *plan, int32_t *slices_host, int64_t capacity,
+                                          int32_t *info_host)
+{
+    if (!plan) return RSDGC_ERR_INVALID;
+    const int64_t n = (int64_t)plan->tail_slices.size();
+    if (slices_host)
+        for (int64_t i = 0; i < n && i < capacity; ++i) {
+            const TailSlice &t = plan->tail_slices[i];
+            int32_t *o = slices_host + 6 * i;
+            o[0] = t.layer, o[1] = t.start, o[2] = t.n, o[3] = t.n_ranks, o[4] = t.rank, o[5] = t.leader;
+        }
+    if (info_host) info_host[0] = plan->n_tail_big, info_host[1] = plan->n_tail_small, info_host[2] = plan->n_tail_clusters;
     return n;
 }
 

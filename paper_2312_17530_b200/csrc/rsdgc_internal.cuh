@@ -30,6 +30,12 @@ constexpr int kMaxLayers = 2048;
 constexpr int kMaxSlot = 4096;
 constexpr int kArenaAlign = 64;      // elements; also the alignment of tile offsets
 constexpr uint32_t kTakeNone = 0xFFFFFFFFu;  // prefix / threshold marker: keep nothing
+// the single-kernel selection + pack for plans of small layers (tail.cu)
+constexpr int kTailCluster = 8;        // CTAs per thread-block cluster = slices a layer may have
+constexpr int kTailKeysBig = 32768;    // keys a CTA of the cluster variant holds in shared memory
+constexpr int kTailThreadsBig = 512;
+constexpr int kTailKeysSmall = 8192;   // layers up to this many tiles take the one-CTA variant
+constexpr int kTailThreadsSmall = 256;
 
 // ---- tables ----------------------------------------------------------------------------
 struct LayerDev {
@@ -83,6 +89,15 @@ struct EChunk {
     int32_t layer, n;
 };
 
+// One CTA's share of the single-kernel selection + pack: keys [start, start + n) of a layer.  The
+// n_ranks CTAs of a layer sit in one cluster, `rank` counts them, `leader` is the cluster rank of
+// the first.  n = 0: a rank of a cluster that holds no slice.
+struct TailSlice {
+    int32_t layer, start, n;
+    int32_t n_ranks, rank, leader;
+    int32_t pad[2];
+};
+
 // Per-layer selection state carried from kernel to kernel (device memory, plan-owned).
 struct LayerState {
     unsigned int ticket[4];  // arrival counters of the four phases; each resets itself
@@ -108,6 +123,7 @@ struct Lane {
     float *resid;
     int32_t *idx;
     void *val;                 // binary32 or bfloat16 payload values
+    int32_t *counts;           // k_l per layer (written by the single-kernel tail; the chained path writes it from the first pass)
 };
 struct LaneTable {
     Lane l[kMaxLanes];
@@ -147,6 +163,11 @@ struct rsdgc_plan {
     std::vector<int32_t> cta_begin_bulk, cta_begin_reg;  // grid + 1 indices into each kernel's item list
     std::vector<rsdgc::Chunk> chunks;
     std::vector<rsdgc::EChunk> echunks;
+    // single-kernel tail (plans of small layers): slices of the cluster variant (n_tail_big of them, a
+    // multiple of the cluster size), then those of the one-CTA variant; n_tail_clusters = 0: not eligible
+    std::vector<rsdgc::TailSlice> tail_slices;
+    int n_tail_big = 0, n_tail_small = 0, n_tail_clusters = 0;
+    int tail_max_clusters = 16;  // clusters of the big variant the device holds at a time
 
     rsdgc_info info{};
 
@@ -154,6 +175,7 @@ struct rsdgc_plan {
     rsdgc::LayerDev *d_layers = nullptr;
     rsdgc::ItemDev *d_items = nullptr;
     int32_t *d_cta_begin_bulk = nullptr, *d_cta_begin_reg = nullptr;
+    rsdgc::TailSlice *d_tail_slices = nullptr;
     rsdgc::Chunk *d_chunks = nullptr;
     rsdgc::EChunk *d_echunks = nullptr;
     rsdgc::LayerState *d_state = nullptr;
@@ -204,12 +226,16 @@ cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const
 cudaError_t launch_payload_to_coo(rsdgc_plan *p, const int32_t *idx, const int32_t *counts, long long *coo,
                                   long long coo_cap, cudaStream_t s);
 cudaError_t launch_selftest_bounded_wait(rsdgc_plan *p, unsigned int polls, cudaStream_t s);
+cudaError_t launch_tail(rsdgc_plan *p, const LaneTable &lanes, int n_lanes, const float *ratios, long long idx_cap,
+                        long long val_cap, int prof, cudaStream_t s, cudaError_t (*mark)(rsdgc_plan *, cudaStream_t));
+int tail_max_active_clusters();
 void count_launch(int n);
 void set_last_cuda_error(int e);
 int k1_reg_ctas_per_sm(int dtype, bool momentum);
 int k1_bulk_ctas_per_sm(bool momentum);
 cudaError_t launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                           float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                          cudaStream_t s, bool after_sibling = false, bool before_sibling = false);
+                          cudaStream_t s, bool after_sibling = false, bool before_sibling = false,
+                          bool no_histogram = false);
 
 }  // namespace rsdgc

@@ -22,11 +22,18 @@ def _lib():
 # config 1: one 512x512 layer, clustered outliers, zero residual, 3x3 tiles, keep 1/64
 # ---------------------------------------------------------------------------------------------
 
-def test_single_layer_512(oracle):
+# Plans of small layers select and pack in one kernel per layer-size class; NO_FUSED_TAIL sends the same
+# plan through the chained selection kernels that large layers take.  Both must match the oracle.
+TAILS = [pytest.param(0, id="fused"), pytest.param(binding.NO_FUSED_TAIL, id="chained")]
+
+
+@pytest.mark.parametrize("tail", TAILS)
+def test_single_layer_512(oracle, tail):
     shapes = [(512, 512, 3, 3)]
     g = [synth.clustered_matrix(512, 512, seed=0)]
     r = [np.zeros(512 * 512, np.float32)]
-    plan = binding.Plan(shapes, alpha=0.5)
+    plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE | tail)
+    assert (len(plan.tail_slices()[0]) > 0) == (tail == 0)
     assert plan.layers[0].n_tiles == 171 * 171
     _, refs, gc = parity.compress_and_check(oracle, plan, shapes, g, r, [1 / 64], 0.5, what="512x512")
     assert refs[0].k == 457
@@ -48,14 +55,16 @@ ZOO = [
 ]
 
 
+@pytest.mark.parametrize("tail", TAILS)
 @pytest.mark.parametrize("alpha", [0.5, 0.0, 1.0, 0.25])
-def test_layer_zoo(oracle, alpha):
+def test_layer_zoo(oracle, alpha, tail):
     rng = np.random.default_rng(int(alpha * 100) + 1)
     shapes = ZOO
     g = [(rng.standard_normal(r * c) * 10 ** rng.uniform(-4, 0)).astype(np.float32) for r, c, _, _ in shapes]
     res = [(rng.standard_normal(r * c) * 10 ** rng.uniform(-5, -1)).astype(np.float32) for r, c, _, _ in shapes]
     ratios = rng.choice([0.001, 0.01, 1 / 64, 0.1, 0.3, 1.0, 0.0], size=len(shapes)).astype(np.float32)
-    plan = binding.Plan(shapes, alpha=alpha)
+    plan = binding.Plan(shapes, alpha=alpha, flags=binding.KEEP_AT_LEAST_ONE | tail)
+    assert (len(plan.tail_slices()[0]) > 0) == (tail == 0)
     new_res, refs, gc = parity.compress_and_check(oracle, plan, shapes, g, res, ratios, alpha, what="zoo")
     # second iteration on the carried residual, same buffers
     g2 = [(rng.standard_normal(r * c) * 1e-2).astype(np.float32) for r, c, _, _ in shapes]
@@ -64,7 +73,8 @@ def test_layer_zoo(oracle, alpha):
     parity.compress_and_check(oracle, plan, shapes, g2, new_res, ratios, alpha, gc=gc, what="zoo it2")
 
 
-def test_degenerate_layers(oracle):
+@pytest.mark.parametrize("tail", TAILS)
+def test_degenerate_layers(oracle, tail):
     rng = np.random.default_rng(5)
     shapes = [(60, 60, 3, 3), (60, 60, 3, 3), (1, 900, 1, 9), (33, 33, 3, 3), (1, 7, 1, 9), (300, 300, 3, 3)]
     g = [np.zeros(3600, np.float32),                                    # all-zero layer: all NSI equal 0
@@ -77,7 +87,7 @@ def test_degenerate_layers(oracle):
     res = [np.zeros(x.size, np.float32) for x in g]
     for ratios, clamp in (([0.1, 0.1, 0.05, 1.0, 0.5, 0.4], True), ([0.0] * 6, True), ([0.0] * 6, False),
                           ([1.0] * 6, True), ([0.5, 1e-9, 2.0, -1.0, 0.0, 0.33], False)):
-        plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE if clamp else 0)
+        plan = binding.Plan(shapes, alpha=0.5, flags=(binding.KEEP_AT_LEAST_ONE if clamp else 0) | tail)
         _, refs, _ = parity.compress_and_check(oracle, plan, shapes, g, res, ratios, 0.5, clamp=clamp, what="degenerate")
         if ratios[0] == 0.1:
             k = oracle.keep_count(400, 0.1)                             # pure ties: the first k tiles
@@ -128,11 +138,12 @@ def test_bounded_wait_gives_up_and_reports_timeout():
     assert st.flags == 0 and int(gc.counts[0]) == 49
 
 
-def test_payload_overflow_is_reported_and_nothing_is_lost(oracle):
+@pytest.mark.parametrize("tail", TAILS)
+def test_payload_overflow_is_reported_and_nothing_is_lost(oracle, tail):
     shapes = [(90, 90, 3, 3), (60, 60, 3, 3)]
     rng = np.random.default_rng(7)
     g = [rng.standard_normal(8100).astype(np.float32), rng.standard_normal(3600).astype(np.float32)]
-    plan = binding.Plan(shapes, alpha=0.5)
+    plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE | tail)
     gc = parity.GpuCompress(plan, max_ratio=0.01)           # room for about 1 % of the tiles only
     cap = gc.idx.numel()
     k0, k1 = oracle.keep_count(900, 0.1), oracle.keep_count(400, 0.1)
@@ -165,10 +176,11 @@ def test_payload_overflow_is_reported_and_nothing_is_lost(oracle):
 # config 2: ResNet-18-shaped set, 10 iterations, residual carried, ratios from the weights
 # ---------------------------------------------------------------------------------------------
 
-def test_resnet18_ten_iterations_with_dynamic_ratios(oracle):
+@pytest.mark.parametrize("tail", TAILS)
+def test_resnet18_ten_iterations_with_dynamic_ratios(oracle, tail):
     tensors = synth.resnet18_tensors()
     shapes = synth.layer_shapes(tensors)
-    plan = binding.Plan(shapes, alpha=0.5)
+    plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE | tail)
     weights = synth.synthetic_weights(tensors, (2,))
     # ratio rule (Eq. 3-5) on the GPU against the oracle's full sort
     d_w = parity.dev(parity.to_arena(plan, weights))
@@ -260,12 +272,13 @@ def test_decompress_accumulate_four_workers(oracle, scale):
 # several workers in one call: the selection kernels run once over all workers
 # ---------------------------------------------------------------------------------------------
 
+@pytest.mark.parametrize("tail", TAILS)
 @pytest.mark.parametrize("n_workers", [1, 3])
-def test_compress_workers_two_iterations(oracle, n_workers):
+def test_compress_workers_two_iterations(oracle, n_workers, tail):
     shapes = [(300, 515, 3, 3), (256, 64 * 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3), (1200, 1536, 3, 3),
               (64, 7 * 7 * 3, 1, 49), (5, 5, 3, 3)]
     tensors = [("t%d" % i, (s[0], s[1])) for i, s in enumerate(shapes)]
-    plan = binding.Plan(shapes, alpha=0.5)
+    plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE | tail)
     sig = synth.log_uniform_scales(len(shapes), (21,))
     ratios = np.array([1 / 16, 1 / 50, 0.3, 1.0, 1 / 64, 0.0, 0.5], np.float32)
     res = [[np.zeros(s[0] * s[1], np.float32) for s in shapes] for _ in range(n_workers)]
@@ -581,11 +594,12 @@ def test_momentum_correction_five_iterations(oracle, bf16):
 # payload with bfloat16 values: q = bfloat16(v) is sent, v - q stays in the accumulator
 # ---------------------------------------------------------------------------------------------
 
-def test_bf16_payload_three_iterations_and_aggregation(oracle):
+@pytest.mark.parametrize("tail", TAILS)
+def test_bf16_payload_three_iterations_and_aggregation(oracle, tail):
     shapes = [(300, 515, 3, 3), (256 * 16, 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3), (64, 147, 1, 49),
               (1200, 1536, 3, 3), (5, 5, 3, 3)]
     tensors = [("t%d" % i, (s[0], s[1])) for i, s in enumerate(shapes)]
-    plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE | binding.PAYLOAD_BF16)
+    plan = binding.Plan(shapes, alpha=0.5, flags=binding.KEEP_AT_LEAST_ONE | binding.PAYLOAD_BF16 | tail)
     sig = synth.log_uniform_scales(len(shapes), (41,))
     ratios = np.array([1 / 16, 1 / 50, 0.3, 1.0, 0.1, 1 / 64, 0.5], np.float32)
     n_workers = 2

@@ -33,7 +33,7 @@ def test_library_exports_every_declared_symbol(lib):
 def test_plan_create_rejects_bad_arguments(lib):
     ok = [(8, 8, 3, 3)]
     for layers, kw in [([], {}), ([(0, 8, 3, 3)], {}), ([(8, 8, 0, 3)], {}), (ok, {"alpha": 1.5}),
-                       (ok, {"alpha": float("nan")}), (ok, {"grad_dtype": 7}), (ok, {"flags": 16})]:
+                       (ok, {"alpha": float("nan")}), (ok, {"grad_dtype": 7}), (ok, {"flags": 32})]:
         with pytest.raises(binding.RsdgcError) as e:
             binding.Plan(layers, device=-1, **kw)
         assert e.value.code == binding.ERR_INVALID
@@ -125,3 +125,50 @@ def test_payload_bound(lib):
     assert ni == (457 + 1) + 2 and nv == 9 * ni
     ni, nv = p.payload_bound(1.0)
     assert ni == 29241 + 8
+
+
+@pytest.mark.parametrize("net", ["resnet18", "resnet50", "odd", "single"])
+def test_tail_slices_cover_every_tile_once(lib, net):
+    """Plans of small layers select and pack in one kernel: every layer's tiles are covered exactly once by
+    slices of at most 32768 keys, a layer's slices sit in one cluster of 8 CTAs on consecutive ranks, and
+    layers of at most 8192 tiles take one CTA each outside the clusters."""
+    if net == "odd":
+        shapes = [(7, 11, 3, 3), (1, 5, 1, 9), (4096, 45, 3, 3), (3, 20000, 3, 3), (100, 4401, 2, 5), (1536, 1536, 3, 3),
+                  (5000, 7, 1, 7), (1, 100000, 1, 9), (64, 64, 64, 64), (9, 9, 1, 1), (70000, 9, 1, 9), (40000, 9, 1, 9)]
+    elif net == "single":
+        shapes = [(512, 512, 3, 3)]
+    else:
+        shapes = synth.layer_shapes(getattr(synth, net + "_tensors")())
+    p = binding.Plan(shapes, device=-1)
+    sl, (n_big, n_small, n_clusters) = p.tail_slices()
+    assert len(sl) == n_big + n_small and n_big == 8 * n_clusters and 0 < n_clusters <= 16
+    tiles = [li.n_tiles for li in p.layers]
+    cover = [np.zeros(t, np.int32) for t in tiles]
+    for i, (layer, start, n, n_ranks, rank, leader) in enumerate(sl.tolist()):
+        if n == 0:
+            assert i < n_big                             # an idle rank of a partly filled cluster
+            continue
+        cover[layer][start:start + n] += 1
+        assert start % 64 == 0
+        if i < n_big:
+            assert tiles[layer] > 8192 and n <= 32768 and 1 <= n_ranks <= 8 and 0 <= rank < n_ranks
+            assert leader == i % 8 - rank and leader + n_ranks <= 8      # consecutive ranks of one cluster
+            assert sl[i - rank, 0] == layer and sl[i - rank, 4] == 0
+        else:
+            assert tiles[layer] <= 8192 and (start, n, n_ranks, rank, leader) == (0, tiles[layer], 1, 0, 0)
+    for c in cover:
+        assert (c == 1).all()
+    # equal slices: no slice of a layer is more than 64 keys larger than another
+    for l in range(len(shapes)):
+        ns = sl[(sl[:, 0] == l) & (sl[:, 2] > 0), 2]
+        assert len(ns) == 0 or ns.max() - ns[:-1].min(initial=ns.max()) <= 64
+    # the flag and layers beyond a cluster's reach give the chained kernels
+    assert len(binding.Plan(shapes, device=-1, flags=binding.NO_FUSED_TAIL).tail_slices()[0]) == 0
+    assert len(binding.Plan(shapes + [(3000, 3000, 3, 3)], device=-1).tail_slices()[0]) == 0
+
+
+def test_tail_not_used_when_clusters_exceed_one_wave(lib):
+    shapes = [(1536, 1536, 3, 3)] * 17                     # 17 layers of 8 slices each: 17 clusters
+    assert len(binding.Plan(shapes, device=-1).tail_slices()[0]) == 0
+    assert len(binding.Plan(shapes[:16], device=-1).tail_slices()[0]) == 128
+    assert len(binding.Plan(synth.layer_shapes(synth.vgg19_tensors()), device=-1).tail_slices()[0]) == 0
