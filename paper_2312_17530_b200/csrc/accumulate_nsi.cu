@@ -20,9 +20,6 @@
 
 namespace rsdgc {
 
-constexpr int kNoHistogram = 4;  // launch mode bit of both kernels: keys only, no level-1 histogram (the kernel
-                                 // that follows selects from the keys alone)
-
 // ------------------------------------------------------------------------------------------
 // NSI of one tile
 // ------------------------------------------------------------------------------------------
@@ -89,7 +86,7 @@ __device__ __forceinline__ void emit_key(float nsi, uint32_t *dst, unsigned int 
         ++nonfinite;
     }
     *dst = key;
-    if (hist_smem) atomicAdd(&hist_smem[key >> kL1Shift], 1u);
+    atomicAdd(&hist_smem[key >> kL1Shift], 1u);
 }
 
 // Keys of all tiles of one item from its v block in shared memory (row pitch d.P).
@@ -131,14 +128,30 @@ struct FlushShared {
 // Adds this CTA's level-1 histogram to the layer's global histogram; the last CTA to do so
 // for the layer computes k_l (Eq. 11) and resolves the first 11 key bits of the threshold.
 // Called by all threads of the CTA.
+// What the flush of a layer needs from the plan's tables and the ratios: loaded when a CTA enters the
+// layer, so that the loads (cold: every layer's entries are read only here) are long complete when the
+// CTA leaves it.
+struct FlushInfo {
+    int K, n_flush1;
+    float ratio;
+};
+__device__ __forceinline__ FlushInfo load_flush_info(const LayerDev *__restrict__ layers,
+                                                     const float *__restrict__ ratios, int layer)
+{
+    FlushInfo f;
+    f.K = __ldg(&layers[layer].K);
+    f.n_flush1 = __ldg(&layers[layer].n_flush1);
+    f.ratio = __ldg(&ratios[layer]);
+    return f;
+}
+
 template <int NTHREADS>
-__device__ void k1_flush_layer(unsigned int *hist_smem, FlushShared &fs, int layer, const LayerDev *layers,
-                               unsigned int *hist, LayerState *state, const float *ratios, int32_t *counts,
-                               unsigned int flags)
+__device__ void k1_flush_layer(unsigned int *hist_smem, FlushShared &fs, int layer, const FlushInfo info,
+                               unsigned int *hist, LayerState *state, int32_t *counts, unsigned int flags)
 {
     __syncthreads();
     unsigned int *gh = hist + (size_t)layer * kHistStride;
-    const bool sole_owner = layers[layer].n_flush1 == 1;  // the whole layer went through this CTA
+    const bool sole_owner = info.n_flush1 == 1;  // the whole layer went through this CTA
     if (!sole_owner) {
         for (int b = threadIdx.x; b < kL1Bins; b += NTHREADS) {
             const unsigned int c = hist_smem[b];
@@ -151,7 +164,7 @@ __device__ void k1_flush_layer(unsigned int *hist_smem, FlushShared &fs, int lay
         __syncthreads();
         if (threadIdx.x == 0) {
             const unsigned int t = atomicAdd(&state[layer].ticket[0], 1u);
-            fs.is_last = (t + 1u == (unsigned int)layers[layer].n_flush1);
+            fs.is_last = (t + 1u == (unsigned int)info.n_flush1);
         }
         __syncthreads();
         if (!fs.is_last) return;  // uniform for the CTA
@@ -168,8 +181,7 @@ __device__ void k1_flush_layer(unsigned int *hist_smem, FlushShared &fs, int lay
         }
     }
     __syncthreads();
-    const int K = layers[layer].K;
-    const int k = keep_count(K, ratios[layer], flags);
+    const int k = keep_count(info.K, info.ratio, flags);
     if (k > 0) find_bin_from_top<kL1Bins, NTHREADS>(hist_smem, (unsigned long long)k, fs.found, fs.scan_tmp);
     if (threadIdx.x == 0) {
         LayerState &st = state[layer];
@@ -426,11 +438,9 @@ __global__ void __launch_bounds__(kThreads)
 k1_reg(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict__ vel, float mom,
        uint32_t *__restrict__ keys, const LayerDev *__restrict__ layers, const ItemDev *__restrict__ items,
        const int32_t *__restrict__ cta_begin, unsigned int *hist, LayerState *state,
-       const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags,
-       int mode)
+       const float *__restrict__ ratios, int32_t *counts, StatusDev *status, float alpha, unsigned int flags)
 {
     extern __shared__ __align__(16) unsigned char k1_smem_raw[];
-    const bool with_hist = (mode & kNoHistogram) == 0;
     K1RegShared &sh = *reinterpret_cast<K1RegShared *>(k1_smem_raw);
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     if (begin >= end) return;
@@ -441,6 +451,7 @@ k1_reg(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict
     K1Regs<MOM> x;
     K1Map map;
     ItemDev cur = load_item(items, begin);
+    FlushInfo finfo = load_flush_info(layers, ratios, cur.layer);
     k1_issue_loads<G, MOM>(cur, grads, resid, vel, x, map);
     int buf = 0;
 
@@ -456,9 +467,11 @@ k1_reg(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict
         // the next item's g and r stream in while this item's tiles are reduced
         if (has_next) k1_issue_loads<G, MOM>(nxt, grads, resid, vel, x, map);
         __syncthreads();
-        nonfinite += item_tile_keys<kThreads>(cur, sv, keys, with_hist ? sh.hist : nullptr, alpha);
-        if (with_hist && (!has_next || nxt.layer != cur.layer))
-            k1_flush_layer<kThreads>(sh.hist, sh.fs, cur.layer, layers, hist, state, ratios, counts, flags);
+        nonfinite += item_tile_keys<kThreads>(cur, sv, keys, sh.hist, alpha);
+        if (!has_next || nxt.layer != cur.layer) {
+            k1_flush_layer<kThreads>(sh.hist, sh.fs, cur.layer, finfo, hist, state, counts, flags);
+            if (has_next) finfo = load_flush_info(layers, ratios, nxt.layer);
+        }
         cur = nxt;
         buf ^= 1;
     }
@@ -607,7 +620,6 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
     K1BulkShared<MOM> &sh = *reinterpret_cast<K1BulkShared<MOM> *>(k1_bulk_smem_raw);
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     const bool wait_late = (overlap & kOverlapPrev) != 0;
-    const bool with_hist = (overlap & kNoHistogram) == 0;
     if (begin >= end) {
         if (wait_late) grid_dependency_wait();
         return;
@@ -647,6 +659,7 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
     // call is then invalid).
     bool dead = false;
     ItemDev cur = load_item(items, begin);
+    FlushInfo finfo = load_flush_info(layers, ratios, cur.layer);
     // the producer thread keeps the descriptor of the next item to load one iteration ahead
     ItemDev ahead = cur;
     if (tid == 0 && begin + kLookahead < end) ahead = load_item(items, begin + kLookahead);
@@ -713,10 +726,12 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
                 }
             }
             // ---- NSI of every tile of the item
-            nonfinite += item_tile_keys<kBulkThreads>(cur, sr, keys, with_hist ? sh.hist : nullptr, alpha);
+            nonfinite += item_tile_keys<kBulkThreads>(cur, sr, keys, sh.hist, alpha);
         }
-        if (with_hist && (!has_next || nxt.layer != cur.layer))
-            k1_flush_layer<kBulkThreads>(sh.hist, sh.fs, cur.layer, layers, hist, state, ratios, counts, flags);
+        if (!has_next || nxt.layer != cur.layer) {
+            k1_flush_layer<kBulkThreads>(sh.hist, sh.fs, cur.layer, finfo, hist, state, counts, flags);
+            if (has_next) finfo = load_flush_info(layers, ratios, nxt.layer);
+        }
         cur = nxt;
     }
     if (dead && tid == 0) {
@@ -851,7 +866,7 @@ static cudaError_t launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *st
     if (p->n_items_reg > 0) {
         k1_reg<G, MOM><<<p->grid_reg, kThreads, sizeof(K1RegShared), s>>>(
             g, resid, vel, mom, keys, p->d_layers, p->d_items + p->n_items_bulk, p->d_cta_begin_reg, hist,
-            state, ratios, counts, p->d_status, p->alpha, p->flags, overlap & kNoHistogram);
+            state, ratios, counts, p->d_status, p->alpha, p->flags);
         e = cudaGetLastError();
         if (e != cudaSuccess) return e;
         ++*launches;
@@ -867,12 +882,11 @@ static cudaError_t launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *st
 // not run on keys no first pass has written.
 cudaError_t launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                                   float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                                  cudaStream_t s, bool after_sibling, bool before_sibling, bool no_histogram)
+                                  cudaStream_t s, bool after_sibling, bool before_sibling)
 {
     int overlap = 0;
     if (p->n_items_reg == 0)  // the register-staged kernel is launched without overlap
         overlap = (after_sibling ? kOverlapPrev : 0) | (before_sibling ? kOverlapNext : 0);
-    if (no_histogram) overlap |= kNoHistogram;
     int launches = 0;
     cudaError_t e = configure_once();
     if (e != cudaSuccess) return e;

@@ -607,11 +607,10 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, floa
     if (prof >= 1) e = record_event(p, s);
     const bool fused = use_fused_tail(p, 1);
     if (e == cudaSuccess)
-        e = launch_accumulate_nsi(p, p->d_hist, p->d_state, grads, resid, vel, mom, ratios, counts, keys, s, false,
-                                  false, fused);
+        e = launch_accumulate_nsi(p, p->d_hist, p->d_state, grads, resid, vel, mom, ratios, counts, keys, s);
     if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
     LaneTable lanes{};
-    lanes.l[0] = Lane{keys, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid, idx, val, counts};
+    lanes.l[0] = Lane{keys, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid, idx, val};
     if (e == cudaSuccess)
         e = fused ? launch_fused_tail(p, lanes, 1, ratios, idx_cap, val_cap, prof, s)
                   : launch_selection(p, lanes, 1, idx_cap, val_cap, prof, s);
@@ -641,15 +640,15 @@ cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *co
             const int w = w0 + j;
             Lane &ln = lanes.l[j];
             if (w == 0) {
-                ln = Lane{keys_all, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid[0], idx[0], val[0], counts[0]};
+                ln = Lane{keys_all, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid[0], idx[0], val[0]};
             } else {
                 const rsdgc_plan::LaneScratch &x = p->extra_lanes[(size_t)w - 1];
                 ln = Lane{keys_all + (size_t)w * key_stride, x.hist, x.state, x.chunk_cnt, x.codes, resid[w], idx[w],
-                          val[w], counts[w]};
+                          val[w]};
             }
             // the first passes of a group's workers share nothing: all but the first start without waiting
             e = launch_accumulate_nsi(p, ln.hist, ln.state, grads[w], ln.resid, nullptr, 0.0f, ratios, counts[w],
-                                      ln.keys, s, j > 0, j + 1 < n, fused);
+                                      ln.keys, s, j > 0, j + 1 < n);
         }
         if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
         if (e == cudaSuccess)

@@ -33,7 +33,7 @@ constexpr uint32_t kTakeNone = 0xFFFFFFFFu;  // prefix / threshold marker: keep 
 // the single-kernel selection + pack for plans of small layers (tail.cu)
 constexpr int kTailCluster = 8;        // CTAs per thread-block cluster = slices a layer may have
 constexpr int kTailKeysBig = 32768;    // keys a CTA of the cluster variant holds in shared memory
-constexpr int kTailThreadsBig = 512;
+constexpr int kTailThreadsBig = 1024;
 constexpr int kTailKeysSmall = 8192;   // layers up to this many tiles take the one-CTA variant
 constexpr int kTailThreadsSmall = 256;
 
@@ -123,7 +123,6 @@ struct Lane {
     float *resid;
     int32_t *idx;
     void *val;                 // binary32 or bfloat16 payload values
-    int32_t *counts;           // k_l per layer (written by the single-kernel tail; the chained path writes it from the first pass)
 };
 struct LaneTable {
     Lane l[kMaxLanes];
@@ -235,7 +234,6 @@ int k1_reg_ctas_per_sm(int dtype, bool momentum);
 int k1_bulk_ctas_per_sm(bool momentum);
 cudaError_t launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                           float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
-                          cudaStream_t s, bool after_sibling = false, bool before_sibling = false,
-                          bool no_histogram = false);
+                          cudaStream_t s, bool after_sibling = false, bool before_sibling = false);
 
 }  // namespace rsdgc

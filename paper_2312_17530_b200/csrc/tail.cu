@@ -1,13 +1,15 @@
 // Everything after the accumulate+NSI pass in ONE kernel per layer-size class, for plans whose layers
-// are small enough to keep a layer's keys on chip: keep count (Eq. 11), the three-level radix
-// selection of the threshold (Algorithm 1's ranking), the payload indices, the gather of the kept
-// values and the clearing of the accumulator (Sec. III-C, Eq. 12).
+// are small enough to keep a layer's keys on chip: levels 2 and 3 of the radix selection of the
+// threshold (Algorithm 1's ranking; level 1 and the keep count of Eq. 11 come with the first pass,
+// whose histogram work is spread over all SMs), the payload indices, the gather of the kept values
+// and the clearing of the accumulator (Sec. III-C, Eq. 12).
 //
 // Why: the chained kernels (two refinement passes, count, mark, gather) each cost a chain of
 // dependent global round trips (table, layer state, keys, histogram flush, ticket, last CTA), about
 // 7 us per kernel whatever the data, which is most of a call on network-sized layer sets.  Here a
 // layer's keys are read from global memory once, into shared memory, and every later step works
-// from there.
+// from there.  (Keys held in registers would need fully unrolled passes: measured, the instruction
+// fetches of the straight-line code, cold after every call, cost more than the shared-memory reads.)
 //
 //  * k_tail<kTailCluster, ...>: a layer of up to kTailCluster * kTailKeysBig tiles is cut into slices
 //    of kTailKeysBig keys, one slice per CTA, all CTAs of a layer in one thread-block cluster.  The
@@ -34,20 +36,28 @@ struct TailShared {
     unsigned int hist[kL2Bins];              // this CTA's histogram; the leader's also receives the others'
     unsigned long long scan_tmp[NT / 32];
     unsigned long long found[2];
-    unsigned int res[2];                     // leader: what the level resolved (bin / prefix, remaining)
+    unsigned int res[2];                     // leader: what the level resolved (bin, remaining)
     unsigned int cnt[kTailCluster][2];       // leader: per rank, keys above the threshold / equal to it
     unsigned int warp_cnt[NT / 32][2];       // per warp of this CTA: the same counts over the warp's keys
     long long idx_off, val_off;              // payload offsets of the layer
-    int k;                                   // tiles to keep (Eq. 11)
 };
 
-// Block-wide sum of one value per thread (every thread gets it).  Two barriers.
+// Block-wide sum of one value per thread (every thread gets it).  Not inlined: these kernels run
+// once per call on cold instruction caches, so their code is kept small (loops with a little
+// unrolling for memory-level parallelism, one copy of every helper).
 template <int NT>
-__device__ __forceinline__ unsigned long long block_sum(unsigned long long x, unsigned long long *tmp)
+__device__ __noinline__ unsigned long long block_sum(unsigned long long x, unsigned long long *tmp)
 {
     unsigned long long total;
     (void)block_exclusive_scan<unsigned long long, NT>(x, tmp, &total);
     return total;
+}
+
+template <int NT>
+__device__ __noinline__ void tail_find_bin(const unsigned int *h, unsigned long long need, unsigned long long *out,
+                                           unsigned long long *tmp)
+{
+    find_bin_from_top<kL2Bins, NT>(h, need, out, tmp);
 }
 
 template <int CS, int KEYS, int NT, bool BF16VAL>
@@ -77,7 +87,8 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
         else return p;
     };
 
-    // ---- what needs only the plan and the ratios: k_l and the layer's payload offsets
+    // ---- what needs only the plan and the ratios: the layer's payload offsets (sums of the k_l of the
+    // preceding layers, Eq. 11)
     for (int b = tid; b < kL2Bins; b += NT) sh.hist[b] = 0;
     if (active) {
         long long si = 0, sv = 0;
@@ -91,7 +102,6 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
         if (tid == 0) {
             sh.idx_off = (long long)ti;
             sh.val_off = (long long)tv;
-            sh.k = keep_count(layers[sl.layer].K, ratios[sl.layer], flags);
         }
     }
     // ---- the first pass has written the keys (a kernel launched right behind a sibling of this one
@@ -99,34 +109,68 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     if (!wait_late) grid_dependency_wait();
     grid_dependency_launch_next();
     const LayerDev L = layers[active ? sl.layer : 0];
+    // it also left k_l and level 1 (key bits 30..21) of the layer's selection in the layer's state
+    int k = 0;
+    uint32_t prefix = kTakeNone;   // key bits resolved so far
+    unsigned int remaining = 0;    // tiles still to take among the keys that carry the prefix
+    const int n4 = (sl.n + 3) >> 2;  // the slice as 128-bit words (the last one padded)
     if (active) {
+        const LayerState &st = ln.state[sl.layer];
+        k = __ldcg(&st.k);
+        prefix = __ldcg(&st.prefix);
+        remaining = (unsigned int)__ldcg(&st.remaining);
         const uint32_t *kp = ln.keys + L.tile_off + sl.start;  // 16-byte aligned: offsets are multiples of 64 keys
         const int nvec = sl.n >> 2;
-        for (int i = tid; i < nvec; i += NT)
-            reinterpret_cast<uint4 *>(skeys)[i] = __ldcg(reinterpret_cast<const uint4 *>(kp) + i);
-        for (int i = (nvec << 2) + tid; i < sl.n; i += NT) skeys[i] = __ldcg(kp + i);
+        constexpr int kLoadBatch = 8;  // 128-bit loads in flight per thread: the slice arrives in one or two round trips
+        for (int base = 0; base < nvec; base += NT * kLoadBatch) {
+            uint4 q[kLoadBatch];
+#pragma unroll
+            for (int u = 0; u < kLoadBatch; ++u) {
+                const int i = base + u * NT + tid;
+                q[u] = (i < nvec) ? __ldcg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int u = 0; u < kLoadBatch; ++u) {
+                const int i = base + u * NT + tid;
+                if (i < nvec) reinterpret_cast<uint4 *>(skeys)[i] = q[u];
+            }
+        }
+        // the last, partial word: keys beyond the slice are all ones, which no prefix or threshold matches
+        if (tid < 4 && (sl.n & 3)) {
+            const int i = (nvec << 2) + tid;
+            skeys[i] = (i < sl.n) ? __ldcg(kp + i) : 0xFFFFFFFFu;
+        }
     }
     __syncthreads();
     sync_all();  // every histogram of the cluster is zero before anything is added to a leader's
-    const int k = active ? sh.k : 0;
 
-    // ---- three radix levels on the key bits 30..21, 20..10, 9..0
-    uint32_t prefix = (k > 0) ? 0u : kTakeNone;  // key bits resolved so far
-    unsigned int remaining = (unsigned int)k;    // tiles still to take among the keys that carry the prefix
-#pragma unroll
-    for (int level = 1; level <= 3; ++level) {
-        const int shift_hi = level == 1 ? 31 : (level == 2 ? kL1Shift : kL2Shift);
-        const int shift_lo = level == 1 ? kL1Shift : (level == 2 ? kL2Shift : 0);
-        const int nbins = level == 2 ? kL2Bins : kL1Bins;
+    // ---- levels 2 and 3: key bits 20..10, 9..0
+#pragma unroll 1
+    for (int level = 2; level <= 3; ++level) {
+        const int shift_hi = level == 2 ? kL1Shift : kL2Shift;
+        const int shift_lo = level == 2 ? kL2Shift : 0;
+        const unsigned int mask = level == 2 ? (unsigned int)(kL2Bins - 1) : (unsigned int)(kL3Bins - 1);
         if (active && prefix != kTakeNone) {
-            for (int i = tid; i < sl.n; i += NT) {
-                const uint32_t key = skeys[i];
-                if ((key >> shift_hi) == prefix) atomicAdd(&sh.hist[(key >> shift_lo) & (nbins - 1)], 1u);
+#pragma unroll 1
+            for (int base = 0; base < n4; base += NT * 2) {
+                uint4 q[2];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    const int i = base + u * NT + tid;
+                    q[u] = (i < n4) ? reinterpret_cast<const uint4 *>(skeys)[i] : make_uint4(~0u, ~0u, ~0u, ~0u);
+                }
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+                    if ((q[u].x >> shift_hi) == prefix) atomicAdd(&sh.hist[(q[u].x >> shift_lo) & mask], 1u);
+                    if ((q[u].y >> shift_hi) == prefix) atomicAdd(&sh.hist[(q[u].y >> shift_lo) & mask], 1u);
+                    if ((q[u].z >> shift_hi) == prefix) atomicAdd(&sh.hist[(q[u].z >> shift_lo) & mask], 1u);
+                    if ((q[u].w >> shift_hi) == prefix) atomicAdd(&sh.hist[(q[u].w >> shift_lo) & mask], 1u);
+                }
             }
             if (CS > 1 && !leader) {
                 __syncthreads();
                 unsigned int *lh = at_leader(&sh.hist[0]);
-                for (int b = tid; b < nbins; b += NT) {
+                for (int b = tid; b <= (int)mask; b += NT) {
                     const unsigned int c = sh.hist[b];
                     if (c) {
                         atomicAdd(lh + b, c);
@@ -137,18 +181,18 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
         }
         sync_all();
         if (leader && prefix != kTakeNone) {
-            if (level == 2) find_bin_from_top<kL2Bins, NT>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
-            else find_bin_from_top<kL1Bins, NT>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
+            // (level 3 fills the lower 1024 of the 2048 bins; the upper ones are zero and change nothing)
+            tail_find_bin<NT>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
             if (tid == 0) {
                 sh.res[0] = (unsigned int)sh.found[0];
                 sh.res[1] = (unsigned int)sh.found[1];
             }
-            for (int b = tid; b < nbins; b += NT) sh.hist[b] = 0;
+            for (int b = tid; b <= (int)mask; b += NT) sh.hist[b] = 0;
         }
         sync_all();
         if (active && prefix != kTakeNone) {
             const unsigned int *res = at_leader(&sh.res[0]);
-            prefix = (prefix << (level == 2 ? kL2Bits : kL1Bits)) | res[0];
+            prefix = (prefix << (level == 2 ? kL2Bits : kL3Bits)) | res[0];
             remaining = res[1];
         }
     }
@@ -158,15 +202,17 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     // ---- per warp, per CTA, per layer: how many keys lie above T and how many equal it
     // warp w owns the keys [w * per_warp, (w + 1) * per_warp) of the slice
     constexpr int per_warp = KEYS / NW;
-    const int w0 = warp * per_warp;
+    const int w0 = warp * per_warp, w1 = min(sl.n, w0 + per_warp);
     {
         unsigned int gt = 0, eq = 0;
-        if (active && T != kTakeNone)
-            for (int i = w0 + lane; i < min(sl.n, w0 + per_warp); i += 32) {
+        if (active && T != kTakeNone) {
+#pragma unroll 4
+            for (int i = w0 + lane; i < w1; i += 32) {
                 const uint32_t key = skeys[i];
                 gt += key > T;
                 eq += key == T;
             }
+        }
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) {
             gt += __shfl_xor_sync(0xFFFFFFFFu, gt, d);
@@ -178,15 +224,20 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
         }
     }
     __syncthreads();
-    if (active && tid == 0) {
-        unsigned int a = 0, b = 0;
-        for (int w = 0; w < NW; ++w) {
-            a += sh.warp_cnt[w][0];
-            b += sh.warp_cnt[w][1];
+    long long gt_before = 0, eq_before = 0, cta_gt = 0, cta_eq = 0;  // in the warps before this one / in the CTA
+#pragma unroll 1
+    for (int w = 0; w < NW; ++w) {
+        if (w < warp) {
+            gt_before += sh.warp_cnt[w][0];
+            eq_before += sh.warp_cnt[w][1];
         }
+        cta_gt += sh.warp_cnt[w][0];
+        cta_eq += sh.warp_cnt[w][1];
+    }
+    if (active && tid == 0) {
         unsigned int *c = at_leader(&sh.cnt[0][0]);
-        c[2 * sl.rank] = a;
-        c[2 * sl.rank + 1] = b;
+        c[2 * sl.rank] = (unsigned int)cta_gt;
+        c[2 * sl.rank + 1] = (unsigned int)cta_eq;
     }
     sync_all();
     long long lay_gt0 = 0, lay_eq0 = 0;  // keys above / equal in the slices of the layer before this one
@@ -204,14 +255,11 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     }
 
     const long long idx_off = sh.idx_off, val_off = sh.val_off;
-    if (leader && tid == 0) {
-        ln.counts[sl.layer] = k;
-        if (sl.layer == n_layers - 1) {
-            const long long need_i = idx_off + k, need_v = val_off + (long long)k * L.slot;
-            status->idx_needed = need_i;
-            status->val_needed = need_v;
-            if (need_i > idx_cap || need_v > val_cap) atomicOr(&status->flags, RSDGC_STATUS_PAYLOAD_OVERFLOW);
-        }
+    if (leader && tid == 0 && sl.layer == n_layers - 1) {
+        const long long need_i = idx_off + k, need_v = val_off + (long long)k * L.slot;
+        status->idx_needed = need_i;
+        status->val_needed = need_v;
+        if (need_i > idx_cap || need_v > val_cap) atomicOr(&status->flags, RSDGC_STATUS_PAYLOAD_OVERFLOW);
     }
     if (T == kTakeNone) {
         if (wait_late) grid_dependency_wait();
@@ -220,29 +268,35 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
 
     // ---- payload indices: a tile is kept if its key is above T, or equals T with fewer than e equal
     // keys before it in the layer; its slot is the number of kept tiles before it
-    long long gt_before = lay_gt0, eq_before = lay_eq0, cta_gt = 0, cta_eq = 0;
-    for (int w = 0; w < NW; ++w) {
-        if (w < warp) {
-            gt_before += sh.warp_cnt[w][0];
-            eq_before += sh.warp_cnt[w][1];
-        }
-        cta_gt += sh.warp_cnt[w][0];
-        cta_eq += sh.warp_cnt[w][1];
-    }
+    gt_before += lay_gt0;
+    eq_before += lay_eq0;
     int32_t *__restrict__ idx = ln.idx;
-    for (int base = w0; base < min(sl.n, w0 + per_warp); base += 32) {
-        const int i = base + lane;
-        const uint32_t key = (i < sl.n) ? skeys[i] : 0u;
-        const bool above = (i < sl.n) && key > T, equal = (i < sl.n) && key == T;
-        const unsigned int ma = __ballot_sync(0xFFFFFFFFu, above), me = __ballot_sync(0xFFFFFFFFu, equal);
-        const unsigned int lower = (1u << lane) - 1u;
-        const long long g_rank = gt_before + __popc(ma & lower), e_rank = eq_before + __popc(me & lower);
-        if (above || (equal && e_rank < e)) {
-            const long long s = idx_off + g_rank + min(e_rank, e);
-            if (s < idx_cap) idx[s] = sl.start + i;
+#pragma unroll 1
+    for (int base = w0; base < w1; base += 128) {  // four groups of 32 keys per round: their loads and votes overlap
+        uint32_t key[4];
+        unsigned int ma[4], me[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int i = base + u * 32 + lane;
+            key[u] = (i < w1) ? skeys[i] : 0xFFFFFFFFu;  // all ones: neither above nor equal (T has bit 31 clear)
         }
-        gt_before += __popc(ma);
-        eq_before += __popc(me);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            ma[u] = __ballot_sync(0xFFFFFFFFu, key[u] != 0xFFFFFFFFu && key[u] > T);
+            me[u] = __ballot_sync(0xFFFFFFFFu, key[u] == T);
+        }
+        const unsigned int lower = (1u << lane) - 1u;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long g_rank = gt_before + __popc(ma[u] & lower), e_rank = eq_before + __popc(me[u] & lower);
+            const bool above = (ma[u] >> lane) & 1u, equal = (me[u] >> lane) & 1u;
+            if (above || (equal && e_rank < e)) {
+                const long long s = idx_off + g_rank + min(e_rank, e);
+                if (s < idx_cap) idx[s] = sl.start + base + u * 32 + lane;
+            }
+            gt_before += __popc(ma[u]);
+            eq_before += __popc(me[u]);
+        }
     }
     __syncthreads();  // the gather below reads the indices this CTA has just written
 
@@ -251,13 +305,17 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     const long long s_first = idx_off + lay_gt0 + min(lay_eq0, e);
     const long long n_kept = cta_gt + (min(lay_eq0 + cta_eq, e) - min(lay_eq0, e));
     const int slot = L.slot;
-    float *__restrict__ resid = ln.resid;
-    float *__restrict__ val = reinterpret_cast<float *>(ln.val);
-    __nv_bfloat16 *__restrict__ val16 = reinterpret_cast<__nv_bfloat16 *>(ln.val);
+    // positions relative to the layer's start in the arena / in the payload fit 32 bits (a layer has
+    // fewer than 2^31 elements)
+    float *__restrict__ resid_l = ln.resid + L.elem_off;
+    float *__restrict__ val_l = reinterpret_cast<float *>(ln.val) + val_off;
+    __nv_bfloat16 *__restrict__ val16_l = reinterpret_cast<__nv_bfloat16 *>(ln.val) + val_off;
     constexpr int kBatch = 4;
     const long long n_vals = n_kept * slot;
+    const int cols = (int)L.cols;
+#pragma unroll 1
     for (long long j0 = 0; j0 < n_vals; j0 += (long long)NT * kBatch) {
-        long long ga[kBatch], vo[kBatch];
+        int ga[kBatch], vo[kBatch];
         float xv[kBatch];
 #pragma unroll
         for (int u = 0; u < kBatch; ++u) {
@@ -265,16 +323,8 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
             ga[u] = -1;
             vo[u] = -1;
             if (j < n_vals) {
-                long long q;
-                int el;
-                if (j < 0x7FFFFFFFll) {
-                    int qq;
-                    divmod_small((int)j, slot, &qq, &el);
-                    q = qq;
-                } else {
-                    q = j / slot;
-                    el = (int)(j - q * slot);
-                }
+                int q, el;
+                divmod_small((int)j, slot, &q, &el);  // n_vals <= the layer's elements < 2^31
                 const long long s = s_first + q;
                 // tiles that do not fit the payload buffers are not sent and stay in the accumulator
                 if (s < idx_cap && val_off + (s - idx_off + 1) * slot <= val_cap) {
@@ -282,29 +332,29 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
                     const int tr = tile / L.TC, tc = tile - tr * L.TC;
                     int a, b;
                     divmod_small(el, L.nw, &a, &b);
-                    const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
-                    if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
-                    vo[u] = val_off + (s - idx_off) * slot + el;
+                    const int i = tr * L.nh + a, jj = tc * L.nw + b;
+                    if (i < (int)L.rows && jj < cols) ga[u] = i * cols + jj;
+                    vo[u] = (int)(s - idx_off) * slot + el;
                 }
             }
         }
         if (BF16VAL) {  // q = bfloat16(v) is sent, v - q stays (exact in binary32)
 #pragma unroll
-            for (int u = 0; u < kBatch; ++u) xv[u] = (ga[u] >= 0) ? resid[ga[u]] : 0.0f;
+            for (int u = 0; u < kBatch; ++u) xv[u] = (ga[u] >= 0) ? resid_l[ga[u]] : 0.0f;
 #pragma unroll
             for (int u = 0; u < kBatch; ++u) {
                 const __nv_bfloat16 q = __float2bfloat16_rn(xv[u]);
-                if (ga[u] >= 0) resid[ga[u]] = __fsub_rn(xv[u], __bfloat162float(q));
-                if (vo[u] >= 0) val16[vo[u]] = q;
+                if (ga[u] >= 0) resid_l[ga[u]] = __fsub_rn(xv[u], __bfloat162float(q));
+                if (vo[u] >= 0) val16_l[vo[u]] = q;
             }
         } else {  // read v and leave +0 in one exchange (see k_gather)
 #pragma unroll
             for (int u = 0; u < kBatch; ++u)
-                xv[u] = (ga[u] >= 0) ? __uint_as_float(atomicExch(reinterpret_cast<unsigned int *>(resid) + ga[u], 0u))
+                xv[u] = (ga[u] >= 0) ? __uint_as_float(atomicExch(reinterpret_cast<unsigned int *>(resid_l) + ga[u], 0u))
                                      : 0.0f;
 #pragma unroll
             for (int u = 0; u < kBatch; ++u)
-                if (vo[u] >= 0) val[vo[u]] = xv[u];
+                if (vo[u] >= 0) val_l[vo[u]] = xv[u];
         }
     }
     if (wait_late) grid_dependency_wait();
@@ -366,7 +416,7 @@ static cudaError_t launch_tail_typed(rsdgc_plan *p, const LaneTable &lanes, int 
         cfg.gridDim = dim3((unsigned)p->n_tail_big, (unsigned)n_lanes);
         cfg.blockDim = dim3(kTailThreadsBig);
         cfg.dynamicSmemBytes = kTailSmemBig;
-        cfg.stream = s;
+            cfg.stream = s;
         cudaLaunchAttribute attr[2];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr[0].val.programmaticStreamSerializationAllowed = 1;

@@ -735,6 +735,73 @@ def test_payload_exchange_through_nccl_one_rank():
     assert out.returncode == 0 and "nccl exchange ok" in out.stdout, out.stdout + out.stderr
 
 
+NCCL_GROUPED_CHILD = r"""
+import os, sys
+sys.path.insert(0, %r); sys.path.insert(0, os.path.join(%r, "tests"))
+import numpy as np, torch
+import torch.distributed as td
+import oracle, parity
+from paper_2312_17530_b200 import binding, sync, synth
+td.init_process_group("nccl", rank=0, world_size=1)
+torch.cuda.set_device(0)
+shapes = [(300, 515, 3, 3), (256, 9, 1, 9), (1, 1000, 1, 9), (77, 45, 3, 3), (640, 1152, 3, 3), (1, 640, 1, 9), (200, 99, 3, 3)]
+tensors = [("t%%d" %% i, (s[0], s[1])) for i, s in enumerate(shapes)]
+ratios = np.array([0.1, 0.3, 0.2, 0.05, 1 / 64, 0.0, 0.02], np.float32)
+n_local = 2
+groups = sync.split_layers(shapes, 3)
+plans = [binding.Plan(shapes[lo:hi], alpha=0.5) for lo, hi in groups]
+gx = sync.GroupedExchange(shapes, groups, plans, n_local, 1, 0, "cuda:0", always_gather=True)
+gx.set_ratios(ratios.tolist())
+sig = synth.log_uniform_scales(len(shapes), (62,))
+res = [[np.zeros(s[0] * s[1], np.float32) for s in shapes] for _ in range(n_local)]
+d_res = [[parity.dev(parity.to_arena(p, res[w][lo:hi])) for w in range(n_local)] for p, (lo, hi) in zip(plans, groups)]
+d_rat = [torch.tensor(ratios[lo:hi], device="cuda:0") for lo, hi in groups]
+ws = [torch.empty(n_local * max(p.info.workspace_bytes, 16), dtype=torch.uint8, device="cuda:0") for p in plans]
+dense = [torch.full((p.info.arena_elems,), float("nan"), device="cuda:0") for p in plans]
+for it in range(2):                                  # residuals carried; the second step reuses streams and events
+    grads = synth.multi_worker_gradients(tensors, n_local, (62, it), sig)
+    d_g = [[parity.dev(parity.to_arena(p, grads[w][lo:hi])) for w in range(n_local)] for p, (lo, hi) in zip(plans, groups)]
+    gx.step(d_g, d_res, d_rat, ws, dense, scale=0.5, assign=True)
+    torch.cuda.synchronize()
+    assert all(p.status().flags == 0 for p in plans)
+    refs = [oracle.compress(shapes, grads[w], res[w], ratios, 0.5) for w in range(n_local)]
+    want = [np.zeros(s[0] * s[1], np.float32) for s in shapes]
+    oracle.decompress_assign(shapes, want, refs, 0.5)        # the ungrouped aggregation of all workers
+    for p, (lo, hi), d in zip(plans, groups, dense):
+        for got, w in zip(parity.from_arena(p, d.cpu().numpy()), want[lo:hi]):
+            assert np.array_equal(got.view(np.uint32), w.view(np.uint32))
+    res = [[l.residual for l in r.layers] for r in refs]
+    for g, (p, (lo, hi)) in enumerate(zip(plans, groups)):
+        for w in range(n_local):
+            for got, w_res in zip(parity.from_arena(p, d_res[g][w].cpu().numpy()), res[w][lo:hi]):
+                assert np.array_equal(got.view(np.uint32), w_res.view(np.uint32))
+k = [oracle.keep_count(oracle.tile_count(*s), float(q)) for s, q in zip(shapes, ratios)]
+# exactly what is sent plus at most 15 bytes of padding per section
+assert gx.message_bytes() <= n_local * (4 * (len(shapes) + sum(k) + sum(a * s[2] * s[3] for a, s in zip(k, shapes))) + 45 * len(groups))
+td.destroy_process_group()
+print("nccl grouped exchange ok")
+"""
+
+
+def test_grouped_overlapped_exchange_through_nccl_one_rank():
+    """Layer groups: group g + 1 is compressed while group g's exact-size payload message goes through a
+    real NCCL all-gather on a second stream, then the groups are aggregated in order; the dense result
+    equals the oracle's ungrouped aggregation bit for bit, over two iterations with carried residuals."""
+    import os
+    import socket
+    import subprocess
+    import sys
+
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    env = dict(os.environ, RANK="0", LOCAL_RANK="0", WORLD_SIZE="1", MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    out = subprocess.run([sys.executable, "-c", NCCL_GROUPED_CHILD % (root, root)], env=env, capture_output=True,
+                         text=True, timeout=300)
+    assert out.returncode == 0 and "nccl grouped exchange ok" in out.stdout, out.stdout + out.stderr
+
+
 # ---------------------------------------------------------------------------------------------
 # more workers than one launch serves (groups of 16): compress_workers and the aggregation
 # ---------------------------------------------------------------------------------------------
