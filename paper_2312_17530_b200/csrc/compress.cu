@@ -607,7 +607,10 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, floa
     if (prof >= 1) e = record_event(p, s);
     const bool fused = use_fused_tail(p, 1);
     if (e == cudaSuccess)
-        e = launch_accumulate_nsi(p, p->d_hist, p->d_state, grads, resid, vel, mom, ratios, counts, keys, s);
+        // ahead of the single-kernel tail the first pass lets its successor be scheduled as its CTAs leave:
+        // that kernel touches only plan tables and the ratios before its own dependency wait
+        e = launch_accumulate_nsi(p, p->d_hist, p->d_state, grads, resid, vel, mom, ratios, counts, keys, s, false,
+                                  fused);
     if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
     LaneTable lanes{};
     lanes.l[0] = Lane{keys, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid, idx, val};

@@ -152,10 +152,13 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
             int64_t ntr_max = kItemElems / band;
             int64_t n_items = ceil_div64(L.TR, ntr_max);
             int64_t ntr = ceil_div64(L.TR, n_items);
-            // multiples of 8 tile rows keep every item start 16-byte aligned in both arenas
-            // (8 bfloat16 or 4 binary32 elements): 128-bit loads and bulk copies
-            if (round_up64(ntr, 8) <= ntr_max) ntr = round_up64(ntr, 8);
-            else if (ntr_max >= 8) ntr = ntr_max & ~(int64_t)7;
+            // every item start must be 16-byte aligned in both arenas (8 bfloat16 or 4 binary32 elements)
+            // for 128-bit loads and bulk copies: a band of a multiple of 8 elements gives that for any
+            // number of tile rows, otherwise multiples of 8 tile rows do
+            if (band % 8 != 0) {
+                if (round_up64(ntr, 8) <= ntr_max) ntr = round_up64(ntr, 8);
+                else if (ntr_max >= 8) ntr = ntr_max & ~(int64_t)7;
+            }
             for (int64_t tr0 = 0; tr0 < L.TR; tr0 += ntr) {
                 Item it{l, (int32_t)tr0, (int32_t)std::min<int64_t>(ntr, L.TR - tr0), 0, L.TC};
                 p->items.push_back(it);
@@ -242,9 +245,12 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
         p->item_path[i] = bulk ? 0 : 1;
         p->item_pitch[i] = d.P;
         p->item_flags[i] = d.flags;
-        cost[i] = (double)d.R * d.W + 512.0;  // elements + a fixed cost per item
-        // the first item of a layer pays for the previous layer's histogram flush in its CTA
-        if (i > 0 && p->items[i - 1].layer != it.layer) cost[i] += 6000.0;
+        // elements + a fixed cost per item: an item takes a CTA about one memory round trip under load
+        // whatever its size (measured: 3.7 us for 4400 elements, hardly less for 3000), the streaming of
+        // its bytes adds to that
+        cost[i] = (double)d.R * d.W + 8000.0;
+        // the first item of a layer pays for the previous layer's histogram flush in its CTA (about 2.5 us)
+        if (i > 0 && p->items[i - 1].layer != it.layer) cost[i] += 12000.0;
     }
 
     // --- each kernel's items in layer order, split into contiguous ranges of equal cost, one

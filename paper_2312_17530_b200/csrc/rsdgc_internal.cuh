@@ -33,7 +33,7 @@ constexpr uint32_t kTakeNone = 0xFFFFFFFFu;  // prefix / threshold marker: keep 
 // the single-kernel selection + pack for plans of small layers (tail.cu)
 constexpr int kTailCluster = 8;        // CTAs per thread-block cluster = slices a layer may have
 constexpr int kTailKeysBig = 32768;    // keys a CTA of the cluster variant holds in shared memory
-constexpr int kTailThreadsBig = 1024;
+constexpr int kTailThreadsBig = 512;
 constexpr int kTailKeysSmall = 8192;   // layers up to this many tiles take the one-CTA variant
 constexpr int kTailThreadsSmall = 256;
 

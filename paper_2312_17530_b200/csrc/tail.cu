@@ -39,6 +39,7 @@ struct TailShared {
     unsigned int res[2];                     // leader: what the level resolved (bin, remaining)
     unsigned int cnt[kTailCluster][2];       // leader: per rank, keys above the threshold / equal to it
     unsigned int warp_cnt[NT / 32][2];       // per warp of this CTA: the same counts over the warp's keys
+    unsigned int warp_pre[NT / 32 + 1][2];   // the counts of the warps before each warp; last entry: the CTA's totals
     long long idx_off, val_off;              // payload offsets of the layer
 };
 
@@ -196,8 +197,8 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
             remaining = res[1];
         }
     }
-    const uint32_t T = prefix;                 // the threshold key, or kTakeNone
-    const long long e = (long long)remaining;  // keys equal to T that are taken, lowest tile index first
+    const uint32_t T = prefix;       // the threshold key, or kTakeNone
+    const int e = (int)remaining;    // keys equal to T that are taken, lowest tile index first
 
     // ---- per warp, per CTA, per layer: how many keys lie above T and how many equal it
     // warp w owns the keys [w * per_warp, (w + 1) * per_warp) of the slice
@@ -224,28 +225,42 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
         }
     }
     __syncthreads();
-    long long gt_before = 0, eq_before = 0, cta_gt = 0, cta_eq = 0;  // in the warps before this one / in the CTA
-#pragma unroll 1
-    for (int w = 0; w < NW; ++w) {
-        if (w < warp) {
-            gt_before += sh.warp_cnt[w][0];
-            eq_before += sh.warp_cnt[w][1];
+    // exclusive prefix of the warps' counts (warp 0, by shuffles); the CTA's totals end up in entry NW
+    if (warp == 0) {
+        unsigned int a = (lane < NW) ? sh.warp_cnt[lane][0] : 0u, b = (lane < NW) ? sh.warp_cnt[lane][1] : 0u;
+        const unsigned int a0 = a, b0 = b;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned int ya = __shfl_up_sync(0xFFFFFFFFu, a, d), yb = __shfl_up_sync(0xFFFFFFFFu, b, d);
+            if (lane >= d) {
+                a += ya;
+                b += yb;
+            }
         }
-        cta_gt += sh.warp_cnt[w][0];
-        cta_eq += sh.warp_cnt[w][1];
+        if (lane < NW) {
+            sh.warp_pre[lane][0] = a - a0;
+            sh.warp_pre[lane][1] = b - b0;
+        }
+        if (lane == NW - 1) {
+            sh.warp_pre[NW][0] = a;
+            sh.warp_pre[NW][1] = b;
+        }
     }
+    __syncthreads();
+    int gt_before = (int)sh.warp_pre[warp][0], eq_before = (int)sh.warp_pre[warp][1];  // in the warps before this one
+    const int cta_gt = (int)sh.warp_pre[NW][0], cta_eq = (int)sh.warp_pre[NW][1];
     if (active && tid == 0) {
         unsigned int *c = at_leader(&sh.cnt[0][0]);
         c[2 * sl.rank] = (unsigned int)cta_gt;
         c[2 * sl.rank + 1] = (unsigned int)cta_eq;
     }
     sync_all();
-    long long lay_gt0 = 0, lay_eq0 = 0;  // keys above / equal in the slices of the layer before this one
+    int lay_gt0 = 0, lay_eq0 = 0;  // keys above / equal in the slices of the layer before this one (< K_l < 2^31)
     if (active) {
         const unsigned int *c = at_leader(&sh.cnt[0][0]);
         for (int r = 0; r < sl.rank; ++r) {
-            lay_gt0 += c[2 * r];
-            lay_eq0 += c[2 * r + 1];
+            lay_gt0 += (int)c[2 * r];
+            lay_eq0 += (int)c[2 * r + 1];
         }
     }
     sync_all();  // nothing of another CTA's shared memory is touched from here on
@@ -288,10 +303,10 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
         const unsigned int lower = (1u << lane) - 1u;
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const long long g_rank = gt_before + __popc(ma[u] & lower), e_rank = eq_before + __popc(me[u] & lower);
+            const int g_rank = gt_before + __popc(ma[u] & lower), e_rank = eq_before + __popc(me[u] & lower);
             const bool above = (ma[u] >> lane) & 1u, equal = (me[u] >> lane) & 1u;
             if (above || (equal && e_rank < e)) {
-                const long long s = idx_off + g_rank + min(e_rank, e);
+                const long long s = idx_off + (g_rank + min(e_rank, e));
                 if (s < idx_cap) idx[s] = sl.start + base + u * 32 + lane;
             }
             gt_before += __popc(ma[u]);

@@ -110,10 +110,17 @@ def test_plan_offsets_and_worklist_cover_every_tile_once(lib, net, dtype):
             continue
         assert (np.diff(sel[:, 6]) >= 0).all()
         cost = np.zeros(grids[path])
-        for l, tr0, ntr, tc0, ntc, _, cta, _, _ in sel.tolist():
+        all_items = items.tolist()
+        for k, (l, tr0, ntr, tc0, ntc, pa, cta, _, _) in enumerate(all_items):
+            if pa != path:
+                continue
             r, c, nh, nw = shapes[l]
-            cost[cta] += (min(r, (tr0 + ntr) * nh) - tr0 * nh) * (min(c, (tc0 + ntc) * nw) - tc0 * nw) + 512
-        assert cost.max() <= cost.sum() / len(cost) + 4400 + 512 + 1
+            # the plan's cost model: elements + a fixed cost per item + the flush a CTA pays when it enters a
+            # new layer
+            cost[cta] += (min(r, (tr0 + ntr) * nh) - tr0 * nh) * (min(c, (tc0 + ntc) * nw) - tc0 * nw) + 8000
+            if k > 0 and all_items[k - 1][0] != l:
+                cost[cta] += 12000
+        assert cost.max() <= cost.sum() / len(cost) + 4400 + 8000 + 12000 + 1
     if net not in ("odd", "wide_tiles"):
         assert (items[:, 5] == 0).mean() > 0.99       # the usual shapes go to the bulk-copy kernel
 
