@@ -74,6 +74,8 @@ typedef enum {
 #define RSDGC_STATUS_NONFINITE 1u         /* some indicator was NaN/Inf (ranked first as +Inf)  */
 #define RSDGC_STATUS_PAYLOAD_OVERFLOW 2u  /* idx/val capacity too small; excess tiles not sent   */
 #define RSDGC_STATUS_TIMEOUT 4u           /* a bounded on-chip wait gave up; results are invalid  */
+#define RSDGC_STATUS_BOUNDS 8u            /* bounds-checked builds (RSDGC_DEBUG) only: a kernel    */
+                                          /* formed an index outside its buffers; access skipped  */
 
 typedef struct {
     int64_t rows, cols; /* row-major 2-D view of the layer (Sec. III-C)            */

@@ -11,7 +11,8 @@ import os
 from typing import List, Optional, Sequence, Tuple
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "librsdgc_b200.so")
+# RSDGC_LIBRARY selects another build of the same library (e.g. the bounds-checked one)
+LIB_PATH = os.environ.get("RSDGC_LIBRARY") or os.path.join(_HERE, "librsdgc_b200.so")
 
 RSDGC_F32, RSDGC_BF16 = 0, 1
 KEEP_AT_LEAST_ONE = 1
@@ -19,7 +20,7 @@ NO_BULK_COPY = 2
 MOMENTUM = 4
 PAYLOAD_BF16 = 8
 NO_FUSED_TAIL = 16
-STATUS_NONFINITE, STATUS_PAYLOAD_OVERFLOW, STATUS_TIMEOUT = 1, 2, 4
+STATUS_NONFINITE, STATUS_PAYLOAD_OVERFLOW, STATUS_TIMEOUT, STATUS_BOUNDS = 1, 2, 4, 8
 OK, ERR_INVALID, ERR_ALIGNMENT, ERR_CAPACITY, ERR_CUDA, ERR_NOMEM = 0, -1, -2, -3, -4, -5
 
 EXPORTS = [

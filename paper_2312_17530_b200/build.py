@@ -21,15 +21,27 @@ def _stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_library(force: bool = False, verbose: bool = False) -> str:
-    """nvcc -> librsdgc_b200.so next to this file; returns its path."""
+DEBUG_LIB_PATH = os.path.join(_HERE, "librsdgc_b200_debug.so")
+
+
+def build_library(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    """nvcc -> librsdgc_b200.so next to this file; returns its path.  ``debug``: the bounds-checked
+    build (-DRSDGC_DEBUG: every index the kernels form is tested against the plan's extents, failures
+    raise RSDGC_STATUS_BOUNDS and skip the access) -> librsdgc_b200_debug.so; load it by pointing the
+    environment variable RSDGC_LIBRARY at it."""
+    if debug:
+        return _compile(DEBUG_LIB_PATH, verbose, ["-DRSDGC_DEBUG"])
     if not force and not _stale():
         return LIB_PATH
+    return _compile(LIB_PATH, verbose, [])
+
+
+def _compile(out_path: str, verbose: bool, extra) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-    tmp = LIB_PATH + ".tmp.%d" % os.getpid()
+    tmp = out_path + ".tmp.%d" % os.getpid()
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC,-Wall", "-shared", "-I", os.path.join(_ROOT, "include"), "-I", CSRC,
-           "-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
+           "-o", tmp] + list(extra) + [os.path.join(CSRC, s) for s in SOURCES]
     # NVTX ranges around the entry points (header-only NVTX 3; RSDGC_NVTX=0 compiles them out)
     if os.environ.get("RSDGC_NVTX", "1") != "0":
         cmd[1:1] = ["-DRSDGC_NVTX"]
@@ -42,9 +54,9 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
         sys.stderr.write(res.stderr)
     if res.returncode != 0:
         raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, out_path)
+    return out_path
 
 
 if __name__ == "__main__":
-    print(build_library(force=True, verbose="-v" in sys.argv))
+    print(build_library(force=True, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -89,6 +89,37 @@ __device__ __forceinline__ void emit_key(float nsi, uint32_t *dst, unsigned int 
     atomicAdd(&hist_smem[key >> kL1Shift], 1u);
 }
 
+// Keys of all tiles of an item none of whose tiles is clipped, for a tile shape known at compile
+// time: two tiles per thread and round, so that the two chains of dependent additions (every sum is
+// sequential by definition) overlap instead of following each other.
+template <int NTHREADS, int HH, int WW>
+__device__ __forceinline__ unsigned int item_tile_keys_fixed(const ItemDev &d, const float *sv,
+                                                             uint32_t *__restrict__ keys, unsigned int *hist_smem,
+                                                             float alpha)
+{
+    const int P = d.P, ntc = d.ntc;
+    const int ntr = d.R / HH;
+    const int ntile = ntr * ntc;
+    uint32_t *kout = keys + d.kbase;
+    unsigned int nonfinite = 0;
+    int t = threadIdx.x;
+    for (; t + NTHREADS < ntile; t += 2 * NTHREADS) {
+        const int ti0 = (ntr == 1) ? 0 : fast_div(t, d.inv_ntc), ti1 = (ntr == 1) ? 0 : fast_div(t + NTHREADS, d.inv_ntc);
+        const int tj0 = t - ti0 * ntc, tj1 = t + NTHREADS - ti1 * ntc;
+        const float nsi0 = tile_nsi_fixed<HH, WW>(sv + (ti0 * HH) * P + tj0 * WW, P, alpha);
+        const float nsi1 = tile_nsi_fixed<HH, WW>(sv + (ti1 * HH) * P + tj1 * WW, P, alpha);
+        emit_key(nsi0, kout + ti0 * d.TC + tj0, hist_smem, nonfinite);
+        emit_key(nsi1, kout + ti1 * d.TC + tj1, hist_smem, nonfinite);
+    }
+    if (t < ntile) {
+        const int ti = (ntr == 1) ? 0 : fast_div(t, d.inv_ntc);
+        const int tj = t - ti * ntc;
+        emit_key(tile_nsi_fixed<HH, WW>(sv + (ti * HH) * P + tj * WW, P, alpha), kout + ti * d.TC + tj, hist_smem,
+                 nonfinite);
+    }
+    return nonfinite;
+}
+
 // Keys of all tiles of one item from its v block in shared memory (row pitch d.P).
 // Returns the number of non-finite indicators this thread saw.
 template <int NTHREADS>
@@ -96,6 +127,10 @@ __device__ __forceinline__ unsigned int item_tile_keys(const ItemDev &d, const f
                                                        unsigned int *hist_smem, float alpha)
 {
     const int nh = d.nh, nw = d.nw, R = d.R, W = d.W, P = d.P;
+    if (d.flags & kItemNoClip) {  // the two usual shapes, every tile whole
+        if (nh == 3 && nw == 3) return item_tile_keys_fixed<NTHREADS, 3, 3>(d, sv, keys, hist_smem, alpha);
+        if (nh == 1 && nw == 9) return item_tile_keys_fixed<NTHREADS, 1, 9>(d, sv, keys, hist_smem, alpha);
+    }
     const int ntr = (R + nh - 1) / nh;
     const int ntc = d.ntc;
     const int ntile = ntr * ntc;
@@ -241,6 +276,24 @@ __device__ __forceinline__ ItemDev load_item(const ItemDev *items, int i)
     u.q[3] = __ldg(p + 3);
     return u.d;
 }
+
+#ifdef RSDGC_DEBUG
+// Bounds-checked build: every item of the CTA's range must lie inside the arenas, the key array and
+// the layer table; called by all threads, the same answer in every thread.
+template <int NTHREADS>
+__device__ bool debug_items_ok(const ItemDev *items, int begin, int end, StatusDev *status)
+{
+    bool ok = begin >= 0 && end <= status->n_items;
+    for (int i = begin + (int)threadIdx.x; ok && i < end; i += NTHREADS) {
+        const ItemDev d = load_item(items, i);
+        const int ntr = (d.R + d.nh - 1) / d.nh;
+        ok = d.R >= 1 && d.W >= 1 && d.gbase >= 0 && d.gbase + (long long)(d.R - 1) * d.cols + d.W <= status->arena_elems &&
+             d.kbase >= 0 && d.kbase + (long long)(ntr - 1) * d.TC + d.ntc <= status->keys_len && d.layer >= 0 &&
+             d.layer < status->n_layers && (long long)d.R * d.P <= kItemElems;  // (every variant's stage holds at most this)
+    }
+    return !__syncthreads_or(!debug_in_bounds(ok, status));
+}
+#endif
 
 // Momentum correction (Eq. 12, first line): u = m * u_prev + g, product then sum, each rounded.
 __device__ __forceinline__ float momentum_step(float m, float u_prev, float g)
@@ -445,6 +498,9 @@ k1_reg(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     if (begin >= end) return;
     const int tid = threadIdx.x;
+#ifdef RSDGC_DEBUG
+    if (!debug_items_ok<kThreads>(items, begin, end, status)) return;
+#endif
     for (int b = tid; b < kL1Bins; b += kThreads) sh.hist[b] = 0;
     unsigned int nonfinite = 0;
 
@@ -497,17 +553,30 @@ k1_reg(const G *__restrict__ grads, float *__restrict__ resid, float *__restrict
 constexpr int kBulkThreads = RSDGC_BULK_THREADS;
 constexpr int kBulkCtasPerSm = RSDGC_BULK_CTAS;
 constexpr int kBulkCtasPerSmMomentum = 2;  // a third block per stage: 110 KB of shared memory per CTA
-constexpr int kStages = RSDGC_BULK_STAGES;  // shared-memory stages; loads run kStages - 1 items ahead
-constexpr int kLookahead = kStages - 1;
+// Shared-memory stages and elements per stage of a (gradient type, momentum) variant; loads run
+// kStages - 1 items ahead.  The pass is bound by the bytes it keeps in flight: with 2-byte gradients an
+// item carries a quarter fewer bytes, so that variant takes three smaller stages (two items ahead) in
+// the same shared memory instead of two.  The plan cuts its items to bulk_item_elems().
+template <typename G, bool MOM>
+struct BulkCfg {
+    static constexpr int kStages = RSDGC_BULK_STAGES;
+    static constexpr int kElems = kItemElems;
+};
+template <>
+struct BulkCfg<__nv_bfloat16, false> {
+    static constexpr int kStages = RSDGC_BF16_STAGES;
+    static constexpr int kElems = kItemElemsBf16;
+};
 constexpr unsigned int kSpinLimit = 1u << 22;  // bounded mbarrier waits
 constexpr int kOverlapPrev = 1;  // k1_bulk: the previous kernel in the stream is another worker's first pass
 constexpr int kOverlapNext = 2;  // k1_bulk: the next one is
 
-template <bool MOM>
+template <typename G, bool MOM>
 struct K1BulkShared {
-    __align__(128) float r[kStages][kItemElems];  // residual block; becomes v in place
-    __align__(128) float g[kStages][kItemElems];  // gradient block (binary32 or bfloat16 packed)
-    __align__(128) float u[MOM ? kStages : 1][MOM ? kItemElems : 4];  // velocity block, updated in place
+    static constexpr int kStages = BulkCfg<G, MOM>::kStages, kElems = BulkCfg<G, MOM>::kElems;
+    __align__(128) float r[kStages][kElems];  // residual block; becomes v in place
+    __align__(128) G g[kStages][kElems];      // gradient block
+    __align__(128) float u[MOM ? kStages : 1][MOM ? kElems : 4];  // velocity block, updated in place
     unsigned int hist[kL1Bins];
     __align__(8) unsigned long long full[kStages];  // mbarriers: stage loaded
     FlushShared fs;
@@ -617,7 +686,8 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
         int overlap)
 {
     extern __shared__ __align__(128) unsigned char k1_bulk_smem_raw[];
-    K1BulkShared<MOM> &sh = *reinterpret_cast<K1BulkShared<MOM> *>(k1_bulk_smem_raw);
+    K1BulkShared<G, MOM> &sh = *reinterpret_cast<K1BulkShared<G, MOM> *>(k1_bulk_smem_raw);
+    constexpr int kStages = BulkCfg<G, MOM>::kStages, kLookahead = kStages - 1;
     const int begin = cta_begin[blockIdx.x], end = cta_begin[blockIdx.x + 1];
     const bool wait_late = (overlap & kOverlapPrev) != 0;
     if (begin >= end) {
@@ -625,6 +695,12 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
         return;
     }
     const int tid = threadIdx.x;
+#ifdef RSDGC_DEBUG
+    if (!debug_items_ok<kBulkThreads>(items, begin, end, status)) {  // nothing is loaded or stored
+        if (wait_late) grid_dependency_wait();
+        return;
+    }
+#endif
     for (int b = tid; b < kL1Bins; b += kBulkThreads) sh.hist[b] = 0;
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) mbar_init(&sh.full[s], 1);
@@ -647,7 +723,7 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
     if (tid == 0) {
         for (int j = 0; j < kLookahead && begin + j < end; ++j) {
             const ItemDev d = load_item(items, begin + j);
-            bulk_issue_item<G, MOM>(d, grads, resid, vel, sh.r[j % kStages], reinterpret_cast<G *>(sh.g[j % kStages]),
+            bulk_issue_item<G, MOM>(d, grads, resid, vel, sh.r[j % kStages], sh.g[j % kStages],
                                     sh.u[MOM ? j % kStages : 0], &sh.full[j % kStages]);
         }
     }
@@ -673,7 +749,7 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
 
         // ---- wait for this item's blocks (bounded), form v in place
         float *sr = sh.r[stage];
-        const G *sg = reinterpret_cast<const G *>(sh.g[stage]);
+        const G *sg = sh.g[stage];
         float *su = sh.u[MOM ? stage : 0];
         const int nb = bulk_elems<G>(cur);
         bool arrived = true;
@@ -717,11 +793,13 @@ k1_bulk(const G *__restrict__ grads, float *__restrict__ resid, float *__restric
                 // ---- producer: item it + kLookahead goes into the stage item it - 1 used.  Every
                 // thread finished that item's tiles before the barrier above, and its bulk store
                 // has finished reading shared memory once only the store just committed is pending.
+                // (Issued earlier, before this item is waited for, so that a CTA has two items in flight:
+                // measured 7 % slower; the memory system is already saturated by one item per CTA.)
                 if (it + kLookahead < end) {
                     bulk_wait_read<1>();
                     const int ps = (rel + kLookahead) % kStages;
-                    bulk_issue_item<G, MOM>(ahead, grads, resid, vel, sh.r[ps], reinterpret_cast<G *>(sh.g[ps]),
-                                            sh.u[MOM ? ps : 0], &sh.full[ps]);
+                    bulk_issue_item<G, MOM>(ahead, grads, resid, vel, sh.r[ps], sh.g[ps], sh.u[MOM ? ps : 0],
+                                            &sh.full[ps]);
                     if (it + 1 + kLookahead < end) ahead = load_item(items, it + 1 + kLookahead);
                 }
             }
@@ -804,10 +882,10 @@ static cudaError_t configure_once()
         if (e == cudaSuccess) e = allow_smem(k1_reg<float, true>, sizeof(K1RegShared));
         if (e == cudaSuccess) e = allow_smem(k1_reg<__nv_bfloat16, false>, sizeof(K1RegShared));
         if (e == cudaSuccess) e = allow_smem(k1_reg<__nv_bfloat16, true>, sizeof(K1RegShared));
-        if (e == cudaSuccess) e = allow_smem(k1_bulk<float, false>, sizeof(K1BulkShared<false>));
-        if (e == cudaSuccess) e = allow_smem(k1_bulk<float, true>, sizeof(K1BulkShared<true>));
-        if (e == cudaSuccess) e = allow_smem(k1_bulk<__nv_bfloat16, false>, sizeof(K1BulkShared<false>));
-        if (e == cudaSuccess) e = allow_smem(k1_bulk<__nv_bfloat16, true>, sizeof(K1BulkShared<true>));
+        if (e == cudaSuccess) e = allow_smem(k1_bulk<float, false>, sizeof(K1BulkShared<float, false>));
+        if (e == cudaSuccess) e = allow_smem(k1_bulk<float, true>, sizeof(K1BulkShared<float, true>));
+        if (e == cudaSuccess) e = allow_smem(k1_bulk<__nv_bfloat16, false>, sizeof(K1BulkShared<__nv_bfloat16, false>));
+        if (e == cudaSuccess) e = allow_smem(k1_bulk<__nv_bfloat16, true>, sizeof(K1BulkShared<__nv_bfloat16, true>));
         return e;
     }();
     if (tracked) done[dev] = (result == cudaSuccess);
@@ -815,6 +893,13 @@ static cudaError_t configure_once()
 }
 
 int k1_bulk_ctas_per_sm(bool momentum) { return momentum ? kBulkCtasPerSmMomentum : kBulkCtasPerSm; }
+
+// Elements an item of the first pass may hold for this gradient type (one stage of the variant's
+// shared memory).
+int bulk_item_elems(int dtype, bool momentum)
+{
+    return (dtype == RSDGC_BF16 && !momentum) ? BulkCfg<__nv_bfloat16, false>::kElems : kItemElems;
+}
 
 // Resident CTAs per SM of the register-staged kernel on the current device.
 int k1_reg_ctas_per_sm(int dtype, bool momentum)
@@ -848,7 +933,7 @@ static cudaError_t launch_k1_typed(rsdgc_plan *p, uint32_t *hist, LayerState *st
         cudaLaunchConfig_t cfg = {};
         cfg.gridDim = dim3((unsigned)p->grid_bulk);
         cfg.blockDim = dim3(kBulkThreads);
-        cfg.dynamicSmemBytes = sizeof(K1BulkShared<MOM>);
+        cfg.dynamicSmemBytes = sizeof(K1BulkShared<G, MOM>);
         cfg.stream = s;
         cudaLaunchAttribute attr[1];
         attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -101,7 +101,7 @@ __device__ __forceinline__ void refine_flush(RefineShared &sh, const Lane &ln, c
 template <int LEVEL>
 __global__ void __launch_bounds__(kThreads, kRefineCtasPerSm)
 k_refine(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
-         const Chunk *__restrict__ chunks, int n_chunks_all)
+         const Chunk *__restrict__ chunks, int n_chunks_all, StatusDev *status)
 {
     __shared__ RefineShared sh;
     const Lane &ln = lanes.l[blockIdx.y];
@@ -130,6 +130,9 @@ k_refine(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ l
         }
         ++n_done;
         if (prefix == kTakeNone) continue;
+        if (!RSDGC_CHECKED(chunk_id < status->n_chunks && c.layer < status->n_layers && c.start >= 0 && c.n >= 0 &&
+                               layers[c.layer].tile_off + c.start + c.n <= status->keys_len, status))
+            continue;
         const uint32_t *kp = keys + layers[c.layer].tile_off + c.start;
         const int nvec = c.n >> 2;
         for (int base = 0; base < nvec; base += kThreads * kKeyVecBatch) {
@@ -186,7 +189,8 @@ k_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ la
     grid_dependency_launch_next();
     const uint32_t T = st.T;
     unsigned int gt = 0, eq = 0;
-    {
+    if (RSDGC_CHECKED((int)blockIdx.x < status->n_chunks && c.layer < status->n_layers && c.start >= 0 && c.n >= 0 &&
+                          L.tile_off + c.start + c.n <= status->keys_len, status)) {
         // one code byte per 128-bit word of keys (bit c: key c above T, bit 4 + c: key c equal
         // to T) is left for k_mark, which then needs no second look at the keys
         const uint32_t *kp = keys + L.tile_off + c.start;
@@ -300,7 +304,7 @@ struct MarkShared {
 
 __global__ void __launch_bounds__(kThreads)
 k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
-       const Chunk *__restrict__ chunks, long long idx_cap)
+       const Chunk *__restrict__ chunks, long long idx_cap, StatusDev *status)
 {
     __shared__ MarkShared sh;
     const Lane &ln = lanes.l[blockIdx.y];
@@ -314,6 +318,9 @@ k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     grid_dependency_launch_next();
     const LayerState st = state[c.layer];
     if (st.k == 0) return;
+    if (!RSDGC_CHECKED((int)blockIdx.x < status->n_chunks && c.layer < status->n_layers &&
+                           layers[c.layer].tile_off + c.start + c.n <= status->keys_len, status))
+        return;
     const uint2 base = chunk_cnt[blockIdx.x];  // tiles above T / equal to T in earlier chunks
     // equal keys of this chunk that are still taken: those with layer-wide equal-rank < e
     const long long eq_room = max(0ll, (long long)st.e - (long long)base.y);
@@ -397,7 +404,7 @@ constexpr int kCopyBatch = RSDGC_COPY_BATCH;
 template <bool BF16VAL>
 __global__ void __launch_bounds__(kThreads)
 k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *__restrict__ layers, int n_layers,
-         long long idx_cap, long long val_cap)
+         long long idx_cap, long long val_cap, StatusDev *status)
 {
     extern __shared__ __align__(16) unsigned char gather_smem_raw[];
     long long *val_off = reinterpret_cast<long long *>(gather_smem_raw);  // n_layers + 1
@@ -480,6 +487,7 @@ k_gather(const __grid_constant__ LaneTable lanes, int n_lanes, const LayerDev *_
                     divmod_small(el[u], L.nw, &a, &b);
                     const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
                     if (i < L.rows && jj < L.cols) ga[u] = L.elem_off + i * L.cols + jj;
+                    if (!RSDGC_CHECKED(tile[u] < L.K && ga[u] < status->arena_elems, status)) ga[u] = -1, vo[u] = -1;
                 }
             }
             if (BF16VAL) {  // q = bfloat16(v) is sent, v - q stays (exact in binary32)
@@ -555,24 +563,25 @@ static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n
                                           : std::max(1, std::min(n_chunks, resident / n_lanes))),
                            (unsigned)n_lanes);
     if (e == cudaSuccess)
-        e = launch_chained(k_refine<2>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks);
+        e = launch_chained(k_refine<2>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks, p->d_status);
     RSDGC_MARK(2);
     if (e == cudaSuccess)
-        e = launch_chained(k_refine<3>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks);
+        e = launch_chained(k_refine<3>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks, p->d_status);
     RSDGC_MARK(2);
     if (e == cudaSuccess)
         e = launch_chained(k_count, grid, 0, s, lanes, p->d_layers, p->d_chunks, p->n_layers, (long long)idx_cap,
                            (long long)val_cap, p->d_status);
     RSDGC_MARK(2);
-    if (e == cudaSuccess) e = launch_chained(k_mark, grid, 0, s, lanes, p->d_layers, p->d_chunks, (long long)idx_cap);
+    if (e == cudaSuccess)
+        e = launch_chained(k_mark, grid, 0, s, lanes, p->d_layers, p->d_chunks, (long long)idx_cap, p->d_status);
     RSDGC_MARK(2);
     const size_t gather_smem = (size_t)(2 * p->n_layers + 1) * sizeof(long long);  // val_off, idx_off tables
     if (e == cudaSuccess)
         e = (p->flags & RSDGC_PAYLOAD_BF16)
                 ? launch_chained(k_gather<true>, grid_gather, gather_smem, s, lanes, n_lanes, p->d_layers, p->n_layers,
-                                 (long long)idx_cap, (long long)val_cap)
+                                 (long long)idx_cap, (long long)val_cap, p->d_status)
                 : launch_chained(k_gather<false>, grid_gather, gather_smem, s, lanes, n_lanes, p->d_layers,
-                                 p->n_layers, (long long)idx_cap, (long long)val_cap);
+                                 p->n_layers, (long long)idx_cap, (long long)val_cap, p->d_status);
     RSDGC_MARK(2);
 #undef RSDGC_MARK
     count_launch(5);

@@ -19,7 +19,8 @@ struct CooShared {
 
 __global__ void __launch_bounds__(kThreads)
 k_payload_to_coo(const int32_t *__restrict__ idx, const int32_t *__restrict__ counts,
-                 const LayerDev *__restrict__ layers, int n_layers, long long *__restrict__ coo, long long coo_cap)
+                 const LayerDev *__restrict__ layers, int n_layers, long long *__restrict__ coo, long long coo_cap,
+                 StatusDev *status)
 {
     __shared__ CooShared sh;
     const int tid = threadIdx.x;
@@ -75,6 +76,7 @@ k_payload_to_coo(const int32_t *__restrict__ idx, const int32_t *__restrict__ co
                 const int a = el / L.nw, b = el - a * L.nw;
                 const long long i = (long long)tr * L.nh + a, jj = (long long)tc * L.nw + b;
                 if (i < L.rows && jj < L.cols) pos = L.elem_off + i * L.cols + jj;
+                if (!RSDGC_CHECKED(pos < status->arena_elems, status)) pos = -1;
             }
             coo[j] = pos;
         }
@@ -84,7 +86,7 @@ k_payload_to_coo(const int32_t *__restrict__ idx, const int32_t *__restrict__ co
 cudaError_t launch_payload_to_coo(rsdgc_plan *p, const int32_t *idx, const int32_t *counts, long long *coo,
                                   long long coo_cap, cudaStream_t s)
 {
-    k_payload_to_coo<<<p->n_sm * 4, kThreads, 0, s>>>(idx, counts, p->d_layers, p->n_layers, coo, coo_cap);
+    k_payload_to_coo<<<p->n_sm * 4, kThreads, 0, s>>>(idx, counts, p->d_layers, p->n_layers, coo, coo_cap, p->d_status);
     count_launch(1);
     return cudaGetLastError();
 }

@@ -101,13 +101,16 @@ __device__ __forceinline__ void zero_chunk(float *__restrict__ dense, const Laye
 template <bool ASSIGN, bool BF16VAL>
 __global__ void __launch_bounds__(kThreads)
 k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restrict__ layers,
-             const Chunk *__restrict__ chunks, float scale, float *__restrict__ dense)
+             const Chunk *__restrict__ chunks, float scale, float *__restrict__ dense, StatusDev *status)
 {
     __shared__ DecompressShared sh;
     const Chunk c = chunks[blockIdx.x];
     const LayerDev L = layers[c.layer];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int W = wp.n_workers;
+    if (!RSDGC_CHECKED((int)blockIdx.x < status->n_chunks && c.layer >= 0 && c.layer < status->n_layers && c.start >= 0 &&
+                           c.start + c.n <= L.K && L.elem_off + L.rows * L.cols <= status->arena_elems, status))
+        return;
     if (ASSIGN) zero_chunk(dense, L, c);  // made visible to the whole CTA by the barrier below
 
     // ---- per worker (one warp each, round-robin): payload offsets of this layer = sums of the
@@ -187,7 +190,8 @@ k_decompress(const __grid_constant__ WorkerPayloads wp, const LayerDev *__restri
                         divmod_small(el, nw, &a, &b);
                         const long long g0 = sh.gbase[q];
                         const int thw = sh.hw[q];
-                        if (g0 >= 0 && a < (thw >> 16) && b < (thw & 0xFFFF)) {
+                        if (g0 >= 0 && a < (thw >> 16) && b < (thw & 0xFFFF) &&
+                            RSDGC_CHECKED(g0 + a * cols + b < status->arena_elems, status)) {
                             ga[u] = g0 + a * cols + b;
                             pv[u] = BF16VAL ? __bfloat162float(val16[v0 + j]) : __ldg(val + v0 + j);
                         }
@@ -213,7 +217,8 @@ cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const
     const int n_chunks = (int)p->chunks.size();
     const bool half = (p->flags & RSDGC_PAYLOAD_BF16) != 0;
     if (assign && n_workers == 0) {  // nothing was sent: the result is all +0
-        k_decompress<true, false><<<n_chunks, kThreads, 0, s>>>(WorkerPayloads{}, p->d_layers, p->d_chunks, scale, dense);
+        k_decompress<true, false><<<n_chunks, kThreads, 0, s>>>(WorkerPayloads{}, p->d_layers, p->d_chunks, scale, dense,
+                                                                p->d_status);
         count_launch(1);
     }
     for (int w0 = 0; w0 < n_workers; w0 += kMaxWorkersPerLaunch) {
@@ -229,7 +234,7 @@ cudaError_t launch_decompress(rsdgc_plan *p, int n_workers, const int32_t *const
         const bool zero_first = assign && w0 == 0;
         auto kernel = zero_first ? (half ? k_decompress<true, true> : k_decompress<true, false>)
                                  : (half ? k_decompress<false, true> : k_decompress<false, false>);
-        kernel<<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense);
+        kernel<<<n_chunks, kThreads, 0, s>>>(wp, p->d_layers, p->d_chunks, scale, dense, p->d_status);
         count_launch(1);
     }
     return cudaGetLastError();

@@ -68,6 +68,20 @@ __device__ __forceinline__ void find_bin_from_top(const unsigned int *h, unsigne
     __syncthreads();
 }
 
+// Bounds-checked build (-DRSDGC_DEBUG): every index a kernel forms into a caller's buffer or a plan
+// table is tested against the extents recorded in the status block; a failure raises
+// RSDGC_STATUS_BOUNDS and the access is skipped.  In the normal build the test is not compiled.
+#ifdef RSDGC_DEBUG
+__device__ __forceinline__ bool debug_in_bounds(bool ok, StatusDev *st)
+{
+    if (!ok) atomicOr(&st->flags, RSDGC_STATUS_BOUNDS);
+    return ok;
+}
+#define RSDGC_CHECKED(cond, st) debug_in_bounds((cond), (st))
+#else
+#define RSDGC_CHECKED(cond, st) true
+#endif
+
 // Programmatic dependent launch: a kernel launched with the "programmatic stream
 // serialization" attribute may start while its predecessor in the stream is still draining.
 // grid_dependency_wait() returns once the predecessor has completed and its writes are visible;

@@ -125,6 +125,7 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
     p->chunks.clear();
     p->echunks.clear();
     std::vector<int64_t> chunk_w(n_layers, 0);  // columns of a regular (not last) column chunk
+    const int64_t item_elems = p->item_elems;
     int64_t elem_off = 0, tile_off = 0, total_elems = 0, total_tiles = 0;
     int max_slot = 0;
     for (int l = 0; l < n_layers; ++l) {
@@ -148,8 +149,8 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
 
         // --- accumulate+NSI items: rectangles of tiles holding at most kItemElems elements
         const int64_t band = (int64_t)d.nh * d.cols;  // one full-width row of tiles
-        if (band <= kItemElems) {
-            int64_t ntr_max = kItemElems / band;
+        if (band <= item_elems) {
+            int64_t ntr_max = item_elems / band;
             int64_t n_items = ceil_div64(L.TR, ntr_max);
             int64_t ntr = ceil_div64(L.TR, n_items);
             // every item start must be 16-byte aligned in both arenas (8 bfloat16 or 4 binary32 elements)
@@ -164,7 +165,7 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
                 p->items.push_back(it);
             }
         } else {
-            int64_t ntc_max = kItemElems / L.slot;
+            int64_t ntc_max = item_elems / L.slot;
             int64_t n_items = ceil_div64(L.TC, ntc_max);
             int64_t ntc = ceil_div64(L.TC, n_items);
             if (round_up64(ntc, 8) <= ntc_max) ntc = round_up64(ntc, 8);
@@ -174,7 +175,7 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
             // elements keeps every row of the block 16-byte aligned there for both element sizes
             // (neighborhoods of more than 550 elements leave fewer than 8 tile columns per item, so
             // the width itself need not be one)
-            if (round_up64(chunk_w[l], 8) * d.nh <= kItemElems) chunk_w[l] = round_up64(chunk_w[l], 8);
+            if (round_up64(chunk_w[l], 8) * d.nh <= item_elems) chunk_w[l] = round_up64(chunk_w[l], 8);
             for (int64_t tr = 0; tr < L.TR; ++tr)
                 for (int64_t tc0 = 0; tc0 < L.TC; tc0 += ntc) {
                     Item it{l, (int32_t)tr, 1, (int32_t)tc0, (int32_t)std::min<int64_t>(ntc, L.TC - tc0)};
@@ -381,6 +382,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
     p->dtype = grad_dtype;
     p->alpha = alpha;
     p->flags = flags;
+    p->item_elems = bulk_item_elems(grad_dtype, (flags & RSDGC_MOMENTUM) != 0);
 
     if (device >= 0) {
         int n_sm = 0;
@@ -424,6 +426,16 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         if (e == cudaSuccess) e = alloc_zero(&p->d_survivors, (size_t)n_layers);
         if (e == cudaSuccess) e = alloc_zero(&p->d_rstate, 1);
         if (e == cudaSuccess) e = alloc_zero(&p->d_status, 1);
+        if (e == cudaSuccess) {
+            StatusDev st{};
+            st.arena_elems = p->info.arena_elems;
+            st.keys_len = p->info.total_tiles_padded;
+            st.n_layers = n_layers;
+            st.n_chunks = (int)p->chunks.size();
+            st.n_echunks = (int)p->echunks.size();
+            st.n_items = (int)p->items_dev.size();
+            e = cudaMemcpy(p->d_status, &st, sizeof st, cudaMemcpyHostToDevice);
+        }
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
         if (e != cudaSuccess) {
             free_device_tables(p);
@@ -867,7 +879,7 @@ extern "C" int rsdgc_get_status(rsdgc_plan *plan, void *stream, rsdgc_status *ou
     cudaStream_t s = (cudaStream_t)stream;
     StatusDev h{};
     cudaError_t e = cudaMemcpyAsync(&h, plan->d_status, sizeof h, cudaMemcpyDeviceToHost, s);
-    if (e == cudaSuccess) e = cudaMemsetAsync(plan->d_status, 0, sizeof(StatusDev), s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(plan->d_status, 0, kStatusResetBytes, s);
     if (e == cudaSuccess) e = cudaStreamSynchronize(s);
     if (e != cudaSuccess) return cuda_fail(e);
     out_host->flags = h.flags;

@@ -21,7 +21,7 @@ template <int LEVEL>
 __global__ void __launch_bounds__(kThreads)
 k_ratio_level(const float *__restrict__ weights, const LayerDev *__restrict__ layers,
               const EChunk *__restrict__ echunks, int n_echunks, int n_layers, unsigned int *hist,
-              RatioState *rs, long long *survivors, float *ratios, long long n_keep)
+              RatioState *rs, long long *survivors, float *ratios, long long n_keep, StatusDev *status)
 {
     __shared__ RatioShared sh;
     constexpr int NBINS = (LEVEL == 1) ? kL1Bins : (LEVEL == 2 ? kL2Bins : kL3Bins);
@@ -32,7 +32,9 @@ k_ratio_level(const float *__restrict__ weights, const LayerDev *__restrict__ la
     const uint32_t prefix = (LEVEL == 1) ? 0u : rs->prefix;  // bit 31 of |w| is 0
     for (int b = tid; b < NBINS; b += kThreads) sh.hist[b] = 0;
     __syncthreads();
-    if (prefix != kTakeNone) {
+    if (prefix != kTakeNone &&
+        RSDGC_CHECKED((int)blockIdx.x < status->n_echunks && c.layer >= 0 && c.layer < status->n_layers && c.start >= 0 &&
+                          layers[c.layer].elem_off + c.start + c.n <= status->arena_elems, status)) {
         const uint32_t *wp = reinterpret_cast<const uint32_t *>(weights) + layers[c.layer].elem_off + c.start;
         const int nvec = c.n >> 2;  // layer starts and chunk starts are multiples of 4 elements
         constexpr int BATCH = 8;
@@ -172,11 +174,11 @@ cudaError_t launch_update_ratios(rsdgc_plan *p, const float *weights, long long 
 {
     const int n = (int)p->echunks.size();
     k_ratio_level<1><<<n, kThreads, 0, s>>>(weights, p->d_layers, p->d_echunks, n, p->n_layers, p->d_hist,
-                                            p->d_rstate, p->d_survivors, ratios, n_keep);
+                                            p->d_rstate, p->d_survivors, ratios, n_keep, p->d_status);
     k_ratio_level<2><<<n, kThreads, 0, s>>>(weights, p->d_layers, p->d_echunks, n, p->n_layers, p->d_hist,
-                                            p->d_rstate, p->d_survivors, ratios, n_keep);
+                                            p->d_rstate, p->d_survivors, ratios, n_keep, p->d_status);
     k_ratio_level<3><<<n, kThreads, 0, s>>>(weights, p->d_layers, p->d_echunks, n, p->n_layers, p->d_hist,
-                                            p->d_rstate, p->d_survivors, ratios, n_keep);
+                                            p->d_rstate, p->d_survivors, ratios, n_keep, p->d_status);
     count_launch(3);
     return cudaGetLastError();
 }

@@ -15,7 +15,15 @@ constexpr int kThreads = 256;        // threads per CTA, every kernel
 #ifndef RSDGC_ITEM_ELEMS
 #define RSDGC_ITEM_ELEMS 4400
 #endif
-constexpr int kItemElems = RSDGC_ITEM_ELEMS;  // elements of one accumulate+NSI work item
+constexpr int kItemElems = RSDGC_ITEM_ELEMS;  // elements of one accumulate+NSI work item (the most any variant takes)
+#ifndef RSDGC_BF16_STAGES
+#define RSDGC_BF16_STAGES 2
+#endif
+#ifndef RSDGC_BF16_ITEM_ELEMS
+#define RSDGC_BF16_ITEM_ELEMS 4400
+#endif
+constexpr int kItemElemsBf16 = RSDGC_BF16_ITEM_ELEMS;  // ... with bfloat16 gradients and no momentum (<= kItemElems)
+static_assert(kItemElemsBf16 <= kItemElems, "the register-staged kernel and the plan size their buffers for kItemElems");
 constexpr int kL1Bits = 10;          // radix level 1: key bits 30..21 (8 exponent + 2 mantissa)
 constexpr int kL1Bins = 1 << kL1Bits;
 constexpr int kL1Shift = 21;
@@ -139,7 +147,12 @@ struct StatusDev {
     unsigned int flags, pad;
     unsigned long long nonfinite;
     long long idx_needed, val_needed;
+    // extents of the plan's arenas and tables (constant after plan creation; rsdgc_get_status() resets
+    // only what lies before them): what the bounds-checked build tests every index against
+    long long arena_elems, keys_len;
+    int n_layers, n_chunks, n_echunks, n_items;
 };
+constexpr size_t kStatusResetBytes = 32;  // flags .. val_needed
 
 }  // namespace rsdgc
 
@@ -151,6 +164,7 @@ struct rsdgc_plan {
     uint32_t flags = 0;
     int n_sm = 148;
     int reg_ctas_per_sm = 2;
+    int item_elems = rsdgc::kItemElems;     // elements an item of the first pass may hold (depends on the gradient type)
     int grid_bulk = 0, grid_reg = 0;        // CTAs of the two accumulate+NSI kernels
     int n_items_bulk = 0, n_items_reg = 0;  // items_dev = [bulk items..., register items...]
 
@@ -232,6 +246,7 @@ void count_launch(int n);
 void set_last_cuda_error(int e);
 int k1_reg_ctas_per_sm(int dtype, bool momentum);
 int k1_bulk_ctas_per_sm(bool momentum);
+int bulk_item_elems(int dtype, bool momentum);
 cudaError_t launch_accumulate_nsi(rsdgc_plan *p, uint32_t *hist, LayerState *state, const void *grads, float *resid,
                           float *vel, float mom, const float *ratios, int32_t *counts, uint32_t *keys,
                           cudaStream_t s, bool after_sibling = false, bool before_sibling = false);

@@ -74,7 +74,12 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     const TailSlice sl = slices[blockIdx.x];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int NW = NT / 32;
-    const bool active = sl.n > 0;  // a rank without a slice only takes part in the cluster's barriers
+    // a rank without a slice only takes part in the cluster's barriers (so does, in the bounds-checked
+    // build, a slice that does not lie inside its layer and the key array)
+    const bool active = sl.n > 0 &&
+                        RSDGC_CHECKED(sl.n <= KEYS && sl.layer >= 0 && sl.layer < status->n_layers && sl.start >= 0 &&
+                                          sl.start + sl.n <= layers[sl.layer].K &&
+                                          layers[sl.layer].tile_off + sl.start + sl.n <= status->keys_len, status);
     const bool leader = active && sl.rank == 0;
 
     // every CTA of a cluster runs the same sequence of barriers
@@ -350,6 +355,8 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
                     const int i = tr * L.nh + a, jj = tc * L.nw + b;
                     if (i < (int)L.rows && jj < cols) ga[u] = i * cols + jj;
                     vo[u] = (int)(s - idx_off) * slot + el;
+                    if (!RSDGC_CHECKED(tile >= 0 && tile < L.K && L.elem_off + ga[u] < status->arena_elems, status))
+                        ga[u] = -1, vo[u] = -1;
                 }
             }
         }
