@@ -31,21 +31,28 @@ namespace cg = cooperative_groups;
 
 namespace rsdgc {
 
-template <int NT>
+constexpr int kTailCand = 1024;  // candidates a CTA can list (keys that share the threshold's upper 21 bits)
+
+template <int NT, int KEYS>
 struct TailShared {
     unsigned int hist[kL2Bins];              // this CTA's histogram; the leader's also receives the others'
     unsigned long long scan_tmp[NT / 32];
     unsigned long long found[2];
-    unsigned int res[2];                     // leader: what the level resolved (bin, remaining)
+    unsigned int res[3];                     // leader: what a level resolved (bin, remaining), fallback flag
     unsigned int cnt[kTailCluster][2];       // leader: per rank, keys above the threshold / equal to it
-    unsigned int warp_cnt[NT / 32][2];       // per warp of this CTA: the same counts over the warp's keys
+    unsigned int overflow[kTailCluster];     // leader: per rank, its candidate list did not hold its candidates
+    unsigned int warp_cnt[NT / 32][2];       // per warp of this CTA: kept-for-sure / equal keys in the warp's range
     unsigned int warp_pre[NT / 32 + 1][2];   // the counts of the warps before each warp; last entry: the CTA's totals
+    unsigned int above[KEYS / 32];           // one bit per key of the slice: above the threshold
+    unsigned int equal[KEYS / 32];           // ... equal to the threshold
+    unsigned int cand[kTailCand];            // candidates: key bits 9..0 << 15 | position in the slice
+    unsigned int n_cand;
     long long idx_off, val_off;              // payload offsets of the layer
 };
 
 // Block-wide sum of one value per thread (every thread gets it).  Not inlined: these kernels run
-// once per call on cold instruction caches, so their code is kept small (loops with a little
-// unrolling for memory-level parallelism, one copy of every helper).
+// once per call, so their code is kept small (loops with a little unrolling for memory-level
+// parallelism, one copy of every helper).
 template <int NT>
 __device__ __noinline__ unsigned long long block_sum(unsigned long long x, unsigned long long *tmp)
 {
@@ -61,6 +68,13 @@ __device__ __noinline__ void tail_find_bin(const unsigned int *h, unsigned long 
     find_bin_from_top<kL2Bins, NT>(h, need, out, tmp);
 }
 
+// How the passes over a slice are kept few: a CTA is one SM, and every pass over up to 32768 keys costs
+// it 2 to 3 us.  Level 2 is histogrammed while the keys arrive.  After level 2 the upper 21 bits of
+// the threshold are known: a key above them is kept, a key below is not, and the few keys that share
+// them ("candidates") decide the rest.  ONE pass writes a bit per key (above) and lists the
+// candidates; level 3, the equal keys and all ranks then come from the list and the bit masks.  If some
+// CTA of the layer has more candidates than its list holds (many equal indicators: constant layers),
+// the layer takes one more pass: level 3 over all its keys, then the masks from the full threshold.
 template <int CS, int KEYS, int NT, bool BF16VAL>
 __global__ void __launch_bounds__(NT, 1)
 k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
@@ -69,11 +83,13 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
 {
     extern __shared__ __align__(16) unsigned char tail_smem_raw[];
     uint32_t *skeys = reinterpret_cast<uint32_t *>(tail_smem_raw);  // KEYS words
-    __shared__ TailShared<NT> sh;
+    __shared__ TailShared<NT, KEYS> sh;
     const Lane &ln = lanes.l[blockIdx.y];
     const TailSlice sl = slices[blockIdx.x];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     constexpr int NW = NT / 32;
+    constexpr int WPW = KEYS / 32 / NW;  // mask words per warp (a warp owns KEYS / NW consecutive keys)
+    static_assert(WPW >= 1 && WPW <= 32 * 2 && (KEYS / 32) % NW == 0, "a lane handles at most two mask words");
     // a rank without a slice only takes part in the cluster's barriers (so does, in the bounds-checked
     // build, a slice that does not lie inside its layer and the key array)
     const bool active = sl.n > 0 &&
@@ -92,10 +108,37 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
         if constexpr (CS > 1) return cg::this_cluster().map_shared_rank(p, (unsigned int)sl.leader);
         else return p;
     };
+    // adds this CTA's histogram (bins 0 .. nbins - 1) to the leader's and clears it
+    auto push_hist = [&](int nbins) {
+        if (CS > 1 && !leader) {
+            __syncthreads();
+            unsigned int *lh = at_leader(&sh.hist[0]);
+            for (int b = tid; b < nbins; b += NT) {
+                const unsigned int c = sh.hist[b];
+                if (c) {
+                    atomicAdd(lh + b, c);
+                    sh.hist[b] = 0;
+                }
+            }
+        }
+    };
+    // the leader finds the bin in which the running count from the top reaches `need`, publishes it and
+    // clears its histogram (level 3 fills the lower 1024 of the 2048 bins; the upper ones are zero)
+    auto resolve = [&](unsigned int need, int nbins) {
+        tail_find_bin<NT>(sh.hist, (unsigned long long)need, sh.found, sh.scan_tmp);
+        if (tid == 0) {
+            sh.res[0] = (unsigned int)sh.found[0];
+            sh.res[1] = (unsigned int)sh.found[1];
+        }
+        for (int b = tid; b < nbins; b += NT) sh.hist[b] = 0;
+    };
 
     // ---- what needs only the plan and the ratios: the layer's payload offsets (sums of the k_l of the
     // preceding layers, Eq. 11)
     for (int b = tid; b < kL2Bins; b += NT) sh.hist[b] = 0;
+    for (int b = tid; b < KEYS / 32; b += NT) sh.above[b] = sh.equal[b] = 0;
+    if (tid == 0) sh.n_cand = 0;
+    if (tid < kTailCluster) sh.overflow[tid] = 0;
     if (active) {
         long long si = 0, sv = 0;
         for (int l = tid; l < sl.layer; l += NT) {
@@ -120,139 +163,226 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     uint32_t prefix = kTakeNone;   // key bits resolved so far
     unsigned int remaining = 0;    // tiles still to take among the keys that carry the prefix
     const int n4 = (sl.n + 3) >> 2;  // the slice as 128-bit words (the last one padded)
+    __syncthreads();                 // the tables cleared above
     if (active) {
         const LayerState &st = ln.state[sl.layer];
         k = __ldcg(&st.k);
         prefix = __ldcg(&st.prefix);
         remaining = (unsigned int)__ldcg(&st.remaining);
+        // keys: global -> shared memory, and level 2 (bits 20..10 of the keys that carry the level-1
+        // prefix) histogrammed on the way
         const uint32_t *kp = ln.keys + L.tile_off + sl.start;  // 16-byte aligned: offsets are multiples of 64 keys
         const int nvec = sl.n >> 2;
         constexpr int kLoadBatch = 8;  // 128-bit loads in flight per thread: the slice arrives in one or two round trips
-        for (int base = 0; base < nvec; base += NT * kLoadBatch) {
+#pragma unroll 1
+        for (int base = 0; base < n4; base += NT * kLoadBatch) {
             uint4 q[kLoadBatch];
 #pragma unroll
             for (int u = 0; u < kLoadBatch; ++u) {
                 const int i = base + u * NT + tid;
-                q[u] = (i < nvec) ? __ldcg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
+                q[u] = (i < nvec) ? __ldcg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(~0u, ~0u, ~0u, ~0u);
+                if (i == nvec && (sl.n & 3)) {  // the last, partial word: keys beyond the slice stay all ones,
+                    q[u].x = __ldcg(kp + 4 * i);  // which no prefix or threshold matches
+                    if ((sl.n & 3) > 1) q[u].y = __ldcg(kp + 4 * i + 1);
+                    if ((sl.n & 3) > 2) q[u].z = __ldcg(kp + 4 * i + 2);
+                }
             }
 #pragma unroll
             for (int u = 0; u < kLoadBatch; ++u) {
                 const int i = base + u * NT + tid;
-                if (i < nvec) reinterpret_cast<uint4 *>(skeys)[i] = q[u];
+                if (i < n4) {
+                    reinterpret_cast<uint4 *>(skeys)[i] = q[u];
+                    if ((q[u].x >> kL1Shift) == prefix) atomicAdd(&sh.hist[(q[u].x >> kL2Shift) & (kL2Bins - 1)], 1u);
+                    if ((q[u].y >> kL1Shift) == prefix) atomicAdd(&sh.hist[(q[u].y >> kL2Shift) & (kL2Bins - 1)], 1u);
+                    if ((q[u].z >> kL1Shift) == prefix) atomicAdd(&sh.hist[(q[u].z >> kL2Shift) & (kL2Bins - 1)], 1u);
+                    if ((q[u].w >> kL1Shift) == prefix) atomicAdd(&sh.hist[(q[u].w >> kL2Shift) & (kL2Bins - 1)], 1u);
+                }
             }
         }
-        // the last, partial word: keys beyond the slice are all ones, which no prefix or threshold matches
-        if (tid < 4 && (sl.n & 3)) {
-            const int i = (nvec << 2) + tid;
-            skeys[i] = (i < sl.n) ? __ldcg(kp + i) : 0xFFFFFFFFu;
+    }
+    sync_all();  // every CTA's tables are cleared before anything is added to a leader's
+    if (active && prefix != kTakeNone) push_hist(kL2Bins);
+    sync_all();
+    if (leader && prefix != kTakeNone) resolve(remaining, kL2Bins);
+    sync_all();
+    if (active && prefix != kTakeNone) {
+        const unsigned int *res = at_leader(&sh.res[0]);
+        prefix = (prefix << kL2Bits) | res[0];   // the upper 21 bits of the threshold
+        remaining = res[1];
+    }
+
+    // ---- one pass: a bit per key above the upper 21 bits, the candidates that share them into the list
+    // (warp w owns the keys [w * per_warp, (w + 1) * per_warp) of the slice; four groups of 32 per round)
+    constexpr int per_warp = KEYS / NW;
+    const int w0 = warp * per_warp, w1 = min(sl.n, w0 + per_warp);
+    if (active && prefix != kTakeNone) {
+#pragma unroll 1
+        for (int base = w0; base < w1; base += 128) {
+            uint32_t key[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + u * 32 + lane;
+                key[u] = (i < w1) ? skeys[i] : 0xFFFFFFFFu;
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = base + u * 32 + lane;
+                const uint32_t hi = key[u] >> kL2Shift;
+                const unsigned int ma = __ballot_sync(0xFFFFFFFFu, key[u] != 0xFFFFFFFFu && hi > prefix);
+                if (lane == 0 && base + u * 32 < w1) sh.above[(base >> 5) + u] = ma;
+                if (hi == prefix) {
+                    const unsigned int pos = atomicAdd(&sh.n_cand, 1u);
+                    if (pos < (unsigned int)kTailCand) sh.cand[pos] = ((key[u] & (kL3Bins - 1)) << 15) | (unsigned int)i;
+                }
+            }
         }
     }
     __syncthreads();
-    sync_all();  // every histogram of the cluster is zero before anything is added to a leader's
-
-    // ---- levels 2 and 3: key bits 20..10, 9..0
+    const unsigned int n_cand_all = sh.n_cand;  // may exceed the list
+    const int n_cand = (int)min(n_cand_all, (unsigned int)kTailCand);
+    if (active && prefix != kTakeNone) {
+        // level 3 (key bits 9..0) over the candidates; an overflowing list is reported to the leader
+        for (int c = tid; c < n_cand; c += NT) atomicAdd(&sh.hist[sh.cand[c] >> 15], 1u);
+        if (tid == 0 && n_cand_all > (unsigned int)kTailCand) at_leader(&sh.overflow[0])[sl.rank] = 1u;
+        push_hist(kL3Bins);
+    }
+    sync_all();
+    if (leader && prefix != kTakeNone) {
+        unsigned int any = 0;
+        for (int r = 0; r < sl.n_ranks; ++r) any |= sh.overflow[r];
+        if (any) {  // some list is incomplete: its histogram is worthless
+            for (int b = tid; b < kL3Bins; b += NT) sh.hist[b] = 0;
+            if (tid == 0) sh.res[2] = 1u;
+        } else {
+            resolve(remaining, kL3Bins);
+            if (tid == 0) sh.res[2] = 0u;
+        }
+    }
+    sync_all();
+    bool fallback = false;
+    uint32_t T = kTakeNone;  // the threshold key
+    int e = 0;               // keys equal to T that are taken, lowest tile index first
+    if (active && prefix != kTakeNone) {
+        const unsigned int *res = at_leader(&sh.res[0]);
+        fallback = res[2] != 0u;
+        if (!fallback) {
+            T = (prefix << kL3Bits) | res[0];
+            e = (int)res[1];
+        }
+    }
+    // ---- the layer's extra pass when a candidate list overflowed: level 3 over all the keys
+    if (fallback) {
 #pragma unroll 1
-    for (int level = 2; level <= 3; ++level) {
-        const int shift_hi = level == 2 ? kL1Shift : kL2Shift;
-        const int shift_lo = level == 2 ? kL2Shift : 0;
-        const unsigned int mask = level == 2 ? (unsigned int)(kL2Bins - 1) : (unsigned int)(kL3Bins - 1);
-        if (active && prefix != kTakeNone) {
-#pragma unroll 1
-            for (int base = 0; base < n4; base += NT * 2) {
-                uint4 q[2];
+        for (int base = 0; base < n4; base += NT * 2) {
+            uint4 q[2];
 #pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    const int i = base + u * NT + tid;
-                    q[u] = (i < n4) ? reinterpret_cast<const uint4 *>(skeys)[i] : make_uint4(~0u, ~0u, ~0u, ~0u);
-                }
-#pragma unroll
-                for (int u = 0; u < 2; ++u) {
-                    if ((q[u].x >> shift_hi) == prefix) atomicAdd(&sh.hist[(q[u].x >> shift_lo) & mask], 1u);
-                    if ((q[u].y >> shift_hi) == prefix) atomicAdd(&sh.hist[(q[u].y >> shift_lo) & mask], 1u);
-                    if ((q[u].z >> shift_hi) == prefix) atomicAdd(&sh.hist[(q[u].z >> shift_lo) & mask], 1u);
-                    if ((q[u].w >> shift_hi) == prefix) atomicAdd(&sh.hist[(q[u].w >> shift_lo) & mask], 1u);
-                }
+            for (int u = 0; u < 2; ++u) {
+                const int i = base + u * NT + tid;
+                q[u] = (i < n4) ? reinterpret_cast<const uint4 *>(skeys)[i] : make_uint4(~0u, ~0u, ~0u, ~0u);
             }
-            if (CS > 1 && !leader) {
-                __syncthreads();
-                unsigned int *lh = at_leader(&sh.hist[0]);
-                for (int b = tid; b <= (int)mask; b += NT) {
-                    const unsigned int c = sh.hist[b];
-                    if (c) {
-                        atomicAdd(lh + b, c);
-                        sh.hist[b] = 0;
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                if ((q[u].x >> kL2Shift) == prefix) atomicAdd(&sh.hist[q[u].x & (kL3Bins - 1)], 1u);
+                if ((q[u].y >> kL2Shift) == prefix) atomicAdd(&sh.hist[q[u].y & (kL3Bins - 1)], 1u);
+                if ((q[u].z >> kL2Shift) == prefix) atomicAdd(&sh.hist[q[u].z & (kL3Bins - 1)], 1u);
+                if ((q[u].w >> kL2Shift) == prefix) atomicAdd(&sh.hist[q[u].w & (kL3Bins - 1)], 1u);
+            }
+        }
+        push_hist(kL3Bins);
+    }
+    sync_all();
+    if (leader && fallback) resolve(remaining, kL3Bins);
+    sync_all();
+    if (fallback) {
+        const unsigned int *res = at_leader(&sh.res[0]);
+        T = (prefix << kL3Bits) | res[0];
+        e = (int)res[1];
+    }
+
+    // ---- the bit masks of the keys above and equal to the full threshold
+    if (active && T != kTakeNone) {
+        if (!fallback) {  // only the candidates can still change a bit
+            const uint32_t t_low = T & (kL3Bins - 1);
+            for (int c = tid; c < n_cand; c += NT) {
+                const unsigned int v = sh.cand[c], low = v >> 15, i = v & 0x7FFFu;
+                if (low > t_low) atomicOr(&sh.above[i >> 5], 1u << (i & 31));
+                else if (low == t_low) atomicOr(&sh.equal[i >> 5], 1u << (i & 31));
+            }
+        } else {
+#pragma unroll 1
+            for (int base = w0; base < w1; base += 128) {
+                uint32_t key[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = base + u * 32 + lane;
+                    key[u] = (i < w1) ? skeys[i] : 0xFFFFFFFFu;
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const unsigned int ma = __ballot_sync(0xFFFFFFFFu, key[u] != 0xFFFFFFFFu && key[u] > T);
+                    const unsigned int me = __ballot_sync(0xFFFFFFFFu, key[u] == T);
+                    if (lane == 0 && base + u * 32 < w1) {
+                        sh.above[(base >> 5) + u] = ma;
+                        sh.equal[(base >> 5) + u] = me;
                     }
                 }
             }
         }
-        sync_all();
-        if (leader && prefix != kTakeNone) {
-            // (level 3 fills the lower 1024 of the 2048 bins; the upper ones are zero and change nothing)
-            tail_find_bin<NT>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
-            if (tid == 0) {
-                sh.res[0] = (unsigned int)sh.found[0];
-                sh.res[1] = (unsigned int)sh.found[1];
-            }
-            for (int b = tid; b <= (int)mask; b += NT) sh.hist[b] = 0;
-        }
-        sync_all();
-        if (active && prefix != kTakeNone) {
-            const unsigned int *res = at_leader(&sh.res[0]);
-            prefix = (prefix << (level == 2 ? kL2Bits : kL3Bits)) | res[0];
-            remaining = res[1];
-        }
     }
-    const uint32_t T = prefix;       // the threshold key, or kTakeNone
-    const int e = (int)remaining;    // keys equal to T that are taken, lowest tile index first
+    __syncthreads();
 
-    // ---- per warp, per CTA, per layer: how many keys lie above T and how many equal it
-    // warp w owns the keys [w * per_warp, (w + 1) * per_warp) of the slice
-    constexpr int per_warp = KEYS / NW;
-    const int w0 = warp * per_warp, w1 = min(sl.n, w0 + per_warp);
-    {
-        unsigned int gt = 0, eq = 0;
-        if (active && T != kTakeNone) {
-#pragma unroll 4
-            for (int i = w0 + lane; i < w1; i += 32) {
-                const uint32_t key = skeys[i];
-                gt += key > T;
-                eq += key == T;
-            }
-        }
+    // ---- per warp, per CTA, per layer: how many keys lie above T and how many equal it.  A lane holds
+    // the mask words lane * WPL .. of its warp's range.
+    constexpr int WPL = (WPW + 31) / 32;  // mask words per lane (1 or 2)
+    unsigned int ab[WPL], eq[WPL];
+    unsigned int my_gt = 0, my_eq = 0;
 #pragma unroll
-        for (int d = 16; d > 0; d >>= 1) {
-            gt += __shfl_xor_sync(0xFFFFFFFFu, gt, d);
-            eq += __shfl_xor_sync(0xFFFFFFFFu, eq, d);
-        }
-        if (lane == 0) {
-            sh.warp_cnt[warp][0] = gt;
-            sh.warp_cnt[warp][1] = eq;
+    for (int j = 0; j < WPL; ++j) {
+        const int wl = lane * WPL + j;  // word within the warp's range
+        ab[j] = (wl < WPW) ? sh.above[warp * WPW + wl] : 0u;
+        eq[j] = (wl < WPW) ? sh.equal[warp * WPW + wl] : 0u;
+        my_gt += __popc(ab[j]);
+        my_eq += __popc(eq[j]);
+    }
+    // exclusive prefix over the lanes of the warp, and the warp's totals
+    unsigned int pg = my_gt, pe = my_eq;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const unsigned int yg = __shfl_up_sync(0xFFFFFFFFu, pg, d), ye = __shfl_up_sync(0xFFFFFFFFu, pe, d);
+        if (lane >= d) {
+            pg += yg;
+            pe += ye;
         }
     }
+    if (lane == 31) {
+        sh.warp_cnt[warp][0] = pg;
+        sh.warp_cnt[warp][1] = pe;
+    }
+    pg -= my_gt;
+    pe -= my_eq;
     __syncthreads();
     // exclusive prefix of the warps' counts (warp 0, by shuffles); the CTA's totals end up in entry NW
     if (warp == 0) {
-        unsigned int a = (lane < NW) ? sh.warp_cnt[lane][0] : 0u, b = (lane < NW) ? sh.warp_cnt[lane][1] : 0u;
-        const unsigned int a0 = a, b0 = b;
+        unsigned int a = (lane < NW) ? sh.warp_cnt[lane][0] : 0u, b2 = (lane < NW) ? sh.warp_cnt[lane][1] : 0u;
+        const unsigned int a0 = a, b0 = b2;
 #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            const unsigned int ya = __shfl_up_sync(0xFFFFFFFFu, a, d), yb = __shfl_up_sync(0xFFFFFFFFu, b, d);
+            const unsigned int ya = __shfl_up_sync(0xFFFFFFFFu, a, d), yb = __shfl_up_sync(0xFFFFFFFFu, b2, d);
             if (lane >= d) {
                 a += ya;
-                b += yb;
+                b2 += yb;
             }
         }
         if (lane < NW) {
             sh.warp_pre[lane][0] = a - a0;
-            sh.warp_pre[lane][1] = b - b0;
+            sh.warp_pre[lane][1] = b2 - b0;
         }
         if (lane == NW - 1) {
             sh.warp_pre[NW][0] = a;
-            sh.warp_pre[NW][1] = b;
+            sh.warp_pre[NW][1] = b2;
         }
     }
     __syncthreads();
-    int gt_before = (int)sh.warp_pre[warp][0], eq_before = (int)sh.warp_pre[warp][1];  // in the warps before this one
     const int cta_gt = (int)sh.warp_pre[NW][0], cta_eq = (int)sh.warp_pre[NW][1];
     if (active && tid == 0) {
         unsigned int *c = at_leader(&sh.cnt[0][0]);
@@ -287,35 +417,27 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     }
 
     // ---- payload indices: a tile is kept if its key is above T, or equals T with fewer than e equal
-    // keys before it in the layer; its slot is the number of kept tiles before it
-    gt_before += lay_gt0;
-    eq_before += lay_eq0;
+    // keys before it in the layer; its slot is the number of kept tiles before it.  Only the set bits
+    // are visited.
     int32_t *__restrict__ idx = ln.idx;
-#pragma unroll 1
-    for (int base = w0; base < w1; base += 128) {  // four groups of 32 keys per round: their loads and votes overlap
-        uint32_t key[4];
-        unsigned int ma[4], me[4];
+    {
+        int g_rank = lay_gt0 + (int)sh.warp_pre[warp][0] + (int)pg, e_rank = lay_eq0 + (int)sh.warp_pre[warp][1] + (int)pe;
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int i = base + u * 32 + lane;
-            key[u] = (i < w1) ? skeys[i] : 0xFFFFFFFFu;  // all ones: neither above nor equal (T has bit 31 clear)
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            ma[u] = __ballot_sync(0xFFFFFFFFu, key[u] != 0xFFFFFFFFu && key[u] > T);
-            me[u] = __ballot_sync(0xFFFFFFFFu, key[u] == T);
-        }
-        const unsigned int lower = (1u << lane) - 1u;
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int g_rank = gt_before + __popc(ma[u] & lower), e_rank = eq_before + __popc(me[u] & lower);
-            const bool above = (ma[u] >> lane) & 1u, equal = (me[u] >> lane) & 1u;
-            if (above || (equal && e_rank < e)) {
-                const long long s = idx_off + (g_rank + min(e_rank, e));
-                if (s < idx_cap) idx[s] = sl.start + base + u * 32 + lane;
+        for (int j = 0; j < WPL; ++j) {
+            const int tile0 = sl.start + (warp * WPW + lane * WPL + j) * 32;
+            unsigned int todo = ab[j] | eq[j];
+            while (todo) {
+                const int bit = __ffs((int)todo) - 1;
+                todo &= todo - 1;
+                const unsigned int below = (1u << bit) - 1u;
+                const int gr = g_rank + __popc(ab[j] & below), er = e_rank + __popc(eq[j] & below);
+                if (((ab[j] >> bit) & 1u) || er < e) {
+                    const long long s = idx_off + (gr + min(er, e));
+                    if (s < idx_cap) idx[s] = tile0 + bit;
+                }
             }
-            gt_before += __popc(ma[u]);
-            eq_before += __popc(me[u]);
+            g_rank += __popc(ab[j]);
+            e_rank += __popc(eq[j]);
         }
     }
     __syncthreads();  // the gather below reads the indices this CTA has just written
