@@ -160,104 +160,95 @@ k_refine(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ l
 }
 
 // ------------------------------------------------------------------------------------------
-// K4: per chunk, how many keys lie above the threshold and how many equal it; the last CTA
-// of a layer turns the layer's chunk counts into exclusive bases and computes the layer's
-// payload offsets (prefix sums of k_l' over the preceding layers).
+// K3 + K4 in one pass over the keys: level 3 of the selection AND everything the index pass needs.
+// When this pass runs, the upper 21 bits of a layer's threshold are known.  A key above them is kept
+// whatever level 3 finds, a key below them is not; only the keys that share them ("in the bin") depend
+// on the low 10 bits.  Per chunk the pass therefore leaves
+//   * one code byte per four keys (bit c: key c above the bin, bit 4 + c: key c in the bin),
+//   * the number of keys above the bin,
+//   * the suffix sums of the chunk's histogram of the low 10 bits of its in-bin keys
+//     (sfx[b] = in-bin keys of the chunk whose low bits are >= b),
+// and adds the chunk's histogram to the layer's.  The CTA that accounts for a layer's last chunk
+// resolves level 3 (T and e), reads two suffix sums per chunk to get every chunk's count of keys
+// above T and equal to T, turns them into exclusive bases and computes the layer's payload offsets:
+// no separate counting pass over the keys.
 // ------------------------------------------------------------------------------------------
 
-struct CountShared {
+struct Refine3Shared {
+    unsigned int hist[kL3Bins];   // level-3 histogram of the current layer over the chunks this CTA took
+    unsigned int chist[kL3Bins];  // ... of the current chunk
     unsigned long long scan_tmp[kThreads / 32];
-    unsigned int red[2][kThreads / 32];
+    unsigned long long found[2];
+    unsigned int red[kThreads / 32];
     int is_last;
 };
 
-__global__ void __launch_bounds__(kThreads)
-k_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
-        const Chunk *__restrict__ chunks, int n_layers, long long idx_cap, long long val_cap, StatusDev *status)
+// Layer `layer` is complete in this CTA (n_done of its chunks): add to the layer's global histogram;
+// the last CTA to do so finishes the layer.
+__device__ __forceinline__ void refine3_flush(Refine3Shared &sh, const Lane &ln, const LayerDev *__restrict__ layers,
+                                              int layer, int n_done, int n_layers, long long idx_cap,
+                                              long long val_cap, StatusDev *status)
 {
-    __shared__ CountShared sh;
-    const Lane &ln = lanes.l[blockIdx.y];
-    const uint32_t *__restrict__ keys = ln.keys;
-    LayerState *state = ln.state;
-    uint2 *chunk_cnt = ln.chunk_cnt;
-    unsigned char *__restrict__ codes = ln.codes;
-    const Chunk c = chunks[blockIdx.x];
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    LayerState &st = state[c.layer];
-    const LayerDev &L = layers[c.layer];
-    grid_dependency_wait();
-    grid_dependency_launch_next();
-    const uint32_t T = st.T;
-    unsigned int gt = 0, eq = 0;
-    if (RSDGC_CHECKED((int)blockIdx.x < status->n_chunks && c.layer < status->n_layers && c.start >= 0 && c.n >= 0 &&
-                          L.tile_off + c.start + c.n <= status->keys_len, status)) {
-        // one code byte per 128-bit word of keys (bit c: key c above T, bit 4 + c: key c equal
-        // to T) is left for k_mark, which then needs no second look at the keys
-        const uint32_t *kp = keys + L.tile_off + c.start;
-        unsigned char *cp = codes + ((L.tile_off + c.start) >> 2);
-        const int nvec = c.n >> 2;
-        const int nvec_all = (c.n + 3) >> 2;
-        for (int base = 0; base < nvec_all; base += kThreads * kKeyVecBatch) {
-            uint4 q[kKeyVecBatch];
-#pragma unroll
-            for (int u = 0; u < kKeyVecBatch; ++u) {
-                const int i = base + u * kThreads + tid;
-                q[u] = (i < nvec) ? __ldg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
-            }
-#pragma unroll
-            for (int u = 0; u < kKeyVecBatch; ++u) {
-                const int i = base + u * kThreads + tid;
-                if (i >= nvec_all) continue;
-                unsigned int code = 0;
-                if (i < nvec) {
-                    code = (q[u].x > T) | ((q[u].y > T) << 1) | ((q[u].z > T) << 2) | ((q[u].w > T) << 3) |
-                           ((q[u].x == T) << 4) | ((q[u].y == T) << 5) | ((q[u].z == T) << 6) | ((q[u].w == T) << 7);
-                } else {  // the last, partial word of the chunk
-                    for (int j = 0; j < (c.n & 3); ++j) {
-                        const uint32_t k1 = kp[(nvec << 2) + j];
-                        code |= ((k1 > T) << j) | ((k1 == T) << (4 + j));
-                    }
-                }
-                cp[i] = (unsigned char)code;
-                gt += __popc(code & 0x0Fu);
-                eq += __popc(code & 0xF0u);
-            }
+    const int tid = threadIdx.x;
+    LayerState &st = ln.state[layer];
+    const LayerDev &L = layers[layer];
+    unsigned int *gh = ln.hist + (size_t)layer * kHistStride;
+    __syncthreads();
+    for (int b = tid; b < kL3Bins; b += kThreads) {
+        const unsigned int n = sh.hist[b];
+        if (n) {
+            atomicAdd(gh + b, n);
+            sh.hist[b] = 0;
         }
     }
-#pragma unroll
-    for (int d = 16; d > 0; d >>= 1) {
-        gt += __shfl_xor_sync(0xFFFFFFFFu, gt, d);
-        eq += __shfl_xor_sync(0xFFFFFFFFu, eq, d);
-    }
-    if (lane == 0) {
-        sh.red[0][warp] = gt;
-        sh.red[1][warp] = eq;
-    }
+    __threadfence();  // also orders this CTA's per-chunk counts and suffix sums before its ticket
     __syncthreads();
     if (tid == 0) {
-        unsigned int a = 0, b = 0;
-        for (int w = 0; w < kThreads / 32; ++w) {
-            a += sh.red[0][w];
-            b += sh.red[1][w];
-        }
-        chunk_cnt[blockIdx.x] = make_uint2(a, b);
-        __threadfence();
-        const unsigned int t = atomicAdd(&st.ticket[3], 1u);
-        sh.is_last = (t + 1u == (unsigned int)L.n_chunks);
+        const unsigned int t = atomicAdd(&st.ticket[2], (unsigned int)n_done);
+        sh.is_last = (t + (unsigned int)n_done == (unsigned int)L.n_chunks);
     }
     __syncthreads();
     if (!sh.is_last) return;
     __threadfence();
+    {
+        unsigned int h[kL3Bins / kThreads];
+#pragma unroll
+        for (int j = 0; j < kL3Bins / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + tid);
+#pragma unroll
+        for (int j = 0; j < kL3Bins / kThreads; ++j) {
+            sh.hist[j * kThreads + tid] = h[j];
+            gh[j * kThreads + tid] = 0;
+        }
+    }
+    __syncthreads();
+    const uint32_t prefix = st.prefix;
+    const int remaining = st.remaining;
+    int bin = 0;
+    if (prefix != kTakeNone) {
+        find_bin_from_top<kL3Bins>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
+        bin = (int)sh.found[0];
+    }
+    if (tid == 0) {
+        st.ticket[2] = 0;
+        st.T = prefix != kTakeNone ? ((prefix << kL3Bits) | (uint32_t)bin) : kTakeNone;
+        st.e = prefix != kTakeNone ? (int32_t)sh.found[1] : 0;
+    }
+    __syncthreads();
+    for (int b = tid; b < kL3Bins; b += kThreads) sh.hist[b] = 0;  // it held the layer's totals
 
-    // exclusive scan of (gt, eq) over the layer's chunks, in chunk order
-    uint2 *cc = chunk_cnt + L.first_chunk;
-    unsigned long long carry = 0;  // gt in the low 32 bits, eq in the high 32 bits
+    // per chunk: keys above T = keys above the bin + in-bin keys with low bits > bin; equal = low bits == bin;
+    // then the exclusive scan over the layer's chunks, in chunk order
+    uint2 *cc = ln.chunk_cnt + L.first_chunk;
+    const unsigned short *sfx = ln.chunk_sfx + (size_t)L.first_chunk * kL3Bins;
+    unsigned long long carry = 0;  // above in the low 32 bits, equal in the high 32 bits
     for (int base = 0; base < L.n_chunks; base += kThreads) {
         const int i = base + tid;
         unsigned long long x = 0;
-        if (i < L.n_chunks) {
-            const unsigned long long raw = __ldcg(reinterpret_cast<const unsigned long long *>(cc + i));
-            x = raw;  // uint2 {x = gt, y = eq} is little-endian: low word gt, high word eq
+        if (i < L.n_chunks && prefix != kTakeNone) {
+            const unsigned int above_bin = __ldcg(&cc[i].x);
+            const unsigned int ge = __ldcg(sfx + (size_t)i * kL3Bins + bin);
+            const unsigned int gt = (bin + 1 < kL3Bins) ? (unsigned int)__ldcg(sfx + (size_t)i * kL3Bins + bin + 1) : 0u;
+            x = ((unsigned long long)(ge - gt) << 32) | (unsigned long long)(above_bin + gt);
         }
         unsigned long long total;
         const unsigned long long ex = block_exclusive_scan<unsigned long long>(x, sh.scan_tmp, &total) + carry;
@@ -267,8 +258,8 @@ k_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ la
 
     // payload offsets of this layer: sums over the preceding layers of k and k * slot
     long long si = 0, sv = 0;
-    for (int l = tid; l < c.layer; l += kThreads) {
-        const long long k = state[l].k;
+    for (int l = tid; l < layer; l += kThreads) {
+        const long long k = ln.state[l].k;
         si += k;
         sv += k * layers[l].slot;
     }
@@ -278,8 +269,7 @@ k_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ la
     if (tid == 0) {
         st.idx_off = (long long)tot_i;
         st.val_off = (long long)tot_v;
-        st.ticket[3] = 0;
-        if (c.layer == n_layers - 1) {
+        if (layer == n_layers - 1) {
             const long long need_i = (long long)tot_i + st.k;
             const long long need_v = (long long)tot_v + (long long)st.k * L.slot;
             status->idx_needed = need_i;
@@ -287,6 +277,116 @@ k_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ la
             if (need_i > idx_cap || need_v > val_cap) atomicOr(&status->flags, RSDGC_STATUS_PAYLOAD_OVERFLOW);
         }
     }
+    __syncthreads();
+}
+
+constexpr int kRefine3CtasPerSm = 4;  // 64 registers per thread
+
+__global__ void __launch_bounds__(kThreads, kRefine3CtasPerSm)
+k_refine3_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
+                const Chunk *__restrict__ chunks, int n_chunks_all, int n_layers, long long idx_cap, long long val_cap,
+                StatusDev *status)
+{
+    __shared__ Refine3Shared sh;
+    const Lane &ln = lanes.l[blockIdx.y];
+    const uint32_t *__restrict__ keys = ln.keys;
+    unsigned char *__restrict__ codes = ln.codes;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int chunk_begin = (int)((long long)blockIdx.x * n_chunks_all / gridDim.x);
+    const int chunk_end = (int)((long long)(blockIdx.x + 1) * n_chunks_all / gridDim.x);
+    for (int b = tid; b < kL3Bins; b += kThreads) sh.hist[b] = sh.chist[b] = 0;
+    grid_dependency_wait();
+    grid_dependency_launch_next();
+    __syncthreads();
+    int cur_layer = -1, n_done = 0;
+    uint32_t prefix = kTakeNone;
+    for (int chunk_id = chunk_begin; chunk_id < chunk_end; ++chunk_id) {
+        const Chunk c = chunks[chunk_id];
+        if (c.layer != cur_layer) {
+            if (n_done) refine3_flush(sh, ln, layers, cur_layer, n_done, n_layers, idx_cap, val_cap, status);
+            cur_layer = c.layer;
+            n_done = 0;
+            prefix = ln.state[c.layer].prefix;  // the upper 21 bits, left by the level-2 pass
+        }
+        ++n_done;
+        if (prefix == kTakeNone) continue;  // nothing of this layer is kept: no code, no count is read
+        const LayerDev &L = layers[c.layer];
+        if (!RSDGC_CHECKED(chunk_id < status->n_chunks && c.layer < status->n_layers && c.start >= 0 && c.n >= 0 &&
+                               L.tile_off + c.start + c.n <= status->keys_len, status))
+            continue;
+        const uint32_t *kp = keys + L.tile_off + c.start;
+        unsigned char *cp = codes + ((L.tile_off + c.start) >> 2);
+        const int nvec = c.n >> 2;
+        const int nvec_all = (c.n + 3) >> 2;
+        unsigned int above = 0;
+        for (int base = 0; base < nvec_all; base += kThreads * kKeyVecBatch) {
+            uint4 q[kKeyVecBatch];  // all loads of a batch are issued before any is consumed
+#pragma unroll
+            for (int u = 0; u < kKeyVecBatch; ++u) {
+                const int i = base + u * kThreads + tid;
+                q[u] = (i < nvec) ? __ldg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
+                if (i == nvec && i < nvec_all) {  // the last, partial word of the chunk; absent keys: all ones
+                    q[u] = make_uint4(~0u, ~0u, ~0u, ~0u);
+                    q[u].x = kp[4 * i];
+                    if ((c.n & 3) > 1) q[u].y = kp[4 * i + 1];
+                    if ((c.n & 3) > 2) q[u].z = kp[4 * i + 2];
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < kKeyVecBatch; ++u) {
+                const int i = base + u * kThreads + tid;
+                if (i >= nvec_all) continue;
+                const uint32_t kx[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
+                unsigned int code = 0;
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t hi = kx[j] >> kL2Shift;
+                    if (kx[j] != 0xFFFFFFFFu && hi > prefix) code |= 1u << j;
+                    if (hi == prefix) {  // (an absent key's upper bits match no prefix)
+                        code |= 16u << j;
+                        atomicAdd(&sh.chist[kx[j] & (kL3Bins - 1)], 1u);
+                    }
+                }
+                cp[i] = (unsigned char)code;
+                above += __popc(code & 0x0Fu);
+            }
+        }
+        // ---- the chunk's count of keys above the bin, the suffix sums of its histogram, and the
+        // histogram into the layer's
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xFFFFFFFFu, above, d);
+        if (lane == 0) sh.red[warp] = above;
+        __syncthreads();  // also: the chunk's histogram is complete
+        if (tid == 0) {
+            unsigned int a = 0;
+            for (int w = 0; w < kThreads / 32; ++w) a += sh.red[w];
+            ln.chunk_cnt[chunk_id] = make_uint2(a, 0u);
+        }
+        {
+            constexpr int PER = kL3Bins / kThreads;  // thread t owns bins [t * PER, (t + 1) * PER)
+            unsigned int h[PER];
+            unsigned long long mine = 0;
+#pragma unroll
+            for (int j = 0; j < PER; ++j) {
+                h[j] = sh.chist[tid * PER + j];
+                mine += h[j];
+            }
+            unsigned long long total;
+            unsigned long long below = block_exclusive_scan<unsigned long long>(mine, sh.scan_tmp, &total);
+            unsigned short *out = ln.chunk_sfx + (size_t)chunk_id * kL3Bins + tid * PER;
+#pragma unroll
+            for (int j = 0; j < PER; ++j) {
+                out[j] = (unsigned short)(total - below);  // in-bin keys with low bits >= this bin (<= 16384)
+                below += h[j];
+                if (h[j]) {
+                    sh.hist[tid * PER + j] += h[j];
+                    sh.chist[tid * PER + j] = 0;
+                }
+            }
+        }
+        __syncthreads();
+    }
+    if (n_done) refine3_flush(sh, ln, layers, cur_layer, n_done, n_layers, idx_cap, val_cap, status);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -311,6 +411,7 @@ k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     const unsigned char *__restrict__ codes = ln.codes;
     const LayerState *__restrict__ state = ln.state;
     const uint2 *__restrict__ chunk_cnt = ln.chunk_cnt;
+    const uint32_t *__restrict__ keys = ln.keys;
     int32_t *__restrict__ idx = ln.idx;
     const Chunk c = chunks[blockIdx.x];
     const int tid = threadIdx.x;
@@ -325,7 +426,7 @@ k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     // equal keys of this chunk that are still taken: those with layer-wide equal-rank < e
     const long long eq_room = max(0ll, (long long)st.e - (long long)base.y);
 
-    // ---- the code bytes k_count left: thread t owns keys [64 t, 64 t + 64) = 16 bytes; bytes
+    // ---- the code bytes the level-3 pass left: thread t owns keys [64 t, 64 t + 64) = 16 bytes; bytes
     // beyond the chunk's last word belong to whatever follows in the array and are masked off
     const unsigned char *cp = codes + ((layers[c.layer].tile_off + c.start) >> 2);
     const int nvec_all = (c.n + 3) >> 2;
@@ -343,16 +444,28 @@ k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
             }
         }
     }
-    // 64-bit masks in key order: bit 4 * byte + c of `above` (`equal`) is set when key c of that
-    // code byte lies above (equals) the threshold
-    unsigned long long above = 0, equal = 0;
+    // 64-bit masks in key order: bit 4 * byte + c of `above` (`inbin`) is set when key c of that
+    // code byte lies above (shares) the upper 21 bits of the threshold
+    unsigned long long above = 0, inbin = 0, equal = 0;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
         const unsigned int lo = w[j] & 0x0F0F0F0Fu, hi = (w[j] >> 4) & 0x0F0F0F0Fu;
         const unsigned int a16 = (lo & 0xFu) | ((lo >> 4) & 0xF0u) | ((lo >> 8) & 0xF00u) | ((lo >> 12) & 0xF000u);
         const unsigned int e16 = (hi & 0xFu) | ((hi >> 4) & 0xF0u) | ((hi >> 8) & 0xF00u) | ((hi >> 12) & 0xF000u);
         above |= (unsigned long long)a16 << (16 * j);
-        equal |= (unsigned long long)e16 << (16 * j);
+        inbin |= (unsigned long long)e16 << (16 * j);
+    }
+    // the few keys in the bin are looked at themselves: their low 10 bits against the threshold's
+    {
+        const uint32_t t_low = st.T & (kL3Bins - 1);
+        const uint32_t *kp = keys + layers[c.layer].tile_off + c.start + tid * kKeysPerThread;
+        while (inbin) {
+            const int p = __ffsll((long long)inbin) - 1;
+            inbin &= inbin - 1;
+            const uint32_t low = __ldg(kp + p) & (kL3Bins - 1);
+            if (low > t_low) above |= 1ull << p;
+            else if (low == t_low) equal |= 1ull << p;
+        }
     }
     const unsigned int gt = __popcll(above), eq = __popcll(equal);
     unsigned long long total;
@@ -557,21 +670,22 @@ static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n
     // the two full key passes: one wave of resident CTAs with a contiguous chunk range each when
     // the chunk list is much longer than that, else one CTA per chunk
     const int n_chunks = (int)p->chunks.size();
-    const int resident = p->n_sm * kRefineCtasPerSm;
-    const dim3 grid_refine((unsigned)((long long)n_chunks * n_lanes <= 2ll * resident
-                                          ? n_chunks
-                                          : std::max(1, std::min(n_chunks, resident / n_lanes))),
-                           (unsigned)n_lanes);
+    auto refine_grid = [&](int ctas_per_sm) {
+        const int resident = p->n_sm * ctas_per_sm;
+        return dim3((unsigned)((long long)n_chunks * n_lanes <= 2ll * resident
+                                   ? n_chunks
+                                   : std::max(1, std::min(n_chunks, resident / n_lanes))),
+                    (unsigned)n_lanes);
+    };
+    const dim3 grid_refine = refine_grid(kRefineCtasPerSm), grid_refine3 = refine_grid(kRefine3CtasPerSm);
     if (e == cudaSuccess)
         e = launch_chained(k_refine<2>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks, p->d_status);
     RSDGC_MARK(2);
     if (e == cudaSuccess)
-        e = launch_chained(k_refine<3>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks, p->d_status);
+        e = launch_chained(k_refine3_count, grid_refine3, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks, p->n_layers,
+                           (long long)idx_cap, (long long)val_cap, p->d_status);
     RSDGC_MARK(2);
-    if (e == cudaSuccess)
-        e = launch_chained(k_count, grid, 0, s, lanes, p->d_layers, p->d_chunks, p->n_layers, (long long)idx_cap,
-                           (long long)val_cap, p->d_status);
-    RSDGC_MARK(2);
+    RSDGC_MARK(2);  // (the slot of the former counting pass: level 3 leaves the counts)
     if (e == cudaSuccess)
         e = launch_chained(k_mark, grid, 0, s, lanes, p->d_layers, p->d_chunks, (long long)idx_cap, p->d_status);
     RSDGC_MARK(2);
@@ -584,7 +698,7 @@ static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n
                                  p->n_layers, (long long)idx_cap, (long long)val_cap, p->d_status);
     RSDGC_MARK(2);
 #undef RSDGC_MARK
-    count_launch(5);
+    count_launch(4);
     return e;
 }
 
@@ -622,7 +736,7 @@ cudaError_t launch_compress(rsdgc_plan *p, const void *grads, float *resid, floa
                                   fused);
     if (prof >= 1 && e == cudaSuccess) e = record_event(p, s);
     LaneTable lanes{};
-    lanes.l[0] = Lane{keys, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid, idx, val};
+    lanes.l[0] = Lane{keys, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_chunk_sfx, p->d_codes, resid, idx, val};
     if (e == cudaSuccess)
         e = fused ? launch_fused_tail(p, lanes, 1, ratios, idx_cap, val_cap, prof, s)
                   : launch_selection(p, lanes, 1, idx_cap, val_cap, prof, s);
@@ -652,10 +766,10 @@ cudaError_t launch_compress_workers(rsdgc_plan *p, int n_workers, const void *co
             const int w = w0 + j;
             Lane &ln = lanes.l[j];
             if (w == 0) {
-                ln = Lane{keys_all, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_codes, resid[0], idx[0], val[0]};
+                ln = Lane{keys_all, p->d_hist, p->d_state, p->d_chunk_cnt, p->d_chunk_sfx, p->d_codes, resid[0], idx[0], val[0]};
             } else {
                 const rsdgc_plan::LaneScratch &x = p->extra_lanes[(size_t)w - 1];
-                ln = Lane{keys_all + (size_t)w * key_stride, x.hist, x.state, x.chunk_cnt, x.codes, resid[w], idx[w],
+                ln = Lane{keys_all + (size_t)w * key_stride, x.hist, x.state, x.chunk_cnt, x.chunk_sfx, x.codes, resid[w], idx[w],
                           val[w]};
             }
             // the first passes of a group's workers share nothing: all but the first start without waiting

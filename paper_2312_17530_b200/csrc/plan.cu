@@ -89,6 +89,7 @@ void free_device_tables(rsdgc_plan *p)
     cudaFree(p->d_state);
     cudaFree(p->d_hist);
     cudaFree(p->d_chunk_cnt);
+    cudaFree(p->d_chunk_sfx);
     cudaFree(p->d_codes);
     cudaFree(p->d_survivors);
     cudaFree(p->d_rstate);
@@ -98,6 +99,7 @@ void free_device_tables(rsdgc_plan *p)
         cudaFree(x.hist);
         cudaFree(x.codes);
         cudaFree(x.chunk_cnt);
+        cudaFree(x.chunk_sfx);
     }
     p->extra_lanes.clear();
     for (cudaEvent_t ev : p->events) cudaEventDestroy(ev);
@@ -422,6 +424,7 @@ extern "C" int rsdgc_plan_create(const rsdgc_layer_desc *layers_host, int32_t n_
         if (e == cudaSuccess) e = alloc_zero(&p->d_state, (size_t)n_layers);
         if (e == cudaSuccess) e = alloc_zero(&p->d_hist, (size_t)n_layers * kHistStride);
         if (e == cudaSuccess) e = alloc_zero(&p->d_chunk_cnt, p->chunks.size());
+        if (e == cudaSuccess) e = alloc_zero(&p->d_chunk_sfx, p->chunks.size() * (size_t)kL3Bins);
         if (e == cudaSuccess) e = alloc_zero(&p->d_codes, (size_t)p->info.total_tiles_padded / 4 + kChunkKeys / 4 + 16);
         if (e == cudaSuccess) e = alloc_zero(&p->d_survivors, (size_t)n_layers);
         if (e == cudaSuccess) e = alloc_zero(&p->d_rstate, 1);
@@ -623,6 +626,7 @@ extern "C" int rsdgc_plan_reserve_workers(rsdgc_plan *plan, int32_t n_workers)
         cudaError_t e = alloc_zero(&x.state, (size_t)plan->n_layers);
         if (e == cudaSuccess) e = alloc_zero(&x.hist, (size_t)plan->n_layers * kHistStride);
         if (e == cudaSuccess) e = alloc_zero(&x.chunk_cnt, plan->chunks.size());
+        if (e == cudaSuccess) e = alloc_zero(&x.chunk_sfx, plan->chunks.size() * (size_t)kL3Bins);
         if (e == cudaSuccess)
             e = alloc_zero(&x.codes, (size_t)plan->info.total_tiles_padded / 4 + kChunkKeys / 4 + 16);
         if (e == cudaSuccess) e = cudaDeviceSynchronize();
@@ -630,6 +634,7 @@ extern "C" int rsdgc_plan_reserve_workers(rsdgc_plan *plan, int32_t n_workers)
             cudaFree(x.state);
             cudaFree(x.hist);
             cudaFree(x.chunk_cnt);
+            cudaFree(x.chunk_sfx);
             cudaFree(x.codes);
             return e == cudaErrorMemoryAllocation ? RSDGC_ERR_NOMEM : cuda_fail(e);
         }

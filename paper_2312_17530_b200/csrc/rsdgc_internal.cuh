@@ -127,6 +127,7 @@ struct Lane {
     unsigned int *hist;        // n_layers * kHistStride
     LayerState *state;         // n_layers
     uint2 *chunk_cnt;          // one entry per key chunk
+    unsigned short *chunk_sfx; // kL3Bins entries per key chunk
     unsigned char *codes;      // one byte per 4 tiles
     float *resid;
     int32_t *idx;
@@ -193,14 +194,16 @@ struct rsdgc_plan {
     rsdgc::EChunk *d_echunks = nullptr;
     rsdgc::LayerState *d_state = nullptr;
     uint32_t *d_hist = nullptr;        // n_layers * kHistStride
-    unsigned char *d_codes = nullptr;  // one byte per 4 tiles: above / equal flags left by k_count for k_mark
-    uint2 *d_chunk_cnt = nullptr;      // per key chunk: (#key > T, #key == T), then exclusive bases
-    // the same four tables for workers 1.. of rsdgc_compress_workers() (worker 0 uses the ones above)
+    unsigned char *d_codes = nullptr;  // one byte per 4 tiles: "above the threshold's bin" / "in it" flags for k_mark
+    uint2 *d_chunk_cnt = nullptr;      // per key chunk: #keys above the bin, then exclusive bases (#key > T, #key == T)
+    unsigned short *d_chunk_sfx = nullptr;  // per key chunk: suffix sums of its level-3 histogram (kL3Bins entries)
+    // the same five tables for workers 1.. of rsdgc_compress_workers() (worker 0 uses the ones above)
     struct LaneScratch {
         rsdgc::LayerState *state = nullptr;
         uint32_t *hist = nullptr;
         unsigned char *codes = nullptr;
         uint2 *chunk_cnt = nullptr;
+        unsigned short *chunk_sfx = nullptr;
     };
     std::vector<LaneScratch> extra_lanes;
     long long *d_survivors = nullptr;  // ratio rule: per-layer survivor counts
