@@ -372,16 +372,17 @@ int64_t rsdgc_plan_tail_slices(const rsdgc_plan *plan, int32_t *slices_host, int
  * Optional per-kernel timing of rsdgc_compress().  While enabled, every rsdgc_compress() on
  * this plan records CUDA events on its stream: with level 1 only before and after the first
  * pass (accumulate+NSI, the kernel that moves all the bytes), with level 2 after each of the
- * RSDGC_N_COMPRESS_KERNELS stages as well (accumulate+NSI, refine level 2, refine level 3,
- * count, mark, gather; on plans that select and pack in one kernel per layer-size class: accumulate+NSI,
- * the cluster kernel, the one-CTA kernel, and three empty stages).  Events between kernels cost about 3 us each, so level 2 is for
+ * RSDGC_N_COMPRESS_KERNELS stages as well (accumulate+NSI, refine level 2, refine level 3 with
+ * the per-chunk counts, mark, gather; on plans that select and pack in one kernel per layer-size
+ * class: accumulate+NSI, the cluster kernel, the one-CTA kernel, and two empty stages).  Events
+ * between kernels cost about 3 us each, so level 2 is for
  * breakdowns, not for throughput numbers.  rsdgc_profile_read() waits for the recorded events,
  * adds the elapsed milliseconds of every timed stage over all recorded calls into
  * ms_per_kernel_host[RSDGC_N_COMPRESS_KERNELS] (untimed stages stay 0), stores the number of
  * calls and forgets them.  Level 0 (the default) records nothing; not for use during stream
  * capture.
  */
-#define RSDGC_N_COMPRESS_KERNELS 6
+#define RSDGC_N_COMPRESS_KERNELS 5
 int rsdgc_profile_enable(rsdgc_plan *plan, int32_t level);
 int rsdgc_profile_read(rsdgc_plan *plan, double *ms_per_kernel_host, int64_t *n_calls_host);
 

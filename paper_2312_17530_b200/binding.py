@@ -33,8 +33,8 @@ EXPORTS = [
     "rsdgc_selftest_bounded_wait", "rsdgc_plan_tail_slices",
 ]
 NOALLOC_MAX_LAYERS = 64
-N_COMPRESS_KERNELS = 6
-COMPRESS_KERNELS = ("accumulate_nsi", "refine2", "refine3", "count", "mark", "gather")
+N_COMPRESS_KERNELS = 5
+COMPRESS_KERNELS = ("accumulate_nsi", "refine2", "refine3_count", "mark", "gather")
 
 
 class LayerDesc(C.Structure):

@@ -289,7 +289,7 @@ __device__ bool debug_items_ok(const ItemDev *items, int begin, int end, StatusD
         const int ntr = (d.R + d.nh - 1) / d.nh;
         ok = d.R >= 1 && d.W >= 1 && d.gbase >= 0 && d.gbase + (long long)(d.R - 1) * d.cols + d.W <= status->arena_elems &&
              d.kbase >= 0 && d.kbase + (long long)(ntr - 1) * d.TC + d.ntc <= status->keys_len && d.layer >= 0 &&
-             d.layer < status->n_layers && (long long)d.R * d.P <= kItemElems;  // (every variant's stage holds at most this)
+             d.layer < status->n_layers && (long long)d.R * d.P <= kItemElemsMax;  // (no variant's stage holds more)
     }
     return !__syncthreads_or(!debug_in_bounds(ok, status));
 }
@@ -335,10 +335,10 @@ __device__ __forceinline__ void k1_tail(const ItemDev &d, int gran, const G *__r
 // k1_reg: register-staged variant (any alignment)
 // ------------------------------------------------------------------------------------------
 
-constexpr int kVecPerThread = (kItemElems + 4 * kThreads - 1) / (4 * kThreads);  // 128-bit loads of g and of r per thread
+constexpr int kVecPerThread = (kItemElemsMax + 4 * kThreads - 1) / (4 * kThreads);  // 128-bit loads of g and of r per thread
 
 struct K1RegShared {
-    float v[2][kItemElems];  // double buffer: tiles of item i are reduced while item i+1 streams in
+    float v[2][kItemElemsMax];  // double buffer: tiles of item i are reduced while item i+1 streams in
     unsigned int hist[kL1Bins];
     FlushShared fs;
 };
@@ -554,9 +554,10 @@ constexpr int kBulkThreads = RSDGC_BULK_THREADS;
 constexpr int kBulkCtasPerSm = RSDGC_BULK_CTAS;
 constexpr int kBulkCtasPerSmMomentum = 2;  // a third block per stage: 110 KB of shared memory per CTA
 // Shared-memory stages and elements per stage of a (gradient type, momentum) variant; loads run
-// kStages - 1 items ahead.  The pass is bound by the bytes it keeps in flight: with 2-byte gradients an
-// item carries a quarter fewer bytes, so that variant takes three smaller stages (two items ahead) in
-// the same shared memory instead of two.  The plan cuts its items to bulk_item_elems().
+// kStages - 1 items ahead.  The pass is bound by the bytes it keeps in flight, and an item costs a CTA
+// about one memory round trip whatever it carries: with 2-byte gradients a stage of the same number of
+// elements is a quarter smaller, so that variant may take more elements per stage within the same
+// shared memory.  The plan cuts its items to bulk_item_elems().
 template <typename G, bool MOM>
 struct BulkCfg {
     static constexpr int kStages = RSDGC_BULK_STAGES;

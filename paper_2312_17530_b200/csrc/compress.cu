@@ -1,5 +1,6 @@
 // Kernels of rsdgc_compress() after the accumulate+NSI pass: two refinement passes of the
-// per-layer radix selection, the per-chunk count/scan, the payload indices and the gather.
+// per-layer radix selection (the second leaves the per-chunk counts and their scan), the payload
+// indices and the gather.
 //
 // Ordering between CTAs comes only from kernel boundaries and from "last arriver finishes
 // the job" tickets (an atomic counter per layer and phase); no thread ever waits on another
@@ -15,11 +16,11 @@
 namespace rsdgc {
 
 // ------------------------------------------------------------------------------------------
-// K2 / K3: refinement passes over the keys (levels 2 and 3 of the radix selection)
+// K2: level 2 of the radix selection, a histogram pass over the keys
 // ------------------------------------------------------------------------------------------
 
 constexpr int kKeyVecBatch = 8;  // 128-bit key loads in flight per thread in the key passes
-constexpr int kRefineCtasPerSm = 6;  // resident CTAs per SM of k_refine (40 registers, 8 KB of shared memory)
+constexpr int kRefineCtasPerSm = 6;  // resident CTAs per SM of k_refine2 (40 registers, 8 KB of shared memory)
 
 struct RefineShared {
     unsigned int hist[kL2Bins];
@@ -30,18 +31,15 @@ struct RefineShared {
 
 // Adds the CTA's histogram of `layer` (it covers n_done chunks of the layer) to the layer's
 // global one and clears it; the CTA that accounts for the layer's last chunk finds the bin the
-// threshold falls into and extends the layer's prefix (level 2) or fixes T and e (level 3).
-template <int LEVEL>
-__device__ __forceinline__ void refine_flush(RefineShared &sh, const Lane &ln, const LayerDev *__restrict__ layers,
-                                             int layer, int n_done)
+// threshold falls into and extends the layer's prefix to 21 bits.
+__device__ __forceinline__ void refine2_flush(RefineShared &sh, const Lane &ln, const LayerDev *__restrict__ layers,
+                                              int layer, int n_done)
 {
-    constexpr int NBITS = (LEVEL == 2) ? kL2Bits : kL3Bits;
-    constexpr int NBINS = 1 << NBITS;
     const int tid = threadIdx.x;
     LayerState &st = ln.state[layer];
     unsigned int *gh = ln.hist + (size_t)layer * kHistStride;
     __syncthreads();
-    for (int b = tid; b < NBINS; b += kThreads) {
+    for (int b = tid; b < kL2Bins; b += kThreads) {
         const unsigned int n = sh.hist[b];
         if (n) {
             atomicAdd(gh + b, n);
@@ -51,18 +49,18 @@ __device__ __forceinline__ void refine_flush(RefineShared &sh, const Lane &ln, c
     __threadfence();
     __syncthreads();
     if (tid == 0) {
-        const unsigned int t = atomicAdd(&st.ticket[LEVEL - 1], (unsigned int)n_done);
+        const unsigned int t = atomicAdd(&st.ticket[1], (unsigned int)n_done);
         sh.is_last = (t + (unsigned int)n_done == (unsigned int)layers[layer].n_chunks);
     }
     __syncthreads();
     if (!sh.is_last) return;
     __threadfence();
     {
-        unsigned int h[NBINS / kThreads];
+        unsigned int h[kL2Bins / kThreads];
 #pragma unroll
-        for (int j = 0; j < NBINS / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + tid);
+        for (int j = 0; j < kL2Bins / kThreads; ++j) h[j] = __ldcg(gh + j * kThreads + tid);
 #pragma unroll
-        for (int j = 0; j < NBINS / kThreads; ++j) {
+        for (int j = 0; j < kL2Bins / kThreads; ++j) {
             sh.hist[j * kThreads + tid] = h[j];
             gh[j * kThreads + tid] = 0;
         }
@@ -71,58 +69,45 @@ __device__ __forceinline__ void refine_flush(RefineShared &sh, const Lane &ln, c
     const uint32_t prefix = st.prefix;
     const int remaining = st.remaining;
     if (prefix != kTakeNone)
-        find_bin_from_top<NBINS>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
+        find_bin_from_top<kL2Bins>(sh.hist, (unsigned long long)remaining, sh.found, sh.scan_tmp);
     if (tid == 0) {
-        st.ticket[LEVEL - 1] = 0;
+        st.ticket[1] = 0;
         if (prefix != kTakeNone) {
-            const uint32_t next = (prefix << NBITS) | (uint32_t)sh.found[0];
-            if (LEVEL == 2) {
-                st.prefix = next;
-                st.remaining = (int32_t)sh.found[1];
-            } else {
-                st.T = next;
-                st.e = (int32_t)sh.found[1];
-            }
-        } else if (LEVEL == 3) {
-            st.T = kTakeNone;
-            st.e = 0;
+            st.prefix = (prefix << kL2Bits) | (uint32_t)sh.found[0];
+            st.remaining = (int32_t)sh.found[1];
         }
     }
     __syncthreads();
-    for (int b = tid; b < NBINS; b += kThreads) sh.hist[b] = 0;  // it held the layer's totals
+    for (int b = tid; b < kL2Bins; b += kThreads) sh.hist[b] = 0;  // it held the layer's totals
     __syncthreads();
 }
 
-// LEVEL 2: among keys whose bits 30..21 equal the layer's prefix, histogram bits 20..10.
-// LEVEL 3: among keys whose bits 30..10 equal the prefix, histogram bits 9..0; the last CTA
-// of the layer then knows the threshold key T and how many keys equal to T are taken.
-// Every CTA takes a contiguous range of the key chunks (one chunk when the grid is as large as
-// the chunk list) and keeps one shared-memory histogram per layer it passes through.
-template <int LEVEL>
+// Among the keys whose bits 30..21 equal the layer's prefix (level 1, resolved by the first pass),
+// histogram bits 20..10.  Every CTA takes a contiguous range of the key chunks (one chunk when the
+// grid is as large as the chunk list) and keeps one shared-memory histogram per layer it passes through.
 __global__ void __launch_bounds__(kThreads, kRefineCtasPerSm)
-k_refine(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
-         const Chunk *__restrict__ chunks, int n_chunks_all, StatusDev *status)
+k_refine2(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ layers,
+          const Chunk *__restrict__ chunks, int n_chunks_all, StatusDev *status)
 {
     __shared__ RefineShared sh;
     const Lane &ln = lanes.l[blockIdx.y];
     const uint32_t *__restrict__ keys = ln.keys;
-    constexpr int SHIFT_HI = (LEVEL == 2) ? kL1Shift : kL2Shift;
-    constexpr int SHIFT_LO = (LEVEL == 2) ? kL2Shift : 0;
-    constexpr int NBITS = (LEVEL == 2) ? kL2Bits : kL3Bits;
-    constexpr int NBINS = 1 << NBITS;
     const int tid = threadIdx.x;
     const int chunk_begin = (int)((long long)blockIdx.x * n_chunks_all / gridDim.x);
     const int chunk_end = (int)((long long)(blockIdx.x + 1) * n_chunks_all / gridDim.x);
-    for (int b = tid; b < NBINS; b += kThreads) sh.hist[b] = 0;
+    for (int b = tid; b < kL2Bins; b += kThreads) sh.hist[b] = 0;
     grid_dependency_wait();
     grid_dependency_launch_next();
     __syncthreads();
     int cur_layer = -1, n_done = 0;
     uint32_t prefix = kTakeNone;
+    auto tally = [&](uint32_t key) {
+        if ((key >> kL1Shift) == prefix) atomicAdd(&sh.hist[(key >> kL2Shift) & (kL2Bins - 1)], 1u);
+    };
     for (int chunk_id = chunk_begin; chunk_id < chunk_end; ++chunk_id) {
         const Chunk c = chunks[chunk_id];
         if (c.layer != cur_layer) {
-            if (n_done) refine_flush<LEVEL>(sh, ln, layers, cur_layer, n_done);
+            if (n_done) refine2_flush(sh, ln, layers, cur_layer, n_done);
             cur_layer = c.layer;
             n_done = 0;
             // not yet extended by this pass: this CTA still owes the layer a chunk
@@ -144,23 +129,20 @@ k_refine(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ l
             }
 #pragma unroll
             for (int u = 0; u < kKeyVecBatch; ++u) {  // the all-ones filler never matches a prefix
-                if ((q[u].x >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].x >> SHIFT_LO) & (NBINS - 1)], 1u);
-                if ((q[u].y >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].y >> SHIFT_LO) & (NBINS - 1)], 1u);
-                if ((q[u].z >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].z >> SHIFT_LO) & (NBINS - 1)], 1u);
-                if ((q[u].w >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q[u].w >> SHIFT_LO) & (NBINS - 1)], 1u);
+                tally(q[u].x);
+                tally(q[u].y);
+                tally(q[u].z);
+                tally(q[u].w);
             }
         }
         const int i = (nvec << 2) + tid;
-        if (i < c.n) {
-            const uint32_t q = kp[i];
-            if ((q >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q >> SHIFT_LO) & (NBINS - 1)], 1u);
-        }
+        if (i < c.n) tally(kp[i]);
     }
-    if (n_done) refine_flush<LEVEL>(sh, ln, layers, cur_layer, n_done);
+    if (n_done) refine2_flush(sh, ln, layers, cur_layer, n_done);
 }
 
 // ------------------------------------------------------------------------------------------
-// K3 + K4 in one pass over the keys: level 3 of the selection AND everything the index pass needs.
+// K3: level 3 of the selection AND everything the index pass needs, in one pass over the keys.
 // When this pass runs, the upper 21 bits of a layer's threshold are known.  A key above them is kept
 // whatever level 3 finds, a key below them is not; only the keys that share them ("in the bin") depend
 // on the low 10 bits.  Per chunk the pass therefore leaves
@@ -390,7 +372,7 @@ k_refine3_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restr
 }
 
 // ------------------------------------------------------------------------------------------
-// K5: mark.  A tile is kept if its key is above T, or equals T and fewer than e equal keys
+// K4: mark.  A tile is kept if its key is above T, or equals T and fewer than e equal keys
 // precede it in the layer.  Its payload slot is its rank among the kept tiles of the layer
 // (ascending tile index).  This kernel writes the tile indices of the payload; the values are
 // moved by k_gather, whose work is spread evenly whatever the spatial pattern of the kept tiles.
@@ -494,7 +476,7 @@ k_mark(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
 }
 
 // ------------------------------------------------------------------------------------------
-// K6: gather.  Payload value j of the whole call belongs to layer l (val_off_l <= j <
+// K5: gather.  Payload value j of the whole call belongs to layer l (val_off_l <= j <
 // val_off_l + k_l * slot_l), payload slot s = (j - val_off_l) / slot_l, element el of the tile
 // idx[idx_off_l + s].  The value is moved from the residual to val and the residual entry
 // becomes +0 (Eq. 12: what is sent leaves the accumulator); with 16-bit payload values
@@ -658,7 +640,7 @@ static cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, size_t sm
     return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
-// The five kernels after the accumulate+NSI pass, one launch each for all the lanes of the call.
+// The four kernels after the accumulate+NSI pass, one launch each for all the lanes of the call.
 static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n_lanes, int64_t idx_cap,
                                     int64_t val_cap, int prof, cudaStream_t s)
 {
@@ -667,25 +649,24 @@ static cudaError_t launch_selection(rsdgc_plan *p, const LaneTable &lanes, int n
     cudaError_t e = cudaSuccess;
 #define RSDGC_MARK(level)                              \
     if (prof >= (level) && e == cudaSuccess) e = record_event(p, s)
-    // the two full key passes: one wave of resident CTAs with a contiguous chunk range each when
-    // the chunk list is much longer than that, else one CTA per chunk
     const int n_chunks = (int)p->chunks.size();
+    // The two key passes.  Contiguous ranges of chunks of EQUAL length (the last CTAs one chunk less) when the list is
+    // longer than the CTAs that fit on the device at once: with ceil(n / resident) chunks per CTA
+    // and only as many CTAs as that takes, nobody is still working on an extra chunk while the
+    // others are done.
     auto refine_grid = [&](int ctas_per_sm) {
-        const int resident = p->n_sm * ctas_per_sm;
-        return dim3((unsigned)((long long)n_chunks * n_lanes <= 2ll * resident
-                                   ? n_chunks
-                                   : std::max(1, std::min(n_chunks, resident / n_lanes))),
-                    (unsigned)n_lanes);
+        const int at_once = std::max(1, p->n_sm * ctas_per_sm / n_lanes);
+        const int per_cta = (n_chunks + at_once - 1) / at_once;
+        return dim3((unsigned)std::max(1, (n_chunks + per_cta - 1) / per_cta), (unsigned)n_lanes);
     };
     const dim3 grid_refine = refine_grid(kRefineCtasPerSm), grid_refine3 = refine_grid(kRefine3CtasPerSm);
     if (e == cudaSuccess)
-        e = launch_chained(k_refine<2>, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks, p->d_status);
+        e = launch_chained(k_refine2, grid_refine, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks, p->d_status);
     RSDGC_MARK(2);
     if (e == cudaSuccess)
         e = launch_chained(k_refine3_count, grid_refine3, 0, s, lanes, p->d_layers, p->d_chunks, n_chunks, p->n_layers,
                            (long long)idx_cap, (long long)val_cap, p->d_status);
     RSDGC_MARK(2);
-    RSDGC_MARK(2);  // (the slot of the former counting pass: level 3 leaves the counts)
     if (e == cudaSuccess)
         e = launch_chained(k_mark, grid, 0, s, lanes, p->d_layers, p->d_chunks, (long long)idx_cap, p->d_status);
     RSDGC_MARK(2);
@@ -716,7 +697,7 @@ static cudaError_t launch_fused_tail(rsdgc_plan *p, const LaneTable &lanes, int 
                                      int64_t idx_cap, int64_t val_cap, int prof, cudaStream_t s)
 {
     cudaError_t e = launch_tail(p, lanes, n_lanes, ratios, (long long)idx_cap, (long long)val_cap, prof, s, record_event);
-    for (int k = 0; k < 3 && prof >= 2 && e == cudaSuccess; ++k) e = record_event(p, s);
+    for (int k = 0; k < 2 && prof >= 2 && e == cudaSuccess; ++k) e = record_event(p, s);
     return e;
 }
 

@@ -20,10 +20,10 @@ constexpr int kItemElems = RSDGC_ITEM_ELEMS;  // elements of one accumulate+NSI 
 #define RSDGC_BF16_STAGES 2
 #endif
 #ifndef RSDGC_BF16_ITEM_ELEMS
-#define RSDGC_BF16_ITEM_ELEMS 4400
+#define RSDGC_BF16_ITEM_ELEMS 5600
 #endif
-constexpr int kItemElemsBf16 = RSDGC_BF16_ITEM_ELEMS;  // ... with bfloat16 gradients and no momentum (<= kItemElems)
-static_assert(kItemElemsBf16 <= kItemElems, "the register-staged kernel and the plan size their buffers for kItemElems");
+constexpr int kItemElemsBf16 = RSDGC_BF16_ITEM_ELEMS;  // ... with bfloat16 gradients and no momentum
+constexpr int kItemElemsMax = kItemElems > kItemElemsBf16 ? kItemElems : kItemElemsBf16;  // what the register-staged kernel holds
 constexpr int kL1Bits = 10;          // radix level 1: key bits 30..21 (8 exponent + 2 mantissa)
 constexpr int kL1Bins = 1 << kL1Bits;
 constexpr int kL1Shift = 21;
