@@ -297,26 +297,45 @@ int build_plan_tables(rsdgc_plan *p, const rsdgc_layer_desc *descs, int n_layers
     for (const LayerDev &L : p->layers)
         if ((int64_t)L.K > (int64_t)kTailCluster * kTailKeysBig) tail_ok = false;
     if (tail_ok) {
-        // layers above the one-CTA size: m slices each, all in one cluster; first fit, largest first
+        // layers above the one-CTA size: m slices each, all in one cluster; first fit, largest first.
+        // A layer needs ceil(K / 32768) slices; it gets more (a pass over a slice is a CTA's time, so
+        // the layer that decides the kernel's duration should be spread over the whole cluster) as long
+        // as the plan then takes no more clusters than with the fewest slices.
         struct Big {
             int layer, m;
         };
-        std::vector<Big> big;
-        for (int l = 0; l < n_layers; ++l)
-            if (p->layers[l].K > kTailKeysSmall)
-                big.push_back(Big{l, (int)ceil_div64(p->layers[l].K, kTailKeysBig)});
-        std::stable_sort(big.begin(), big.end(), [](const Big &a, const Big &b) { return a.m > b.m; });
         std::vector<std::vector<Big>> clusters;
-        std::vector<int> used;
-        for (const Big &b : big) {
-            size_t c = 0;
-            while (c < clusters.size() && used[c] + b.m > kTailCluster) ++c;
-            if (c == clusters.size()) {
-                clusters.emplace_back();
-                used.push_back(0);
+        auto pack = [&](int64_t slice_keys) {
+            std::vector<Big> big;
+            for (int l = 0; l < n_layers; ++l)
+                if (p->layers[l].K > kTailKeysSmall) {
+                    const int64_t K = p->layers[l].K;
+                    const int m = (int)std::max<int64_t>(ceil_div64(K, kTailKeysBig),
+                                                         std::min<int64_t>(kTailCluster, ceil_div64(K, slice_keys)));
+                    big.push_back(Big{l, m});
+                }
+            std::stable_sort(big.begin(), big.end(), [](const Big &a, const Big &b) { return a.m > b.m; });
+            std::vector<std::vector<Big>> cl;
+            std::vector<int> used;
+            for (const Big &b : big) {
+                size_t c = 0;
+                while (c < cl.size() && used[c] + b.m > kTailCluster) ++c;
+                if (c == cl.size()) {
+                    cl.emplace_back();
+                    used.push_back(0);
+                }
+                cl[c].push_back(b);
+                used[c] += b.m;
             }
-            clusters[c].push_back(b);
-            used[c] += b.m;
+            return cl;
+        };
+        clusters = pack(kTailKeysBig);
+        for (int64_t slice_keys = kTailKeysBig / 8; slice_keys < kTailKeysBig; slice_keys *= 2) {
+            std::vector<std::vector<Big>> finer = pack(slice_keys);
+            if (finer.size() <= clusters.size()) {
+                clusters = std::move(finer);
+                break;
+            }
         }
         for (const std::vector<Big> &cl : clusters) {
             int rank = 0;

@@ -153,6 +153,9 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
             sh.val_off = (long long)tv;
         }
     }
+    // every CTA's tables are cleared before anything is added to a leader's: this barrier still runs
+    // while the first pass does
+    sync_all();
     // ---- the first pass has written the keys (a kernel launched right behind a sibling of this one
     // starts only after that sibling's CTAs have passed this wait, and waits itself before it exits)
     if (!wait_late) grid_dependency_wait();
@@ -163,7 +166,6 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     uint32_t prefix = kTakeNone;   // key bits resolved so far
     unsigned int remaining = 0;    // tiles still to take among the keys that carry the prefix
     const int n4 = (sl.n + 3) >> 2;  // the slice as 128-bit words (the last one padded)
-    __syncthreads();                 // the tables cleared above
     if (active) {
         const LayerState &st = ln.state[sl.layer];
         k = __ldcg(&st.k);
@@ -200,7 +202,6 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
             }
         }
     }
-    sync_all();  // every CTA's tables are cleared before anything is added to a leader's
     if (active && prefix != kTakeNone) push_hist(kL2Bins);
     sync_all();
     if (leader && prefix != kTakeNone) resolve(remaining, kL2Bins);
@@ -212,24 +213,24 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     }
 
     // ---- one pass: a bit per key above the upper 21 bits, the candidates that share them into the list
-    // (warp w owns the keys [w * per_warp, (w + 1) * per_warp) of the slice; four groups of 32 per round)
-    constexpr int per_warp = KEYS / NW;
-    const int w0 = warp * per_warp, w1 = min(sl.n, w0 + per_warp);
+    // (a group of 32 keys is one mask word; the warps take four groups at a time, round robin, so a
+    // short slice is spread over all of them)
+    const int n_groups = (sl.n + 31) >> 5;
     if (active && prefix != kTakeNone) {
 #pragma unroll 1
-        for (int base = w0; base < w1; base += 128) {
+        for (int g0 = warp * 4; g0 < n_groups; g0 += NW * 4) {
             uint32_t key[4];
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int i = base + u * 32 + lane;
-                key[u] = (i < w1) ? skeys[i] : 0xFFFFFFFFu;
+                const int i = (g0 + u) * 32 + lane;
+                key[u] = (i < sl.n) ? skeys[i] : 0xFFFFFFFFu;
             }
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
-                const int i = base + u * 32 + lane;
+                const int i = (g0 + u) * 32 + lane;
                 const uint32_t hi = key[u] >> kL2Shift;
                 const unsigned int ma = __ballot_sync(0xFFFFFFFFu, key[u] != 0xFFFFFFFFu && hi > prefix);
-                if (lane == 0 && base + u * 32 < w1) sh.above[(base >> 5) + u] = ma;
+                if (lane == 0 && g0 + u < n_groups) sh.above[g0 + u] = ma;
                 if (hi == prefix) {
                     const unsigned int pos = atomicAdd(&sh.n_cand, 1u);
                     if (pos < (unsigned int)kTailCand) sh.cand[pos] = ((key[u] & (kL3Bins - 1)) << 15) | (unsigned int)i;
@@ -310,20 +311,20 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
             }
         } else {
 #pragma unroll 1
-            for (int base = w0; base < w1; base += 128) {
+            for (int g0 = warp * 4; g0 < n_groups; g0 += NW * 4) {
                 uint32_t key[4];
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
-                    const int i = base + u * 32 + lane;
-                    key[u] = (i < w1) ? skeys[i] : 0xFFFFFFFFu;
+                    const int i = (g0 + u) * 32 + lane;
+                    key[u] = (i < sl.n) ? skeys[i] : 0xFFFFFFFFu;
                 }
 #pragma unroll
                 for (int u = 0; u < 4; ++u) {
                     const unsigned int ma = __ballot_sync(0xFFFFFFFFu, key[u] != 0xFFFFFFFFu && key[u] > T);
                     const unsigned int me = __ballot_sync(0xFFFFFFFFu, key[u] == T);
-                    if (lane == 0 && base + u * 32 < w1) {
-                        sh.above[(base >> 5) + u] = ma;
-                        sh.equal[(base >> 5) + u] = me;
+                    if (lane == 0 && g0 + u < n_groups) {
+                        sh.above[g0 + u] = ma;
+                        sh.equal[g0 + u] = me;
                     }
                 }
             }
