@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "librsdgc_b200.so")
 SOURCES = ["plan.cu", "accumulate_nsi.cu", "compress.cu", "ratio.cu", "decompress.cu", "ratio_noalloc.cu", "coo.cu", "tail.cu"]
-HEADERS = ["rsdgc_internal.cuh", "device_utils.cuh"]
+HEADERS = ["rsdgc_internal.cuh", "device_utils.cuh", "ratio_common.cuh"]
 
 
 def _stale() -> bool:

@@ -6,7 +6,7 @@
 #include <cmath>
 #include <mutex>
 
-#include "device_utils.cuh"
+#include "ratio_common.cuh"
 
 namespace rsdgc {
 
@@ -31,25 +31,12 @@ struct NoAllocScratch {
 // until the process exits.  All calls on a device share it.
 static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
 
-struct NoAllocShared {
-    unsigned int hist[kHistStride];
-    unsigned long long gh64[kHistStride];
-    unsigned long long scan_tmp[kThreads / 32];
-    unsigned long long found[2];
-    int is_last;
-};
-
 template <int LEVEL>
 __global__ void __launch_bounds__(kThreads)
 k_ratio_noalloc(const float *__restrict__ weights, const __grid_constant__ NoAllocLayers t, NoAllocScratch *sc,
                 float *ratios, long long n_keep)
 {
-    __shared__ NoAllocShared sh;
-    constexpr int NBINS = (LEVEL == 1) ? kL1Bins : (LEVEL == 2 ? kL2Bins : kL3Bins);
-    constexpr int SHIFT_HI = (LEVEL == 1) ? 31 : (LEVEL == 2 ? kL1Shift : kL2Shift);
-    constexpr int SHIFT_LO = (LEVEL == 1) ? kL1Shift : (LEVEL == 2 ? kL2Shift : 0);
-    constexpr int BATCH = 8;
-    const int tid = threadIdx.x;
+    __shared__ RatioShared sh;
     const int n_layers = t.n_layers;
     const int n_chunks = t.chunk_begin[n_layers];
 
@@ -63,130 +50,12 @@ k_ratio_noalloc(const float *__restrict__ weights, const __grid_constant__ NoAll
     const long long start = (long long)((int)blockIdx.x - t.chunk_begin[layer]) * kChunkKeys;
     const int n = (int)min((long long)kChunkKeys, t.size[layer] - start);
 
-    const uint32_t prefix = (LEVEL == 1) ? 0u : sc->rs.prefix;  // bit 31 of |w| is 0
-    for (int b = tid; b < NBINS; b += kThreads) sh.hist[b] = 0;
-    __syncthreads();
-    if (prefix != kTakeNone) {
-        const uint32_t *wp = reinterpret_cast<const uint32_t *>(weights) + t.off[layer] + start;
-        const int nvec = n >> 2;
-        for (int base = 0; base < nvec; base += kThreads * BATCH) {
-            uint4 q[BATCH];  // all loads of a batch are issued before any is consumed
-#pragma unroll
-            for (int u = 0; u < BATCH; ++u) {
-                const int i = base + u * kThreads + tid;
-                q[u] = (i < nvec) ? __ldcs(reinterpret_cast<const uint4 *>(wp) + i) : make_uint4(0u, 0u, 0u, 0u);
-            }
-#pragma unroll
-            for (int u = 0; u < BATCH; ++u) {
-                const int i = base + u * kThreads + tid;
-                if (i < nvec) {
-                    const uint32_t k0 = q[u].x & 0x7FFFFFFFu, k1 = q[u].y & 0x7FFFFFFFu;
-                    const uint32_t k2 = q[u].z & 0x7FFFFFFFu, k3 = q[u].w & 0x7FFFFFFFu;
-                    if ((k0 >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(k0 >> SHIFT_LO) & (NBINS - 1)], 1u);
-                    if ((k1 >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(k1 >> SHIFT_LO) & (NBINS - 1)], 1u);
-                    if ((k2 >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(k2 >> SHIFT_LO) & (NBINS - 1)], 1u);
-                    if ((k3 >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(k3 >> SHIFT_LO) & (NBINS - 1)], 1u);
-                }
-            }
-        }
-        const int i = (nvec << 2) + tid;
-        if (i < n) {
-            const uint32_t q = wp[i] & 0x7FFFFFFFu;
-            if ((q >> SHIFT_HI) == prefix) atomicAdd(&sh.hist[(q >> SHIFT_LO) & (NBINS - 1)], 1u);
-        }
-    }
-    __syncthreads();
-    unsigned int *gh = sc->hist[layer];
-    for (int b = tid; b < NBINS; b += kThreads) {
-        const unsigned int c = sh.hist[b];
-        if (c) atomicAdd(gh + b, c);
-    }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const unsigned int ticket = atomicAdd(&sc->rs.ticket, 1u);
-        sh.is_last = (ticket + 1u == (unsigned int)n_chunks);
-    }
-    __syncthreads();
-    if (!sh.is_last) return;
-    __threadfence();
-
-    // ---- last CTA to arrive: totals over the layers, the bin holding the n_keep-th magnitude
-    const long long remaining = (LEVEL == 1) ? n_keep : sc->rs.remaining;
-    const bool active = (LEVEL == 1) ? (n_keep > 0) : (prefix != kTakeNone);
-    constexpr int PER = NBINS / kThreads;
-    unsigned long long gsum[PER];
-#pragma unroll
-    for (int j = 0; j < PER; ++j) gsum[j] = 0;
-    for (int l = 0; l < n_layers; ++l) {
-#pragma unroll
-        for (int j = 0; j < PER; ++j) gsum[j] += __ldcg(&sc->hist[l][j * kThreads + tid]);
-    }
-#pragma unroll
-    for (int j = 0; j < PER; ++j) sh.gh64[j * kThreads + tid] = gsum[j];
-    if (tid == 0) {
-        sh.found[0] = 0;
-        sh.found[1] = 0;
-    }
-    __syncthreads();
-    unsigned long long local = 0;
-#pragma unroll
-    for (int j = 0; j < PER; ++j) local += sh.gh64[NBINS - 1 - (tid * PER + j)];
-    unsigned long long total;
-    const unsigned long long excl = block_exclusive_scan<unsigned long long>(local, sh.scan_tmp, &total);
-    if (active && excl < (unsigned long long)remaining && (unsigned long long)remaining <= excl + local) {
-        unsigned long long run = excl;
-#pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            const int b = NBINS - 1 - (tid * PER + j);
-            const unsigned long long c = sh.gh64[b];
-            if (run < (unsigned long long)remaining && (unsigned long long)remaining <= run + c) {
-                sh.found[0] = (unsigned long long)b;
-                sh.found[1] = (unsigned long long)remaining - run;
-            }
-            run += c;
-        }
-    }
-    __syncthreads();
-    const int bin = (int)sh.found[0];
-    const long long rem_next = (long long)sh.found[1];
-
-    // ---- every layer is credited with its entries above the bin
-    const int lane = tid & 31, warp = tid >> 5;
-    for (int l = warp; l < n_layers; l += kThreads / 32) {
-        long long above = 0;
-        if (active)
-            for (int b = bin + 1 + lane; b < NBINS; b += 32) above += __ldcg(&sc->hist[l][b]);
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xFFFFFFFFu, above, d);
-        if (lane == 0) sc->survivors[l] = (LEVEL == 1 ? 0 : sc->survivors[l]) + above;
-    }
-    __syncthreads();
-    if (LEVEL == 3 && tid == 0) {
-        // entries equal to the threshold magnitude go to the layers in arena order (Eq. 4)
-        long long left = active ? rem_next : 0;
-        for (int l = 0; l < n_layers; ++l) {
-            long long take = active ? (long long)__ldcg(&sc->hist[l][bin]) : 0;
-            if (take > left) take = left;
-            left -= take;
-            const long long cl = sc->survivors[l] + take;
-            ratios[l] = (float)((double)cl / (double)t.size[l]);  // Eq. 5
-        }
-    }
-    __syncthreads();
-    // ---- the histograms and the ticket start the next level from zero
-    for (int l = 0; l < n_layers; ++l)
-        for (int b = tid; b < NBINS; b += kThreads) sc->hist[l][b] = 0;
-    if (tid == 0) {
-        sc->rs.ticket = 0;
-        if (LEVEL == 1) {
-            sc->rs.prefix = active ? (uint32_t)bin : kTakeNone;
-            sc->rs.remaining = rem_next;
-        } else if (LEVEL == 2) {
-            if (active) sc->rs.prefix = (prefix << kL2Bits) | (uint32_t)bin;
-            sc->rs.remaining = rem_next;
-        }
-    }
+    const uint32_t prefix = (LEVEL == 1) ? 0u : sc->rs.prefix;
+    ratio_histogram_chunk<LEVEL>(sh, reinterpret_cast<const uint32_t *>(weights) + t.off[layer] + start, n, prefix, true);
+    if (!ratio_flush_and_ticket<LEVEL>(sh, sc->hist[layer], &sc->rs, n_chunks)) return;
+    ratio_resolve_level<LEVEL>(
+        sh, n_layers, [&](int l) { return sc->hist[l]; }, [&](int l) { return t.size[l]; }, &sc->rs, sc->survivors,
+        ratios, n_keep, prefix);
 }
 
 // Device address of the scratch array on the current device, looked up once per device.
