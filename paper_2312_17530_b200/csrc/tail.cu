@@ -421,6 +421,11 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
     // keys before it in the layer; its slot is the number of kept tiles before it.  Only the set bits
     // are visited.
     int32_t *__restrict__ idx = ln.idx;
+    // kept tiles of this CTA: payload slots [s_first, s_first + n_kept) of the call; their indices also
+    // stay in shared memory (the keys are no longer needed), where the gather below finds them
+    const long long s_first = idx_off + lay_gt0 + min(lay_eq0, e);
+    const long long n_kept = cta_gt + (min(lay_eq0 + cta_eq, e) - min(lay_eq0, e));
+    int32_t *sidx = reinterpret_cast<int32_t *>(skeys);
     {
         int g_rank = lay_gt0 + (int)sh.warp_pre[warp][0] + (int)pg, e_rank = lay_eq0 + (int)sh.warp_pre[warp][1] + (int)pe;
 #pragma unroll
@@ -434,6 +439,7 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
                 const int gr = g_rank + __popc(ab[j] & below), er = e_rank + __popc(eq[j] & below);
                 if (((ab[j] >> bit) & 1u) || er < e) {
                     const long long s = idx_off + (gr + min(er, e));
+                    sidx[s - s_first] = tile0 + bit;
                     if (s < idx_cap) idx[s] = tile0 + bit;
                 }
             }
@@ -441,12 +447,9 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
             e_rank += __popc(eq[j]);
         }
     }
-    __syncthreads();  // the gather below reads the indices this CTA has just written
+    __syncthreads();  // the gather below reads the indices this CTA has just left in shared memory
 
     // ---- gather: the values of the kept tiles leave the accumulator (Eq. 12)
-    // kept tiles of this CTA: payload slots [s_first, s_first + n_kept) of the call
-    const long long s_first = idx_off + lay_gt0 + min(lay_eq0, e);
-    const long long n_kept = cta_gt + (min(lay_eq0 + cta_eq, e) - min(lay_eq0, e));
     const int slot = L.slot;
     // positions relative to the layer's start in the arena / in the payload fit 32 bits (a layer has
     // fewer than 2^31 elements)
@@ -471,7 +474,7 @@ k_tail(const __grid_constant__ LaneTable lanes, const LayerDev *__restrict__ lay
                 const long long s = s_first + q;
                 // tiles that do not fit the payload buffers are not sent and stay in the accumulator
                 if (s < idx_cap && val_off + (s - idx_off + 1) * slot <= val_cap) {
-                    const int tile = __ldcg(idx + s);
+                    const int tile = sidx[q];
                     const int tr = tile / L.TC, tc = tile - tr * L.TC;
                     int a, b;
                     divmod_small(el, L.nw, &a, &b);
