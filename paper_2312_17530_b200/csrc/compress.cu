@@ -227,10 +227,13 @@ __device__ __forceinline__ void refine3_flush(Refine3Shared &sh, const Lane &ln,
         const int i = base + tid;
         unsigned long long x = 0;
         if (i < L.n_chunks && prefix != kTakeNone) {
-            const unsigned int above_bin = __ldcg(&cc[i].x);
-            const unsigned int ge = __ldcg(sfx + (size_t)i * kL3Bins + bin);
-            const unsigned int gt = (bin + 1 < kL3Bins) ? (unsigned int)__ldcg(sfx + (size_t)i * kL3Bins + bin + 1) : 0u;
-            x = ((unsigned long long)(ge - gt) << 32) | (unsigned long long)(above_bin + gt);
+            const uint2 a = __ldcg(cc + i);  // (keys above the 21 bits, keys sharing them)
+            unsigned int ge = 0, gt = 0;
+            if (a.y) {
+                ge = __ldcg(sfx + (size_t)i * kL3Bins + bin);
+                if (bin + 1 < kL3Bins) gt = __ldcg(sfx + (size_t)i * kL3Bins + bin + 1);
+            }
+            x = ((unsigned long long)(ge - gt) << 32) | (unsigned long long)(a.x + gt);
         }
         unsigned long long total;
         const unsigned long long ex = block_exclusive_scan<unsigned long long>(x, sh.scan_tmp, &total) + carry;
@@ -282,7 +285,9 @@ k_refine3_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restr
     __syncthreads();
     int cur_layer = -1, n_done = 0;
     uint32_t prefix = kTakeNone;
-    for (int chunk_id = chunk_begin; chunk_id < chunk_end; ++chunk_id) {
+    // (the CTA walks its range backwards: the level-2 pass walked it forwards, so what that pass read last
+    // - about half of the keys when they exceed the L2 - is read first here and still found there)
+    for (int chunk_id = chunk_end - 1; chunk_id >= chunk_begin; --chunk_id) {
         const Chunk c = chunks[chunk_id];
         if (c.layer != cur_layer) {
             if (n_done) refine3_flush(sh, ln, layers, cur_layer, n_done, n_layers, idx_cap, val_cap, status);
@@ -299,52 +304,62 @@ k_refine3_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restr
         const uint32_t *kp = keys + L.tile_off + c.start;
         unsigned char *cp = codes + ((L.tile_off + c.start) >> 2);
         const int nvec = c.n >> 2;
-        const int nvec_all = (c.n + 3) >> 2;
-        unsigned int above = 0;
-        for (int base = 0; base < nvec_all; base += kThreads * kKeyVecBatch) {
+        // keys in [lo_key, hi_key) share the threshold's upper 21 bits, keys >= hi_key lie above them
+        // (prefix < 2^21, so hi_key <= 2^31 does not wrap)
+        const uint32_t lo_key = prefix << kL3Bits, hi_key = lo_key + (uint32_t)kL3Bins;
+        unsigned int above = 0, sharing = 0;
+        auto code_of = [&](uint32_t k0, uint32_t k1, uint32_t k2, uint32_t k3) {
+            unsigned int code = (unsigned int)(k0 >= hi_key) | ((unsigned int)(k1 >= hi_key) << 1) |
+                                ((unsigned int)(k2 >= hi_key) << 2) | ((unsigned int)(k3 >= hi_key) << 3);
+            const bool s0 = (k0 - lo_key) < (uint32_t)kL3Bins, s1 = (k1 - lo_key) < (uint32_t)kL3Bins;
+            const bool s2 = (k2 - lo_key) < (uint32_t)kL3Bins, s3 = (k3 - lo_key) < (uint32_t)kL3Bins;
+            if (s0 | s1 | s2 | s3) {  // rare: a layer has few keys that close to its threshold
+                if (s0) atomicAdd(&sh.chist[k0 & (kL3Bins - 1)], 1u);
+                if (s1) atomicAdd(&sh.chist[k1 & (kL3Bins - 1)], 1u);
+                if (s2) atomicAdd(&sh.chist[k2 & (kL3Bins - 1)], 1u);
+                if (s3) atomicAdd(&sh.chist[k3 & (kL3Bins - 1)], 1u);
+                code |= ((unsigned int)s0 << 4) | ((unsigned int)s1 << 5) | ((unsigned int)s2 << 6) | ((unsigned int)s3 << 7);
+                sharing += (unsigned int)s0 + (unsigned int)s1 + (unsigned int)s2 + (unsigned int)s3;
+            }
+            above += __popc(code & 0x0Fu);
+            return (unsigned char)code;
+        };
+        for (int base = 0; base < nvec; base += kThreads * kKeyVecBatch) {
             uint4 q[kKeyVecBatch];  // all loads of a batch are issued before any is consumed
 #pragma unroll
             for (int u = 0; u < kKeyVecBatch; ++u) {
                 const int i = base + u * kThreads + tid;
                 q[u] = (i < nvec) ? __ldg(reinterpret_cast<const uint4 *>(kp) + i) : make_uint4(0u, 0u, 0u, 0u);
-                if (i == nvec && i < nvec_all) {  // the last, partial word of the chunk; absent keys: all ones
-                    q[u] = make_uint4(~0u, ~0u, ~0u, ~0u);
-                    q[u].x = kp[4 * i];
-                    if ((c.n & 3) > 1) q[u].y = kp[4 * i + 1];
-                    if ((c.n & 3) > 2) q[u].z = kp[4 * i + 2];
-                }
             }
 #pragma unroll
             for (int u = 0; u < kKeyVecBatch; ++u) {
                 const int i = base + u * kThreads + tid;
-                if (i >= nvec_all) continue;
-                const uint32_t kx[4] = {q[u].x, q[u].y, q[u].z, q[u].w};
-                unsigned int code = 0;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t hi = kx[j] >> kL2Shift;
-                    if (kx[j] != 0xFFFFFFFFu && hi > prefix) code |= 1u << j;
-                    if (hi == prefix) {  // (an absent key's upper bits match no prefix)
-                        code |= 16u << j;
-                        atomicAdd(&sh.chist[kx[j] & (kL3Bins - 1)], 1u);
-                    }
-                }
-                cp[i] = (unsigned char)code;
-                above += __popc(code & 0x0Fu);
+                if (i < nvec) cp[i] = code_of(q[u].x, q[u].y, q[u].z, q[u].w);
             }
         }
-        // ---- the chunk's count of keys above the bin, the suffix sums of its histogram, and the
-        // histogram into the layer's
+        if ((c.n & 3) && tid == 0) {  // the last, partial word of the chunk; absent keys get no flag
+            unsigned int code = 0;
+            for (int j = 0; j < (c.n & 3); ++j) {
+                const uint32_t k = kp[4 * nvec + j];
+                if (k >= hi_key) {
+                    code |= 1u << j;
+                    ++above;
+                } else if (k - lo_key < (uint32_t)kL3Bins) {
+                    code |= 16u << j;
+                    atomicAdd(&sh.chist[k & (kL3Bins - 1)], 1u);
+                    ++sharing;
+                }
+            }
+            cp[nvec] = (unsigned char)code;
+        }
+        // ---- the chunk's count of keys above the bin; when it has keys that share the 21 bits, the suffix
+        // sums of its histogram, and the histogram into the layer's
+        const int any_sharing = __syncthreads_or((int)sharing);  // also: the chunk's histogram is complete
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) above += __shfl_xor_sync(0xFFFFFFFFu, above, d);
         if (lane == 0) sh.red[warp] = above;
-        __syncthreads();  // also: the chunk's histogram is complete
-        if (tid == 0) {
-            unsigned int a = 0;
-            for (int w = 0; w < kThreads / 32; ++w) a += sh.red[w];
-            ln.chunk_cnt[chunk_id] = make_uint2(a, 0u);
-        }
-        {
+        unsigned long long total = 0;
+        if (any_sharing) {
             constexpr int PER = kL3Bins / kThreads;  // thread t owns bins [t * PER, (t + 1) * PER)
             unsigned int h[PER];
             unsigned long long mine = 0;
@@ -353,12 +368,11 @@ k_refine3_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restr
                 h[j] = sh.chist[tid * PER + j];
                 mine += h[j];
             }
-            unsigned long long total;
             unsigned long long below = block_exclusive_scan<unsigned long long>(mine, sh.scan_tmp, &total);
             unsigned short *out = ln.chunk_sfx + (size_t)chunk_id * kL3Bins + tid * PER;
 #pragma unroll
             for (int j = 0; j < PER; ++j) {
-                out[j] = (unsigned short)(total - below);  // in-bin keys with low bits >= this bin (<= 16384)
+                out[j] = (unsigned short)(total - below);  // sharing keys with low bits >= this bin (<= 16384)
                 below += h[j];
                 if (h[j]) {
                     sh.hist[tid * PER + j] += h[j];
@@ -367,6 +381,11 @@ k_refine3_count(const __grid_constant__ LaneTable lanes, const LayerDev *__restr
             }
         }
         __syncthreads();
+        if (tid == 0) {
+            unsigned int a = 0;
+            for (int w = 0; w < kThreads / 32; ++w) a += sh.red[w];
+            ln.chunk_cnt[chunk_id] = make_uint2(a, (unsigned int)total);  // (keys above the 21 bits, keys sharing them)
+        }
     }
     if (n_done) refine3_flush(sh, ln, layers, cur_layer, n_done, n_layers, idx_cap, val_cap, status);
 }
