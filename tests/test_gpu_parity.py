@@ -76,22 +76,26 @@ def test_layer_zoo(oracle, alpha, tail):
 @pytest.mark.parametrize("tail", TAILS)
 def test_degenerate_layers(oracle, tail):
     rng = np.random.default_rng(5)
-    shapes = [(60, 60, 3, 3), (60, 60, 3, 3), (1, 900, 1, 9), (33, 33, 3, 3), (1, 7, 1, 9), (300, 300, 3, 3)]
+    shapes = [(60, 60, 3, 3), (60, 60, 3, 3), (1, 900, 1, 9), (33, 33, 3, 3), (1, 7, 1, 9), (300, 300, 3, 3),
+              (9, 15, 3, 3), (9, 18, 3, 3)]
     g = [np.zeros(3600, np.float32),                                    # all-zero layer: all NSI equal 0
          np.full(3600, 0.125, np.float32),                              # constant: all NSI equal, pure ties
          np.tile(np.arange(9, dtype=np.float32), 100),                  # identical tiles
          rng.standard_normal(33 * 33).astype(np.float32),
          rng.standard_normal(7).astype(np.float32),                    # a single clipped tile
          np.repeat(rng.integers(0, 3, 100 * 100), 9).reshape(100, 100, 3, 3).transpose(0, 2, 1, 3)
-         .reshape(-1).astype(np.float32)]                               # three distinct NSI values: many ties
+         .reshape(-1).astype(np.float32),                               # three distinct NSI values: many ties
+         np.full(9 * 15, -0.5, np.float32),                             # 15 and 18 equal keys: the tie is cut inside
+         np.full(9 * 18, 3.0, np.float32)]                              # the last, partial group of four keys
     res = [np.zeros(x.size, np.float32) for x in g]
-    for ratios, clamp in (([0.1, 0.1, 0.05, 1.0, 0.5, 0.4], True), ([0.0] * 6, True), ([0.0] * 6, False),
-                          ([1.0] * 6, True), ([0.5, 1e-9, 2.0, -1.0, 0.0, 0.33], False)):
+    for ratios, clamp in (([0.1, 0.1, 0.05, 1.0, 0.5, 0.4, 0.9, 0.9], True), ([0.0] * 8, True), ([0.0] * 8, False),
+                          ([1.0] * 8, True), ([0.5, 1e-9, 2.0, -1.0, 0.0, 0.33, 0.95, 0.5], False)):
         plan = binding.Plan(shapes, alpha=0.5, flags=(binding.KEEP_AT_LEAST_ONE if clamp else 0) | tail)
         _, refs, _ = parity.compress_and_check(oracle, plan, shapes, g, res, ratios, 0.5, clamp=clamp, what="degenerate")
         if ratios[0] == 0.1:
             k = oracle.keep_count(400, 0.1)                             # pure ties: the first k tiles
             assert refs[0].idx.tolist() == list(range(k)) and refs[1].idx.tolist() == list(range(k))
+            assert refs[6].idx.tolist() == list(range(14)) and refs[7].idx.tolist() == list(range(17))
         if not clamp and ratios[0] == 0.0:
             assert sum(r.k for r in refs) == 0
 
